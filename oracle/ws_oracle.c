@@ -1,0 +1,338 @@
+/*
+ * ws_oracle.c - CPU oracle for the sharded weight update.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition that the
+ * CUDA library is checked against.  It shares no code, header or table with
+ * the CUDA path and must never be linked into, or called from, the product.
+ *
+ * All floating-point work is done in double and every stored fp32 output is
+ * rounded exactly once (the cast at the store).  Nothing here is blocked,
+ * fused or reordered beyond what the cited passage states.  The OpenMP
+ * pragmas only split loops whose iterations are independent; every
+ * reduction (gradient sum over replicas, norm sums) runs in one fixed,
+ * ascending order on one thread.
+ *
+ * What the paper fixes and where:
+ *   - replicas sum their gradients and apply the same update      (Section 2.2)
+ *   - reduce-scatter leaves replica r one fully reduced shard, the
+ *     update runs on that shard, all-gather rebuilds the weights  (Section 2.2,
+ *     "Sharding with decomposed all-reduce")
+ *   - a tensor is reformatted (dimensions combined, then padded so
+ *     that it divides by the shard count) and dynamic-sliced by
+ *     replica id; gradient, weight and slots use one format        (Section 4.1)
+ *   - reduces over sharded data mask pads with the identity by
+ *     comparing element locations with the pad area, then combine
+ *     per-replica partial results                                  (Section 4.1,
+ *     "Non-elementwise operators")
+ *   - one combined shard holds one shard of every tensor           (Section 5.2,
+ *     "Batched communication operators")
+ *   - update in fp32, full weight gathered in bfloat16             (Section 4.2)
+ * The paper cites but does not print the optimizer formulas; the readings
+ * used here are: momentum-SGD with L2 decay added to the gradient
+ * (m' = mu m + g + wd w; w' = w - lr m'), Adam with bias correction and eps
+ * outside the root, LAMB = Adam direction plus decoupled decay, scaled per
+ * tensor by ||w|| / ||u|| (1 when either norm is zero).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+enum { WSO_SGDM = 0, WSO_ADAM = 1, WSO_LAMB = 2 };
+enum { WSO_F32 = 0, WSO_BF16 = 1 };
+
+typedef struct {
+    int32_t opt;
+    double lr, beta1, beta2, eps, weight_decay, momentum, grad_scale;
+    int64_t step; /* 1-based index of the update being applied */
+} wso_hyper;
+
+/* ---------------------------------------------------------------- bf16 -- */
+
+/* bfloat16 is the upper half of an IEEE binary32; widening is exact. */
+double wso_bf16_to_double(uint16_t h) {
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return (double)f;
+}
+
+/* binary32 -> bfloat16, round to nearest, ties to even (Section 4.2 is silent
+ * on the mode; nearest-even is the reading).  NaN stays NaN (quiet). */
+uint16_t wso_f32_to_bf16(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    if ((u & 0x7f800000u) == 0x7f800000u && (u & 0x007fffffu) != 0u)
+        return (uint16_t)((u >> 16) | 0x0040u);
+    uint32_t lower = u & 0xffffu;      /* the 16 bits that are dropped */
+    uint32_t upper = u >> 16;
+    if (lower > 0x8000u || (lower == 0x8000u && (upper & 1u))) upper += 1u;
+    return (uint16_t)upper;
+}
+
+static double load_grad(const void *p, int32_t dtype, int64_t i) {
+    if (dtype == WSO_BF16) return wso_bf16_to_double(((const uint16_t *)p)[i]);
+    return (double)((const float *)p)[i];
+}
+
+/* ---------------------------------------------------------------- plan -- */
+
+/* Sharding format of tensor t (Section 4.1): all dimensions are combined
+ * (row-major flatten, free on linear memory), the shard count R divides the
+ * flattened length after padding, and every shard ("piece") is additionally
+ * rounded up to a multiple of A elements.  One combined shard is one piece of
+ * every tensor, in tensor order (Section 5.2).  Returns S, the combined shard
+ * length; piece[t] = p_t, off[t] = start of tensor t's piece inside a shard. */
+int64_t wso_plan(const int64_t *numel, int32_t T, int32_t R, int32_t A,
+                 int64_t *piece, int64_t *off) {
+    int64_t S = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        int64_t per = (numel[t] + R - 1) / R;      /* ceil(n_t / R)        */
+        int64_t p = ((per + A - 1) / A) * A;       /* up to a multiple of A */
+        piece[t] = p;
+        off[t] = S;
+        S += p;
+    }
+    return S;
+}
+
+/* ------------------------------------------------------- pack / unpack -- */
+
+/* flat[r*S + off_t + q] = X_t[r*p_t + q] when that location exists in the
+ * tensor, else an all-zero-bits pad (Section 4.1: pad, then dynamic-slice by
+ * replica id).  elem_bytes is 4 or 2; data are copied as bits. */
+void wso_pack(const void *const *tensors, const int64_t *numel, const int64_t *piece,
+              const int64_t *off, int32_t T, int32_t R, int64_t S, int32_t elem_bytes,
+              void *flat) {
+    for (int32_t r = 0; r < R; ++r)
+        for (int32_t t = 0; t < T; ++t)
+            for (int64_t q = 0; q < piece[t]; ++q) {
+                int64_t loc = (int64_t)r * piece[t] + q;
+                char *dst = (char *)flat + ((int64_t)r * S + off[t] + q) * elem_bytes;
+                if (loc < numel[t])
+                    memcpy(dst, (const char *)tensors[t] + loc * elem_bytes, (size_t)elem_bytes);
+                else
+                    memset(dst, 0, (size_t)elem_bytes);
+            }
+}
+
+/* X_t[i] = gathered[(i div p_t)*S + off_t + i mod p_t]  (reverse formatting
+ * after the all-gather, Section 4.2). */
+void wso_unpack(const void *flat, const int64_t *numel, const int64_t *piece,
+                const int64_t *off, int32_t T, int64_t S, int32_t elem_bytes,
+                void *const *tensors) {
+    for (int32_t t = 0; t < T; ++t)
+        for (int64_t i = 0; i < numel[t]; ++i) {
+            int64_t r = i / piece[t], q = i % piece[t];
+            memcpy((char *)tensors[t] + i * elem_bytes,
+                   (const char *)flat + (r * S + off[t] + q) * elem_bytes, (size_t)elem_bytes);
+        }
+}
+
+/* -------------------------------------------------- per-element update -- */
+
+typedef struct { double bc1, bc2; } bias_corr;
+
+static bias_corr bias_of(const wso_hyper *h) {
+    bias_corr b;
+    b.bc1 = 1.0 - pow(h->beta1, (double)h->step);
+    b.bc2 = 1.0 - pow(h->beta2, (double)h->step);
+    return b;
+}
+
+/* momentum-SGD with weight decay. */
+static void sgdm_elem(const wso_hyper *h, double g, double *w, double *m) {
+    double gp = g + h->weight_decay * (*w);
+    double mn = h->momentum * (*m) + gp;
+    *m = mn;
+    *w = *w - h->lr * mn;
+}
+
+/* Adam moments; returns the bias-corrected direction mhat / (sqrt(vhat)+eps). */
+static double adam_moments(const wso_hyper *h, bias_corr b, double g, double *m, double *v) {
+    double mn = h->beta1 * (*m) + (1.0 - h->beta1) * g;
+    double vn = h->beta2 * (*v) + (1.0 - h->beta2) * g * g;
+    *m = mn;
+    *v = vn;
+    return (mn / b.bc1) / (sqrt(vn / b.bc2) + h->eps);
+}
+
+/* ------------------------------------------- unsharded definition (O) -- */
+
+/* The plain definition the sharded method must reproduce (Section 3.1: every
+ * replica would compute the same values): all-reduce = sum the R gradient
+ * copies of a whole tensor, then apply the optimizer to the whole tensor.
+ * grads[k] is replica k's gradient for THIS tensor (n elements).  w, m, v are
+ * updated in place (v unused for SGDM).  *rho receives the LAMB trust ratio
+ * (1 for the other optimizers). */
+void wso_update_tensor(const wso_hyper *h, int64_t n, int32_t R, const void *const *grads,
+                       int32_t g_dtype, float *w, float *m, float *v, double *rho) {
+    bias_corr b = bias_of(h);
+    if (rho) *rho = 1.0;
+    if (h->opt == WSO_SGDM || h->opt == WSO_ADAM) {
+#pragma omp parallel for schedule(static)
+        for (int64_t i = 0; i < n; ++i) {
+            double g = 0.0;
+            for (int32_t k = 0; k < R; ++k) g += load_grad(grads[k], g_dtype, i);
+            g *= h->grad_scale;
+            double wd = (double)w[i], md = (double)m[i];
+            if (h->opt == WSO_SGDM) {
+                sgdm_elem(h, g, &wd, &md);
+            } else {
+                double vd = (double)v[i];
+                double dir = adam_moments(h, b, g, &md, &vd);
+                wd = wd - h->lr * dir;
+                v[i] = (float)vd;
+            }
+            m[i] = (float)md;
+            w[i] = (float)wd;
+        }
+        return;
+    }
+    /* LAMB: u over the whole tensor, then the two norms, then the step. */
+    double *u = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) {
+        double g = 0.0;
+        for (int32_t k = 0; k < R; ++k) g += load_grad(grads[k], g_dtype, i);
+        g *= h->grad_scale;
+        double md = (double)m[i], vd = (double)v[i];
+        double dir = adam_moments(h, b, g, &md, &vd);
+        u[i] = dir + h->weight_decay * (double)w[i];
+        m[i] = (float)md;
+        v[i] = (float)vd;
+    }
+    double a = 0.0, bb = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        a += (double)w[i] * (double)w[i];
+        bb += u[i] * u[i];
+    }
+    double ratio = (a > 0.0 && bb > 0.0) ? sqrt(a) / sqrt(bb) : 1.0;
+    if (rho) *rho = ratio;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < n; ++i) w[i] = (float)((double)w[i] - h->lr * ratio * u[i]);
+    free(u);
+}
+
+/* ------------------------------------------ sharded route, step by step -- */
+
+/* The method's own steps on packed buffers, in the paper's order:
+ *   for every shard r: reduce the R gradient copies of slice r (reduce-scatter
+ *   arithmetic), masking pads by location; update the 1/R slice of w, m, v;
+ *   LAMB: per-(shard, tensor) partial sums of w^2 and u^2 over valid
+ *   locations, combined over shards in ascending r (the scalar all-reduce),
+ *   then the step; write w' into slot r of the gathered layout (fp32, or
+ *   bf16 rounded from the fp32 master).
+ * gpacked[k]: replica k's packed gradients, R*S elements, pads arbitrary.
+ * w, m, v: [R][S] fp32 shard-major, updated in place, pads written +0.
+ * gathered: [R][S] of out_dtype, or NULL.  rho: T doubles or NULL.
+ * partials: [R][T][2] doubles (a, b) or NULL. */
+void wso_sharded_update(const wso_hyper *h, int32_t T, const int64_t *numel,
+                        const int64_t *piece, const int64_t *off, int64_t S, int32_t R,
+                        const void *const *gpacked, int32_t g_dtype, float *w, float *m,
+                        float *v, void *gathered, int32_t out_dtype, double *rho,
+                        double *partials) {
+    bias_corr b = bias_of(h);
+    int lamb = (h->opt == WSO_LAMB);
+    double *u = NULL, *part = NULL;
+    if (lamb) {
+        u = (double *)calloc((size_t)R * (size_t)S + 1, sizeof(double));
+        part = (double *)calloc((size_t)R * (size_t)T * 2 + 1, sizeof(double));
+    }
+    for (int32_t r = 0; r < R; ++r) {
+        for (int32_t t = 0; t < T; ++t) {
+            double pa = 0.0, pb = 0.0;
+            for (int64_t q = 0; q < piece[t]; ++q) {
+                int64_t j = (int64_t)r * S + off[t] + q;   /* position in [R][S] */
+                int64_t loc = (int64_t)r * piece[t] + q;   /* iota + start offset */
+                if (loc >= numel[t]) {                      /* pad: identity / +0 */
+                    w[j] = 0.0f;
+                    m[j] = 0.0f;
+                    if (v) v[j] = 0.0f;
+                    continue;
+                }
+                double g = 0.0;
+                for (int32_t k = 0; k < R; ++k) g += load_grad(gpacked[k], g_dtype, j);
+                g *= h->grad_scale;
+                double wd = (double)w[j], md = (double)m[j];
+                if (h->opt == WSO_SGDM) {
+                    sgdm_elem(h, g, &wd, &md);
+                    w[j] = (float)wd;
+                } else {
+                    double vd = (double)v[j];
+                    double dir = adam_moments(h, b, g, &md, &vd);
+                    v[j] = (float)vd;
+                    if (lamb) {
+                        double uu = dir + h->weight_decay * wd;
+                        u[j] = uu;
+                        pa += wd * wd;
+                        pb += uu * uu;
+                    } else {
+                        w[j] = (float)(wd - h->lr * dir);
+                    }
+                }
+                m[j] = (float)md;
+            }
+            if (lamb) {
+                part[((size_t)r * T + t) * 2 + 0] = pa;
+                part[((size_t)r * T + t) * 2 + 1] = pb;
+            }
+        }
+    }
+    for (int32_t t = 0; t < T; ++t) {
+        double ratio = 1.0;
+        if (lamb) {
+            double a = 0.0, bb = 0.0;
+            for (int32_t r = 0; r < R; ++r) {              /* combine partials */
+                a += part[((size_t)r * T + t) * 2 + 0];
+                bb += part[((size_t)r * T + t) * 2 + 1];
+            }
+            ratio = (a > 0.0 && bb > 0.0) ? sqrt(a) / sqrt(bb) : 1.0;
+            for (int32_t r = 0; r < R; ++r)
+                for (int64_t q = 0; q < piece[t]; ++q) {
+                    int64_t j = (int64_t)r * S + off[t] + q;
+                    if ((int64_t)r * piece[t] + q >= numel[t]) continue;
+                    w[j] = (float)((double)w[j] - h->lr * ratio * u[j]);
+                }
+        }
+        if (rho) rho[t] = ratio;
+    }
+    if (partials && lamb) memcpy(partials, part, sizeof(double) * (size_t)R * T * 2);
+    if (gathered) {
+        int64_t G = (int64_t)R * S;
+        if (out_dtype == WSO_BF16)
+            for (int64_t j = 0; j < G; ++j) ((uint16_t *)gathered)[j] = wso_f32_to_bf16(w[j]);
+        else
+            memcpy(gathered, w, sizeof(float) * (size_t)G);
+    }
+    free(u);
+    free(part);
+}
+
+/* Reduce step alone (reduce-scatter arithmetic for shard r): out[j] =
+ * grad_scale * sum_k G_k[r*S + j] over valid locations, 0 on pads; rounded
+ * once to fp32. */
+void wso_shard_reduce(int32_t T, const int64_t *numel, const int64_t *piece, const int64_t *off,
+                      int64_t S, int32_t R, int32_t r, const void *const *gpacked,
+                      int32_t g_dtype, double grad_scale, float *out) {
+    for (int32_t t = 0; t < T; ++t)
+        for (int64_t q = 0; q < piece[t]; ++q) {
+            int64_t loc = (int64_t)r * piece[t] + q;
+            double g = 0.0;
+            if (loc < numel[t]) {
+                for (int32_t k = 0; k < R; ++k)
+                    g += load_grad(gpacked[k], g_dtype, (int64_t)r * S + off[t] + q);
+                g *= grad_scale;
+            }
+            out[off[t] + q] = (float)g;
+        }
+}
+
+int32_t wso_num_threads(void) {
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

@@ -1,0 +1,199 @@
+"""ctypes front end of the CPU oracle (``ws_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by the tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  The product package never imports this module
+and this module never imports the product's kernels or bindings.
+
+Arrays are numpy; fp32 data are ``float32`` arrays, bf16 data are ``uint16``
+arrays holding the raw bits.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+from typing import List, Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ws_oracle.c")
+_SO = os.path.join(_HERE, "libws_oracle.so")
+
+SGDM, ADAM, LAMB = 0, 1, 2
+F32, BF16 = 0, 1
+OPT_CODE = {"sgdm": SGDM, "adam": ADAM, "lamb": LAMB}
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (plain C, -O2, IEEE arithmetic, OpenMP only
+    for loops with independent iterations)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-fopenmp", "-ffp-contract=off",
+               "-o", _SO, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _SO
+
+
+class Hyper(C.Structure):
+    _fields_ = [("opt", C.c_int32), ("lr", C.c_double), ("beta1", C.c_double),
+                ("beta2", C.c_double), ("eps", C.c_double), ("weight_decay", C.c_double),
+                ("momentum", C.c_double), ("grad_scale", C.c_double), ("step", C.c_int64)]
+
+
+def make_hyper(opt, hyper: dict) -> Hyper:
+    code = OPT_CODE[opt] if isinstance(opt, str) else int(opt)
+    return Hyper(code, hyper["lr"], hyper["beta1"], hyper["beta2"], hyper["eps"],
+                 hyper["weight_decay"], hyper["momentum"], hyper["grad_scale"],
+                 int(hyper["step"]))
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        i64p, vpp = C.POINTER(C.c_int64), C.POINTER(C.c_void_p)
+        L.wso_plan.restype = C.c_int64
+        L.wso_plan.argtypes = [i64p, C.c_int32, C.c_int32, C.c_int32, i64p, i64p]
+        L.wso_pack.restype = None
+        L.wso_pack.argtypes = [vpp, i64p, i64p, i64p, C.c_int32, C.c_int32, C.c_int64,
+                               C.c_int32, C.c_void_p]
+        L.wso_unpack.restype = None
+        L.wso_unpack.argtypes = [C.c_void_p, i64p, i64p, i64p, C.c_int32, C.c_int64,
+                                 C.c_int32, vpp]
+        L.wso_update_tensor.restype = None
+        L.wso_update_tensor.argtypes = [C.POINTER(Hyper), C.c_int64, C.c_int32, vpp, C.c_int32,
+                                        C.c_void_p, C.c_void_p, C.c_void_p,
+                                        C.POINTER(C.c_double)]
+        L.wso_sharded_update.restype = None
+        L.wso_sharded_update.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p,
+                                         C.c_int64, C.c_int32, vpp, C.c_int32, C.c_void_p,
+                                         C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                         C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        L.wso_shard_reduce.restype = None
+        L.wso_shard_reduce.argtypes = [C.c_int32, i64p, i64p, i64p, C.c_int64, C.c_int32,
+                                       C.c_int32, vpp, C.c_int32, C.c_double, C.c_void_p]
+        L.wso_f32_to_bf16.restype = C.c_uint16
+        L.wso_f32_to_bf16.argtypes = [C.c_float]
+        L.wso_bf16_to_double.restype = C.c_double
+        L.wso_bf16_to_double.argtypes = [C.c_uint16]
+        L.wso_num_threads.restype = C.c_int32
+        _lib = L
+    return _lib
+
+
+def _i64(a) -> np.ndarray:
+    return np.ascontiguousarray(np.asarray(a, dtype=np.int64))
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(C.POINTER(C.c_int64))
+
+
+def _ptrs(arrs: Sequence[np.ndarray]):
+    out = (C.c_void_p * max(1, len(arrs)))()
+    for i, a in enumerate(arrs):
+        assert a.flags["C_CONTIGUOUS"]
+        out[i] = a.ctypes.data
+    return out
+
+
+def _dtype_code(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return F32
+    if a.dtype == np.uint16:
+        return BF16
+    raise TypeError(f"oracle takes float32 or uint16(bf16 bits) arrays, got {a.dtype}")
+
+
+class Plan:
+    """O1: piece sizes, in-shard offsets and the combined shard length."""
+
+    def __init__(self, numel: Sequence[int], R: int, A: int):
+        self.numel = _i64(numel)
+        self.T, self.R, self.A = len(self.numel), int(R), int(A)
+        self.piece = np.zeros(self.T, dtype=np.int64)
+        self.off = np.zeros(self.T, dtype=np.int64)
+        self.S = int(lib().wso_plan(_p(self.numel), self.T, self.R, self.A,
+                                    _p(self.piece), _p(self.off)))
+        self.G = self.R * self.S
+        self.N = int(self.numel.sum())
+
+
+def pack(plan: Plan, tensors: Sequence[np.ndarray]) -> np.ndarray:
+    dt = tensors[0].dtype if len(tensors) else np.float32
+    flat = np.empty(plan.G, dtype=dt)
+    lib().wso_pack(_ptrs(tensors), _p(plan.numel), _p(plan.piece), _p(plan.off), plan.T,
+                   plan.R, plan.S, np.dtype(dt).itemsize, flat.ctypes.data)
+    return flat
+
+
+def unpack(plan: Plan, flat: np.ndarray) -> List[np.ndarray]:
+    outs = [np.empty(int(n), dtype=flat.dtype) for n in plan.numel]
+    lib().wso_unpack(flat.ctypes.data, _p(plan.numel), _p(plan.piece), _p(plan.off), plan.T,
+                     plan.S, flat.dtype.itemsize, _ptrs(outs))
+    return outs
+
+
+def update_tensor(h: Hyper, grads: Sequence[np.ndarray], w: np.ndarray, m: np.ndarray,
+                  v: Optional[np.ndarray]) -> float:
+    """Unsharded definition on one whole tensor, in place; returns rho."""
+    rho = C.c_double(1.0)
+    n = w.size
+    lib().wso_update_tensor(C.byref(h), n, len(grads), _ptrs(grads), _dtype_code(grads[0]),
+                            w.ctypes.data, m.ctypes.data,
+                            v.ctypes.data if v is not None else None, C.byref(rho))
+    return rho.value
+
+
+def update_unsharded(h: Hyper, grads: Sequence[Sequence[np.ndarray]], w, m, v):
+    """All tensors of a model; grads[k][t].  In place.  Returns rho per tensor."""
+    T = len(w)
+    return [update_tensor(h, [g[t] for g in grads], w[t], m[t], v[t] if v is not None else None)
+            for t in range(T)]
+
+
+def sharded_update(h: Hyper, plan: Plan, gpacked: Sequence[np.ndarray], w: np.ndarray,
+                   m: np.ndarray, v: Optional[np.ndarray], out_dtype: Optional[int] = None):
+    """Sharded route on packed [R][S] buffers, in place.  Returns
+    (gathered or None, rho[T], partials[R][T][2])."""
+    rho = np.ones(plan.T, dtype=np.float64)
+    partials = np.zeros((plan.R, plan.T, 2), dtype=np.float64)
+    gathered = None
+    if out_dtype is not None:
+        gathered = np.empty(plan.G, dtype=np.uint16 if out_dtype == BF16 else np.float32)
+    lib().wso_sharded_update(
+        C.byref(h), plan.T, _p(plan.numel), _p(plan.piece), _p(plan.off), plan.S, plan.R,
+        _ptrs(gpacked), _dtype_code(gpacked[0]), w.ctypes.data, m.ctypes.data,
+        v.ctypes.data if v is not None else None,
+        gathered.ctypes.data if gathered is not None else None,
+        out_dtype if out_dtype is not None else F32,
+        rho.ctypes.data_as(C.POINTER(C.c_double)),
+        partials.ctypes.data_as(C.POINTER(C.c_double)))
+    return gathered, rho, partials
+
+
+def shard_reduce(plan: Plan, r: int, gpacked: Sequence[np.ndarray], grad_scale: float = 1.0):
+    out = np.empty(plan.S, dtype=np.float32)
+    lib().wso_shard_reduce(plan.T, _p(plan.numel), _p(plan.piece), _p(plan.off), plan.S,
+                           plan.R, r, _ptrs(gpacked), _dtype_code(gpacked[0]),
+                           float(grad_scale), out.ctypes.data)
+    return out
+
+
+def f32_to_bf16_bits(x: np.ndarray) -> np.ndarray:
+    f = lib().wso_f32_to_bf16
+    flat = np.ascontiguousarray(x, dtype=np.float32).ravel()
+    return np.array([f(float(a)) if not np.isnan(a) else f(C.c_float(float("nan")))
+                     for a in flat], dtype=np.uint16).reshape(np.shape(x))
+
+
+def bf16_bits_to_f64(x: np.ndarray) -> np.ndarray:
+    return (np.ascontiguousarray(x, dtype=np.uint16).astype(np.uint32) << 16).view(np.float32).astype(np.float64)
+
+
+def num_threads() -> int:
+    return int(lib().wso_num_threads())
