@@ -1,0 +1,224 @@
+/*
+ * ws.h - C ABI of the sharded weight update for data-parallel training.
+ *
+ * The library implements the data path of cross-replica weight-update
+ * sharding on one GPU: R logical replicas are R gradient buffers in device
+ * memory; the summed gradient of shard r (reduce-scatter arithmetic) drives a
+ * fused optimizer update of the r-th 1/R slice of weights and optimizer
+ * slots, and the updated weights are written in the all-gather output layout
+ * (paper Section 2.2, "Sharding with decomposed all-reduce").
+ *
+ * Conventions for every call
+ *   - `stream` is a cudaStream_t passed as void*.  Calls enqueue work on it and
+ *     return; they never synchronise and never allocate or free device memory.
+ *   - "device pointer" arguments must be 16-byte aligned; "host array"
+ *     arguments are read before the call returns and may be freed afterwards.
+ *   - Nothing throws or aborts across this boundary; every failure is a
+ *     ws_status.  Argument errors are found on the host before any launch.
+ *   - The caller owns every buffer.  The library owns only ws_plan objects.
+ *   - dtype arguments say how 2- or 4-byte elements are interpreted.
+ *
+ * Layout vocabulary (Section 4.1 "Sharding representation", Section 5.2
+ * "Batched communication operators"):
+ *   tensor t has n_t elements (row-major, flattened - all dimensions combined);
+ *   its piece size is p_t = A * ceil(ceil(n_t / R) / A); shard r of tensor t is
+ *   elements [r p_t, (r+1) p_t), positions >= n_t being padding;
+ *   one combined shard is piece r of every tensor back to back, tensor t at
+ *   offset off_t, so the shard length is S = sum_t p_t and a packed buffer has
+ *   G = R * S elements laid out shard-major [R][S] - the layout an all-gather
+ *   of R equal contributions produces.
+ */
+#ifndef WS_H_
+#define WS_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    WS_OK = 0,
+    WS_ERR_INVALID_ARG = 1, /* null pointer, bad count, r out of range, bad enum        */
+    WS_ERR_ALIGNMENT = 2,   /* a device pointer is not 16-byte aligned                  */
+    WS_ERR_DTYPE = 3,       /* dtype combination not supported                          */
+    WS_ERR_WORKSPACE = 4,   /* workspace missing or smaller than ws_workspace_bytes     */
+    WS_ERR_NOT_UPLOADED = 5,/* plan tables are not on the device yet (ws_plan_upload)   */
+    WS_ERR_CUDA = 6,        /* a CUDA runtime call or a launch failed                   */
+    WS_ERR_TOO_LARGE = 7    /* size beyond a documented fixed limit                     */
+} ws_status;
+
+typedef enum { WS_F32 = 0, WS_BF16 = 1 } ws_dtype;
+typedef enum { WS_SGDM = 0, WS_ADAM = 1, WS_LAMB = 2 } ws_opt;
+
+#define WS_MAX_DIMS 8
+typedef struct {
+    int32_t ndim;               /* 0..WS_MAX_DIMS; ndim == 0 is a scalar (1 element) */
+    int64_t dims[WS_MAX_DIMS];  /* every dim >= 1                                      */
+    uint32_t flags;             /* reserved, pass 0                                    */
+} ws_tensor_desc;
+
+/* One row of the segment table: tensor t inside a combined shard. */
+typedef struct {
+    int64_t numel;      /* n_t                                   */
+    int64_t piece;      /* p_t, a multiple of the alignment A    */
+    int64_t shard_off;  /* off_t, start of the piece in a shard  */
+} ws_segment;
+
+typedef struct ws_plan ws_plan;
+
+/* ---------------------------------------------------------------- plan ---
+ * Shard planner (Section 4.1: combine dimensions, pad so the shard count
+ * divides, dynamic-slice by replica id; Section 5.2: a combined shard holds
+ * one shard of every tensor).  Host only, no CUDA call.
+ *   descs       host array of T tensor descriptors, in the caller's order
+ *   R           shard count = replica count, >= 1
+ *   align_elems A: power of two >= 8, every piece is a multiple of A elements
+ *   tile_elems  work-tile length in elements used by the kernels; 0 = default
+ *               (2048); otherwise a multiple of 1024
+ *   out         receives a new plan; release with ws_plan_destroy
+ * Errors: WS_ERR_INVALID_ARG for null/empty input, bad R, A or tile size. */
+ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int32_t R, int32_t align_elems,
+                         int32_t tile_elems, ws_plan** out);
+void ws_plan_destroy(ws_plan* plan);
+
+int32_t ws_plan_num_tensors(const ws_plan* plan); /* T */
+int32_t ws_plan_num_shards(const ws_plan* plan);  /* R */
+int32_t ws_plan_align(const ws_plan* plan);       /* A */
+int64_t ws_plan_shard_elems(const ws_plan* plan); /* S */
+int64_t ws_plan_valid_elems(const ws_plan* plan); /* N = sum n_t */
+int64_t ws_plan_num_tiles(const ws_plan* plan);   /* work tiles per shard */
+/* Host view of the segment table; plan-owned, valid until ws_plan_destroy. */
+ws_status ws_plan_segments(const ws_plan* plan, const ws_segment** segs, int32_t* T);
+
+/* The kernels read the plan from device memory.  The caller provides a buffer
+ * of at least ws_plan_device_bytes(plan) bytes (16-byte aligned) that must
+ * stay alive and unmodified while the plan is in use; ws_plan_upload copies
+ * the tables into it with one cudaMemcpyAsync on `stream`.  Upload once per
+ * plan; afterwards the plan is immutable and may be shared between threads. */
+size_t ws_plan_device_bytes(const ws_plan* plan);
+ws_status ws_plan_upload(ws_plan* plan, void* dev_buf, size_t bytes, void* stream);
+
+/* ------------------------------------------------------- pack / unpack ---
+ * ws_pack: flat[r S + off_t + q] = X_t[r p_t + q] where that location exists,
+ * +0 (all-zero bits) otherwise.  This is the "sharding program" for weights
+ * and optimizer slots (Section 4.2, out-of-loop placement) and the formatting
+ * step in front of the reduce-scatter for gradients (Section 5.1).  Padding
+ * is produced in place; the tensors are never read beyond n_t.
+ *   tensor_ptrs host array of T device pointers (tensor t has n_t elements of
+ *               `dtype`, contiguous)
+ *   flat        device buffer of G = R*S elements of `dtype`, fully overwritten
+ * ws_unpack is the reverse formatting after the all-gather (the "unsharding
+ * program"): X_t[i] = flat[(i div p_t) S + off_t + i mod p_t]; pads are not
+ * read.  Both are bit copies. */
+ws_status ws_pack(const ws_plan* plan, const void* const* tensor_ptrs, ws_dtype dtype, void* flat,
+                  void* stream);
+ws_status ws_unpack(const ws_plan* plan, const void* flat, ws_dtype dtype,
+                    void* const* tensor_ptrs, void* stream);
+
+/* ------------------------------------------------------ sharded update --- */
+
+/* The R gradient copies (one per logical replica).
+ *   slice_mode 0: ptrs[k] is replica k's packed buffer of G elements; the call
+ *                 for shard r reads elements [r S, (r+1) S) of each.
+ *   slice_mode 1: ptrs[k] is the S-element slice for the shard being updated
+ *                 (what a reduce-scatter receive buffer holds); only valid with
+ *                 a single shard r >= 0.
+ * Gradient pads may hold anything: they are masked by location, never read
+ * into the result (Section 4.1, "Non-elementwise operators"). */
+typedef struct {
+    const void* const* ptrs; /* host array of R device pointers */
+    int32_t R;               /* must equal the plan's R unless slice_mode == 1 */
+    ws_dtype dtype;          /* WS_F32 or WS_BF16 */
+    int32_t slice_mode;
+} ws_grads;
+
+/* fp32 master weights and optimizer slots, kept sharded between steps
+ * (Section 2.2: auxiliary variables stay sharded across iterations).
+ * With r >= 0 each pointer is the S-element shard r.  With r == -1 each is
+ * the shard-major [R][S] buffer of all shards.  Updated in place; pads are
+ * written +0.  v is unused (may be NULL) for WS_SGDM. */
+typedef struct {
+    void* w;
+    void* m;
+    void* v;
+} ws_state;
+
+/* Hyper-parameters.  The paper cites the optimizers without printing them;
+ * the library computes, per valid element, with g = grad_scale * sum_k g_k:
+ *   WS_SGDM  m' = momentum m + g + weight_decay w;        w' = w - lr m'
+ *   WS_ADAM  m' = beta1 m + (1-beta1) g;  v' = beta2 v + (1-beta2) g^2;
+ *            w' = w - lr (m'/(1-beta1^step)) / (sqrt(v'/(1-beta2^step)) + eps)
+ *   WS_LAMB  m', v' as Adam; u = Adam direction + weight_decay w;
+ *            rho_t = ||w_t|| / ||u_t|| over tensor t (1 if either norm is 0);
+ *            w' = w - lr rho_t u
+ * `step` is the 1-based index of the update being applied.  Derived constants
+ * are formed in double on the host and narrowed to fp32 for the kernels. */
+typedef struct {
+    ws_opt opt;
+    double lr, beta1, beta2, eps, weight_decay, momentum, grad_scale;
+    int64_t step;
+} ws_hyper;
+
+/* Where the updated weights go in the all-gather output layout (Section 2.2;
+ * Section 4.2: the full weight is only needed in bfloat16 while the update
+ * stays fp32).  `gathered` is the base of a G-element buffer of `dtype`; the
+ * call for shard r overwrites slot [r S, (r+1) S) completely, pads with +0.
+ * bf16 values are the fp32 results rounded to nearest-even.  gathered may be
+ * NULL: then nothing extra is written (with r == -1 the fp32 [R][S] weight
+ * state already is the gathered layout). */
+typedef struct {
+    void* gathered;
+    ws_dtype dtype;
+} ws_out;
+
+/* Bytes of caller-provided scratch (device, 16-byte aligned) the update needs:
+ * 0 for WS_SGDM / WS_ADAM.  For WS_LAMB it holds, in this order:
+ *   float  rho[T]            trust ratios written by ws_lamb_finalize
+ *   (padding to 16 bytes)
+ *   double norms[T][2]       squared norms (sum w^2, sum u^2) per tensor
+ *   float  partials[R][tiles][2]   per-tile partial sums from phase 1
+ * so a caller can read rho and the norms back for logging. */
+size_t ws_workspace_bytes(const ws_plan* plan, ws_opt opt);
+
+/* Fused reduce + optimizer update + gathered-layout write for shard r
+ * (0 <= r < R), or for all R shards in one launch when r == -1.
+ * Reads the r-th slice of each of the R gradient buffers exactly once, w/m/v
+ * once, writes w/m/v (and the gathered slot) once (Section 2.2: the update is
+ * memory bound - read gradient, weight, auxiliaries; write weight,
+ * auxiliaries).  With opt == WS_LAMB only r == -1 is accepted here (phase 1
+ * over all shards, finalize, phase 2 over all shards): the trust ratio needs
+ * every shard's partial norms before any shard can apply (Section 4.1). */
+ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_grads* grads,
+                          const ws_state* state, const ws_hyper* hyper, const ws_out* out,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/* LAMB shard by shard (what one replica would run).  Phase 1 for shard r:
+ * reduce, moments m'/v' written, per-tile partial sums of w^2 and u^2 over
+ * valid locations stored to workspace (pads masked with the identity by
+ * comparing locations with n_t).  ws_lamb_finalize sums every shard's
+ * partials in a fixed order in double and writes rho[T]; it stands where the
+ * paper has the combined scalar all-reduce (Section 5.2), so call it after
+ * phase 1 of ALL shards.  Phase 2 for shard r recomputes u from w, m', v' and
+ * applies w' = w - lr rho u, writing the gathered slot.  `grads` is ignored
+ * by ws_lamb_apply and may be NULL there. */
+ws_status ws_lamb_partial(const ws_plan* plan, int32_t r, const ws_grads* grads,
+                          const ws_state* state, const ws_hyper* hyper, void* workspace,
+                          size_t workspace_bytes, void* stream);
+ws_status ws_lamb_finalize(const ws_plan* plan, void* workspace, size_t workspace_bytes,
+                           void* stream);
+ws_status ws_lamb_apply(const ws_plan* plan, int32_t r, const ws_state* state,
+                        const ws_hyper* hyper, const ws_out* out, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
+/* Static, never NULL. */
+const char* ws_status_string(ws_status s);
+/* Text of the last CUDA error seen by the calling thread inside this library
+ * ("" if none).  Static storage per thread. */
+const char* ws_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WS_H_ */

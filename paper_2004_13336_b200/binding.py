@@ -1,0 +1,265 @@
+"""Thin ctypes binding of libws.so: same names as the C ABI (include/ws.h),
+argument marshalling only.  Every step of the path runs in the CUDA library;
+there is no CPU fallback - loading fails loudly when the library is missing.
+
+Tensors are torch tensors used purely as device memory (``data_ptr()``) and
+streams come from ``torch.cuda.current_stream()``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libws.so")
+
+WS_OK = 0
+WS_F32, WS_BF16 = 0, 1
+WS_SGDM, WS_ADAM, WS_LAMB = 0, 1, 2
+OPT_CODE = {"sgdm": WS_SGDM, "adam": WS_ADAM, "lamb": WS_LAMB}
+WS_MAX_DIMS = 8
+
+
+class WsError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        msg = lib().ws_status_string(status).decode()
+        extra = lib().ws_last_cuda_error().decode()
+        super().__init__(f"{what}: {msg}" + (f" ({extra})" if status == 6 and extra else ""))
+
+
+class ws_tensor_desc(C.Structure):
+    _fields_ = [("ndim", C.c_int32), ("dims", C.c_int64 * WS_MAX_DIMS), ("flags", C.c_uint32)]
+
+
+class ws_segment(C.Structure):
+    _fields_ = [("numel", C.c_int64), ("piece", C.c_int64), ("shard_off", C.c_int64)]
+
+
+class ws_grads(C.Structure):
+    _fields_ = [("ptrs", C.POINTER(C.c_void_p)), ("R", C.c_int32), ("dtype", C.c_int32),
+                ("slice_mode", C.c_int32)]
+
+
+class ws_state(C.Structure):
+    _fields_ = [("w", C.c_void_p), ("m", C.c_void_p), ("v", C.c_void_p)]
+
+
+class ws_hyper(C.Structure):
+    _fields_ = [("opt", C.c_int32), ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double),
+                ("eps", C.c_double), ("weight_decay", C.c_double), ("momentum", C.c_double),
+                ("grad_scale", C.c_double), ("step", C.c_int64)]
+
+
+class ws_out(C.Structure):
+    _fields_ = [("gathered", C.c_void_p), ("dtype", C.c_int32)]
+
+
+EXPORTS = [
+    "ws_plan_create", "ws_plan_destroy", "ws_plan_num_tensors", "ws_plan_num_shards", "ws_plan_align",
+    "ws_plan_shard_elems", "ws_plan_valid_elems", "ws_plan_num_tiles", "ws_plan_segments",
+    "ws_plan_device_bytes", "ws_plan_upload", "ws_pack", "ws_unpack", "ws_workspace_bytes",
+    "ws_shard_update", "ws_lamb_partial", "ws_lamb_finalize", "ws_lamb_apply", "ws_status_string",
+    "ws_last_cuda_error",
+]
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libws.so from the package directory.  Raises if it has not been
+    built (``python -m paper_2004_13336_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2004_13336_b200.build` "
+                          "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, vpp = C.c_void_p, C.POINTER(C.c_void_p)
+    L.ws_plan_create.restype = C.c_int
+    L.ws_plan_create.argtypes = [C.POINTER(ws_tensor_desc), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                 C.POINTER(vp)]
+    L.ws_plan_destroy.restype = None
+    L.ws_plan_destroy.argtypes = [vp]
+    for name, rt in (("ws_plan_num_tensors", C.c_int32), ("ws_plan_num_shards", C.c_int32),
+                     ("ws_plan_align", C.c_int32), ("ws_plan_shard_elems", C.c_int64),
+                     ("ws_plan_valid_elems", C.c_int64), ("ws_plan_num_tiles", C.c_int64),
+                     ("ws_plan_device_bytes", C.c_size_t)):
+        getattr(L, name).restype = rt
+        getattr(L, name).argtypes = [vp]
+    L.ws_plan_segments.restype = C.c_int
+    L.ws_plan_segments.argtypes = [vp, C.POINTER(C.POINTER(ws_segment)), C.POINTER(C.c_int32)]
+    L.ws_plan_upload.restype = C.c_int
+    L.ws_plan_upload.argtypes = [vp, vp, C.c_size_t, vp]
+    L.ws_pack.restype = C.c_int
+    L.ws_pack.argtypes = [vp, vpp, C.c_int, vp, vp]
+    L.ws_unpack.restype = C.c_int
+    L.ws_unpack.argtypes = [vp, vp, C.c_int, vpp, vp]
+    L.ws_workspace_bytes.restype = C.c_size_t
+    L.ws_workspace_bytes.argtypes = [vp, C.c_int]
+    L.ws_shard_update.restype = C.c_int
+    L.ws_shard_update.argtypes = [vp, C.c_int32, C.POINTER(ws_grads), C.POINTER(ws_state),
+                                  C.POINTER(ws_hyper), C.POINTER(ws_out), vp, C.c_size_t, vp]
+    L.ws_lamb_partial.restype = C.c_int
+    L.ws_lamb_partial.argtypes = [vp, C.c_int32, C.POINTER(ws_grads), C.POINTER(ws_state),
+                                  C.POINTER(ws_hyper), vp, C.c_size_t, vp]
+    L.ws_lamb_finalize.restype = C.c_int
+    L.ws_lamb_finalize.argtypes = [vp, vp, C.c_size_t, vp]
+    L.ws_lamb_apply.restype = C.c_int
+    L.ws_lamb_apply.argtypes = [vp, C.c_int32, C.POINTER(ws_state), C.POINTER(ws_hyper),
+                                C.POINTER(ws_out), vp, C.c_size_t, vp]
+    L.ws_status_string.restype = C.c_char_p
+    L.ws_status_string.argtypes = [C.c_int]
+    L.ws_last_cuda_error.restype = C.c_char_p
+    L.ws_last_cuda_error.argtypes = []
+    _lib = L
+    return L
+
+
+def _check(status: int, what: str):
+    if status != WS_OK:
+        raise WsError(status, what)
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.float32:
+        return WS_F32
+    if dt == torch.bfloat16:
+        return WS_BF16
+    raise TypeError(f"unsupported dtype {dt}")
+
+
+def _ptr_array(tensors: Sequence[torch.Tensor]):
+    arr = (C.c_void_p * max(1, len(tensors)))()
+    for i, t in enumerate(tensors):
+        arr[i] = t.data_ptr()
+    return arr
+
+
+def make_hyper(opt, hyper: dict) -> ws_hyper:
+    code = OPT_CODE[opt] if isinstance(opt, str) else int(opt)
+    return ws_hyper(code, hyper["lr"], hyper["beta1"], hyper["beta2"], hyper["eps"],
+                    hyper["weight_decay"], hyper["momentum"], hyper["grad_scale"], int(hyper["step"]))
+
+
+class Plan:
+    """Owns a ws_plan and the device buffer that holds its tables."""
+
+    def __init__(self, shapes: Sequence[Sequence[int]], R: int, align_elems: int = 32, tile_elems: int = 0,
+                 device: Optional[torch.device] = None, upload: bool = True):
+        T = len(shapes)
+        descs = (ws_tensor_desc * max(1, T))()
+        for i, s in enumerate(shapes):
+            s = tuple(int(x) for x in s)
+            if len(s) > WS_MAX_DIMS:
+                s = (int(torch.Size(s).numel()),)
+            descs[i].ndim = len(s)
+            for j, d in enumerate(s):
+                descs[i].dims[j] = d
+        self._h = C.c_void_p()
+        _check(lib().ws_plan_create(descs, T, R, align_elems, tile_elems, C.byref(self._h)), "ws_plan_create")
+        L = lib()
+        self.T, self.R, self.A = L.ws_plan_num_tensors(self._h), L.ws_plan_num_shards(self._h), L.ws_plan_align(self._h)
+        self.S, self.N = L.ws_plan_shard_elems(self._h), L.ws_plan_valid_elems(self._h)
+        self.G = self.R * self.S
+        self.ntiles = L.ws_plan_num_tiles(self._h)
+        self.dev_buf = None
+        if upload:
+            self.upload(device)
+
+    @property
+    def handle(self):
+        return self._h
+
+    def segments(self) -> List[ws_segment]:
+        segs, T = C.POINTER(ws_segment)(), C.c_int32()
+        _check(lib().ws_plan_segments(self._h, C.byref(segs), C.byref(T)), "ws_plan_segments")
+        return [segs[i] for i in range(T.value)]
+
+    def upload(self, device=None):
+        nbytes = lib().ws_plan_device_bytes(self._h)
+        self.dev_buf = torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
+        _check(lib().ws_plan_upload(self._h, self.dev_buf.data_ptr(), nbytes, _stream()), "ws_plan_upload")
+
+    def workspace_bytes(self, opt) -> int:
+        code = OPT_CODE[opt] if isinstance(opt, str) else int(opt)
+        return lib().ws_workspace_bytes(self._h, code)
+
+    def __del__(self):
+        try:
+            if self._h:
+                lib().ws_plan_destroy(self._h)
+                self._h = None
+        except Exception:
+            pass
+
+
+def ws_pack(plan: Plan, tensors: Sequence[torch.Tensor], flat: torch.Tensor):
+    dt = _dtype_code(flat.dtype)
+    _check(lib().ws_pack(plan.handle, _ptr_array(tensors), dt, flat.data_ptr(), _stream()), "ws_pack")
+
+
+def ws_unpack(plan: Plan, flat: torch.Tensor, tensors: Sequence[torch.Tensor]):
+    dt = _dtype_code(flat.dtype)
+    _check(lib().ws_unpack(plan.handle, flat.data_ptr(), dt, _ptr_array(tensors), _stream()), "ws_unpack")
+
+
+def _grads(gbufs: Sequence[torch.Tensor], slice_mode: int):
+    arr = _ptr_array(gbufs)
+    g = ws_grads(C.cast(arr, C.POINTER(C.c_void_p)), len(gbufs), _dtype_code(gbufs[0].dtype), slice_mode)
+    g._keep = arr
+    return g
+
+
+def _state(w, m, v):
+    return ws_state(w.data_ptr(), m.data_ptr(), v.data_ptr() if v is not None else None)
+
+
+def _out(gathered):
+    if gathered is None:
+        return None
+    return ws_out(gathered.data_ptr(), _dtype_code(gathered.dtype))
+
+
+def ws_shard_update(plan: Plan, r: int, gbufs: Sequence[torch.Tensor], w, m, v, hyper: ws_hyper,
+                    gathered: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None,
+                    slice_mode: int = 0):
+    g, s, o = _grads(gbufs, slice_mode), _state(w, m, v), _out(gathered)
+    _check(lib().ws_shard_update(plan.handle, r, C.byref(g), C.byref(s), C.byref(hyper),
+                                 C.byref(o) if o is not None else None,
+                                 workspace.data_ptr() if workspace is not None else None,
+                                 workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                 _stream()), "ws_shard_update")
+
+
+def ws_lamb_partial(plan: Plan, r: int, gbufs, w, m, v, hyper: ws_hyper, workspace: torch.Tensor,
+                    slice_mode: int = 0):
+    g, s = _grads(gbufs, slice_mode), _state(w, m, v)
+    _check(lib().ws_lamb_partial(plan.handle, r, C.byref(g), C.byref(s), C.byref(hyper), workspace.data_ptr(),
+                                 workspace.numel() * workspace.element_size(), _stream()), "ws_lamb_partial")
+
+
+def ws_lamb_finalize(plan: Plan, workspace: torch.Tensor):
+    _check(lib().ws_lamb_finalize(plan.handle, workspace.data_ptr(),
+                                  workspace.numel() * workspace.element_size(), _stream()), "ws_lamb_finalize")
+
+
+def ws_lamb_apply(plan: Plan, r: int, w, m, v, hyper: ws_hyper, workspace: torch.Tensor,
+                  gathered: Optional[torch.Tensor] = None):
+    s, o = _state(w, m, v), _out(gathered)
+    _check(lib().ws_lamb_apply(plan.handle, r, C.byref(s), C.byref(hyper),
+                               C.byref(o) if o is not None else None, workspace.data_ptr(),
+                               workspace.numel() * workspace.element_size(), _stream()), "ws_lamb_apply")
+
+
+def lamb_ratios(plan: Plan, workspace: torch.Tensor) -> torch.Tensor:
+    """The trust ratios rho[T] that ws_lamb_finalize left at the start of the workspace."""
+    return workspace[: 4 * plan.T].view(torch.float32)

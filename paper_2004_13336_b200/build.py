@@ -1,0 +1,84 @@
+"""Builds libws.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
+
+    python -m paper_2004_13336_b200.build [--force] [--verbose]
+
+Each .cu file is compiled to an object in csrc/build/ (in parallel) and the
+objects are linked into paper_2004_13336_b200/libws.so.  nvcc cross-compiles
+without a GPU.
+"""
+from __future__ import annotations
+
+import concurrent.futures as cf
+import os
+import subprocess
+import sys
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_ROOT = os.path.dirname(_PKG)
+_CSRC = os.path.join(_PKG, "csrc")
+_OBJ = os.path.join(_CSRC, "build")
+LIB_PATH = os.path.join(_PKG, "libws.so")
+
+NVCC_FLAGS = [
+    "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+    "-Xcompiler", "-fPIC",
+    "-I", os.path.join(_ROOT, "include"), "-I", _CSRC,
+]
+
+
+def _nvcc() -> str:
+    for cand in (os.environ.get("NVCC"), "/usr/local/cuda/bin/nvcc", "nvcc"):
+        if cand and (os.path.isabs(cand) and os.path.exists(cand) or not os.path.isabs(cand)):
+            return cand
+    return "nvcc"
+
+
+def _sources():
+    return sorted(f for f in os.listdir(_CSRC) if f.endswith(".cu"))
+
+
+def _deps_mtime() -> float:
+    paths = [os.path.join(_CSRC, f) for f in os.listdir(_CSRC) if f.endswith((".cu", ".h", ".cuh"))]
+    paths.append(os.path.join(_ROOT, "include", "ws.h"))
+    return max(os.path.getmtime(p) for p in paths)
+
+
+def up_to_date() -> bool:
+    return os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= _deps_mtime()
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    if not force and up_to_date():
+        return LIB_PATH
+    os.makedirs(_OBJ, exist_ok=True)
+    nvcc = _nvcc()
+    extra = ["-Xptxas", "-v"] if verbose else []
+    hdr_mtime = max(os.path.getmtime(os.path.join(_CSRC, f)) for f in os.listdir(_CSRC) if f.endswith(".h"))
+    hdr_mtime = max(hdr_mtime, os.path.getmtime(os.path.join(_ROOT, "include", "ws.h")))
+
+    def compile_one(src: str) -> str:
+        obj = os.path.join(_OBJ, src[:-3] + ".o")
+        spath = os.path.join(_CSRC, src)
+        if (not force and os.path.exists(obj)
+                and os.path.getmtime(obj) >= max(os.path.getmtime(spath), hdr_mtime)):
+            return obj
+        cmd = [nvcc, *NVCC_FLAGS, *extra, "-c", spath, "-o", obj]
+        res = subprocess.run(cmd, capture_output=True, text=True)
+        if verbose:
+            sys.stderr.write(res.stderr)
+        if res.returncode != 0:
+            raise RuntimeError(f"nvcc failed for {src}:\n{res.stdout}\n{res.stderr}")
+        return obj
+
+    with cf.ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
+        objs = list(ex.map(compile_one, _sources()))
+    cmd = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB_PATH, *objs]
+    res = subprocess.run(cmd, capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError(f"link failed:\n{res.stdout}\n{res.stderr}")
+    return LIB_PATH
+
+
+if __name__ == "__main__":
+    path = build(force="--force" in sys.argv, verbose="--verbose" in sys.argv)
+    print(path)

@@ -1,0 +1,63 @@
+// Internal declarations shared by the translation units of libws.so.
+// Nothing here is part of the public ABI (see include/ws.h).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <vector>
+
+#include "ws.h"
+
+// One work tile: a run of at most `tile_elems` consecutive shard positions that
+// lies inside one tensor's piece.  A tile carries everything a kernel needs to
+// address and mask its elements, so the kernels never search the segment table.
+//   shard position of element e of the tile : pos + e
+//   index of that element in tensor `seg`    : r*piece + poff + e      (shard r)
+//   it exists in the tensor iff              : e < vt - r*piece
+struct __align__(16) WsTile {
+    long long pos;    // start inside a shard, multiple of 8
+    long long vt;     // numel - poff: valid elements from the tile start in shard 0
+    long long piece;  // p_t
+    long long poff;   // pos - off_t: start inside the piece
+    int len;          // elements in the tile, multiple of 8, <= tile_elems
+    int seg;          // tensor index t
+    int pad0, pad1;
+};
+static_assert(sizeof(WsTile) == 48, "WsTile is read as three 16-byte words");
+
+// Per tensor: which tiles of a shard belong to it (contiguous range).
+struct WsSegTiles {
+    int tile_begin;
+    int tile_count;
+};
+
+struct ws_plan {
+    int T = 0, R = 0, A = 0, K = 0;
+    long long S = 0, N = 0, ntiles = 0;
+    std::vector<ws_segment> segs;
+    std::vector<WsTile> tiles;
+    std::vector<WsSegTiles> segtiles;
+    // device copies (caller-owned memory, set by ws_plan_upload)
+    const WsTile* d_tiles = nullptr;
+    const WsSegTiles* d_segtiles = nullptr;
+};
+
+// Optimizer constants narrowed to fp32 for the kernels.
+struct WsConsts {
+    float lr, beta1, omb1, beta2, omb2, eps, wd, mu, gscale, inv_bc1, inv_bc2;
+};
+
+// LAMB workspace layout (see ws_workspace_bytes in ws.h).
+struct WsLambWs {
+    float* rho;        // [T]
+    double* norms;     // [T][2]
+    float2* partials;  // [R][ntiles]
+    size_t bytes;
+};
+WsLambWs ws_lamb_layout(const ws_plan* plan, void* workspace);
+
+// error bookkeeping
+ws_status ws_cuda_fail(cudaError_t e, const char* what);
+ws_status ws_check_launch(const char* what);
+
+static inline bool ws_aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }

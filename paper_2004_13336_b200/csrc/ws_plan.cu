@@ -1,0 +1,162 @@
+// Shard planner and plan upload (host code).
+//
+// Sharding format (paper Section 4.1): a tensor's dimensions are combined,
+// the result is padded so that the shard count divides it, and shard r is the
+// r-th equal slice.  On linear GPU memory combining ALL dimensions is free, so
+// the format is "flatten, pad, slice"; each slice (piece) is also rounded up
+// to A elements so that 16-byte vectors never straddle two tensors.
+// One combined shard is piece r of every tensor, in order (Section 5.2).
+#include <stdio.h>
+#include <string.h>
+
+#include <new>
+
+#include "ws_internal.h"
+
+static thread_local char g_cuda_err[256] = "";
+
+ws_status ws_cuda_fail(cudaError_t e, const char* what) {
+    snprintf(g_cuda_err, sizeof(g_cuda_err), "%s: %s", what, cudaGetErrorString(e));
+    return WS_ERR_CUDA;
+}
+
+ws_status ws_check_launch(const char* what) {
+    cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? WS_OK : ws_cuda_fail(e, what);
+}
+
+extern "C" const char* ws_last_cuda_error(void) { return g_cuda_err; }
+
+extern "C" const char* ws_status_string(ws_status s) {
+    switch (s) {
+        case WS_OK: return "ok";
+        case WS_ERR_INVALID_ARG: return "invalid argument";
+        case WS_ERR_ALIGNMENT: return "device pointer not 16-byte aligned";
+        case WS_ERR_DTYPE: return "unsupported dtype combination";
+        case WS_ERR_WORKSPACE: return "workspace missing or too small";
+        case WS_ERR_NOT_UPLOADED: return "plan not uploaded to the device";
+        case WS_ERR_CUDA: return "CUDA error";
+        case WS_ERR_TOO_LARGE: return "size beyond a fixed limit";
+    }
+    return "unknown status";
+}
+
+extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int32_t R,
+                                    int32_t align_elems, int32_t tile_elems, ws_plan** out) {
+    if (!out) return WS_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (!descs || T < 1 || R < 1) return WS_ERR_INVALID_ARG;
+    if (align_elems < 8 || (align_elems & (align_elems - 1)) != 0) return WS_ERR_INVALID_ARG;
+    if (tile_elems == 0) tile_elems = 2048;
+    if (tile_elems < 1024 || tile_elems % 1024 != 0 || tile_elems > (1 << 20)) return WS_ERR_INVALID_ARG;
+
+    ws_plan* p = new (std::nothrow) ws_plan;
+    if (!p) return WS_ERR_INVALID_ARG;
+    p->T = T;
+    p->R = R;
+    p->A = align_elems;
+    p->K = tile_elems;
+    try {
+        p->segs.resize(T);
+        p->segtiles.resize(T);
+        long long off = 0;
+        for (int t = 0; t < T; ++t) {
+            const ws_tensor_desc& d = descs[t];
+            if (d.ndim < 0 || d.ndim > WS_MAX_DIMS) { delete p; return WS_ERR_INVALID_ARG; }
+            long long n = 1;
+            for (int i = 0; i < d.ndim; ++i) {
+                if (d.dims[i] < 1 || n > (1LL << 46) / d.dims[i]) { delete p; return WS_ERR_INVALID_ARG; }
+                n *= d.dims[i];
+            }
+            long long per = (n + R - 1) / R;
+            long long piece = (per + align_elems - 1) / align_elems * align_elems;
+            p->segs[t].numel = n;
+            p->segs[t].piece = piece;
+            p->segs[t].shard_off = off;
+            p->N += n;
+            // cut the piece into tiles that stay inside it
+            long long ntile = (piece + tile_elems - 1) / tile_elems;
+            if ((long long)p->tiles.size() + ntile > 0x7fffffffLL) { delete p; return WS_ERR_TOO_LARGE; }
+            p->segtiles[t].tile_begin = (int)p->tiles.size();
+            p->segtiles[t].tile_count = (int)ntile;
+            for (long long i = 0; i < ntile; ++i) {
+                WsTile tl;
+                memset(&tl, 0, sizeof(tl));
+                tl.poff = i * tile_elems;
+                tl.pos = off + tl.poff;
+                tl.vt = n - tl.poff;
+                tl.piece = piece;
+                long long len = piece - tl.poff;
+                tl.len = (int)(len < tile_elems ? len : tile_elems);
+                tl.seg = t;
+                p->tiles.push_back(tl);
+            }
+            off += piece;
+        }
+        p->S = off;
+        p->ntiles = (long long)p->tiles.size();
+    } catch (...) {
+        delete p;
+        return WS_ERR_INVALID_ARG;
+    }
+    *out = p;
+    return WS_OK;
+}
+
+extern "C" void ws_plan_destroy(ws_plan* plan) { delete plan; }
+extern "C" int32_t ws_plan_num_tensors(const ws_plan* p) { return p ? p->T : 0; }
+extern "C" int32_t ws_plan_num_shards(const ws_plan* p) { return p ? p->R : 0; }
+extern "C" int32_t ws_plan_align(const ws_plan* p) { return p ? p->A : 0; }
+extern "C" int64_t ws_plan_shard_elems(const ws_plan* p) { return p ? p->S : 0; }
+extern "C" int64_t ws_plan_valid_elems(const ws_plan* p) { return p ? p->N : 0; }
+extern "C" int64_t ws_plan_num_tiles(const ws_plan* p) { return p ? p->ntiles : 0; }
+
+extern "C" ws_status ws_plan_segments(const ws_plan* p, const ws_segment** segs, int32_t* T) {
+    if (!p || !segs || !T) return WS_ERR_INVALID_ARG;
+    *segs = p->segs.data();
+    *T = p->T;
+    return WS_OK;
+}
+
+static size_t round16(size_t x) { return (x + 15) & ~(size_t)15; }
+
+extern "C" size_t ws_plan_device_bytes(const ws_plan* p) {
+    if (!p) return 0;
+    return round16(p->tiles.size() * sizeof(WsTile)) + round16(p->segtiles.size() * sizeof(WsSegTiles));
+}
+
+extern "C" ws_status ws_plan_upload(ws_plan* p, void* dev_buf, size_t bytes, void* stream) {
+    if (!p || !dev_buf) return WS_ERR_INVALID_ARG;
+    if (!ws_aligned16(dev_buf)) return WS_ERR_ALIGNMENT;
+    if (bytes < ws_plan_device_bytes(p)) return WS_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    size_t tb = p->tiles.size() * sizeof(WsTile);
+    char* base = (char*)dev_buf;
+    cudaError_t e = cudaMemcpyAsync(base, p->tiles.data(), tb, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return ws_cuda_fail(e, "ws_plan_upload(tiles)");
+    e = cudaMemcpyAsync(base + round16(tb), p->segtiles.data(), p->segtiles.size() * sizeof(WsSegTiles),
+                        cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return ws_cuda_fail(e, "ws_plan_upload(segments)");
+    p->d_tiles = (const WsTile*)base;
+    p->d_segtiles = (const WsSegTiles*)(base + round16(tb));
+    return WS_OK;
+}
+
+WsLambWs ws_lamb_layout(const ws_plan* p, void* workspace) {
+    WsLambWs L;
+    char* b = (char*)workspace;
+    size_t o = 0;
+    L.rho = (float*)(b + o);
+    o = round16(o + sizeof(float) * (size_t)p->T);
+    L.norms = (double*)(b + o);
+    o = round16(o + sizeof(double) * 2 * (size_t)p->T);
+    L.partials = (float2*)(b + o);
+    o = round16(o + sizeof(float2) * (size_t)p->R * (size_t)p->ntiles);
+    L.bytes = o;
+    return L;
+}
+
+extern "C" size_t ws_workspace_bytes(const ws_plan* p, ws_opt opt) {
+    if (!p || opt != WS_LAMB) return 0;
+    return ws_lamb_layout(p, nullptr).bytes;
+}

@@ -1,0 +1,310 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on
+the same seeded inputs.  Layout work (pack, unpack, pads, reduce on integers)
+is bit-exact; floating-point outputs use the per-tensor error metric of
+tests/_util.py with the tolerances 1e-6 (fp32 momentum-SGD / Adam), 1e-5 (LAMB
+weights and trust ratios) and 1e-2 (bf16 outputs)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import ws_oracle as O
+from paper_2004_13336_b200 import binding as B
+from paper_2004_13336_b200 import workloads as W
+from tests._util import TOL_BF16, TOL_FP32, TOL_LAMB, bf16_to_f64, err, to_np
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+# several tiles (tile = 2048 elements) per piece at small R, ragged tails, tiny and prime sizes
+SHAPES = [(1,), (7,), (3, 3, 16, 32), (64, 128), (1031,), (5, 1, 9), (4099, 3), (300, 301), (32,), (20011,)]
+RS = [1, 2, 3, 4, 7, 8, 10, 16, 64, 1024]
+
+
+def _hyper(opt, **kw):
+    h = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, momentum=0.0, grad_scale=1.0, step=10)
+    if opt == "sgdm":
+        h.update(lr=0.1, momentum=0.9, weight_decay=5e-5)
+    if opt == "lamb":
+        h.update(eps=1e-6, weight_decay=0.01)
+    h.update(kw)
+    return h
+
+
+def _model(shapes, R, gdtype=torch.float32, seed=0, gstd=1e-2):
+    wl = W.Workload("t", list(shapes), R=R, opt="adam", hyper={}, grad_dtype=gdtype, grad_std=gstd, seed=seed)
+    w, m, v = W.make_state(wl, DEV)
+    g = W.make_grads(wl, DEV)
+    return wl, w, m, v, g
+
+
+def _guarded(n, dtype, fill):
+    """n-element buffer with 64-element guard zones on both sides."""
+    big = torch.full((n + 128,), fill, dtype=dtype, device=DEV)
+    return big, big[64:64 + n]
+
+
+def _guards_intact(big, n, fill):
+    ref = torch.full((64,), fill, dtype=big.dtype, device=DEV)
+    return bool(torch.equal(big[:64], ref) and torch.equal(big[64 + n:], ref))
+
+
+def _pack_all(plan, w, m, v, g):
+    pw = torch.empty(plan.G, dtype=torch.float32, device=DEV)
+    pm, pv = torch.empty_like(pw), torch.empty_like(pw)
+    B.ws_pack(plan, w, pw)
+    B.ws_pack(plan, m, pm)
+    B.ws_pack(plan, v, pv)
+    pg = []
+    for gk in g:
+        b = torch.empty(plan.G, dtype=gk[0].dtype, device=DEV)
+        B.ws_pack(plan, gk, b)
+        pg.append(b)
+    return pw, pm, pv, pg
+
+
+def _oracle_unsharded(opt, h, w, m, v, g):
+    hs = O.make_hyper(opt, h)
+    ow, om, ov = [to_np(x) for x in w], [to_np(x) for x in m], [to_np(x) for x in v]
+    og = [[to_np(x) for x in gk] for gk in g]
+    rho = O.update_unsharded(hs, og, ow, om, ov if opt != "sgdm" else None)
+    return ow, om, ov, rho
+
+
+def _compare_state(oplan, opt, gpu_bufs, ref_lists, tol):
+    names = ["w", "m", "v"] if opt != "sgdm" else ["w", "m"]
+    for name, buf, ref in zip(names, gpu_bufs, ref_lists):
+        got = O.unpack(oplan, to_np(buf))
+        for t, (a, b) in enumerate(zip(got, ref)):
+            e = err(a, b)
+            assert e <= tol, f"{name}[{t}] err {e:.3e} > {tol}"
+
+
+def _pads_are_zero(oplan, buf):
+    valid = O.pack(oplan, [np.ones(int(n), np.float32) for n in oplan.numel]) != 0
+    a = to_np(buf)
+    bits = a.view(np.uint32) if a.dtype == np.float32 else a
+    return bool((bits[~valid] == 0).all())
+
+
+# ------------------------------------------------------------ pack/unpack ---
+@pytest.mark.parametrize("R", RS)
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("A", [8, 32])
+def test_pack_unpack_bit_exact(R, dtype, A):
+    plan = B.Plan(SHAPES, R, A)
+    oplan = O.Plan([int(np.prod(s)) for s in SHAPES], R, A)
+    gen = torch.Generator(device=DEV).manual_seed(R)
+    tensors = [torch.randn(int(n), device=DEV, generator=gen).to(dtype) for n in oplan.numel]
+    fill = 7.0
+    big, flat = _guarded(plan.G, dtype, fill)
+    B.ws_pack(plan, tensors, flat)
+    ref = O.pack(oplan, [to_np(t) for t in tensors])
+    assert to_np(flat).tobytes() == ref.tobytes()
+    assert _guards_intact(big, plan.G, fill)
+    # unpack into guarded, pre-filled tensors
+    outs = [_guarded(int(n), dtype, fill) for n in oplan.numel]
+    B.ws_unpack(plan, flat, [o[1] for o in outs])
+    for (bg, o), t, n in zip(outs, tensors, oplan.numel):
+        assert torch.equal(o, t)
+        assert _guards_intact(bg, int(n), fill)
+
+
+def test_unpack_never_reads_pads():
+    plan = B.Plan(SHAPES, 7, 32)
+    oplan = O.Plan([int(np.prod(s)) for s in SHAPES], 7, 32)
+    tensors = [torch.randn(int(n), device=DEV) for n in oplan.numel]
+    flat = torch.empty(plan.G, device=DEV)
+    B.ws_pack(plan, tensors, flat)
+    valid = torch.from_numpy(O.pack(oplan, [np.ones(int(n), np.float32) for n in oplan.numel]) != 0).to(DEV)
+    flat[~valid] = float("nan")
+    outs = [torch.empty_like(t) for t in tensors]
+    B.ws_unpack(plan, flat, outs)
+    for o, t in zip(outs, tensors):
+        assert torch.equal(o, t)
+
+
+# ------------------------------------------------------------------ reduce ---
+@pytest.mark.parametrize("R", [1, 2, 5, 8, 33, 128])
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+def test_reduce_is_exact_on_integer_gradients(R, gdtype):
+    # plain SGD with lr=1 from w=0: w' = -sum_k g_k, exact for small integers in any order
+    plan = B.Plan(SHAPES, R, 8)
+    numel = [int(np.prod(s)) for s in SHAPES]
+    gen = torch.Generator(device=DEV).manual_seed(R)
+    g = [[torch.randint(-64, 64, (n,), device=DEV, generator=gen).to(gdtype) for n in numel] for _ in range(R)]
+    w = [torch.zeros(n, device=DEV) for n in numel]
+    pw, pm, pv, pg = _pack_all(plan, w, w, w, g)
+    h = _hyper("sgdm", lr=1.0, momentum=0.0, weight_decay=0.0)
+    B.ws_shard_update(plan, -1, pg, pw, pm, None, B.make_hyper("sgdm", h))
+    outs = [torch.empty(n, device=DEV) for n in numel]
+    B.ws_unpack(plan, pw, outs)
+    for t in range(len(numel)):
+        expect = -sum(gk[t].double() for gk in g)
+        assert torch.equal(outs[t].double(), expect)
+
+
+# ------------------------------------------------------------------ update ---
+@pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb"])
+@pytest.mark.parametrize("R", [1, 2, 3, 4, 8, 10, 16, 64])
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+def test_update_all_shards_matches_oracle(opt, R, gdtype):
+    A = 32
+    wl, w, m, v, g = _model(SHAPES, R, gdtype, seed=R)
+    plan = B.Plan(SHAPES, R, A)
+    oplan = O.Plan(wl.numels, R, A)
+    h = _hyper(opt)
+    ow, om, ov, orho = _oracle_unsharded(opt, h, w, m, v, g)
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    gath32 = torch.full((plan.G,), 9.0, device=DEV)
+    ws = torch.empty(max(16, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv if opt != "sgdm" else None, B.make_hyper(opt, h), gath32, ws)
+    tol = TOL_LAMB if opt == "lamb" else TOL_FP32
+    bufs = [pw, pm, pv] if opt != "sgdm" else [pw, pm]
+    refs = [ow, om, ov] if opt != "sgdm" else [ow, om]
+    # moments are plain Adam arithmetic for LAMB too
+    _compare_state(oplan, opt, bufs[1:], refs[1:], TOL_FP32)
+    _compare_state(oplan, opt, bufs[:1], refs[:1], tol)
+    for b in bufs:
+        assert _pads_are_zero(oplan, b)
+    assert torch.equal(gath32, pw)            # fp32 gathered slot == fp32 master, pads +0
+    if opt == "lamb":
+        rho = B.lamb_ratios(plan, ws).cpu().numpy().astype(np.float64)
+        rel = np.abs(rho - np.array(orho)) / np.array(orho)
+        assert rel.max() <= TOL_LAMB, rel.max()
+
+
+@pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb"])
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+def test_bf16_gathered_copy(opt, gdtype):
+    R, A = 4, 32
+    wl, w, m, v, g = _model(SHAPES, R, gdtype, seed=11)
+    plan = B.Plan(SHAPES, R, A)
+    oplan = O.Plan(wl.numels, R, A)
+    h = _hyper(opt)
+    ow, _, _, _ = _oracle_unsharded(opt, h, w, m, v, g)
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    gath = torch.full((plan.G,), 3.0, dtype=torch.bfloat16, device=DEV)
+    ws = torch.empty(max(16, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv if opt != "sgdm" else None, B.make_hyper(opt, h), gath, ws)
+    # bit-exact self-consistency: bf16 copy == round-to-nearest-even of the fp32 master
+    assert torch.equal(gath, pw.to(torch.bfloat16))
+    assert to_np(gath).tobytes() == O.f32_to_bf16_bits(to_np(pw)).tobytes()
+    assert _pads_are_zero(oplan, gath)
+    got = O.unpack(oplan, to_np(gath))
+    for a, b in zip(got, ow):
+        assert err(bf16_to_f64(a), b) <= TOL_BF16
+
+
+@pytest.mark.parametrize("opt", ["sgdm", "adam"])
+@pytest.mark.parametrize("R", [1, 3, 8])
+@pytest.mark.parametrize("slice_mode", [0, 1])
+def test_per_shard_calls_equal_all_shard_launch(opt, R, slice_mode):
+    wl, w, m, v, g = _model(SHAPES, R, seed=5)
+    plan = B.Plan(SHAPES, R, 32)
+    h = B.make_hyper(opt, _hyper(opt))
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    aw, am, av = pw.clone(), pm.clone(), pv.clone()
+    ga = torch.zeros(plan.G, device=DEV)
+    B.ws_shard_update(plan, -1, pg, aw, am, av if opt != "sgdm" else None, h, ga)
+    gb = torch.zeros(plan.G, device=DEV)
+    S = plan.S
+    for r in range(R):
+        sl = slice(r * S, (r + 1) * S)
+        gr = [b[sl] for b in pg] if slice_mode == 1 else pg
+        B.ws_shard_update(plan, r, gr, pw[sl], pm[sl], pv[sl] if opt != "sgdm" else None, h, gb,
+                          slice_mode=slice_mode)
+    assert torch.equal(aw, pw) and torch.equal(am, pm) and torch.equal(ga, gb)
+    if opt == "adam":
+        assert torch.equal(av, pv)
+
+
+@pytest.mark.parametrize("R", [1, 3, 8])
+def test_lamb_shard_by_shard_phases(R):
+    wl, w, m, v, g = _model(SHAPES, R, seed=6)
+    plan = B.Plan(SHAPES, R, 32)
+    h = B.make_hyper("lamb", _hyper("lamb"))
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    aw, am, av = pw.clone(), pm.clone(), pv.clone()
+    wsa = torch.zeros(plan.workspace_bytes("lamb"), dtype=torch.uint8, device=DEV)
+    wsb = torch.zeros_like(wsa)
+    ga = torch.zeros(plan.G, dtype=torch.bfloat16, device=DEV)
+    gb = torch.zeros_like(ga)
+    B.ws_shard_update(plan, -1, pg, aw, am, av, h, ga, wsa)
+    S = plan.S
+    for r in range(R):
+        sl = slice(r * S, (r + 1) * S)
+        B.ws_lamb_partial(plan, r, pg, pw[sl], pm[sl], pv[sl], h, wsb)
+    B.ws_lamb_finalize(plan, wsb)
+    for r in range(R):
+        sl = slice(r * S, (r + 1) * S)
+        B.ws_lamb_apply(plan, r, pw[sl], pm[sl], pv[sl], h, wsb, gb)
+    assert torch.equal(wsa, wsb)
+    assert torch.equal(aw, pw) and torch.equal(am, pm) and torch.equal(av, pv) and torch.equal(ga, gb)
+
+
+@pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb"])
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+def test_poisoned_pads_never_leak(opt, gdtype):
+    R, A = 7, 32
+    wl, w, m, v, g = _model(SHAPES, R, gdtype, seed=3)
+    plan = B.Plan(SHAPES, R, A)
+    oplan = O.Plan(wl.numels, R, A)
+    hy = B.make_hyper(opt, _hyper(opt))
+    valid = torch.from_numpy(O.pack(oplan, [np.ones(int(n), np.float32) for n in oplan.numel]) != 0).to(DEV)
+    results = []
+    for poison in (False, True):
+        pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+        if poison:
+            for b in [pw, pm, pv] + pg:
+                b[~valid] = float("nan")
+        gath = torch.full((plan.G,), 5.0, dtype=torch.bfloat16, device=DEV)
+        ws = torch.zeros(max(16, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+        B.ws_shard_update(plan, -1, pg, pw, pm, pv if opt != "sgdm" else None, hy, gath, ws)
+        out = [pw, pm, gath] + ([pv] if opt != "sgdm" else [])
+        if opt == "lamb":
+            out.append(B.lamb_ratios(plan, ws).clone())
+        results.append(out)
+    for a, b in zip(*results):
+        assert torch.equal(a, b)
+    for b in results[1][:4 if opt != "sgdm" else 3]:
+        assert _pads_are_zero(oplan, b)
+
+
+@pytest.mark.parametrize("R,mode", [(128, "sum"), (1024, "sum"), (1024, "mean")])
+def test_many_replicas_small_shards(R, mode):
+    # tiny shards (pieces of one alignment unit) and a long gradient sum
+    shapes = [(1024,), (1,), (257, 33), (64, 64)]
+    wl, w, m, v, g = _model(shapes, R, seed=R, gstd=1e-3)
+    plan = B.Plan(shapes, R, 8)
+    oplan = O.Plan(wl.numels, R, 8)
+    h = _hyper("adam", grad_scale=1.0 if mode == "sum" else 1.0 / R)
+    ow, om, ov, _ = _oracle_unsharded("adam", h, w, m, v, g)
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv, B.make_hyper("adam", h))
+    _compare_state(oplan, "adam", [pw, pm, pv], [ow, om, ov], TOL_FP32)
+
+
+def test_argument_errors_are_status_codes():
+    import ctypes as C
+    plan = B.Plan([(64,), (100,)], 2, 8)
+    L = B.lib()
+    buf = torch.zeros(plan.G + 8, device=DEV)
+    hy = B.make_hyper("adam", _hyper("adam"))
+    s = B.ws_state(buf.data_ptr(), buf.data_ptr(), buf.data_ptr())
+    ptrs = (C.c_void_p * 2)(buf.data_ptr(), buf.data_ptr())
+    g = B.ws_grads(C.cast(ptrs, C.POINTER(C.c_void_p)), 2, 0, 0)
+    call = lambda r, gg, ss: L.ws_shard_update(plan.handle, r, C.byref(gg), C.byref(ss), C.byref(hy), None, None, 0, None)
+    assert call(2, g, s) == 1 and call(-2, g, s) == 1                       # r out of range
+    bad = B.ws_state(buf.data_ptr() + 4, buf.data_ptr(), buf.data_ptr())
+    assert call(0, g, bad) == 2                                              # misaligned
+    g3 = B.ws_grads(C.cast(ptrs, C.POINTER(C.c_void_p)), 3, 0, 0)
+    assert call(0, g3, s) == 1                                               # R mismatch
+    g1 = B.ws_grads(C.cast(ptrs, C.POINTER(C.c_void_p)), 2, 0, 1)
+    assert call(-1, g1, s) == 1                                              # slice mode needs one shard
+    gd = B.ws_grads(C.cast(ptrs, C.POINTER(C.c_void_p)), 2, 7, 0)
+    assert call(0, gd, s) == 3                                               # dtype
+    hl = B.make_hyper("lamb", _hyper("lamb"))
+    assert L.ws_shard_update(plan.handle, -1, C.byref(g), C.byref(s), C.byref(hl), None, None, 0, None) == 4
+    assert L.ws_shard_update(plan.handle, 0, C.byref(g), C.byref(s), C.byref(hl), None, None, 0, None) == 1
+    torch.cuda.synchronize()
+    assert float(buf.abs().sum()) == 0.0                                     # nothing was launched

@@ -1,0 +1,110 @@
+"""Host-side checks that need no GPU: the C-ABI library loads and exports every
+symbol the public header declares, the shard planner (pure host code) agrees
+bit for bit with the oracle's independent planner, and argument errors are
+reported as status codes before any launch."""
+import ctypes as C
+import os
+import re
+
+import numpy as np
+import pytest
+
+from oracle import ws_oracle as O
+from paper_2004_13336_b200 import binding as B
+from paper_2004_13336_b200 import build as ws_build
+from paper_2004_13336_b200 import workloads as W
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    ws_build.build()
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "ws.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ws_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = _declared_symbols()
+    assert len(names) >= 18
+    raw = C.CDLL(B.LIB_PATH)
+    for n in names:
+        assert hasattr(raw, n), f"{n} declared in ws.h but not exported"
+    assert sorted(B.EXPORTS) == names
+
+
+def test_status_strings():
+    L = B.lib()
+    assert L.ws_status_string(0) == b"ok"
+    for s in range(1, 8):
+        assert len(L.ws_status_string(s)) > 0
+
+
+@pytest.mark.parametrize("R", [1, 2, 3, 8, 10, 64, 1024])
+@pytest.mark.parametrize("A", [8, 32, 128])
+def test_planner_matches_oracle_planner(R, A):
+    shapes = [(1,), (7,), (3, 3, 16, 32), (64, 128), (1031,), (5, 1, 9), (4096, 3)]
+    plan = B.Plan(shapes, R, A, upload=False)
+    ref = O.Plan([int(np.prod(s)) for s in shapes], R, A)
+    assert (plan.S, plan.N, plan.T, plan.R, plan.A) == (ref.S, ref.N, ref.T, R, A)
+    for t, sg in enumerate(plan.segments()):
+        assert (sg.numel, sg.piece, sg.shard_off) == (ref.numel[t], ref.piece[t], ref.off[t])
+
+
+def test_planner_on_model_shaped_workloads():
+    for name in ("tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b"):
+        wl = W.WORKLOADS[name]()
+        plan = B.Plan(wl.shapes, wl.R, 32, upload=False)
+        ref = O.Plan(wl.numels, wl.R, 32)
+        assert (plan.S, plan.N) == (ref.S, ref.N)
+        segs = plan.segments()
+        assert [s.piece for s in segs] == list(ref.piece)
+        assert [s.shard_off for s in segs] == list(ref.off)
+        # tiles cover each piece exactly once, in order
+        assert plan.ntiles == sum(-(-int(p) // 2048) for p in ref.piece)
+
+
+def test_paper_worked_numbers_through_the_library():
+    # Section 5.2 (4 MB / 2048 ways = 2 KB) and Section 4.1 ([3,3,256,256] at 8, 10 and 64 ways)
+    p = B.Plan([(1024, 1024)], 2048, 8, upload=False)
+    assert p.S * 4 == 2048
+    assert B.Plan([(3, 3, 256, 256)], 64, 8, upload=False).S == 9216
+    assert B.Plan([(3, 3, 256, 256)], 8, 8, upload=False).S == 73728
+    assert B.Plan([(3, 3, 256, 256)], 10, 32, upload=False).S * 10 <= 10 * 256 * 256
+
+
+def test_plan_create_rejects_bad_arguments():
+    L = B.lib()
+    d = (B.ws_tensor_desc * 1)()
+    d[0].ndim = 1
+    d[0].dims[0] = 10
+    h = C.c_void_p()
+    assert L.ws_plan_create(d, 1, 0, 32, 0, C.byref(h)) == 1          # R < 1
+    assert L.ws_plan_create(d, 1, 4, 12, 0, C.byref(h)) == 1          # A not a power of two
+    assert L.ws_plan_create(d, 1, 4, 4, 0, C.byref(h)) == 1           # A < 8
+    assert L.ws_plan_create(d, 0, 4, 32, 0, C.byref(h)) == 1          # empty list
+    assert L.ws_plan_create(d, 1, 4, 32, 1000, C.byref(h)) == 1       # tile not a multiple of 1024
+    assert L.ws_plan_create(None, 1, 4, 32, 0, C.byref(h)) == 1
+    d[0].dims[0] = 0
+    assert L.ws_plan_create(d, 1, 4, 32, 0, C.byref(h)) == 1          # empty dimension
+    assert not h.value
+
+
+def test_calls_fail_cleanly_before_upload():
+    # no device buffer yet: every data call must refuse without touching CUDA
+    L = B.lib()
+    plan = B.Plan([(64,)], 2, 8, upload=False)
+    ptrs = (C.c_void_p * 1)(16)
+    assert L.ws_pack(plan.handle, ptrs, 0, 16, None) == 5
+    assert L.ws_unpack(plan.handle, 16, 0, ptrs, None) == 5
+    g = B.ws_grads(C.cast((C.c_void_p * 2)(16, 16), C.POINTER(C.c_void_p)), 2, 0, 0)
+    s = B.ws_state(16, 16, 16)
+    hy = B.make_hyper("adam", W.tiny().hyper)
+    assert L.ws_shard_update(plan.handle, 0, C.byref(g), C.byref(s), C.byref(hy), None, None, 0, None) == 5
+    assert L.ws_shard_update(None, 0, C.byref(g), C.byref(s), C.byref(hy), None, None, 0, None) == 1
+    assert plan.workspace_bytes("adam") == 0 and plan.workspace_bytes("sgdm") == 0
+    assert plan.workspace_bytes("lamb") >= 4 * 1 + 16 * 1 + 8 * 2 * plan.ntiles
