@@ -1,0 +1,449 @@
+#!/usr/bin/env python
+"""Benchmark of the sharded weight update (one JSON line on stdout).
+
+A step is one pass of the whole hot path over one model-shaped set of synthetic
+tensors: pack each of the R replicas' gradient lists into the shard-major
+layout, run the fused reduce + optimizer update for all R shards, unpack the
+updated weights back to the tensor list.  `value` is updated (valid)
+parameters per second with everything resident in HBM; `e2e` is the same step
+through the host-buffer entry point with host<->device copies inside the timed
+region; `roofline` is the dominant kernel against the measured HBM copy
+bandwidth; `cpu_baseline` is the CPU oracle timed on this machine's host cores.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+With N > 1 (launched by torch.distributed.run) every rank runs the same
+workload on its own independently seeded tensor set: the update has no
+data-path collective, so ranks only meet at the timing barriers.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "updated_params_per_sec"
+UNIT = "params/s"
+FALLBACK_HBM_GBS = 6650.0
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
+# captures summarised under profiles/, keyed by (workload, kernel); None = not captured.
+NCU_TRAFFIC_BYTES = {}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet50",
+                    choices=["tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b"])
+    ap.add_argument("--R", type=int, default=0, help="override the workload's replica count")
+    ap.add_argument("--align", type=int, default=32)
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def get_workload(args):
+    from paper_2004_13336_b200 import workloads as W
+    wl = W.WORKLOADS[args.workload]()
+    if args.R:
+        wl.R = args.R
+    return wl
+
+
+def bytes_per_param(wl):
+    """Algorithmic bytes per valid parameter of the fused update (read R gradients, the weight
+    and its slots once; write weight and slots once; plus the gathered copy when it is a
+    separate bf16 buffer) and of one pack / unpack launch."""
+    gb = 2 if str(wl.grad_dtype).endswith("bfloat16") else 4
+    slots = 1 if wl.opt == "sgdm" else 2
+    upd = gb * wl.R + 4 * (1 + slots) * 2
+    if wl.opt == "lamb":
+        upd += 12          # plain two-pass: phase 2 reads w, m', v' again and rewrites w
+    out_b = 2 if str(wl.out_dtype).endswith("bfloat16") else 0
+    upd += out_b
+    return {"update": upd, "pack": 2 * gb, "unpack": 2 * (2 if out_b else 4)}
+
+
+# ----------------------------------------------------------------------------
+# clocks
+# ----------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.samples = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
+                 "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.samples.append((time.time(), line.strip()))
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=2)
+            except Exception:
+                pass
+
+    def summary(self, t0, t1):
+        def parse(window):
+            sm, mx, reasons = [], [], set()
+            for ts, line in self.samples:
+                if not (window[0] <= ts <= window[1]):
+                    continue
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 7:
+                    continue
+                try:
+                    sm.append(float(p[0]))
+                    mx.append(float(p[1]))
+                except ValueError:
+                    continue
+                for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), p[3:7]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+            return sm, mx, reasons
+        sm, mx, reasons = parse((t0, t1))
+        window = "timed"
+        if len(sm) < 3 and self.samples:
+            sm, mx, reasons = parse((self.samples[0][0], t1 + 1.0))
+            window = "warmup+timed"
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": window}
+        sm.sort()
+        return {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                "samples": len(sm), "window": window}
+
+
+# ----------------------------------------------------------------------------
+# CPU oracle legs
+# ----------------------------------------------------------------------------
+def oracle_step_inputs(wl, stride, align):
+    """Host copies of every `stride`-th tensor of the workload (the bounded sample)."""
+    import torch
+    from oracle import ws_oracle as O
+    from paper_2004_13336_b200 import workloads as W
+    idx = list(range(0, wl.T, stride))
+    sub = W.Workload(**{**wl.__dict__})
+    sub.shapes = [wl.shapes[i] for i in idx]
+    w, m, v = W.make_state(sub, "cpu")
+    g = W.make_grads(sub, "cpu")
+
+    def np_(t):
+        if t.dtype == torch.bfloat16:
+            import numpy as np
+            return t.view(torch.int16).numpy().view(np.uint16)
+        return t.numpy()
+    plan = O.Plan(sub.numels, sub.R, align)
+    w, m, v = ([np_(x) for x in lst] for lst in (w, m, v))
+    g = [[np_(x) for x in gk] for gk in g]
+    pw, pm, pv = O.pack(plan, w), O.pack(plan, m), O.pack(plan, v)
+    return sub, plan, g, pw, pm, pv
+
+
+def oracle_one_step(sub, plan, g, pw, pm, pv):
+    """The whole path as the oracle states it: pack R gradient sets, sharded update, unpack."""
+    from oracle import ws_oracle as O
+    hs = O.make_hyper(sub.opt, sub.hyper)
+    t0 = time.perf_counter()
+    pg = [O.pack(plan, gk) for gk in g]
+    out_dt = O.BF16 if str(sub.out_dtype).endswith("bfloat16") else None
+    gathered, _, _ = O.sharded_update(hs, plan, pg, pw, pm, pv if sub.opt != "sgdm" else None, out_dt)
+    O.unpack(plan, gathered if gathered is not None else pw)
+    return time.perf_counter() - t0
+
+
+def cpu_baseline(wl, align, target_params=26_000_000, min_seconds=10.0, max_steps=20):
+    from oracle import ws_oracle as O
+    stride = max(1, round(wl.N / target_params))
+    sub, plan, g, pw, pm, pv = oracle_step_inputs(wl, stride, align)
+    dt, steps = 0.0, 0
+    while steps < max_steps and (steps == 0 or dt < min_seconds):
+        dt += oracle_one_step(sub, plan, g, pw, pm, pv)
+        steps += 1
+    return {"value": sub.N * steps / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{steps} step(s) (pack {sub.R} gradient sets, sharded update, unpack) over every "
+                      f"{stride}-th tensor of {wl.name}: {sub.T} tensors, {sub.N} params, {dt:.2f} s; "
+                      f"the sharded route of the oracle runs on one thread",
+            "host_cores": len(os.sched_getaffinity(0))}
+
+
+def run_reference(args):
+    """--impl reference: the CPU oracle, as it stands, on this machine's host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import ws_oracle as O
+    O.build()
+    wl = get_workload(args)
+    stride = max(1, round(wl.N / 1_500_000))
+    sub, plan, g, pw, pm, pv = oracle_step_inputs(wl, stride, args.align)
+    for _ in range(args.warmup):
+        oracle_one_step(sub, plan, g, pw, pm, pv)
+    t = 0.0
+    for _ in range(args.steps):
+        t += oracle_one_step(sub, plan, g, pw, pm, pv)
+    val = sub.N * args.steps / t
+    sample = (f"each step = whole path over every {stride}-th tensor of {wl.name} "
+              f"({sub.T} tensors, {sub.N} params)")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic", "config": config_of(wl, args, extra={"sample": sample}),
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def config_of(wl, args, extra=None):
+    c = {"workload": f"{wl.name}: {wl.T} tensors, {wl.N} params, R={wl.R} replicas, {wl.opt}, "
+                     f"grads {str(wl.grad_dtype).split('.')[-1]}, gathered {str(wl.out_dtype).split('.')[-1]}",
+         "R": wl.R, "optimizer": wl.opt, "align_elems": args.align,
+         "step": "pack R gradient sets + fused reduce/update of all shards + unpack weights",
+         "l2": "inputs exceed L2 (no flush)" if wl.N * 4 * (wl.R + 3) > 256e6 else "flush between steps"}
+    if extra:
+        c.update(extra)
+    return c
+
+
+# ----------------------------------------------------------------------------
+# GPU arm
+# ----------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2004_13336_b200 import binding as B
+    from paper_2004_13336_b200 import build as ws_build
+    from paper_2004_13336_b200 import workloads as W
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the sharded update has no CPU fallback")
+    if not ws_build.up_to_date():
+        if rank == 0:
+            ws_build.build()
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+        dist.barrier()
+    B.lib()
+
+    wl = get_workload(args)
+    wl.seed = wl.seed + 1000 * rank           # every rank owns its own tensor set
+    R, T, N = wl.R, wl.T, wl.N
+    plan = B.Plan(wl.shapes, R, args.align, device=dev)
+    gdt, odt = wl.grad_dtype, wl.out_dtype
+    numels = wl.numels
+    A_el = plan.arena_elems
+
+    # ---- device-resident inputs: per replica one gradient arena, viewed tensor by tensor
+    w, m, v = W.make_state(wl, dev)
+    pw = torch.empty(plan.G, device=dev)
+    pm, pv = torch.empty_like(pw), torch.empty_like(pw)
+    for src, dst in ((w, pw), (m, pm), (v, pv)):
+        B.ws_pack(plan, src, dst)
+    if wl.opt == "sgdm":
+        pv = None
+    del m, v
+    g_arena = [torch.zeros(A_el, dtype=gdt, device=dev) for _ in range(R)]
+    g_views = [B.PtrList(plan.arena_views(a, numels)) for a in g_arena]
+    for k in range(R):
+        gk = W.make_grads_one(wl, k, dev)
+        for dst, src in zip(g_views[k], gk):
+            dst.copy_(src)
+        del gk
+    pg = B.PtrList([torch.empty(plan.G, dtype=gdt, device=dev) for _ in range(R)])
+    gathered = torch.empty(plan.G, dtype=odt, device=dev) if odt != torch.float32 else None
+    w_arena = torch.zeros(A_el, dtype=odt, device=dev)
+    w_views = B.PtrList(plan.arena_views(w_arena, numels))
+    ws = torch.empty(max(16, plan.workspace_bytes(wl.opt)), dtype=torch.uint8, device=dev)
+    hy = B.make_hyper(wl.opt, wl.hyper)
+    del w
+    flush = None
+    if N * 4 * (R + 3) <= 256e6:
+        flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
+
+    def step(ev=None):
+        if flush is not None:
+            flush.zero_()
+        if ev:
+            ev[0].record()
+        for k in range(R):
+            B.ws_pack(plan, g_views[k], pg[k])
+        if ev:
+            ev[1].record()
+        B.ws_shard_update(plan, -1, pg, pw, pm, pv, hy, gathered, ws)
+        if ev:
+            ev[2].record()
+        B.ws_unpack(plan, gathered if gathered is not None else pw, w_views)
+        if ev:
+            ev[3].record()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    for _ in range(max(3, args.warmup)):
+        step()
+    K = args.steps
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
+    barrier()
+    t_host0 = time.time()
+    for i in range(K):
+        step(evs[i])
+    barrier()
+    t_host1 = time.time()
+    total_ms = evs[0][0].elapsed_time(evs[-1][3])
+    if flush is not None:
+        total_ms = sum(e[0].elapsed_time(e[3]) for e in evs)   # leave the L2 flush out of the step time
+    phase_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / K for i in range(3)]
+    if world > 1:
+        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    ms_per_step = total_ms / K
+    value = world * N / (ms_per_step * 1e-3)
+
+    # ---- end to end through the host-buffer entry point
+    e2e = None
+    if not args.no_e2e:
+        host_g = [torch.empty(A_el, dtype=gdt).pin_memory() for _ in range(R)]
+        for k in range(R):
+            host_g[k].copy_(g_arena[k])
+        host_g = B.PtrList(host_g)
+        host_w = torch.empty(A_el, dtype=odt).pin_memory()
+        stage = torch.empty(A_el, dtype=gdt, device=dev)
+
+        def e2e_step():
+            B.ws_step_host(plan, host_g, stage, pg, pw, pm, pv, hy, w_arena, host_w, gathered, ws)
+        for _ in range(2):
+            e2e_step()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record()
+        barrier()
+        e2e_ms = e0.elapsed_time(e1)
+        if world > 1:
+            tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_ms = float(tt.item())
+        gb = 2 if gdt == torch.bfloat16 else 4
+        wb = 2 if odt == torch.bfloat16 else 4
+        e2e = {"value": world * N * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": R * A_el * gb, "d2h_bytes_per_step": A_el * wb,
+               "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps,
+               "api": "ws_step_host (pinned host arenas)"}
+        del host_g, host_w, stage
+    sampler.stop()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel
+    peak, peak_src = FALLBACK_HBM_GBS, "fallback"
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        pass
+    bpp = bytes_per_param(wl)
+    n_upd_launch = 3 if wl.opt == "lamb" else 1
+    chunks = -(-T // 1024)
+    kernels = [
+        {"kernel": "pack_kernel (gradients)", "launches_per_step": R * chunks,
+         "ms_per_step": phase_ms[0], "bytes_per_step": R * N * bpp["pack"]},
+        {"kernel": "update_kernel (fused reduce+update)" if wl.opt != "lamb" else
+                   "update_kernel phase 1 + lamb_finalize + update_kernel phase 2",
+         "launches_per_step": n_upd_launch, "ms_per_step": phase_ms[1], "bytes_per_step": N * bpp["update"]},
+        {"kernel": "pack_kernel (unpack weights)", "launches_per_step": chunks,
+         "ms_per_step": phase_ms[2], "bytes_per_step": N * bpp["unpack"]},
+    ]
+    for kz in kernels:
+        kz["achieved_gbs"] = kz["bytes_per_step"] / (kz["ms_per_step"] * 1e-3) / 1e9
+        kz["frac"] = kz["achieved_gbs"] / peak
+        kz["share"] = kz["ms_per_step"] / sum(phase_ms)
+    dom = max(kernels, key=lambda z: z["ms_per_step"])
+    per_launch_bytes = dom["bytes_per_step"] / dom["launches_per_step"] if "phase 1" not in dom["kernel"] else dom["bytes_per_step"]
+    roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["achieved_gbs"], "peak": peak,
+                "peak_source": f"{peak_src} copy bandwidth", "unit": "GB/s", "frac": dom["frac"],
+                "algorithmic_bytes_per_launch": per_launch_bytes,
+                "avg_launch_ms": dom["ms_per_step"] / (dom["launches_per_step"] if "phase 1" not in dom["kernel"] else 1),
+                "traffic": NCU_TRAFFIC_BYTES.get((wl.name, dom["kernel"].split(" ")[0])),
+                "frac_of_nominal_8TBs": dom["achieved_gbs"] / 8000.0}
+    clocks = sampler.summary(t_host0, t_host1)
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": config_of(wl, args), "roofline": roofline, "kernels": kernels, "clocks": clocks,
+        "gpu_launches": K * sum(kz["launches_per_step"] for kz in kernels),
+        "update_only": {"value": N / (phase_ms[1] * 1e-3), "unit": UNIT,
+                        "bytes_per_param": bpp["update"], "achieved_gbs": kernels[1]["achieved_gbs"],
+                        "frac_of_measured_peak": kernels[1]["frac"],
+                        "frac_of_nominal_8TBs": kernels[1]["achieved_gbs"] / 8000.0},
+    }
+    if e2e is not None:
+        line["e2e"] = e2e
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import ws_oracle as O
+        O.build()
+        line["cpu_baseline"] = cpu_baseline(wl, args.align)
+    print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -212,6 +212,43 @@ ws_status ws_lamb_apply(const ws_plan* plan, int32_t r, const ws_state* state,
                         const ws_hyper* hyper, const ws_out* out, void* workspace,
                         size_t workspace_bytes, void* stream);
 
+/* ------------------------------------------------- host-buffer step ---
+ * One whole step for callers whose gradients and weights live in HOST memory
+ * (the end-to-end form of the path of Section 2.2: local gradients in, full
+ * updated weights out).  A "tensor arena" is the model's tensors back to back
+ * in the caller's order, each tensor's start rounded up to a multiple of 8
+ * elements; ws_plan_arena_elems gives its length and ws_plan_arena_offsets the
+ * start of every tensor (plan-owned array of T offsets, in elements).
+ *
+ * ws_step_host enqueues on `stream`, for k = 0..R-1: copy host_grads[k]
+ * (arena of grad_dtype) to dev_grad_arena, pack it into dev_packed_grads[k];
+ * then the fused update of all shards (as ws_shard_update with r == -1 on
+ * `state`, writing `out` if out->gathered is set); then unpack the updated
+ * weights (from out->gathered if set, else from state->w) into
+ * dev_weight_arena and copy that to host_weights.  Copies are
+ * cudaMemcpyAsync: with pinned host memory the call returns before the work
+ * is done, and host_weights is valid after the stream is synchronised.
+ * Nothing is allocated; all device buffers are the caller's:
+ *   dev_grad_arena    arena_elems elements of grad_dtype (staging, reused)
+ *   dev_packed_grads  host array of R device pointers, G elements each
+ *   dev_weight_arena  arena_elems elements of the weight dtype
+ * The weight dtype is out->dtype when out->gathered is set, else WS_F32. */
+int64_t ws_plan_arena_elems(const ws_plan* plan);
+ws_status ws_plan_arena_offsets(const ws_plan* plan, const int64_t** offsets, int32_t* T);
+
+typedef struct {
+    const void* const* host_grads; /* host array of R HOST pointers */
+    ws_dtype grad_dtype;
+    void* dev_grad_arena;
+    void* const* dev_packed_grads;
+    void* dev_weight_arena;
+    void* host_weights;            /* HOST arena, arena_elems elements */
+} ws_host_io;
+
+ws_status ws_step_host(const ws_plan* plan, const ws_host_io* io, const ws_state* state,
+                       const ws_hyper* hyper, const ws_out* out, void* workspace,
+                       size_t workspace_bytes, void* stream);
+
 /* Static, never NULL. */
 const char* ws_status_string(ws_status s);
 /* Text of the last CUDA error seen by the calling thread inside this library

@@ -58,12 +58,18 @@ class ws_out(C.Structure):
     _fields_ = [("gathered", C.c_void_p), ("dtype", C.c_int32)]
 
 
+class ws_host_io(C.Structure):
+    _fields_ = [("host_grads", C.POINTER(C.c_void_p)), ("grad_dtype", C.c_int32),
+                ("dev_grad_arena", C.c_void_p), ("dev_packed_grads", C.POINTER(C.c_void_p)),
+                ("dev_weight_arena", C.c_void_p), ("host_weights", C.c_void_p)]
+
+
 EXPORTS = [
     "ws_plan_create", "ws_plan_destroy", "ws_plan_num_tensors", "ws_plan_num_shards", "ws_plan_align",
     "ws_plan_shard_elems", "ws_plan_valid_elems", "ws_plan_num_tiles", "ws_plan_segments",
     "ws_plan_device_bytes", "ws_plan_upload", "ws_pack", "ws_unpack", "ws_workspace_bytes",
     "ws_shard_update", "ws_lamb_partial", "ws_lamb_finalize", "ws_lamb_apply", "ws_status_string",
-    "ws_last_cuda_error",
+    "ws_last_cuda_error", "ws_plan_arena_elems", "ws_plan_arena_offsets", "ws_step_host",
 ]
 
 _lib = None
@@ -112,6 +118,13 @@ def lib() -> C.CDLL:
     L.ws_lamb_apply.restype = C.c_int
     L.ws_lamb_apply.argtypes = [vp, C.c_int32, C.POINTER(ws_state), C.POINTER(ws_hyper),
                                 C.POINTER(ws_out), vp, C.c_size_t, vp]
+    L.ws_plan_arena_elems.restype = C.c_int64
+    L.ws_plan_arena_elems.argtypes = [vp]
+    L.ws_plan_arena_offsets.restype = C.c_int
+    L.ws_plan_arena_offsets.argtypes = [vp, C.POINTER(C.POINTER(C.c_int64)), C.POINTER(C.c_int32)]
+    L.ws_step_host.restype = C.c_int
+    L.ws_step_host.argtypes = [vp, C.POINTER(ws_host_io), C.POINTER(ws_state), C.POINTER(ws_hyper),
+                               C.POINTER(ws_out), vp, C.c_size_t, vp]
     L.ws_status_string.restype = C.c_char_p
     L.ws_status_string.argtypes = [C.c_int]
     L.ws_last_cuda_error.restype = C.c_char_p
@@ -137,7 +150,25 @@ def _dtype_code(dt: torch.dtype) -> int:
     raise TypeError(f"unsupported dtype {dt}")
 
 
-def _ptr_array(tensors: Sequence[torch.Tensor]):
+class PtrList:
+    """A tensor list with its C pointer array built once, for callers that pass
+    the same tensors every step (keeps the per-call host cost to one ctypes call)."""
+
+    def __init__(self, tensors: Sequence[torch.Tensor]):
+        self.tensors = list(tensors)
+        self.arr = _ptr_array(self.tensors)
+        self.dtype = self.tensors[0].dtype if self.tensors else torch.float32
+
+    def __len__(self):
+        return len(self.tensors)
+
+    def __getitem__(self, i):
+        return self.tensors[i]
+
+
+def _ptr_array(tensors):
+    if isinstance(tensors, PtrList):
+        return tensors.arr
     arr = (C.c_void_p * max(1, len(tensors)))()
     for i, t in enumerate(tensors):
         arr[i] = t.data_ptr()
@@ -188,6 +219,19 @@ class Plan:
         nbytes = lib().ws_plan_device_bytes(self._h)
         self.dev_buf = torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
         _check(lib().ws_plan_upload(self._h, self.dev_buf.data_ptr(), nbytes, _stream()), "ws_plan_upload")
+
+    @property
+    def arena_elems(self) -> int:
+        return lib().ws_plan_arena_elems(self._h)
+
+    def arena_offsets(self) -> List[int]:
+        offs, T = C.POINTER(C.c_int64)(), C.c_int32()
+        _check(lib().ws_plan_arena_offsets(self._h, C.byref(offs), C.byref(T)), "ws_plan_arena_offsets")
+        return [offs[i] for i in range(T.value)]
+
+    def arena_views(self, arena: torch.Tensor, numels: Sequence[int]) -> List[torch.Tensor]:
+        """Per-tensor views of a tensor arena (host or device)."""
+        return [arena[o:o + n] for o, n in zip(self.arena_offsets(), numels)]
 
     def workspace_bytes(self, opt) -> int:
         code = OPT_CODE[opt] if isinstance(opt, str) else int(opt)
@@ -263,3 +307,20 @@ def ws_lamb_apply(plan: Plan, r: int, w, m, v, hyper: ws_hyper, workspace: torch
 def lamb_ratios(plan: Plan, workspace: torch.Tensor) -> torch.Tensor:
     """The trust ratios rho[T] that ws_lamb_finalize left at the start of the workspace."""
     return workspace[: 4 * plan.T].view(torch.float32)
+
+
+def ws_step_host(plan: Plan, host_grads: Sequence[torch.Tensor], dev_grad_arena: torch.Tensor,
+                 dev_packed_grads: Sequence[torch.Tensor], w, m, v, hyper: ws_hyper,
+                 dev_weight_arena: torch.Tensor, host_weights: torch.Tensor,
+                 gathered: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None):
+    """Host gradient arenas in, host weight arena out (pinned memory for overlap-free async copies)."""
+    hg, dp = _ptr_array(host_grads), _ptr_array(dev_packed_grads)
+    io = ws_host_io(C.cast(hg, C.POINTER(C.c_void_p)), _dtype_code(host_grads[0].dtype),
+                    dev_grad_arena.data_ptr(), C.cast(dp, C.POINTER(C.c_void_p)),
+                    dev_weight_arena.data_ptr(), host_weights.data_ptr())
+    s, o = _state(w, m, v), _out(gathered)
+    _check(lib().ws_step_host(plan.handle, C.byref(io), C.byref(s), C.byref(hyper),
+                              C.byref(o) if o is not None else None,
+                              workspace.data_ptr() if workspace is not None else None,
+                              workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                              _stream()), "ws_step_host")

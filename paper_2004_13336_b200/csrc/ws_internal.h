@@ -37,6 +37,9 @@ struct ws_plan {
     std::vector<ws_segment> segs;
     std::vector<WsTile> tiles;
     std::vector<WsSegTiles> segtiles;
+    // tensor arena: tensors back to back, each start rounded up to 8 elements
+    std::vector<long long> arena_off;
+    long long arena_elems = 0;
     // device copies (caller-owned memory, set by ws_plan_upload)
     const WsTile* d_tiles = nullptr;
     const WsSegTiles* d_segtiles = nullptr;

@@ -74,6 +74,8 @@ extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int3
             p->segs[t].piece = piece;
             p->segs[t].shard_off = off;
             p->N += n;
+            p->arena_off.push_back(p->arena_elems);
+            p->arena_elems += (n + 7) / 8 * 8;
             // cut the piece into tiles that stay inside it
             long long ntile = (piece + tile_elems - 1) / tile_elems;
             if ((long long)p->tiles.size() + ntile > 0x7fffffffLL) { delete p; return WS_ERR_TOO_LARGE; }
