@@ -249,6 +249,43 @@ ws_status ws_step_host(const ws_plan* plan, const ws_host_io* io, const ws_state
                        const ws_hyper* hyper, const ws_out* out, void* workspace,
                        size_t workspace_bytes, void* stream);
 
+/* ------------------------------------- LAMB without a caller workspace ---
+ * (No counterpart in the paper: this entry point exists for deployment
+ * reasons only.)
+ *
+ * ws_lamb_update_static_scratch does exactly what ws_shard_update does for
+ * opt == WS_LAMB and r == -1 (phase 1 over all shards, finalize, phase 2 over
+ * all shards; same arguments, same results), but needs no `workspace`: the
+ * trust ratios, norms and per-tile partial sums go to an array of
+ * WS_STATIC_SCRATCH_BYTES that is built into the library.  It is meant for
+ * callers that cannot get device memory when the update runs - an optimizer
+ * plug-in inside a framework whose allocator already owns the whole GPU, a step
+ * loop that must stay out of the CUDA allocator because cudaMalloc can stall
+ * the device, a binding layer that can forward buffers but not create them.
+ * The call performs no device allocation or free of any kind.
+ *
+ * Limits and rules:
+ *   - ws_workspace_bytes(plan, WS_LAMB) must not exceed WS_STATIC_SCRATCH_BYTES
+ *     (4 MiB; enough for BERT-large at R = 16 with the default tile size),
+ *     otherwise WS_ERR_TOO_LARGE is returned and nothing is launched.
+ *   - Every GPU that loads the library carries the array until the process
+ *     exits, whether or not this entry point is ever called.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current) and caches it; make that first call outside any
+ *     stream capture.  Later calls on the same device skip the lookup.
+ *   - All calls on one device share the one array, and it keeps whatever the
+ *     previous call left in it.  Nothing in it needs clearing (each call
+ *     overwrites every entry it later reads), but two calls whose kernels can
+ *     run at the same time on one GPU - different streams, different threads -
+ *     would overwrite each other's partial sums: serialise them.
+ *   - The caller still owns and passes gradients, state and the gathered
+ *     output exactly as for ws_shard_update. */
+#define WS_STATIC_SCRATCH_BYTES (4u * 1024u * 1024u)
+size_t ws_static_scratch_bytes(void); /* == WS_STATIC_SCRATCH_BYTES of the loaded library */
+ws_status ws_lamb_update_static_scratch(const ws_plan* plan, const ws_grads* grads,
+                                        const ws_state* state, const ws_hyper* hyper,
+                                        const ws_out* out, void* stream);
+
 /* Static, never NULL. */
 const char* ws_status_string(ws_status s);
 /* Text of the last CUDA error seen by the calling thread inside this library

@@ -70,6 +70,7 @@ EXPORTS = [
     "ws_plan_device_bytes", "ws_plan_upload", "ws_pack", "ws_unpack", "ws_workspace_bytes",
     "ws_shard_update", "ws_lamb_partial", "ws_lamb_finalize", "ws_lamb_apply", "ws_status_string",
     "ws_last_cuda_error", "ws_plan_arena_elems", "ws_plan_arena_offsets", "ws_step_host",
+    "ws_static_scratch_bytes", "ws_lamb_update_static_scratch",
 ]
 
 _lib = None
@@ -125,6 +126,11 @@ def lib() -> C.CDLL:
     L.ws_step_host.restype = C.c_int
     L.ws_step_host.argtypes = [vp, C.POINTER(ws_host_io), C.POINTER(ws_state), C.POINTER(ws_hyper),
                                C.POINTER(ws_out), vp, C.c_size_t, vp]
+    L.ws_static_scratch_bytes.restype = C.c_size_t
+    L.ws_static_scratch_bytes.argtypes = []
+    L.ws_lamb_update_static_scratch.restype = C.c_int
+    L.ws_lamb_update_static_scratch.argtypes = [vp, C.POINTER(ws_grads), C.POINTER(ws_state),
+                                                C.POINTER(ws_hyper), C.POINTER(ws_out), vp]
     L.ws_status_string.restype = C.c_char_p
     L.ws_status_string.argtypes = [C.c_int]
     L.ws_last_cuda_error.restype = C.c_char_p
@@ -324,3 +330,13 @@ def ws_step_host(plan: Plan, host_grads: Sequence[torch.Tensor], dev_grad_arena:
                               workspace.data_ptr() if workspace is not None else None,
                               workspace.numel() * workspace.element_size() if workspace is not None else 0,
                               _stream()), "ws_step_host")
+
+
+def ws_lamb_update_static_scratch(plan: Plan, gbufs, w, m, v, hyper: ws_hyper,
+                                  gathered: Optional[torch.Tensor] = None):
+    """LAMB update of all shards for callers that cannot provide a workspace: the scratch
+    is a fixed array inside the library (see ws.h for its size limit and sharing rules)."""
+    g, s, o = _grads(gbufs, 0), _state(w, m, v), _out(gathered)
+    _check(lib().ws_lamb_update_static_scratch(plan.handle, C.byref(g), C.byref(s), C.byref(hyper),
+                                               C.byref(o) if o is not None else None, _stream()),
+           "ws_lamb_update_static_scratch")
