@@ -49,6 +49,7 @@ def parse_args():
                     choices=["tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b"])
     ap.add_argument("--R", type=int, default=0, help="override the workload's replica count")
     ap.add_argument("--align", type=int, default=32)
+    ap.add_argument("--tile", type=int, default=0, help="work-tile elements (0 = library default)")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -266,7 +267,7 @@ def run_ours(args):
     wl = get_workload(args)
     wl.seed = wl.seed + 1000 * rank           # every rank owns its own tensor set
     R, T, N = wl.R, wl.T, wl.N
-    plan = B.Plan(wl.shapes, R, args.align, device=dev)
+    plan = B.Plan(wl.shapes, R, args.align, args.tile, device=dev)
     gdt, odt = wl.grad_dtype, wl.out_dtype
     numels = wl.numels
     A_el = plan.arena_elems

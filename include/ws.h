@@ -76,7 +76,8 @@ typedef struct ws_plan ws_plan;
  *   R           shard count = replica count, >= 1
  *   align_elems A: power of two >= 8, every piece is a multiple of A elements
  *   tile_elems  work-tile length in elements used by the kernels; 0 = default
- *               (2048); otherwise a multiple of 1024
+ *               (2048, 4096, 8192 or 16384, the largest that leaves at least
+ *               20000 tiles over all shards); otherwise a multiple of 1024
  *   out         receives a new plan; release with ws_plan_destroy
  * Errors: WS_ERR_INVALID_ARG for null/empty input, bad R, A or tile size. */
 ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int32_t R, int32_t align_elems,
@@ -211,6 +212,50 @@ ws_status ws_lamb_finalize(const ws_plan* plan, void* workspace, size_t workspac
 ws_status ws_lamb_apply(const ws_plan* plan, int32_t r, const ws_state* state,
                         const ws_hyper* hyper, const ws_out* out, void* workspace,
                         size_t workspace_bytes, void* stream);
+
+/* ------------------------------------- formatting fused into the update ---
+ * Section 5.1: padding the gradient before the reduce-scatter costs every
+ * replica a read and a write of the full data, so the paper fuses the
+ * formatting into the reduce-scatter and the all-gather and pads in place.
+ * ws_fused_update is that fusion on one GPU: the kernel reads the R replicas'
+ * gradients straight from their tensor lists (element r p_t + q of tensor t
+ * for shard position off_t + q; positions past n_t are never read), updates
+ * the sharded fp32 state exactly as ws_shard_update does, and writes the
+ * updated weights straight into the weight tensors (fp32, or bf16 rounded to
+ * nearest-even, Section 4.2).  No packed gradient buffer and no gathered
+ * buffer exist; results are bit-identical to ws_pack of every gradient list,
+ * ws_shard_update, ws_unpack.
+ *
+ * Tensor pointers reach the kernel through a device-resident table that is
+ * uploaded once (the tensors of a training job stay where they are):
+ *   ws_tensor_table_upload copies `nsets` lists of T device pointers (host
+ *   array, set-major: ptrs[k*T + t]) into the caller's device buffer of at
+ *   least ws_tensor_table_bytes(plan, nsets) bytes with one cudaMemcpyAsync and
+ *   fills *out, which the caller passes to ws_fused_update and keeps alive,
+ *   together with the device buffer, while it is in use.  Every tensor pointer
+ *   must be 16-byte aligned; 32-byte alignment of all of them lets the kernels
+ *   use 256-bit accesses.
+ * ws_fused_update arguments: `grads` is a table of R sets (the R replicas'
+ * gradient lists), `weights` a table of one set (the weight tensors that
+ * receive the result), `state` as for ws_shard_update (r >= 0: one shard;
+ * r == -1: all shards, the only form accepted for WS_LAMB), `workspace` as for
+ * ws_shard_update. */
+typedef struct {
+    void* dev;        /* device table, layout [T][nsets] */
+    int32_t nsets;
+    int32_t T;
+    ws_dtype dtype;   /* element type of the tensors the table points to */
+    int32_t min_align;/* largest power of two (<= 256) dividing every pointer */
+} ws_tensor_table;
+
+size_t ws_tensor_table_bytes(const ws_plan* plan, int32_t nsets);
+ws_status ws_tensor_table_upload(const ws_plan* plan, const void* const* ptrs, int32_t nsets,
+                                 ws_dtype dtype, void* dev_buf, size_t bytes, void* stream,
+                                 ws_tensor_table* out);
+ws_status ws_fused_update(const ws_plan* plan, int32_t r, const ws_tensor_table* grads,
+                          const ws_state* state, const ws_hyper* hyper,
+                          const ws_tensor_table* weights, void* workspace, size_t workspace_bytes,
+                          void* stream);
 
 /* ------------------------------------------------- host-buffer step ---
  * One whole step for callers whose gradients and weights live in HOST memory

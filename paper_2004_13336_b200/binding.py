@@ -58,6 +58,11 @@ class ws_out(C.Structure):
     _fields_ = [("gathered", C.c_void_p), ("dtype", C.c_int32)]
 
 
+class ws_tensor_table(C.Structure):
+    _fields_ = [("dev", C.c_void_p), ("nsets", C.c_int32), ("T", C.c_int32), ("dtype", C.c_int32),
+                ("min_align", C.c_int32)]
+
+
 class ws_host_io(C.Structure):
     _fields_ = [("host_grads", C.POINTER(C.c_void_p)), ("grad_dtype", C.c_int32),
                 ("dev_grad_arena", C.c_void_p), ("dev_packed_grads", C.POINTER(C.c_void_p)),
@@ -71,6 +76,7 @@ EXPORTS = [
     "ws_shard_update", "ws_lamb_partial", "ws_lamb_finalize", "ws_lamb_apply", "ws_status_string",
     "ws_last_cuda_error", "ws_plan_arena_elems", "ws_plan_arena_offsets", "ws_step_host",
     "ws_static_scratch_bytes", "ws_lamb_update_static_scratch",
+    "ws_tensor_table_bytes", "ws_tensor_table_upload", "ws_fused_update",
 ]
 
 _lib = None
@@ -131,6 +137,14 @@ def lib() -> C.CDLL:
     L.ws_lamb_update_static_scratch.restype = C.c_int
     L.ws_lamb_update_static_scratch.argtypes = [vp, C.POINTER(ws_grads), C.POINTER(ws_state),
                                                 C.POINTER(ws_hyper), C.POINTER(ws_out), vp]
+    L.ws_tensor_table_bytes.restype = C.c_size_t
+    L.ws_tensor_table_bytes.argtypes = [vp, C.c_int32]
+    L.ws_tensor_table_upload.restype = C.c_int
+    L.ws_tensor_table_upload.argtypes = [vp, vpp, C.c_int32, C.c_int, vp, C.c_size_t, vp,
+                                         C.POINTER(ws_tensor_table)]
+    L.ws_fused_update.restype = C.c_int
+    L.ws_fused_update.argtypes = [vp, C.c_int32, C.POINTER(ws_tensor_table), C.POINTER(ws_state),
+                                  C.POINTER(ws_hyper), C.POINTER(ws_tensor_table), vp, C.c_size_t, vp]
     L.ws_status_string.restype = C.c_char_p
     L.ws_status_string.argtypes = [C.c_int]
     L.ws_last_cuda_error.restype = C.c_char_p
@@ -340,3 +354,29 @@ def ws_lamb_update_static_scratch(plan: Plan, gbufs, w, m, v, hyper: ws_hyper,
     _check(lib().ws_lamb_update_static_scratch(plan.handle, C.byref(g), C.byref(s), C.byref(hyper),
                                                C.byref(o) if o is not None else None, _stream()),
            "ws_lamb_update_static_scratch")
+
+
+class TensorTable:
+    """Device-resident table of tensor pointers for ws_fused_update: `sets` is a list of
+    tensor lists (R gradient lists, or one weight list).  Keeps the device buffer alive."""
+
+    def __init__(self, plan: Plan, sets: Sequence[Sequence[torch.Tensor]]):
+        nsets = len(sets)
+        flat = [t for s in sets for t in s]
+        assert len(flat) == nsets * plan.T
+        self.sets = [list(s) for s in sets]
+        nbytes = lib().ws_tensor_table_bytes(plan.handle, nsets)
+        self.dev_buf = torch.empty(nbytes, dtype=torch.uint8, device=flat[0].device)
+        self.c = ws_tensor_table()
+        _check(lib().ws_tensor_table_upload(plan.handle, _ptr_array(flat), nsets, _dtype_code(flat[0].dtype),
+                                            self.dev_buf.data_ptr(), nbytes, _stream(), C.byref(self.c)),
+               "ws_tensor_table_upload")
+
+
+def ws_fused_update(plan: Plan, r: int, grads: TensorTable, w, m, v, hyper: ws_hyper, weights: TensorTable,
+                    workspace: Optional[torch.Tensor] = None):
+    s = _state(w, m, v)
+    _check(lib().ws_fused_update(plan.handle, r, C.byref(grads.c), C.byref(s), C.byref(hyper), C.byref(weights.c),
+                                 workspace.data_ptr() if workspace is not None else None,
+                                 workspace.numel() * workspace.element_size() if workspace is not None else 0,
+                                 _stream()), "ws_fused_update")

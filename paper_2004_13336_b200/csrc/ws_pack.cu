@@ -85,9 +85,6 @@ ws_status run(const ws_plan* p, void* const* tensor_ptrs, ws_dtype dtype, void* 
         if (!ws_aligned16(tensor_ptrs[t])) return WS_ERR_ALIGNMENT;
     }
     cudaStream_t st = (cudaStream_t)stream;
-    int dev = 0, sms = 148;
-    cudaGetDevice(&dev);
-    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     for (int seg_lo = 0; seg_lo < p->T; seg_lo += kPtrChunk) {
         const int seg_hi = seg_lo + kPtrChunk < p->T ? seg_lo + kPtrChunk : p->T;
         PtrChunk tab;
@@ -100,9 +97,8 @@ ws_status run(const ws_plan* p, void* const* tensor_ptrs, ws_dtype dtype, void* 
         P.nitems = P.ntl * p->R;
         P.S = p->S;
         P.seg_lo = seg_lo;
-        long long grid = P.nitems;
-        const long long cap = (long long)sms * 32;
-        if (grid > cap) grid = cap;
+        long long grid = P.nitems;   // one CTA per (shard, tile): the CTA scheduler walks the buffers in order
+        if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;
         if (grid < 1) continue;
         if (dtype == WS_F32) pack_kernel<4, PACK><<<(unsigned)grid, kBlock, 0, st>>>(P, tab, (char*)flat);
         else                 pack_kernel<2, PACK><<<(unsigned)grid, kBlock, 0, st>>>(P, tab, (char*)flat);

@@ -47,7 +47,20 @@ extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int3
     *out = nullptr;
     if (!descs || T < 1 || R < 1) return WS_ERR_INVALID_ARG;
     if (align_elems < 8 || (align_elems & (align_elems - 1)) != 0) return WS_ERR_INVALID_ARG;
-    if (tile_elems == 0) tile_elems = 2048;
+    if (tile_elems == 0) {
+        // Default: the largest tile that still leaves >= 20000 work items for an all-shard
+        // launch.  A CTA reads its tile descriptor before it can issue any data load, so a
+        // large tile amortises that latency; small models keep small tiles so that the
+        // grid still spreads evenly over the SMs.
+        long long total = 0;
+        for (int t = 0; t < T; ++t) {
+            long long n = 1;
+            for (int i = 0; i < descs[t].ndim && i < WS_MAX_DIMS; ++i) n *= (descs[t].dims[i] > 0 ? descs[t].dims[i] : 1);
+            total += n;
+        }
+        tile_elems = 2048;
+        while (tile_elems < 16384 && total / (2 * tile_elems) >= 20000) tile_elems *= 2;
+    }
     if (tile_elems < 1024 || tile_elems % 1024 != 0 || tile_elems > (1 << 20)) return WS_ERR_INVALID_ARG;
 
     ws_plan* p = new (std::nothrow) ws_plan;

@@ -22,6 +22,14 @@
 
 #include "ws_internal.h"
 
+#ifndef WS_TUNE_MINB
+#define WS_TUNE_MINB 3   // resident CTAs per SM the compiler must allow for (register budget);
+                         // the bf16-gradient wide kernel is given 2 (measured faster with more registers)
+#endif
+#ifndef WS_TUNE_U4
+#define WS_TUNE_U4 1     // 128-bit accesses per thread per pass
+#endif
+
 namespace {
 
 constexpr int kBlock = 256;
@@ -46,31 +54,161 @@ struct UpdParams {
     float* m;
     float* v;
     void* gathered;         // base of the G-element gathered buffer, or null
+    const void* const* gtab; // fused formatting: device table [T][R] of gradient tensor pointers
+    void* const* wtab;       // fused formatting: device table [T] of weight tensor pointers (outputs)
     float2* partials;       // LAMB: [R][ntiles]
     const float* rho;       // LAMB phase 2: [T]
     WsConsts c;
 };
 
 // ---------------------------------------------------------------- memory ---
-__device__ __forceinline__ float4 ldg_f4(const float* p) { return __ldcs(reinterpret_cast<const float4*>(p)); }
-__device__ __forceinline__ void stg_f4(float* p, float4 v) { __stcs(reinterpret_cast<float4*>(p), v); }
+// A thread moves VEC consecutive elements at a time: VEC = 4 as one 128-bit access,
+// VEC = 8 as one 256-bit access (ld/st.global.v8.b32, new with sm_100) for fp32 data
+// and one 128-bit access for bf16 data.
+template <int VEC>
+struct Fv {
+    float f[VEC];
+};
 
-template <bool BF16>
-__device__ __forceinline__ float4 load_grad4(const void* base, long long idx) {
-    if (BF16) {
-        const uint2 u = __ldcs(reinterpret_cast<const uint2*>(reinterpret_cast<const unsigned short*>(base) + idx));
-        float4 g;  // bf16 -> fp32 widening is a 16-bit shift, exact
-        g.x = __uint_as_float(u.x << 16);
-        g.y = __uint_as_float(u.x & 0xffff0000u);
-        g.z = __uint_as_float(u.y << 16);
-        g.w = __uint_as_float(u.y & 0xffff0000u);
-        return g;
+#ifndef WS_TUNE_LD8
+#define WS_TUNE_LD8 "ld.global.L1::no_allocate.L2::evict_first.v8.b32"
+#endif
+#ifndef WS_TUNE_ST8
+#define WS_TUNE_ST8 "st.global.v8.b32"
+#endif
+
+template <int VEC>
+__device__ __forceinline__ Fv<VEC> load_f32(const float* p) {
+    Fv<VEC> o;
+    if (VEC == 4) {
+        const float4 v = __ldcs(reinterpret_cast<const float4*>(p));
+        o.f[0] = v.x; o.f[1] = v.y; o.f[2] = v.z; o.f[3] = v.w;
     } else {
-        return ldg_f4(reinterpret_cast<const float*>(base) + idx);
+        unsigned r[8];
+        asm volatile(WS_TUNE_LD8 " {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+                     : "l"(p));
+#pragma unroll
+        for (int i = 0; i < 8; ++i) o.f[i % VEC] = __uint_as_float(r[i]);
+    }
+    return o;
+}
+
+template <int VEC>
+__device__ __forceinline__ void store_f32(float* p, const Fv<VEC>& x) {
+    if (VEC == 4) {
+        __stcs(reinterpret_cast<float4*>(p), make_float4(x.f[0], x.f[1], x.f[2], x.f[3]));
+    } else {
+        asm volatile(WS_TUNE_ST8 " [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                     :: "l"(p), "r"(__float_as_uint(x.f[0])), "r"(__float_as_uint(x.f[1])), "r"(__float_as_uint(x.f[2])),
+                        "r"(__float_as_uint(x.f[3])), "r"(__float_as_uint(x.f[4 % VEC])), "r"(__float_as_uint(x.f[5 % VEC])),
+                        "r"(__float_as_uint(x.f[6 % VEC])), "r"(__float_as_uint(x.f[7 % VEC]))
+                     : "memory");
     }
 }
 
-__device__ __forceinline__ float4 add4(float4 a, float4 b) { return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w); }
+// Gradients as they come from memory (bf16 stays packed until it is summed).
+template <bool GBF, int VEC>
+struct GradRaw {
+    float f[VEC];
+};
+template <>
+struct GradRaw<true, 4> {
+    uint2 u;
+};
+template <>
+struct GradRaw<true, 8> {
+    uint4 u;
+};
+
+template <bool GBF, int VEC>
+__device__ __forceinline__ GradRaw<GBF, VEC> load_grad(const void* base, long long idx) {
+    GradRaw<GBF, VEC> g;
+    if constexpr (GBF) {
+        const unsigned short* p = reinterpret_cast<const unsigned short*>(base) + idx;
+        if constexpr (VEC == 4) g.u = __ldcs(reinterpret_cast<const uint2*>(p));
+        else g.u = __ldcs(reinterpret_cast<const uint4*>(p));
+    } else {
+        const Fv<VEC> v = load_f32<VEC>(reinterpret_cast<const float*>(base) + idx);
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) g.f[i] = v.f[i];
+    }
+    return g;
+}
+
+// The one vector of a tensor that holds its last element: only the first n elements exist.
+template <bool GBF, int VEC>
+__device__ __forceinline__ GradRaw<GBF, VEC> load_grad_partial(const void* base, long long idx, int n) {
+    GradRaw<GBF, VEC> g;
+    if constexpr (GBF) {
+        const unsigned short* p = reinterpret_cast<const unsigned short*>(base) + idx;
+        unsigned w[VEC / 2];
+#pragma unroll
+        for (int i = 0; i < VEC / 2; ++i) {
+            const unsigned lo = (2 * i < n) ? p[2 * i] : 0u;
+            const unsigned hi = (2 * i + 1 < n) ? p[2 * i + 1] : 0u;
+            w[i] = lo | (hi << 16);
+        }
+        if constexpr (VEC == 4) g.u = make_uint2(w[0], w[1]);
+        else g.u = make_uint4(w[0], w[1], w[2], w[3]);
+    } else {
+        const float* p = reinterpret_cast<const float*>(base) + idx;
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) g.f[i] = (i < n) ? p[i] : 0.f;
+    }
+    return g;
+}
+
+template <int VEC>
+__device__ __forceinline__ void store_f32_partial(float* p, const Fv<VEC>& x, int n) {
+#pragma unroll
+    for (int i = 0; i < VEC; ++i)
+        if (i < n) p[i] = x.f[i];
+}
+
+template <int VEC>
+__device__ __forceinline__ void store_bf16_partial(unsigned short* p, const Fv<VEC>& x, int n) {
+#pragma unroll
+    for (int i = 0; i < VEC; ++i)
+        if (i < n) {
+            const __nv_bfloat16 b = __float2bfloat16_rn(x.f[i]);
+            p[i] = *reinterpret_cast<const unsigned short*>(&b);
+        }
+}
+
+// bf16 -> fp32 widening is a 16-bit shift, exact
+template <bool GBF, int VEC>
+__device__ __forceinline__ Fv<VEC> widen(const GradRaw<GBF, VEC>& g) {
+    Fv<VEC> o;
+    if constexpr (GBF) {
+        o.f[0] = __uint_as_float(g.u.x << 16);
+        o.f[1] = __uint_as_float(g.u.x & 0xffff0000u);
+        o.f[2] = __uint_as_float(g.u.y << 16);
+        o.f[3] = __uint_as_float(g.u.y & 0xffff0000u);
+        if constexpr (VEC == 8) {
+            o.f[4] = __uint_as_float(g.u.z << 16);
+            o.f[5] = __uint_as_float(g.u.z & 0xffff0000u);
+            o.f[6] = __uint_as_float(g.u.w << 16);
+            o.f[7] = __uint_as_float(g.u.w & 0xffff0000u);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) o.f[i] = g.f[i];
+    }
+    return o;
+}
+
+template <int VEC>
+__device__ __forceinline__ void store_bf16(unsigned short* p, const Fv<VEC>& x) {
+    unsigned pk[VEC / 2];
+#pragma unroll
+    for (int i = 0; i < VEC / 2; ++i) {
+        const __nv_bfloat162 b = __floats2bfloat162_rn(x.f[2 * i], x.f[2 * i + 1]);
+        pk[i] = *reinterpret_cast<const unsigned int*>(&b);
+    }
+    if constexpr (VEC == 4) __stcs(reinterpret_cast<uint2*>(p), make_uint2(pk[0], pk[1]));
+    else __stcs(reinterpret_cast<uint4*>(p), make_uint4(pk[0], pk[1], pk[2], pk[3]));
+}
 
 // Kahan step: (sum, comp) += x
 __device__ __forceinline__ void kahan1(float& s, float& c, float x) {
@@ -128,74 +266,120 @@ __device__ __forceinline__ float block_sum(float x, float* smem /* kBlock/32 flo
 
 // ---------------------------------------------------------------- kernel ---
 // OPT: optimizer / phase.  GBF: gradients are bf16.  OUT: gathered dtype.
-// U: quads per thread per pass.  RB: gradients summed per tree block.
-// NP: capacity of the by-value gradient pointer table.
-template <int OPT, bool GBF, int OUT, int U, int RB, int NP>
-__global__ void __launch_bounds__(kBlock) update_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp) {
+// VEC: elements per thread access.  U: accesses per thread per pass.
+// RB: gradients summed per tree block.  NP: capacity of the by-value pointer table.
+// FUSED: the formatting steps are fused in (Section 5.1) - gradients are read straight
+// from the replicas' tensor lists and the updated weights are written straight to the
+// weight tensors, so no packed gradient buffer and no gathered buffer exist.
+// One CTA handles one (shard, tile) work item; the grid is the item count, so the
+// hardware CTA scheduler walks the buffers front to back.
+template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED>
+__global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF) ? 2 : WS_TUNE_MINB) update_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp) {
     constexpr bool HAS_V = (OPT != K_SGDM);
     constexpr bool READS_G = (OPT != K_LAMB2);
+    constexpr bool LOOPK = (NP > RB);   // R may exceed one tree block: loop and compensate
     __shared__ float red[2][kBlock / 32];
 
     for (long long item = blockIdx.x; item < P.nitems; item += gridDim.x) {
         const long long rs = item / P.ntiles;              // shard index inside this launch
         const long long ti = item - rs * P.ntiles;
         const long long r = P.r0 + rs;
+#ifdef WS_TUNE_NODESC   /* development experiment: single-tensor plans only */
+        WsTile tl;
+        tl.pos = ti * WS_TUNE_NODESC; tl.poff = tl.pos; tl.piece = P.S; tl.vt = (long long)P.R * P.S - tl.pos;
+        tl.len = (int)((P.S - tl.pos) < WS_TUNE_NODESC ? (P.S - tl.pos) : WS_TUNE_NODESC); tl.seg = 0;
+#else
         const WsTile tl = P.tiles[ti];
+#endif
+        {   // pull the next work item's descriptor towards this SM while this one is processed
+            const long long nitem = item + gridDim.x;
+            if (nitem < P.nitems) {
+                const WsTile* nt = P.tiles + (nitem % P.ntiles);
+                asm volatile("prefetch.global.L1 [%0];" ::"l"(nt));
+                asm volatile("prefetch.global.L1 [%0];" ::"l"(reinterpret_cast<const char*>(nt) + 32));
+            }
+        }
         long long nvl = tl.vt - r * tl.piece;              // valid elements in this tile for shard r
         const int nvalid = nvl < 0 ? 0 : (nvl > tl.len ? tl.len : (int)nvl);
         const long long gbase = rs * P.g_stride + tl.pos;  // into each gradient buffer
         const long long sbase = rs * P.st_stride + tl.pos; // into w/m/v
         const long long obase = r * P.S + tl.pos;          // into the gathered buffer
-        const int nquad = tl.len >> 2;
+        const long long toff = r * tl.piece + tl.poff;     // element index inside tensor tl.seg (fused formatting)
+        const void* const* gt = nullptr;
+        char* wt = nullptr;
+        if constexpr (FUSED) {
+            if (READS_G) gt = P.gtab + (long long)tl.seg * P.R;
+            if (OUT != O_NONE) wt = reinterpret_cast<char*>(P.wtab[tl.seg]);
+        }
+        const int nvec = tl.len / VEC;
         float lr_rho = 0.f;
         if (OPT == K_LAMB2) lr_rho = P.c.lr * P.rho[tl.seg];
         float sw = 0.f, su = 0.f;
 
-        for (int q0 = 0; q0 < nquad; q0 += U * kBlock) {
+        for (int q0 = 0; q0 < nvec; q0 += U * kBlock) {
             int e0[U];
             int nv[U];
-            float4 w4[U], m4[U], v4[U], g4[U], gc[U];
+            Fv<VEC> wv[U], mv[U], vv[U], gv[U], gc[U];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int q = q0 + u * kBlock + threadIdx.x;
-                e0[u] = q << 2;
+                e0[u] = q * VEC;
                 const int left = nvalid - e0[u];
-                nv[u] = q < nquad ? (left < 0 ? 0 : (left > 4 ? 4 : left)) : -1;  // -1: no quad here
-                w4[u] = m4[u] = v4[u] = g4[u] = gc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                nv[u] = q < nvec ? (left < 0 ? 0 : (left > VEC ? VEC : left)) : -1;  // -1: nothing here
+#pragma unroll
+                for (int j = 0; j < VEC; ++j) wv[u].f[j] = mv[u].f[j] = vv[u].f[j] = gv[u].f[j] = gc[u].f[j] = 0.f;
             }
             // issue every load of the pass before any arithmetic
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 if (nv[u] > 0) {
-                    w4[u] = ldg_f4(P.w + sbase + e0[u]);
-                    m4[u] = ldg_f4(P.m + sbase + e0[u]);
-                    if (HAS_V) v4[u] = ldg_f4(P.v + sbase + e0[u]);
+                    wv[u] = load_f32<VEC>(P.w + sbase + e0[u]);
+                    mv[u] = load_f32<VEC>(P.m + sbase + e0[u]);
+                    if (HAS_V) vv[u] = load_f32<VEC>(P.v + sbase + e0[u]);
                 }
             }
             if (READS_G) {
-                for (int k0 = 0; k0 < P.R; k0 += RB) {
-                    float4 gb[U][RB];
+                for (int k0 = 0; k0 < (LOOPK ? P.R : 1); k0 += RB) {
+                    GradRaw<GBF, VEC> raw[U][RB];
+                    bool have[RB];
 #pragma unroll
                     for (int j = 0; j < RB; ++j) {
+                        have[j] = (RB == 1) || (k0 + j < P.R);
 #pragma unroll
-                        for (int u = 0; u < U; ++u) {
-                            gb[u][j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                            if (k0 + j < P.R && nv[u] > 0) gb[u][j] = load_grad4<GBF>(gp.p[k0 + j], gbase + e0[u]);
-                        }
+                        for (int u = 0; u < U; ++u)
+                            if (have[j] && nv[u] > 0) {
+                                if constexpr (FUSED) {
+                                    const void* gk = gt[k0 + j];
+                                    if (nv[u] == VEC) raw[u][j] = load_grad<GBF, VEC>(gk, toff + e0[u]);
+                                    else raw[u][j] = load_grad_partial<GBF, VEC>(gk, toff + e0[u], nv[u]);
+                                } else {
+                                    raw[u][j] = load_grad<GBF, VEC>(gp.p[k0 + j], gbase + e0[u]);
+                                }
+                            }
                     }
 #pragma unroll
                     for (int u = 0; u < U; ++u) {
+                        Fv<VEC> gb[RB];
+#pragma unroll
+                        for (int j = 0; j < RB; ++j) {
+                            if (have[j] && nv[u] > 0) {
+                                gb[j] = widen<GBF, VEC>(raw[u][j]);
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < VEC; ++i) gb[j].f[i] = 0.f;
+                            }
+                        }
 #pragma unroll
                         for (int s = 1; s < RB; s <<= 1)
 #pragma unroll
-                            for (int j = 0; j + s < RB; j += 2 * s) gb[u][j] = add4(gb[u][j], gb[u][j + s]);
-                        if (k0 == 0) {
-                            g4[u] = gb[u][0];
+                            for (int j = 0; j + s < RB; j += 2 * s)
+#pragma unroll
+                                for (int i = 0; i < VEC; ++i) gb[j].f[i] += gb[j + s].f[i];
+                        if (!LOOPK || k0 == 0) {
+                            gv[u] = gb[0];
                         } else {
-                            kahan1(g4[u].x, gc[u].x, gb[u][0].x);
-                            kahan1(g4[u].y, gc[u].y, gb[u][0].y);
-                            kahan1(g4[u].z, gc[u].z, gb[u][0].z);
-                            kahan1(g4[u].w, gc[u].w, gb[u][0].w);
+#pragma unroll
+                            for (int i = 0; i < VEC; ++i) kahan1(gv[u].f[i], gc[u].f[i], gb[0].f[i]);
                         }
                     }
                 }
@@ -203,34 +387,34 @@ __global__ void __launch_bounds__(kBlock) update_kernel(const UpdParams P, const
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 if (nv[u] < 0) continue;
-                float wv[4] = {w4[u].x, w4[u].y, w4[u].z, w4[u].w};
-                float mv[4] = {m4[u].x, m4[u].y, m4[u].z, m4[u].w};
-                float vv[4] = {v4[u].x, v4[u].y, v4[u].z, v4[u].w};
-                const float gv[4] = {g4[u].x, g4[u].y, g4[u].z, g4[u].w};
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < VEC; ++j) {
                     if (j < nv[u]) {
-                        update_elem<OPT>(P.c, gv[j] * P.c.gscale, wv[j], mv[j], vv[j], lr_rho, sw, su);
+                        update_elem<OPT>(P.c, gv[u].f[j] * P.c.gscale, wv[u].f[j], mv[u].f[j], vv[u].f[j], lr_rho, sw, su);
                     } else {  // pad: identity for the sums, +0 for every output
-                        wv[j] = 0.f; mv[j] = 0.f; vv[j] = 0.f;
+                        wv[u].f[j] = 0.f; mv[u].f[j] = 0.f; vv[u].f[j] = 0.f;
                     }
                 }
                 const long long so = sbase + e0[u];
-                if (OPT != K_LAMB1) stg_f4(P.w + so, make_float4(wv[0], wv[1], wv[2], wv[3]));
-                if (OPT == K_LAMB1 && nv[u] < 4) stg_f4(P.w + so, make_float4(wv[0], wv[1], wv[2], wv[3]));
+                if (OPT != K_LAMB1 || nv[u] < VEC) store_f32<VEC>(P.w + so, wv[u]);
                 if (OPT != K_LAMB2) {
-                    stg_f4(P.m + so, make_float4(mv[0], mv[1], mv[2], mv[3]));
-                    if (HAS_V) stg_f4(P.v + so, make_float4(vv[0], vv[1], vv[2], vv[3]));
+                    store_f32<VEC>(P.m + so, mv[u]);
+                    if (HAS_V) store_f32<VEC>(P.v + so, vv[u]);
                 }
-                if (OUT == O_F32) {
-                    stg_f4(reinterpret_cast<float*>(P.gathered) + obase + e0[u], make_float4(wv[0], wv[1], wv[2], wv[3]));
+                if constexpr (FUSED) {
+                    if (OUT == O_F32) {
+                        float* dst = reinterpret_cast<float*>(wt) + toff + e0[u];
+                        if (nv[u] == VEC) store_f32<VEC>(dst, wv[u]);
+                        else store_f32_partial<VEC>(dst, wv[u], nv[u]);
+                    } else if (OUT == O_BF16) {
+                        unsigned short* dst = reinterpret_cast<unsigned short*>(wt) + toff + e0[u];
+                        if (nv[u] == VEC) store_bf16<VEC>(dst, wv[u]);
+                        else store_bf16_partial<VEC>(dst, wv[u], nv[u]);
+                    }
+                } else if (OUT == O_F32) {
+                    store_f32<VEC>(reinterpret_cast<float*>(P.gathered) + obase + e0[u], wv[u]);
                 } else if (OUT == O_BF16) {
-                    const __nv_bfloat162 lo = __floats2bfloat162_rn(wv[0], wv[1]);
-                    const __nv_bfloat162 hi = __floats2bfloat162_rn(wv[2], wv[3]);
-                    uint2 pk;
-                    pk.x = *reinterpret_cast<const unsigned int*>(&lo);
-                    pk.y = *reinterpret_cast<const unsigned int*>(&hi);
-                    __stcs(reinterpret_cast<uint2*>(reinterpret_cast<unsigned short*>(P.gathered) + obase + e0[u]), pk);
+                    store_bf16<VEC>(reinterpret_cast<unsigned short*>(P.gathered) + obase + e0[u], wv[u]);
                 }
             }
         }
@@ -278,56 +462,83 @@ __global__ void __launch_bounds__(kBlock) lamb_finalize_kernel(const WsSegTiles*
 }
 
 // -------------------------------------------------------------- dispatch ---
-int sm_count() {
-    static thread_local int dev_cached = -1, sms = 148;
-    int dev = 0;
-    cudaGetDevice(&dev);
-    if (dev != dev_cached) {
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        dev_cached = dev;
-    }
-    return sms;
-}
-
-template <int OPT, bool GBF, int OUT, int U, int RB, int NP>
+#ifndef WS_TUNE_GRID
+#define WS_TUNE_GRID 0
+#endif
+template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED>
 ws_status launch(const UpdParams& P, const void* const* gptrs, cudaStream_t st) {
     GradPtrs<NP> gp;
-    for (int k = 0; k < NP; ++k) gp.p[k] = (gptrs && k < P.R) ? gptrs[k] : nullptr;
+    for (int k = 0; k < NP; ++k) gp.p[k] = (!FUSED && gptrs && k < P.R) ? gptrs[k] : nullptr;
     long long grid = P.nitems;
-    const long long cap = (long long)sm_count() * 32;
-    if (grid > cap) grid = cap;
     if (grid < 1) return WS_OK;
-    update_kernel<OPT, GBF, OUT, U, RB, NP><<<(unsigned)grid, kBlock, 0, st>>>(P, gp);
-    return ws_check_launch("ws_shard_update");
+    if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;
+    update_kernel<OPT, GBF, OUT, VEC, U, RB, NP, FUSED><<<(unsigned)grid, kBlock, 0, st>>>(P, gp);
+    return ws_check_launch(FUSED ? "ws_fused_update" : "ws_shard_update");
 }
 
-template <int OPT, bool GBF, int OUT>
-ws_status launch_r(const UpdParams& P, const void* const* gptrs, cudaStream_t st) {
-    if (OPT == K_LAMB2) return launch<OPT, GBF, OUT, 2, 1, 1>(P, gptrs, st);
-    if (P.R <= 2) return launch<OPT, GBF, OUT, 2, 2, 8>(P, gptrs, st);
-    if (P.R <= 4) return launch<OPT, GBF, OUT, 2, 4, 8>(P, gptrs, st);
-    if (P.R <= 32) return launch<OPT, GBF, OUT, 1, 8, 32>(P, gptrs, st);
-    if (P.R <= 1024) return launch<OPT, GBF, OUT, 1, 8, 1024>(P, gptrs, st);
-    return WS_ERR_TOO_LARGE;
+// Wide (256-bit) accesses need 32-byte aligned buffers; they pay off when the
+// gradients are bf16 (a 128-bit gradient load then covers 8 elements) and for
+// small R, where the fp32 streams dominate.
+template <int OPT, bool GBF, int OUT, bool FUSED>
+ws_status launch_r(const UpdParams& P, const void* const* gptrs, bool wide_ok, cudaStream_t st) {
+    if constexpr (OPT == K_LAMB2) {
+        if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 1, 1, FUSED>(P, gptrs, st);
+        return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 1, 1, FUSED>(P, gptrs, st);
+    } else {
+        if (P.R <= 2) {
+            if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 2, 2, FUSED>(P, gptrs, st);
+            return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 2, 2, FUSED>(P, gptrs, st);
+        }
+        if (P.R <= 4) {
+            if constexpr (GBF) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 4, 4, FUSED>(P, gptrs, st);
+            return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 4, 4, FUSED>(P, gptrs, st);
+        }
+        if (P.R <= 8) {
+            if constexpr (GBF) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 8, 8, FUSED>(P, gptrs, st);
+            return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 8, 8, FUSED>(P, gptrs, st);
+        }
+        if (P.R <= 32) {
+            if constexpr (GBF) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 8, 32, FUSED>(P, gptrs, st);
+            return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 8, 32, FUSED>(P, gptrs, st);
+        }
+        if (P.R <= 1024) return launch<OPT, GBF, OUT, 4, 1, 8, 1024, FUSED>(P, gptrs, st);
+        return WS_ERR_TOO_LARGE;
+    }
 }
 
-template <int OPT, bool GBF>
-ws_status launch_o(const UpdParams& P, const void* const* gptrs, int out, cudaStream_t st) {
-    if (OPT == K_LAMB1) return launch_r<OPT, GBF, O_NONE>(P, gptrs, st);
-    switch (out) {
-        case O_NONE: return launch_r<OPT, GBF, O_NONE>(P, gptrs, st);
-        case O_F32: return launch_r<OPT, GBF, O_F32>(P, gptrs, st);
-        default: return launch_r<OPT, GBF, O_BF16>(P, gptrs, st);
+bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) == 0; }
+
+// `wide` on entry: whether the caller-side tensors (fused formatting) allow 256-bit accesses.
+template <int OPT, bool GBF, bool FUSED>
+ws_status launch_o(const UpdParams& P, const void* const* gptrs, int out, bool wide, cudaStream_t st) {
+    wide = wide && aligned32(P.w) && aligned32(P.m) && aligned32(P.v) && aligned32(P.gathered);
+    if (!FUSED && OPT != K_LAMB2)
+        for (int k = 0; k < P.R && wide; ++k) wide = aligned32(gptrs[k]);
+    if constexpr (OPT == K_LAMB1) {
+        return launch_r<OPT, GBF, O_NONE, FUSED>(P, gptrs, wide, st);
+    } else {
+        switch (out) {
+            case O_NONE:
+                if constexpr (FUSED) return WS_ERR_INVALID_ARG;
+                else return launch_r<OPT, GBF, O_NONE, FUSED>(P, gptrs, wide, st);
+            case O_F32: return launch_r<OPT, GBF, O_F32, FUSED>(P, gptrs, wide, st);
+            default: return launch_r<OPT, GBF, O_BF16, FUSED>(P, gptrs, wide, st);
+        }
+    }
+}
+
+template <bool FUSED>
+ws_status launch_f(int opt, bool gbf, int out, const UpdParams& P, const void* const* gptrs, bool wide, cudaStream_t st) {
+    switch (opt) {
+        case K_SGDM: return gbf ? launch_o<K_SGDM, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_SGDM, false, FUSED>(P, gptrs, out, wide, st);
+        case K_ADAM: return gbf ? launch_o<K_ADAM, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_ADAM, false, FUSED>(P, gptrs, out, wide, st);
+        case K_LAMB1: return gbf ? launch_o<K_LAMB1, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_LAMB1, false, FUSED>(P, gptrs, out, wide, st);
+        default: return launch_o<K_LAMB2, false, FUSED>(P, gptrs, out, wide, st);
     }
 }
 
 ws_status launch_any(int opt, bool gbf, int out, const UpdParams& P, const void* const* gptrs, cudaStream_t st) {
-    switch (opt) {
-        case K_SGDM: return gbf ? launch_o<K_SGDM, true>(P, gptrs, out, st) : launch_o<K_SGDM, false>(P, gptrs, out, st);
-        case K_ADAM: return gbf ? launch_o<K_ADAM, true>(P, gptrs, out, st) : launch_o<K_ADAM, false>(P, gptrs, out, st);
-        case K_LAMB1: return gbf ? launch_o<K_LAMB1, true>(P, gptrs, out, st) : launch_o<K_LAMB1, false>(P, gptrs, out, st);
-        default: return launch_o<K_LAMB2, false>(P, gptrs, out, st);
-    }
+    return launch_f<false>(opt, gbf, out, P, gptrs, true, st);
 }
 
 WsConsts make_consts(const ws_hyper* h) {
@@ -350,7 +561,7 @@ WsConsts make_consts(const ws_hyper* h) {
 
 // Argument checks shared by the entry points; fills P.  phase: K_* kernel id.
 ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state* s, const ws_hyper* h,
-                  const ws_out* out, int phase, UpdParams& P, int& out_kind, bool& gbf) {
+                  const ws_out* out, int phase, UpdParams& P, int& out_kind, bool& gbf, bool fused = false) {
     if (!p || !s || !h) return WS_ERR_INVALID_ARG;
     if (!p->d_tiles) return WS_ERR_NOT_UPLOADED;
     if (r < -1 || r >= p->R) return WS_ERR_INVALID_ARG;
@@ -359,7 +570,9 @@ ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state
     if (!s->w || !s->m || (needs_v && !s->v)) return WS_ERR_INVALID_ARG;
     if (!ws_aligned16(s->w) || !ws_aligned16(s->m) || (needs_v && !ws_aligned16(s->v))) return WS_ERR_ALIGNMENT;
     gbf = false;
-    if (phase != K_LAMB2) {
+    P.gtab = nullptr;
+    P.wtab = nullptr;
+    if (phase != K_LAMB2 && !fused) {
         if (!g || !g->ptrs || g->R < 1) return WS_ERR_INVALID_ARG;
         if (g->dtype != WS_F32 && g->dtype != WS_BF16) return WS_ERR_DTYPE;
         if (g->slice_mode != 0 && g->slice_mode != 1) return WS_ERR_INVALID_ARG;
@@ -388,7 +601,7 @@ ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state
     P.r0 = (r < 0) ? 0 : r;
     P.nitems = (long long)nshards * p->ntiles;
     P.st_stride = (r < 0) ? p->S : 0;
-    if (g && phase != K_LAMB2) {
+    if (g && phase != K_LAMB2 && !fused) {
         // slice mode 0: pointer is the packed buffer; the launch starts at shard r0
         P.g_stride = (g->slice_mode == 0) ? p->S : 0;
     } else {
@@ -482,4 +695,95 @@ extern "C" ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_gr
     std::vector<const void*> gp;
     offset_grad_ptrs(plan, r, grads, gp);
     return launch_any(phase, gbf, ok, P, gp.data(), (cudaStream_t)stream);
+}
+
+// ------------------------------------------------ fused formatting path ---
+
+extern "C" size_t ws_tensor_table_bytes(const ws_plan* plan, int32_t nsets) {
+    if (!plan || nsets < 1) return 0;
+    return ((size_t)plan->T * (size_t)nsets * sizeof(void*) + 15) & ~(size_t)15;
+}
+
+extern "C" ws_status ws_tensor_table_upload(const ws_plan* plan, const void* const* ptrs, int32_t nsets, ws_dtype dtype,
+                                            void* dev_buf, size_t bytes, void* stream, ws_tensor_table* out) {
+    if (!plan || !ptrs || !dev_buf || !out || nsets < 1 || nsets > 1024) return WS_ERR_INVALID_ARG;
+    if (dtype != WS_F32 && dtype != WS_BF16) return WS_ERR_DTYPE;
+    if (!ws_aligned16(dev_buf)) return WS_ERR_ALIGNMENT;
+    if (bytes < ws_tensor_table_bytes(plan, nsets)) return WS_ERR_WORKSPACE;
+    const int T = plan->T;
+    std::vector<const void*> host((size_t)T * nsets);
+    int min_align = 256;
+    for (int k = 0; k < nsets; ++k)
+        for (int t = 0; t < T; ++t) {
+            const void* q = ptrs[(size_t)k * T + t];
+            if (!q) return WS_ERR_INVALID_ARG;
+            if (!ws_aligned16(q)) return WS_ERR_ALIGNMENT;
+            while (min_align > 16 && (reinterpret_cast<uintptr_t>(q) & (uintptr_t)(min_align - 1)) != 0) min_align >>= 1;
+            host[(size_t)t * nsets + k] = q;   // device layout [T][nsets]: a tile finds its pointers side by side
+        }
+    cudaError_t e = cudaMemcpyAsync(dev_buf, host.data(), host.size() * sizeof(void*), cudaMemcpyHostToDevice,
+                                    (cudaStream_t)stream);
+    if (e != cudaSuccess) return ws_cuda_fail(e, "ws_tensor_table_upload");
+    // the host vector is pageable: the runtime has staged it before cudaMemcpyAsync returns
+    out->dev = dev_buf;
+    out->nsets = nsets;
+    out->T = T;
+    out->dtype = dtype;
+    out->min_align = min_align;
+    return WS_OK;
+}
+
+namespace {
+
+ws_status fused_phase(const ws_plan* plan, int32_t r, const ws_tensor_table* grads, const ws_state* state,
+                      const ws_hyper* hyper, const ws_tensor_table* weights, int phase, void* workspace,
+                      cudaStream_t st) {
+    UpdParams P;
+    int ok;
+    bool gbf;
+    ws_status s = prepare(plan, r, nullptr, state, hyper, nullptr, phase, P, ok, gbf, true);
+    if (s != WS_OK) return s;
+    bool wide = true;
+    int out_kind = O_NONE;
+    if (phase != K_LAMB2) {
+        P.gtab = (const void* const*)grads->dev;
+        P.R = grads->nsets;
+        gbf = grads->dtype == WS_BF16;
+        wide = wide && (gbf || grads->min_align >= 32);
+    }
+    if (phase != K_LAMB1) {
+        P.wtab = (void* const*)weights->dev;
+        out_kind = weights->dtype == WS_F32 ? O_F32 : O_BF16;
+        wide = wide && (weights->dtype == WS_BF16 || weights->min_align >= 32);
+    }
+    if (phase == K_LAMB1 || phase == K_LAMB2) {
+        WsLambWs L = ws_lamb_layout(plan, workspace);
+        P.partials = L.partials;
+        P.rho = L.rho;
+    }
+    return launch_f<true>(phase, gbf, out_kind, P, nullptr, wide, st);
+}
+
+}  // namespace
+
+extern "C" ws_status ws_fused_update(const ws_plan* plan, int32_t r, const ws_tensor_table* grads, const ws_state* state,
+                                     const ws_hyper* hyper, const ws_tensor_table* weights, void* workspace,
+                                     size_t workspace_bytes, void* stream) {
+    if (!plan || !grads || !weights || !hyper || !state) return WS_ERR_INVALID_ARG;
+    if (!grads->dev || !weights->dev) return WS_ERR_INVALID_ARG;
+    if (grads->T != plan->T || weights->T != plan->T || grads->nsets != plan->R || weights->nsets != 1)
+        return WS_ERR_INVALID_ARG;
+    if ((grads->dtype != WS_F32 && grads->dtype != WS_BF16) || (weights->dtype != WS_F32 && weights->dtype != WS_BF16))
+        return WS_ERR_DTYPE;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (hyper->opt == WS_LAMB) {
+        if (r != -1) return WS_ERR_INVALID_ARG;
+        ws_status s = check_ws(plan, workspace, workspace_bytes);
+        if (s != WS_OK) return s;
+        if ((s = fused_phase(plan, -1, grads, state, hyper, weights, K_LAMB1, workspace, st)) != WS_OK) return s;
+        if ((s = ws_lamb_finalize(plan, workspace, workspace_bytes, stream)) != WS_OK) return s;
+        return fused_phase(plan, -1, grads, state, hyper, weights, K_LAMB2, workspace, st);
+    }
+    if (hyper->opt != WS_SGDM && hyper->opt != WS_ADAM) return WS_ERR_INVALID_ARG;
+    return fused_phase(plan, r, grads, state, hyper, weights, hyper->opt == WS_SGDM ? K_SGDM : K_ADAM, nullptr, st);
 }

@@ -173,6 +173,36 @@ def test_update_all_shards_matches_oracle(opt, R, gdtype):
         assert rel.max() <= TOL_LAMB, rel.max()
 
 
+@pytest.mark.parametrize("tile", [1024, 4096, 16384])
+@pytest.mark.parametrize("opt,gdtype", [("sgdm", torch.float32), ("adam", torch.bfloat16), ("lamb", torch.float32)])
+def test_tile_sizes_give_the_same_result(tile, opt, gdtype):
+    # pieces of 1, 1.3 and 5.2 tiles at the largest tile size; the result may not depend on the tiling
+    shapes = [(3, 7), (40000,), (17, 4099), (9,), (171, 1000)]
+    R = 2
+    wl, w, m, v, g = _model(shapes, R, gdtype, seed=tile)
+    h = B.make_hyper(opt, _hyper(opt))
+    outs = []
+    for t in (2048, tile):
+        plan = B.Plan(shapes, R, 32, t)
+        pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+        gath = torch.zeros(plan.G, dtype=torch.bfloat16, device=DEV)
+        ws = torch.zeros(max(16, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+        B.ws_shard_update(plan, -1, pg, pw, pm, pv if opt != "sgdm" else None, h, gath, ws)
+        back = [torch.empty_like(x) for x in w]
+        B.ws_unpack(plan, pw, back)
+        outs.append((pw, pm, pv, gath, back))
+    a, b = outs
+    assert torch.equal(a[1], b[1]) and torch.equal(a[2], b[2])          # moments: elementwise, tiling-free
+    if opt != "lamb":
+        assert torch.equal(a[0], b[0]) and torch.equal(a[3], b[3])
+    else:   # the norm partial sums are grouped by tile: last-bit differences in rho only
+        oplan = O.Plan(wl.numels, R, 32)
+        for x, y in zip(O.unpack(oplan, to_np(a[0])), O.unpack(oplan, to_np(b[0]))):
+            assert err(x, y) <= 2e-7
+    for x, y in zip(a[4], b[4]):
+        assert err(to_np(x), to_np(y)) <= 2e-7
+
+
 @pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb"])
 @pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
 def test_bf16_gathered_copy(opt, gdtype):
@@ -308,3 +338,104 @@ def test_argument_errors_are_status_codes():
     assert L.ws_shard_update(plan.handle, 0, C.byref(g), C.byref(s), C.byref(hl), None, None, 0, None) == 1
     torch.cuda.synchronize()
     assert float(buf.abs().sum()) == 0.0                                     # nothing was launched
+
+
+# ------------------------------------------------- fused formatting path ---
+def _views_with_guards(numels, dtype, fill, misalign):
+    """One buffer per tensor with 64-element guards; `misalign` shifts the view by 16 bytes so
+    that tensors are 16- but not 32-byte aligned."""
+    shift = (16 // torch.empty(0, dtype=dtype).element_size()) if misalign else 0
+    bigs, views = [], []
+    for n in numels:
+        big = torch.full((n + 128 + shift,), fill, dtype=dtype, device=DEV)
+        bigs.append(big)
+        views.append(big[64 + shift:64 + shift + n])
+    return bigs, views
+
+
+@pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb"])
+@pytest.mark.parametrize("R", [1, 3, 8, 40])
+@pytest.mark.parametrize("gdtype,odtype,misalign", [(torch.float32, torch.float32, False),
+                                                     (torch.bfloat16, torch.bfloat16, False),
+                                                     (torch.float32, torch.bfloat16, True),
+                                                     (torch.bfloat16, torch.float32, True)])
+def test_fused_update_equals_pack_update_unpack(opt, R, gdtype, odtype, misalign):
+    wl, w, m, v, g = _model(SHAPES, R, gdtype, seed=R + 50)
+    plan = B.Plan(SHAPES, R, 32)
+    h = B.make_hyper(opt, _hyper(opt))
+    numels = wl.numels
+    # reference: pack every gradient list, update, unpack the gathered buffer
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    fw, fm, fv = pw.clone(), pm.clone(), pv.clone()
+    gathered = torch.zeros(plan.G, dtype=odtype, device=DEV)
+    ws = torch.zeros(max(16, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv if opt != "sgdm" else None, h, gathered, ws)
+    ref_w = [torch.empty(n, dtype=odtype, device=DEV) for n in numels]
+    B.ws_unpack(plan, gathered, ref_w)
+    # fused: gradient tensors (optionally only 16-byte aligned) in, weight tensors out
+    gb = [_views_with_guards(numels, gdtype, float("nan"), misalign) for _ in range(R)]
+    for (bigs, views), gk in zip(gb, g):
+        for dst, src in zip(views, gk):
+            dst.copy_(src)
+    wb_bigs, wb_views = _views_with_guards(numels, odtype, 7.0, misalign)
+    gt = B.TensorTable(plan, [views for _, views in gb])
+    wt = B.TensorTable(plan, [wb_views])
+    assert gt.c.min_align >= (32 if not misalign else 16)
+    ws2 = torch.zeros_like(ws)
+    B.ws_fused_update(plan, -1, gt, fw, fm, fv if opt != "sgdm" else None, h, wt, ws2)
+    # With 16-byte-only alignment the fused kernel runs its 128-bit variant while the packed path
+    # runs the 256-bit one: elementwise results are identical, but LAMB's norm partial sums are
+    # grouped differently, so rho (hence w') may differ in the last bit.
+    exact = not (opt == "lamb" and misalign)
+    assert torch.equal(fm, pm)
+    if opt != "sgdm":
+        assert torch.equal(fv, pv)
+    if exact:
+        assert torch.equal(fw, pw)
+    else:
+        assert err(to_np(fw), to_np(pw)) <= 2e-7
+    shift = (16 // ref_w[0].element_size()) if misalign else 0
+    for big, view, ref, n in zip(wb_bigs, wb_views, ref_w, numels):
+        if exact:
+            assert torch.equal(view, ref)
+        else:
+            assert err(to_np(view.float()), to_np(ref.float())) <= (TOL_BF16 if odtype == torch.bfloat16 else 2e-7)
+        guard = torch.full((64 + shift,), 7.0, dtype=odtype, device=DEV)
+        assert torch.equal(big[:64 + shift], guard) and torch.equal(big[64 + shift + n:], guard[:64])
+
+
+@pytest.mark.parametrize("opt", ["sgdm", "adam"])
+def test_fused_update_shard_by_shard(opt):
+    R = 5
+    wl, w, m, v, g = _model(SHAPES, R, seed=77)
+    plan = B.Plan(SHAPES, R, 32)
+    h = B.make_hyper(opt, _hyper(opt))
+    pw, pm, pv, _ = _pack_all(plan, w, m, v, g)
+    aw, am, av = pw.clone(), pm.clone(), pv.clone()
+    gt = B.TensorTable(plan, g)
+    out_all = [torch.zeros_like(x) for x in w]
+    out_one = [torch.zeros_like(x) for x in w]
+    B.ws_fused_update(plan, -1, gt, aw, am, av if opt != "sgdm" else None, h, B.TensorTable(plan, [out_all]))
+    wt = B.TensorTable(plan, [out_one])
+    S = plan.S
+    for r in range(R):
+        sl = slice(r * S, (r + 1) * S)
+        B.ws_fused_update(plan, r, gt, pw[sl], pm[sl], pv[sl] if opt != "sgdm" else None, h, wt)
+    assert torch.equal(aw, pw) and torch.equal(am, pm)
+    for a, b in zip(out_all, out_one):
+        assert torch.equal(a, b)
+
+
+def test_fused_update_matches_oracle_unsharded():
+    # the fused path straight against the plain definition (no packed buffers anywhere)
+    wl = W.scaled_down(W.resnet50(), 48)
+    w, m, v = W.make_state(wl, DEV)
+    g = W.make_grads(wl, DEV)
+    plan = B.Plan(wl.shapes, wl.R, 32)
+    ow, om, _, _ = _oracle_unsharded(wl.opt, wl.hyper, w, m, v, g)
+    pw, pm, pv, _ = _pack_all(plan, w, m, v, [])
+    outs = [torch.zeros_like(x) for x in w]
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), pw, pm, None, B.make_hyper(wl.opt, wl.hyper),
+                      B.TensorTable(plan, [outs]))
+    for a, b in zip(outs, ow):
+        assert err(to_np(a), b) <= TOL_FP32

@@ -58,14 +58,19 @@ def test_planner_matches_oracle_planner(R, A):
 def test_planner_on_model_shaped_workloads():
     for name in ("tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b"):
         wl = W.WORKLOADS[name]()
-        plan = B.Plan(wl.shapes, wl.R, 32, upload=False)
         ref = O.Plan(wl.numels, wl.R, 32)
-        assert (plan.S, plan.N) == (ref.S, ref.N)
-        segs = plan.segments()
-        assert [s.piece for s in segs] == list(ref.piece)
-        assert [s.shard_off for s in segs] == list(ref.off)
-        # tiles cover each piece exactly once, in order
-        assert plan.ntiles == sum(-(-int(p) // 2048) for p in ref.piece)
+        for tile in (0, 2048, 8192):
+            plan = B.Plan(wl.shapes, wl.R, 32, tile, upload=False)
+            assert (plan.S, plan.N) == (ref.S, ref.N)
+            segs = plan.segments()
+            assert [s.piece for s in segs] == list(ref.piece)
+            assert [s.shard_off for s in segs] == list(ref.off)
+            if tile:    # tiles cover each piece exactly once, in order
+                assert plan.ntiles == sum(-(-int(p) // tile) for p in ref.piece)
+            else:       # default tile: between 2048 and 16384 elements
+                lo = sum(-(-int(p) // 16384) for p in ref.piece)
+                hi = sum(-(-int(p) // 2048) for p in ref.piece)
+                assert lo <= plan.ntiles <= hi
 
 
 def test_paper_worked_numbers_through_the_library():

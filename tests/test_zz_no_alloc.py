@@ -66,7 +66,7 @@ def test_static_scratch_lamb_equals_workspace_lamb_on_two_steps(R, gdtype):
 
 def test_static_scratch_rejects_plans_beyond_its_size():
     # 4 MiB of scratch cannot hold the partial sums of this plan: refused, nothing launched
-    plan = B.Plan([(32768, 32768)] * 2, 16, 32, upload=False)      # 2.1e9 parameters
+    plan = B.Plan([(32768, 32768)] * 2, 16, 32, 2048, upload=False)      # 2.1e9 parameters, 2048-element tiles
     assert plan.workspace_bytes("lamb") > B.lib().ws_static_scratch_bytes()
     buf = torch.zeros(8, device=DEV)
     ptrs = (C.c_void_p * 16)(*([buf.data_ptr()] * 16))
