@@ -50,6 +50,9 @@ def parse_args():
     ap.add_argument("--R", type=int, default=0, help="override the workload's replica count")
     ap.add_argument("--align", type=int, default=32)
     ap.add_argument("--tile", type=int, default=0, help="work-tile elements (0 = library default)")
+    ap.add_argument("--path", default="both", choices=["both", "fused", "unfused"],
+                    help="fused: one kernel reads the gradient tensors and writes the weight tensors; "
+                         "unfused: pack, update, unpack as separate kernels; both: time both, headline = fused")
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -74,8 +77,10 @@ def bytes_per_param(wl):
     if wl.opt == "lamb":
         upd += 12          # plain two-pass: phase 2 reads w, m', v' again and rewrites w
     out_b = 2 if str(wl.out_dtype).endswith("bfloat16") else 0
+    # fused formatting: same reads and state writes, plus the weight tensors written directly
+    fused = upd + (2 if out_b else 4)
     upd += out_b
-    return {"update": upd, "pack": 2 * gb, "unpack": 2 * (2 if out_b else 4)}
+    return {"update": upd, "fused": fused, "pack": 2 * gb, "unpack": 2 * (2 if out_b else 4)}
 
 
 # ----------------------------------------------------------------------------
@@ -227,11 +232,14 @@ def run_reference(args):
     print(json.dumps(line))
 
 
-def config_of(wl, args, extra=None):
+def config_of(wl, args, extra=None, path="unfused"):
+    steps = {"unfused": "pack R gradient sets + fused reduce/update of all shards + unpack weights (separate kernels)",
+             "fused": "one kernel: gradients read from the R replicas' tensor lists (formatting fused in), reduce, "
+                      "update of all shards, weights written to the weight tensors"}
     c = {"workload": f"{wl.name}: {wl.T} tensors, {wl.N} params, R={wl.R} replicas, {wl.opt}, "
                      f"grads {str(wl.grad_dtype).split('.')[-1]}, gathered {str(wl.out_dtype).split('.')[-1]}",
          "R": wl.R, "optimizer": wl.opt, "align_elems": args.align,
-         "step": "pack R gradient sets + fused reduce/update of all shards + unpack weights",
+         "step": steps[path],
          "l2": "inputs exceed L2 (no flush)" if wl.N * 4 * (wl.R + 3) > 256e6 else "flush between steps"}
     if extra:
         c.update(extra)
@@ -269,8 +277,19 @@ def run_ours(args):
     R, T, N = wl.R, wl.T, wl.N
     plan = B.Plan(wl.shapes, R, args.align, args.tile, device=dev)
     gdt, odt = wl.grad_dtype, wl.out_dtype
+    gb = 2 if gdt == torch.bfloat16 else 4
+    wb = 2 if odt == torch.bfloat16 else 4
     numels = wl.numels
     A_el = plan.arena_elems
+    total_mem = torch.cuda.get_device_properties(dev).total_memory
+    run_unfused = args.path in ("both", "unfused")
+    run_fused = args.path in ("both", "fused")
+    need_unfused = R * (A_el + plan.G) * gb + 3 * plan.G * 4 + plan.G * wb + A_el * wb
+    unfused_skipped = None
+    if run_unfused and need_unfused > 0.85 * total_mem:
+        unfused_skipped = f"needs {need_unfused / 1e9:.0f} GB of device memory (tensor lists plus packed gradient buffers)"
+        run_unfused = False
+        run_fused = True
 
     # ---- device-resident inputs: per replica one gradient arena, viewed tensor by tensor
     w, m, v = W.make_state(wl, dev)
@@ -280,7 +299,7 @@ def run_ours(args):
         B.ws_pack(plan, src, dst)
     if wl.opt == "sgdm":
         pv = None
-    del m, v
+    del w, m, v
     g_arena = [torch.zeros(A_el, dtype=gdt, device=dev) for _ in range(R)]
     g_views = [B.PtrList(plan.arena_views(a, numels)) for a in g_arena]
     for k in range(R):
@@ -288,18 +307,23 @@ def run_ours(args):
         for dst, src in zip(g_views[k], gk):
             dst.copy_(src)
         del gk
-    pg = B.PtrList([torch.empty(plan.G, dtype=gdt, device=dev) for _ in range(R)])
-    gathered = torch.empty(plan.G, dtype=odt, device=dev) if odt != torch.float32 else None
     w_arena = torch.zeros(A_el, dtype=odt, device=dev)
     w_views = B.PtrList(plan.arena_views(w_arena, numels))
     ws = torch.empty(max(16, plan.workspace_bytes(wl.opt)), dtype=torch.uint8, device=dev)
     hy = B.make_hyper(wl.opt, wl.hyper)
-    del w
+    pg = gathered = None
+    if run_unfused:
+        pg = B.PtrList([torch.empty(plan.G, dtype=gdt, device=dev) for _ in range(R)])
+        gathered = torch.empty(plan.G, dtype=odt, device=dev) if odt != torch.float32 else None
+    gtab = wtab = None
+    if run_fused:
+        gtab = B.TensorTable(plan, [gv.tensors for gv in g_views])
+        wtab = B.TensorTable(plan, [w_views.tensors])
     flush = None
     if N * 4 * (R + 3) <= 256e6:
         flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device=dev)
 
-    def step(ev=None):
+    def step_unfused(ev=None):
         if flush is not None:
             flush.zero_()
         if ev:
@@ -315,38 +339,61 @@ def run_ours(args):
         if ev:
             ev[3].record()
 
+    def step_fused(ev=None):
+        if flush is not None:
+            flush.zero_()
+        if ev:
+            ev[0].record()
+        B.ws_fused_update(plan, -1, gtab, pw, pm, pv, hy, wtab, ws)
+        if ev:
+            ev[1].record()
+
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
+    K = args.steps
+    W_ = max(3, args.warmup)
+
+    def time_path(step, nev):
+        for _ in range(W_):
+            step()
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nev)] for _ in range(K)]
+        barrier()
+        t0 = time.time()
+        for i in range(K):
+            step(evs[i])
+        barrier()
+        t1 = time.time()
+        total_ms = evs[0][0].elapsed_time(evs[-1][nev - 1])
+        if flush is not None:   # leave the L2 flush out of the step time
+            total_ms = sum(e[0].elapsed_time(e[nev - 1]) for e in evs)
+        phase_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / K for i in range(nev - 1)]
+        if world > 1:
+            tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            total_ms = float(tt.item())
+        return total_ms / K, phase_ms, (t0, t1)
+
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    for _ in range(max(3, args.warmup)):
-        step()
-    K = args.steps
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(K)]
-    barrier()
-    t_host0 = time.time()
-    for i in range(K):
-        step(evs[i])
-    barrier()
-    t_host1 = time.time()
-    total_ms = evs[0][0].elapsed_time(evs[-1][3])
-    if flush is not None:
-        total_ms = sum(e[0].elapsed_time(e[3]) for e in evs)   # leave the L2 flush out of the step time
-    phase_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / K for i in range(3)]
-    if world > 1:
-        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
-    ms_per_step = total_ms / K
+    res = {}
+    if run_unfused:
+        res["unfused"] = time_path(step_unfused, 4)
+    if run_fused:
+        res["fused"] = time_path(step_fused, 2)
+    primary = "fused" if run_fused else "unfused"
+    ms_per_step, _, window = res[primary]
     value = world * N / (ms_per_step * 1e-3)
 
     # ---- end to end through the host-buffer entry point
     e2e = None
     if not args.no_e2e:
+        if pg is None:
+            pg = B.PtrList([torch.empty(plan.G, dtype=gdt, device=dev) for _ in range(R)])
+            gathered = torch.empty(plan.G, dtype=odt, device=dev) if odt != torch.float32 else None
         host_g = [torch.empty(A_el, dtype=gdt).pin_memory() for _ in range(R)]
         for k in range(R):
             host_g[k].copy_(g_arena[k])
@@ -370,8 +417,6 @@ def run_ours(args):
             tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
             dist.all_reduce(tt, op=dist.ReduceOp.MAX)
             e2e_ms = float(tt.item())
-        gb = 2 if gdt == torch.bfloat16 else 4
-        wb = 2 if odt == torch.bfloat16 else 4
         e2e = {"value": world * N * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": R * A_el * gb, "d2h_bytes_per_step": A_el * wb,
                "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps,
@@ -383,7 +428,7 @@ def run_ours(args):
             dist.destroy_process_group()
         return
 
-    # ---- roofline of the dominant kernel
+    # ---- per-kernel rates and the roofline of the dominant kernel
     peak, peak_src = FALLBACK_HBM_GBS, "fallback"
     try:
         with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
@@ -393,40 +438,53 @@ def run_ours(args):
     bpp = bytes_per_param(wl)
     n_upd_launch = 3 if wl.opt == "lamb" else 1
     chunks = -(-T // 1024)
-    kernels = [
-        {"kernel": "pack_kernel (gradients)", "launches_per_step": R * chunks,
-         "ms_per_step": phase_ms[0], "bytes_per_step": R * N * bpp["pack"]},
-        {"kernel": "update_kernel (fused reduce+update)" if wl.opt != "lamb" else
-                   "update_kernel phase 1 + lamb_finalize + update_kernel phase 2",
-         "launches_per_step": n_upd_launch, "ms_per_step": phase_ms[1], "bytes_per_step": N * bpp["update"]},
-        {"kernel": "pack_kernel (unpack weights)", "launches_per_step": chunks,
-         "ms_per_step": phase_ms[2], "bytes_per_step": N * bpp["unpack"]},
-    ]
-    for kz in kernels:
-        kz["achieved_gbs"] = kz["bytes_per_step"] / (kz["ms_per_step"] * 1e-3) / 1e9
-        kz["frac"] = kz["achieved_gbs"] / peak
-        kz["share"] = kz["ms_per_step"] / sum(phase_ms)
+    upd_name = ("update_kernel" if wl.opt != "lamb" else "update_kernel phase 1 + lamb_finalize_kernel + update_kernel phase 2")
+
+    def kernel_rows(path):
+        ph = res[path][1]
+        if path == "fused":
+            rows = [{"kernel": upd_name + " (formatting fused in)", "launches_per_step": n_upd_launch,
+                     "ms_per_step": ph[0], "bytes_per_step": N * bpp["fused"]}]
+        else:
+            rows = [{"kernel": "pack_kernel (gradients)", "launches_per_step": R * chunks,
+                     "ms_per_step": ph[0], "bytes_per_step": R * N * bpp["pack"]},
+                    {"kernel": upd_name, "launches_per_step": n_upd_launch, "ms_per_step": ph[1],
+                     "bytes_per_step": N * bpp["update"]},
+                    {"kernel": "pack_kernel (unpack weights)", "launches_per_step": chunks,
+                     "ms_per_step": ph[2], "bytes_per_step": N * bpp["unpack"]}]
+        tot = sum(r_["ms_per_step"] for r_ in rows)
+        for r_ in rows:
+            r_["achieved_gbs"] = r_["bytes_per_step"] / (r_["ms_per_step"] * 1e-3) / 1e9
+            r_["frac"] = r_["achieved_gbs"] / peak
+            r_["share"] = r_["ms_per_step"] / tot
+        return rows
+
+    kernels = kernel_rows(primary)
     dom = max(kernels, key=lambda z: z["ms_per_step"])
-    per_launch_bytes = dom["bytes_per_step"] / dom["launches_per_step"] if "phase 1" not in dom["kernel"] else dom["bytes_per_step"]
+    one_launch = dom["launches_per_step"] if "phase 1" not in dom["kernel"] else 1
     roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["achieved_gbs"], "peak": peak,
                 "peak_source": f"{peak_src} copy bandwidth", "unit": "GB/s", "frac": dom["frac"],
-                "algorithmic_bytes_per_launch": per_launch_bytes,
-                "avg_launch_ms": dom["ms_per_step"] / (dom["launches_per_step"] if "phase 1" not in dom["kernel"] else 1),
-                "traffic": NCU_TRAFFIC_BYTES.get((wl.name, dom["kernel"].split(" ")[0])),
+                "algorithmic_bytes_per_launch": dom["bytes_per_step"] / one_launch,
+                "avg_launch_ms": dom["ms_per_step"] / one_launch,
+                "traffic": NCU_TRAFFIC_BYTES.get((wl.name, primary)),
                 "frac_of_nominal_8TBs": dom["achieved_gbs"] / 8000.0}
-    clocks = sampler.summary(t_host0, t_host1)
+    clocks = sampler.summary(*window)
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
-        "warmup": max(3, args.warmup), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "warmup": W_, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": config_of(wl, args), "roofline": roofline, "kernels": kernels, "clocks": clocks,
+        "config": config_of(wl, args, path=primary), "roofline": roofline, "kernels": kernels, "clocks": clocks,
         "gpu_launches": K * sum(kz["launches_per_step"] for kz in kernels),
-        "update_only": {"value": N / (phase_ms[1] * 1e-3), "unit": UNIT,
-                        "bytes_per_param": bpp["update"], "achieved_gbs": kernels[1]["achieved_gbs"],
-                        "frac_of_measured_peak": kernels[1]["frac"],
-                        "frac_of_nominal_8TBs": kernels[1]["achieved_gbs"] / 8000.0},
     }
+    if "unfused" in res and primary != "unfused":
+        rows = kernel_rows("unfused")
+        line["unfused_path"] = {
+            "step": "ws_pack x R + ws_shard_update(all shards) + ws_unpack as separate kernels",
+            "value": world * N / (res["unfused"][0] * 1e-3), "unit": UNIT, "ms_per_step": res["unfused"][0],
+            "kernels": rows, "gpu_launches": K * sum(kz["launches_per_step"] for kz in rows)}
+    if unfused_skipped:
+        line["unfused_path"] = {"skipped": unfused_skipped}
     if e2e is not None:
         line["e2e"] = e2e
     if world == 1 and not args.no_cpu_baseline:

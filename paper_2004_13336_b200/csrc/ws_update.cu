@@ -279,6 +279,9 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF) ? 2 : WS_TUNE_MINB) 
     constexpr bool READS_G = (OPT != K_LAMB2);
     constexpr bool LOOPK = (NP > RB);   // R may exceed one tree block: loop and compensate
     __shared__ float red[2][kBlock / 32];
+    // fused formatting: this tile's R gradient tensor pointers, fetched once per work item (the
+    // streaming data would push the table's lines out of L1 between passes)
+    __shared__ const void* sgp[(FUSED && READS_G) ? NP : 1];
 
     for (long long item = blockIdx.x; item < P.nitems; item += gridDim.x) {
         const long long rs = item / P.ntiles;              // shard index inside this launch
@@ -308,8 +311,13 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF) ? 2 : WS_TUNE_MINB) 
         const void* const* gt = nullptr;
         char* wt = nullptr;
         if constexpr (FUSED) {
-            if (READS_G) gt = P.gtab + (long long)tl.seg * P.R;
             if (OUT != O_NONE) wt = reinterpret_cast<char*>(P.wtab[tl.seg]);
+            if constexpr (READS_G) {
+                gt = P.gtab + (long long)tl.seg * P.R;
+                __syncthreads();   // the previous item's readers are done with sgp
+                for (int k = threadIdx.x; k < P.R; k += kBlock) sgp[k] = gt[k];
+                __syncthreads();
+            }
         }
         const int nvec = tl.len / VEC;
         float lr_rho = 0.f;
@@ -349,7 +357,7 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF) ? 2 : WS_TUNE_MINB) 
                         for (int u = 0; u < U; ++u)
                             if (have[j] && nv[u] > 0) {
                                 if constexpr (FUSED) {
-                                    const void* gk = gt[k0 + j];
+                                    const void* gk = sgp[k0 + j];
                                     if (nv[u] == VEC) raw[u][j] = load_grad<GBF, VEC>(gk, toff + e0[u]);
                                     else raw[u][j] = load_grad_partial<GBF, VEC>(gk, toff + e0[u], nv[u]);
                                 } else {
