@@ -36,14 +36,14 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
 # captures summarised under profiles/, keyed by (workload, kernel); None = not captured.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {("resnet50", "fused"): 1.2987e9}   # profiles/fused_update_kernel_resnet50_sgdm_R8.md
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50",
                     choices=["tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b"])
