@@ -247,6 +247,30 @@ def config_of(wl, args, extra=None, path="unfused"):
 
 
 # ----------------------------------------------------------------------------
+# multi-rank plumbing (one process per GPU; no data-path collective)
+# ----------------------------------------------------------------------------
+def rank_seed(base_seed: int, rank: int) -> int:
+    """Each rank updates its own, independently seeded tensor set of the same workload."""
+    return base_seed + 1000 * rank
+
+
+def reduce_max(x: float, device) -> float:
+    """Max over ranks of a per-rank time (the job is as slow as its slowest rank)."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(x)
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(n_params_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Whole-job throughput: every rank updates n parameters per step (weak scaling)."""
+    return world * n_params_per_rank / (ms_per_step * 1e-3)
+
+
+# ----------------------------------------------------------------------------
 # GPU arm
 # ----------------------------------------------------------------------------
 def run_ours(args):
@@ -273,7 +297,7 @@ def run_ours(args):
     B.lib()
 
     wl = get_workload(args)
-    wl.seed = wl.seed + 1000 * rank           # every rank owns its own tensor set
+    wl.seed = rank_seed(wl.seed, rank)        # every rank owns its own tensor set
     R, T, N = wl.R, wl.T, wl.N
     plan = B.Plan(wl.shapes, R, args.align, args.tile, device=dev)
     gdt, odt = wl.grad_dtype, wl.out_dtype
@@ -370,10 +394,7 @@ def run_ours(args):
         if flush is not None:   # leave the L2 flush out of the step time
             total_ms = sum(e[0].elapsed_time(e[nev - 1]) for e in evs)
         phase_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / K for i in range(nev - 1)]
-        if world > 1:
-            tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            total_ms = float(tt.item())
+        total_ms = reduce_max(total_ms, dev)
         return total_ms / K, phase_ms, (t0, t1)
 
     sampler = ClockSampler(local)
@@ -386,7 +407,7 @@ def run_ours(args):
         res["fused"] = time_path(step_fused, 2)
     primary = "fused" if run_fused else "unfused"
     ms_per_step, _, window = res[primary]
-    value = world * N / (ms_per_step * 1e-3)
+    value = job_value(N, world, ms_per_step)
 
     # ---- end to end through the host-buffer entry point
     e2e = None
@@ -413,10 +434,7 @@ def run_ours(args):
         e1.record()
         barrier()
         e2e_ms = e0.elapsed_time(e1)
-        if world > 1:
-            tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tt.item())
+        e2e_ms = reduce_max(e2e_ms, dev)
         e2e = {"value": world * N * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                "h2d_bytes_per_step": R * A_el * gb, "d2h_bytes_per_step": A_el * wb,
                "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps,

@@ -34,8 +34,11 @@ def _gather(t, idx_dev):
     return to_np(t[idx_dev])
 
 
-def _run_sampled(wl, samples_per_tensor=1500):
-    """Elementwise optimizers: full-size GPU step, oracle on sampled elements."""
+def _run_sampled(wl, samples_per_tensor=1500, path="unfused"):
+    """Elementwise optimizers: full-size GPU step, oracle on sampled elements.
+    path "unfused": ws_pack of every gradient list, ws_shard_update, ws_unpack;
+    path "fused":   ws_fused_update straight from the gradient lists into weight tensors
+                    (the configuration the benchmark reports)."""
     torch.cuda.empty_cache()
     rng = np.random.default_rng(wl.seed)
     plan = B.Plan(wl.shapes, wl.R, A)
@@ -50,38 +53,52 @@ def _run_sampled(wl, samples_per_tensor=1500):
     for src, dst in ((w, pw), (m, pm), (v, pv)):
         B.ws_pack(plan, src, dst)
     del m, v
-    pg, sg = [], []
+    pg, sg, glists = [], [], []
     for k in range(wl.R):
         gk = W.make_grads_one(wl, k, DEV)
         sg.append([_gather(x, i) for x, i in zip(gk, idx_dev)])
-        b = torch.empty(plan.G, dtype=wl.grad_dtype, device=DEV)
-        B.ws_pack(plan, gk, b)
-        pg.append(b)
+        if path == "fused":
+            glists.append(gk)
+        else:
+            b = torch.empty(plan.G, dtype=wl.grad_dtype, device=DEV)
+            B.ws_pack(plan, gk, b)
+            pg.append(b)
         del gk
-    gathered = torch.empty(plan.G, dtype=wl.out_dtype, device=DEV) if wl.out_dtype != torch.float32 else None
-    B.ws_shard_update(plan, -1, pg, pw, pm, pv if wl.opt != "sgdm" else None, B.make_hyper(wl.opt, wl.hyper), gathered)
-    del pg
+    hy = B.make_hyper(wl.opt, wl.hyper)
+    gathered = None
+    wout = [torch.zeros(n, dtype=wl.out_dtype, device=DEV) for n in wl.numels]
+    if path == "fused":
+        B.ws_fused_update(plan, -1, B.TensorTable(plan, glists), pw, pm, pv if wl.opt != "sgdm" else None, hy,
+                          B.TensorTable(plan, [wout]))
+        del glists
+    else:
+        gathered = torch.empty(plan.G, dtype=wl.out_dtype, device=DEV) if wl.out_dtype != torch.float32 else None
+        B.ws_shard_update(plan, -1, pg, pw, pm, pv if wl.opt != "sgdm" else None, hy, gathered)
+        B.ws_unpack(plan, gathered if gathered is not None else pw, wout)
+        del pg
     # oracle on the sampled elements (each tensor's sample is a small pseudo-tensor)
     hs = O.make_hyper(wl.opt, wl.hyper)
     for t in range(wl.T):
         O.update_tensor(hs, [sg[k][t] for k in range(wl.R)], sw[t], sm[t], sv[t] if wl.opt != "sgdm" else None)
     # GPU outputs back in tensor form
-    worst = {"w": 0.0, "m": 0.0, "v": 0.0, "bf16": 0.0}
+    worst = {"w": 0.0, "m": 0.0, "v": 0.0, "out": 0.0}
     for name, buf, ref in (("w", pw, sw), ("m", pm, sm), ("v", pv, sv)):
         if name == "v" and wl.opt == "sgdm":
             continue
         B.ws_unpack(plan, buf, w)           # reuse the weight tensors as the unpack target
         for t in range(wl.T):
             worst[name] = max(worst[name], err(_gather(w[t], idx_dev[t]), ref[t]))
-    if gathered is not None:
-        assert torch.equal(gathered, pw.to(torch.bfloat16))     # RNE of the fp32 master, pads +0
-        outs = [torch.empty(n, dtype=torch.bfloat16, device=DEV) for n in wl.numels]
-        B.ws_unpack(plan, gathered, outs)
-        for t in range(wl.T):
-            worst["bf16"] = max(worst["bf16"], err(bf16_to_f64(_gather(outs[t], idx_dev[t])), sw[t]))
-    print(f"{wl.name} R={wl.R}: max err w {worst['w']:.2e} m {worst['m']:.2e} v {worst['v']:.2e} bf16 {worst['bf16']:.2e}")
+        if name == "w":                     # the emitted weights: fp32 copy of, or RNE bf16 of, the fp32 master
+            for t in range(wl.T):
+                assert torch.equal(wout[t], w[t].to(wl.out_dtype)), f"tensor {t}"
+    bf = wl.out_dtype == torch.bfloat16
+    for t in range(wl.T):
+        got = _gather(wout[t], idx_dev[t])
+        worst["out"] = max(worst["out"], err(bf16_to_f64(got) if bf else got, sw[t]))
+    print(f"{wl.name} R={wl.R} {path}: max err w {worst['w']:.2e} m {worst['m']:.2e} v {worst['v']:.2e} "
+          f"out {worst['out']:.2e}")
     assert worst["w"] <= TOL_FP32 and worst["m"] <= TOL_FP32 and worst["v"] <= TOL_FP32
-    assert worst["bf16"] <= TOL_BF16
+    assert worst["out"] <= (TOL_BF16 if bf else TOL_FP32)
     return worst
 
 
@@ -118,21 +135,31 @@ def test_resnet50_full_model_every_element():
     assert (to_np(pw).view(np.uint32)[~valid] == 0).all() and (to_np(pm).view(np.uint32)[~valid] == 0).all()
 
 
+@pytest.mark.parametrize("path", ["unfused", "fused"])
 @pytest.mark.parametrize("R", [1, 2, 8, 32])
-def test_transformer_adam_sampled(R):
-    _run_sampled(W.transformer(R))
+def test_transformer_adam_sampled(R, path):
+    _run_sampled(W.transformer(R), path=path)
 
 
-def test_transformer_adam_R128_sampled():
-    """108 GB of packed gradients: the largest replica count that fits one GPU."""
+@pytest.mark.parametrize("path", ["unfused", "fused"])
+def test_transformer_adam_R128_sampled(path):
+    """108 GB of gradients: the largest replica count that fits one GPU."""
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
     free, _ = torch.cuda.mem_get_info()
     if free < 130e9:
         pytest.skip("needs ~120 GB of free device memory")
-    _run_sampled(W.transformer(128), samples_per_tensor=300)
+    _run_sampled(W.transformer(128), samples_per_tensor=300, path=path)
 
 
-def test_decoder_1p5b_bf16_grads_bf16_gathered_sampled():
-    _run_sampled(W.decoder_1p5b(), samples_per_tensor=500)
+@pytest.mark.parametrize("path", ["unfused", "fused"])
+def test_decoder_1p5b_bf16_grads_bf16_gathered_sampled(path):
+    _run_sampled(W.decoder_1p5b(), samples_per_tensor=500, path=path)
+
+
+def test_resnet50_fused_path_sampled():
+    _run_sampled(W.resnet50(), samples_per_tensor=4000, path="fused")
 
 
 def test_transformer_R1024_window_of_shards():
@@ -218,3 +245,38 @@ def test_bert_large_lamb_whole_tensors():
         worst_mv = max(worst_mv, err(outs["m"][t], rm), err(outs["v"][t], rv))
     print(f"bert_large LAMB: err w {worst_w:.2e} m/v {worst_mv:.2e} rho {worst_rho:.2e}")
     assert worst_rho <= TOL_LAMB and worst_w <= TOL_LAMB and worst_mv <= TOL_FP32
+
+
+def test_bert_large_lamb_fused_equals_unfused():
+    """The benchmark's configuration for config 4: ws_fused_update (three launches) from the 16
+    gradient lists.  Same arithmetic and same tiling as the packed path, so every output is
+    bit-identical to ws_pack + ws_shard_update + ws_unpack (which the test above ties to the oracle)."""
+    wl = W.bert_large()
+    torch.cuda.empty_cache()
+    plan = B.Plan(wl.shapes, wl.R, A)
+    hy = B.make_hyper(wl.opt, wl.hyper)
+    w, m, v = W.make_state(wl, DEV)
+    pw = torch.empty(plan.G, device=DEV)
+    pm, pv = torch.empty_like(pw), torch.empty_like(pw)
+    for src, dst in ((w, pw), (m, pm), (v, pv)):
+        B.ws_pack(plan, src, dst)
+    fw, fm, fv = pw.clone(), pm.clone(), pv.clone()
+    del m, v
+    glists, pg = [], []
+    for k in range(wl.R):
+        gk = W.make_grads_one(wl, k, DEV)
+        b = torch.empty(plan.G, device=DEV)
+        B.ws_pack(plan, gk, b)
+        pg.append(b)
+        glists.append(gk)
+    ws = torch.empty(plan.workspace_bytes("lamb"), dtype=torch.uint8, device=DEV)
+    ws2 = torch.empty_like(ws)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv, hy, None, ws)
+    del pg
+    ref = [torch.empty_like(x) for x in w]
+    B.ws_unpack(plan, pw, ref)
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, glists), fw, fm, fv, hy, B.TensorTable(plan, [w]), ws2)
+    assert torch.equal(B.lamb_ratios(plan, ws), B.lamb_ratios(plan, ws2))
+    assert torch.equal(fw, pw) and torch.equal(fm, pm) and torch.equal(fv, pv)
+    for a, b in zip(w, ref):
+        assert torch.equal(a, b)
