@@ -76,8 +76,9 @@ typedef struct ws_plan ws_plan;
  *   R           shard count = replica count, >= 1
  *   align_elems A: power of two >= 8, every piece is a multiple of A elements
  *   tile_elems  work-tile length in elements used by the kernels; 0 = default
- *               (2048, 4096, 8192 or 16384, the largest that leaves at least
- *               20000 tiles over all shards); otherwise a multiple of 1024
+ *               (1024 ... 16384: the largest power of two that leaves at
+ *               least 20000 tiles over all shards and 600 per shard);
+ *               otherwise a multiple of 1024
  *   out         receives a new plan; release with ws_plan_destroy
  * Errors: WS_ERR_INVALID_ARG for null/empty input, bad R, A or tile size. */
 ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int32_t R, int32_t align_elems,

@@ -58,8 +58,13 @@ extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int3
             for (int i = 0; i < descs[t].ndim && i < WS_MAX_DIMS; ++i) n *= (descs[t].dims[i] > 0 ? descs[t].dims[i] : 1);
             total += n;
         }
-        tile_elems = 2048;
-        while (tile_elems < 16384 && total / (2 * tile_elems) >= 20000) tile_elems *= 2;
+        // ... and >= 600 items for a single-shard launch (many replicas make tiny shards; a CTA
+        // then walks all R gradient slices for its tile, so the grid needs the parallelism).
+        tile_elems = 1024;
+        if (total / R / 2048 >= 600) tile_elems = 2048;
+        while (tile_elems >= 2048 && tile_elems < 16384 && total / (2 * tile_elems) >= 20000 &&
+               total / R / (2 * tile_elems) >= 600)
+            tile_elems *= 2;
     }
     if (tile_elems < 1024 || tile_elems % 1024 != 0 || tile_elems > (1 << 20)) return WS_ERR_INVALID_ARG;
 

@@ -67,9 +67,9 @@ def test_planner_on_model_shaped_workloads():
             assert [s.shard_off for s in segs] == list(ref.off)
             if tile:    # tiles cover each piece exactly once, in order
                 assert plan.ntiles == sum(-(-int(p) // tile) for p in ref.piece)
-            else:       # default tile: between 2048 and 16384 elements
+            else:       # default tile: between 1024 and 16384 elements
                 lo = sum(-(-int(p) // 16384) for p in ref.piece)
-                hi = sum(-(-int(p) // 2048) for p in ref.piece)
+                hi = sum(-(-int(p) // 1024) for p in ref.piece)
                 assert lo <= plan.ntiles <= hi
 
 
