@@ -76,7 +76,7 @@ typedef struct ws_plan ws_plan;
  *   R           shard count = replica count, >= 1
  *   align_elems A: power of two >= 8, every piece is a multiple of A elements
  *   tile_elems  work-tile length in elements used by the kernels; 0 = default
- *               (1024 ... 16384: the largest power of two that leaves at
+ *               (1024 ... 8192: the largest power of two that leaves at
  *               least 20000 tiles over all shards and 600 per shard);
  *               otherwise a multiple of 1024
  *   out         receives a new plan; release with ws_plan_destroy

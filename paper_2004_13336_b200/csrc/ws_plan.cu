@@ -62,7 +62,7 @@ extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int3
         // then walks all R gradient slices for its tile, so the grid needs the parallelism).
         tile_elems = 1024;
         if (total / R / 2048 >= 600) tile_elems = 2048;
-        while (tile_elems >= 2048 && tile_elems < 16384 && total / (2 * tile_elems) >= 20000 &&
+        while (tile_elems >= 2048 && tile_elems < 8192 && total / (2 * tile_elems) >= 20000 &&
                total / R / (2 * tile_elems) >= 600)
             tile_elems *= 2;
     }

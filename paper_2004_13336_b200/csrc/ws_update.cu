@@ -24,7 +24,14 @@
 
 #ifndef WS_TUNE_MINB
 #define WS_TUNE_MINB 3   // resident CTAs per SM the compiler must allow for (register budget);
-                         // the bf16-gradient wide kernel is given 2 (measured faster with more registers)
+                         // the bf16-gradient wide kernel on packed buffers is given WS_TUNE_MINB8 = 2
+                         // (measured faster with more registers; the fused variant is faster with 3)
+#endif
+#ifndef WS_TUNE_MINB8
+#define WS_TUNE_MINB8 2
+#endif
+#ifndef WS_TUNE_U8
+#define WS_TUNE_U8 1
 #endif
 #ifndef WS_TUNE_U4
 #define WS_TUNE_U4 1     // 128-bit accesses per thread per pass
@@ -274,7 +281,7 @@ __device__ __forceinline__ float block_sum(float x, float* smem /* kBlock/32 flo
 // One CTA handles one (shard, tile) work item; the grid is the item count, so the
 // hardware CTA scheduler walks the buffers front to back.
 template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED>
-__global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF) ? 2 : WS_TUNE_MINB) update_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp) {
+__global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_MINB8 : WS_TUNE_MINB) update_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp) {
     constexpr bool HAS_V = (OPT != K_SGDM);
     constexpr bool READS_G = (OPT != K_LAMB2);
     constexpr bool LOOPK = (NP > RB);   // R may exceed one tree block: loop and compensate
@@ -498,7 +505,7 @@ ws_status launch_r(const UpdParams& P, const void* const* gptrs, bool wide_ok, c
             return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 2, 2, FUSED>(P, gptrs, st);
         }
         if (P.R <= 4) {
-            if constexpr (GBF) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 4, 4, FUSED>(P, gptrs, st);
+            if constexpr (GBF) if (wide_ok) return launch<OPT, GBF, OUT, 8, WS_TUNE_U8, 4, 4, FUSED>(P, gptrs, st);
             return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 4, 4, FUSED>(P, gptrs, st);
         }
         if (P.R <= 8) {
