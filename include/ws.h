@@ -55,7 +55,7 @@ typedef enum { WS_SGDM = 0, WS_ADAM = 1, WS_LAMB = 2 } ws_opt;
 #define WS_MAX_DIMS 8
 typedef struct {
     int32_t ndim;               /* 0..WS_MAX_DIMS; ndim == 0 is a scalar (1 element) */
-    int64_t dims[WS_MAX_DIMS];  /* every dim >= 1                                      */
+    int64_t dims[WS_MAX_DIMS];  /* every dim >= 0; a zero dim makes an empty tensor   */
     uint32_t flags;             /* reserved, pass 0                                    */
 } ws_tensor_desc;
 

@@ -81,6 +81,7 @@ ws_status run(const ws_plan* p, void* const* tensor_ptrs, ws_dtype dtype, void* 
     if (!p->d_tiles) return WS_ERR_NOT_UPLOADED;
     if (!ws_aligned16(flat)) return WS_ERR_ALIGNMENT;
     for (int t = 0; t < p->T; ++t) {
+        if (p->segs[t].numel == 0) continue;   // empty tensor: never dereferenced, may be null
         if (!tensor_ptrs[t]) return WS_ERR_INVALID_ARG;
         if (!ws_aligned16(tensor_ptrs[t])) return WS_ERR_ALIGNMENT;
     }

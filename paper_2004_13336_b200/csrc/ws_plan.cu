@@ -55,7 +55,7 @@ extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int3
         long long total = 0;
         for (int t = 0; t < T; ++t) {
             long long n = 1;
-            for (int i = 0; i < descs[t].ndim && i < WS_MAX_DIMS; ++i) n *= (descs[t].dims[i] > 0 ? descs[t].dims[i] : 1);
+            for (int i = 0; i < descs[t].ndim && i < WS_MAX_DIMS; ++i) n *= (descs[t].dims[i] > 0 ? descs[t].dims[i] : 0);
             total += n;
         }
         // ... and >= 600 items for a single-shard launch (many replicas make tiny shards; a CTA
@@ -83,8 +83,8 @@ extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int3
             if (d.ndim < 0 || d.ndim > WS_MAX_DIMS) { delete p; return WS_ERR_INVALID_ARG; }
             long long n = 1;
             for (int i = 0; i < d.ndim; ++i) {
-                if (d.dims[i] < 1 || n > (1LL << 46) / d.dims[i]) { delete p; return WS_ERR_INVALID_ARG; }
-                n *= d.dims[i];
+                if (d.dims[i] < 0 || (d.dims[i] > 0 && n > (1LL << 46) / d.dims[i])) { delete p; return WS_ERR_INVALID_ARG; }
+                n *= d.dims[i];   // a zero dimension makes an empty tensor: no piece, no tiles
             }
             long long per = (n + R - 1) / R;
             long long piece = (per + align_elems - 1) / align_elems * align_elems;

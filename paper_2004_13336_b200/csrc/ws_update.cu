@@ -7,16 +7,25 @@
 // fp32 result, Section 4.2).  Intermediates live in registers only (the
 // "fusion" of Section 2.1); every operand crosses HBM exactly once.
 //
-// Work item = (shard r, tile); a thread owns quads of 4 consecutive elements
-// and moves them as 16-byte vectors.  Pads are recognised by location
-// (element index within the tile vs. the tile's valid length for shard r), so
-// gradient pads are never read into a result and output pads are +0
-// (Section 4.1, "Non-elementwise operators": mask with the identity).
+// Work item = (shard r, tile), one CTA each; a thread owns runs of 4 or 8
+// consecutive elements and moves them as 128- or 256-bit vectors.  Pads are
+// recognised by location (element index within the tile vs. the tile's valid
+// length for shard r), so gradient pads are never read into a result and
+// output pads are +0 (Section 4.1, "Non-elementwise operators": mask with the
+// identity).
 //
-// The R-way sum is formed as tree sums over blocks of RB gradients combined by
-// a compensated (Kahan) accumulation, never as one sequential fp32 chain: the
-// loads of a block are independent (memory-level parallelism) and the rounding
-// error stays near one ulp for R up to 1024.
+// The R-way sum is formed as tree sums over blocks of RB gradients; when R
+// exceeds one block the blocks are combined by a compensated (Kahan)
+// accumulation, never as one sequential fp32 chain: the loads of a block are
+// independent (memory-level parallelism) and the rounding error stays near one
+// ulp for R up to 1024.
+//
+// With FUSED the formatting steps are part of the same kernel (Section 5.1):
+// gradients come straight from the replicas' tensor lists and the updated
+// weights go straight to the weight tensors.
+//
+// The WS_TUNE_* macros are build-time tuning constants; their defaults are the
+// values measured best on a B200.
 #include <cuda_bf16.h>
 #include <math.h>
 
@@ -294,21 +303,7 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_
         const long long rs = item / P.ntiles;              // shard index inside this launch
         const long long ti = item - rs * P.ntiles;
         const long long r = P.r0 + rs;
-#ifdef WS_TUNE_NODESC   /* development experiment: single-tensor plans only */
-        WsTile tl;
-        tl.pos = ti * WS_TUNE_NODESC; tl.poff = tl.pos; tl.piece = P.S; tl.vt = (long long)P.R * P.S - tl.pos;
-        tl.len = (int)((P.S - tl.pos) < WS_TUNE_NODESC ? (P.S - tl.pos) : WS_TUNE_NODESC); tl.seg = 0;
-#else
         const WsTile tl = P.tiles[ti];
-#endif
-        {   // pull the next work item's descriptor towards this SM while this one is processed
-            const long long nitem = item + gridDim.x;
-            if (nitem < P.nitems) {
-                const WsTile* nt = P.tiles + (nitem % P.ntiles);
-                asm volatile("prefetch.global.L1 [%0];" ::"l"(nt));
-                asm volatile("prefetch.global.L1 [%0];" ::"l"(reinterpret_cast<const char*>(nt) + 32));
-            }
-        }
         long long nvl = tl.vt - r * tl.piece;              // valid elements in this tile for shard r
         const int nvalid = nvl < 0 ? 0 : (nvl > tl.len ? tl.len : (int)nvl);
         const long long gbase = rs * P.g_stride + tl.pos;  // into each gradient buffer
@@ -477,9 +472,6 @@ __global__ void __launch_bounds__(kBlock) lamb_finalize_kernel(const WsSegTiles*
 }
 
 // -------------------------------------------------------------- dispatch ---
-#ifndef WS_TUNE_GRID
-#define WS_TUNE_GRID 0
-#endif
 template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED>
 ws_status launch(const UpdParams& P, const void* const* gptrs, cudaStream_t st) {
     GradPtrs<NP> gp;
@@ -731,10 +723,11 @@ extern "C" ws_status ws_tensor_table_upload(const ws_plan* plan, const void* con
     for (int k = 0; k < nsets; ++k)
         for (int t = 0; t < T; ++t) {
             const void* q = ptrs[(size_t)k * T + t];
+            host[(size_t)t * nsets + k] = q;   // device layout [T][nsets]: a tile finds its pointers side by side
+            if (plan->segs[t].numel == 0) continue;   // empty tensor: never dereferenced, may be null
             if (!q) return WS_ERR_INVALID_ARG;
             if (!ws_aligned16(q)) return WS_ERR_ALIGNMENT;
             while (min_align > 16 && (reinterpret_cast<uintptr_t>(q) & (uintptr_t)(min_align - 1)) != 0) min_align >>= 1;
-            host[(size_t)t * nsets + k] = q;   // device layout [T][nsets]: a tile finds its pointers side by side
         }
     cudaError_t e = cudaMemcpyAsync(dev_buf, host.data(), host.size() * sizeof(void*), cudaMemcpyHostToDevice,
                                     (cudaStream_t)stream);

@@ -439,3 +439,64 @@ def test_fused_update_matches_oracle_unsharded():
                       B.TensorTable(plan, [outs]))
     for a, b in zip(outs, ow):
         assert err(to_np(a), b) <= TOL_FP32
+
+
+@pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb"])
+def test_empty_tensors_in_the_list(opt):
+    shapes = [(64, 33), (0,), (5, 0, 2), (4099,), (0, 7)]
+    R = 3
+    wl, w, m, v, g = _model(shapes, R, seed=9)
+    plan = B.Plan(shapes, R, 32)
+    oplan = O.Plan(wl.numels, R, 32)
+    assert plan.S == oplan.S
+    h = _hyper(opt)
+    ow, om, ov, orho = _oracle_unsharded(opt, h, w, m, v, g)
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    fw, fm, fv = pw.clone(), pm.clone(), pv.clone()
+    ws = torch.zeros(max(16, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv if opt != "sgdm" else None, B.make_hyper(opt, h), None, ws)
+    tol = TOL_LAMB if opt == "lamb" else TOL_FP32
+    _compare_state(oplan, opt, [pw, pm, pv][:3 if opt != "sgdm" else 2], [ow, om, ov][:3 if opt != "sgdm" else 2], tol)
+    if opt == "lamb":
+        rho = B.lamb_ratios(plan, ws).cpu().numpy()
+        assert rho[1] == 1.0 and rho[2] == 1.0 and rho[4] == 1.0
+    outs = [torch.full_like(x, 3.0) for x in w]
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), fw, fm, fv if opt != "sgdm" else None,
+                      B.make_hyper(opt, h), B.TensorTable(plan, [outs]), ws)
+    assert torch.equal(fw, pw) and torch.equal(fm, pm)
+    back = [torch.empty_like(x) for x in w]
+    B.ws_unpack(plan, pw, back)
+    for a, b in zip(outs, back):
+        assert torch.equal(a, b)
+
+
+def test_step_can_be_captured_in_a_cuda_graph():
+    # calls take pointers and a stream, allocate nothing and never synchronise, so a whole step
+    # (here: the fused update, and pack + update + unpack) can be captured once and replayed
+    wl, w, m, v, g = _model(SHAPES, 4, seed=4)
+    plan = B.Plan(SHAPES, 4, 32)
+    hy = B.make_hyper("adam", _hyper("adam"))
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    ew, em, ev = pw.clone(), pm.clone(), pv.clone()
+    outs = [torch.zeros_like(x) for x in w]
+    gt, wt = B.TensorTable(plan, g), B.TensorTable(plan, [outs])
+    gl = B.PtrList(pg)
+    B.ws_fused_update(plan, -1, gt, ew, em, ev, hy, wt)        # eager reference: two steps
+    B.ws_fused_update(plan, -1, gt, ew, em, ev, hy, wt)
+    expect = [o.clone() for o in outs]
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            for gk, b in zip(g, pg):
+                B.ws_pack(plan, gk, b)
+            B.ws_shard_update(plan, -1, gl, pw, pm, pv, hy)
+            B.ws_unpack(plan, pw, outs)
+    torch.cuda.current_stream().wait_stream(side)
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(pw, ew) and torch.equal(pm, em) and torch.equal(pv, ev)
+    for a, b in zip(outs, expect):
+        assert torch.equal(a, b)

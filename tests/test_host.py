@@ -94,9 +94,21 @@ def test_plan_create_rejects_bad_arguments():
     assert L.ws_plan_create(d, 0, 4, 32, 0, C.byref(h)) == 1          # empty list
     assert L.ws_plan_create(d, 1, 4, 32, 1000, C.byref(h)) == 1       # tile not a multiple of 1024
     assert L.ws_plan_create(None, 1, 4, 32, 0, C.byref(h)) == 1
-    d[0].dims[0] = 0
-    assert L.ws_plan_create(d, 1, 4, 32, 0, C.byref(h)) == 1          # empty dimension
+    d[0].dims[0] = -3
+    assert L.ws_plan_create(d, 1, 4, 32, 0, C.byref(h)) == 1          # negative dimension
     assert not h.value
+
+
+def test_empty_tensors_take_no_room():
+    # a zero dimension makes an empty tensor: no piece, no tiles, neighbours unaffected
+    shapes = [(5, 7), (0,), (3, 0, 4), (100,)]
+    plan = B.Plan(shapes, 4, 8, upload=False)
+    ref = O.Plan([35, 0, 0, 100], 4, 8)
+    assert (plan.S, plan.N) == (ref.S, ref.N) == (16 + 32, 135)
+    segs = plan.segments()
+    assert [s.piece for s in segs] == [16, 0, 0, 32] == list(ref.piece)
+    assert [s.shard_off for s in segs] == [0, 16, 16, 16] == list(ref.off)
+    assert plan.arena_offsets() == [0, 40, 40, 40] and plan.arena_elems == 144
 
 
 def test_calls_fail_cleanly_before_upload():

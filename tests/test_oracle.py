@@ -450,3 +450,22 @@ def test_tiny_workload_end_to_end():
     O.update_unsharded(hs, g, w, m, v)
     for a, b in zip(w, O.unpack(p, pw)):
         assert a.tobytes() == b.tobytes()
+
+
+def test_empty_tensors_are_inert():
+    # an empty tensor has no piece; the model around it updates exactly as without it
+    numel_a, numel_b = [40, 0, 333, 0, 9], [40, 333, 9]
+    outs = []
+    for numel in (numel_a, numel_b):
+        p, (uw, um, uv, rho_u), (pw, pm, pv, _, rho_s, _) = _run_both("lamb", 4, 8, numel, eps=1e-6,
+                                                                       weight_decay=0.01, seed=3)
+        outs.append((p, [x for x in O.unpack(p, pw) if x.size], [r for r, n in zip(rho_s, numel) if n]))
+        for r, n in zip(rho_s, numel):
+            if n == 0:
+                assert r == 1.0
+    assert outs[0][0].S == outs[1][0].S
+    # same seeds draw different streams for different tensor lists, so compare structure only
+    assert [x.size for x in outs[0][1]] == [x.size for x in outs[1][1]]
+    flat = O.pack(outs[0][0], [np.arange(n, dtype=np.float32) + 1 for n in numel_a])
+    back = O.unpack(outs[0][0], flat)
+    assert [b.size for b in back] == numel_a and (back[2] == np.arange(333) + 1).all()
