@@ -128,10 +128,16 @@ ws_status ws_unpack(const ws_plan* plan, const void* flat, ws_dtype dtype,
  *                 (what a reduce-scatter receive buffer holds); only valid with
  *                 a single shard r >= 0.
  * Gradient pads may hold anything: they are masked by location, never read
- * into the result (Section 4.1, "Non-elementwise operators"). */
+ * into the result (Section 4.1, "Non-elementwise operators").
+ * The number of gradient copies is normally the plan's shard count, but any
+ * count from 1 to 1024 is accepted: with partial sharding (Section 5.2) the
+ * replicas form N groups that each shard the update M ways, so a plan with M
+ * shards is fed N*M copies - the per-group reduce-scatter followed by the
+ * cross-group all-reduce is the sum of all N*M slices of shard j.  The same
+ * holds for the number of sets in ws_fused_update's gradient table. */
 typedef struct {
     const void* const* ptrs; /* host array of R device pointers */
-    int32_t R;               /* must equal the plan's R unless slice_mode == 1 */
+    int32_t R;               /* number of gradient copies, 1..1024 */
     ws_dtype dtype;          /* WS_F32 or WS_BF16 */
     int32_t slice_mode;
 } ws_grads;

@@ -223,13 +223,16 @@ void wso_update_tensor(const wso_hyper *h, int64_t n, int32_t R, const void *con
  *   locations, combined over shards in ascending r (the scalar all-reduce),
  *   then the step; write w' into slot r of the gathered layout (fp32, or
  *   bf16 rounded from the fp32 master).
- * gpacked[k]: replica k's packed gradients, R*S elements, pads arbitrary.
+ * gpacked[k]: gradient copy k, packed, R*S elements, pads arbitrary; there are
+ *   K copies.  K == R in the basic scheme; with partial sharding (Section 5.2:
+ *   groups of replicas each shard R ways, then an all-reduce across groups adds
+ *   the groups' partial results) K = groups * R and shard r sums all K slices.
  * w, m, v: [R][S] fp32 shard-major, updated in place, pads written +0.
  * gathered: [R][S] of out_dtype, or NULL.  rho: T doubles or NULL.
  * partials: [R][T][2] doubles (a, b) or NULL. */
 void wso_sharded_update(const wso_hyper *h, int32_t T, const int64_t *numel,
                         const int64_t *piece, const int64_t *off, int64_t S, int32_t R,
-                        const void *const *gpacked, int32_t g_dtype, float *w, float *m,
+                        int32_t K, const void *const *gpacked, int32_t g_dtype, float *w, float *m,
                         float *v, void *gathered, int32_t out_dtype, double *rho,
                         double *partials) {
     bias_corr b = bias_of(h);
@@ -252,7 +255,7 @@ void wso_sharded_update(const wso_hyper *h, int32_t T, const int64_t *numel,
                     continue;
                 }
                 double g = 0.0;
-                for (int32_t k = 0; k < R; ++k) g += load_grad(gpacked[k], g_dtype, j);
+                for (int32_t k = 0; k < K; ++k) g += load_grad(gpacked[k], g_dtype, j);
                 g *= h->grad_scale;
                 double wd = (double)w[j], md = (double)m[j];
                 if (h->opt == WSO_SGDM) {
@@ -313,14 +316,14 @@ void wso_sharded_update(const wso_hyper *h, int32_t T, const int64_t *numel,
  * grad_scale * sum_k G_k[r*S + j] over valid locations, 0 on pads; rounded
  * once to fp32. */
 void wso_shard_reduce(int32_t T, const int64_t *numel, const int64_t *piece, const int64_t *off,
-                      int64_t S, int32_t R, int32_t r, const void *const *gpacked,
+                      int64_t S, int32_t K, int32_t r, const void *const *gpacked,
                       int32_t g_dtype, double grad_scale, float *out) {
     for (int32_t t = 0; t < T; ++t)
         for (int64_t q = 0; q < piece[t]; ++q) {
             int64_t loc = (int64_t)r * piece[t] + q;
             double g = 0.0;
             if (loc < numel[t]) {
-                for (int32_t k = 0; k < R; ++k)
+                for (int32_t k = 0; k < K; ++k)
                     g += load_grad(gpacked[k], g_dtype, (int64_t)r * S + off[t] + q);
                 g *= grad_scale;
             }

@@ -70,7 +70,7 @@ def lib():
                                         C.POINTER(C.c_double)]
         L.wso_sharded_update.restype = None
         L.wso_sharded_update.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p,
-                                         C.c_int64, C.c_int32, vpp, C.c_int32, C.c_void_p,
+                                         C.c_int64, C.c_int32, C.c_int32, vpp, C.c_int32, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                          C.POINTER(C.c_double), C.POINTER(C.c_double)]
         L.wso_shard_reduce.restype = None
@@ -167,7 +167,7 @@ def sharded_update(h: Hyper, plan: Plan, gpacked: Sequence[np.ndarray], w: np.nd
         gathered = np.empty(plan.G, dtype=np.uint16 if out_dtype == BF16 else np.float32)
     lib().wso_sharded_update(
         C.byref(h), plan.T, _p(plan.numel), _p(plan.piece), _p(plan.off), plan.S, plan.R,
-        _ptrs(gpacked), _dtype_code(gpacked[0]), w.ctypes.data, m.ctypes.data,
+        len(gpacked), _ptrs(gpacked), _dtype_code(gpacked[0]), w.ctypes.data, m.ctypes.data,
         v.ctypes.data if v is not None else None,
         gathered.ctypes.data if gathered is not None else None,
         out_dtype if out_dtype is not None else F32,
@@ -179,7 +179,7 @@ def sharded_update(h: Hyper, plan: Plan, gpacked: Sequence[np.ndarray], w: np.nd
 def shard_reduce(plan: Plan, r: int, gpacked: Sequence[np.ndarray], grad_scale: float = 1.0):
     out = np.empty(plan.S, dtype=np.float32)
     lib().wso_shard_reduce(plan.T, _p(plan.numel), _p(plan.piece), _p(plan.off), plan.S,
-                           plan.R, r, _ptrs(gpacked), _dtype_code(gpacked[0]),
+                           len(gpacked), r, _ptrs(gpacked), _dtype_code(gpacked[0]),
                            float(grad_scale), out.ctypes.data)
     return out
 

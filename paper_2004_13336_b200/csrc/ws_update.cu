@@ -583,7 +583,8 @@ ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state
         if (!g || !g->ptrs || g->R < 1) return WS_ERR_INVALID_ARG;
         if (g->dtype != WS_F32 && g->dtype != WS_BF16) return WS_ERR_DTYPE;
         if (g->slice_mode != 0 && g->slice_mode != 1) return WS_ERR_INVALID_ARG;
-        if (g->slice_mode == 0 && g->R != p->R) return WS_ERR_INVALID_ARG;
+        // g->R need not equal the plan's shard count: with partial sharding (Section 5.2) the
+        // replicas form groups that each shard M ways, and shard j sums all groups' copies
         if (g->slice_mode == 1 && r < 0) return WS_ERR_INVALID_ARG;
         if (g->R > 1024) return WS_ERR_TOO_LARGE;
         for (int k = 0; k < g->R; ++k) {
@@ -779,7 +780,7 @@ extern "C" ws_status ws_fused_update(const ws_plan* plan, int32_t r, const ws_te
                                      size_t workspace_bytes, void* stream) {
     if (!plan || !grads || !weights || !hyper || !state) return WS_ERR_INVALID_ARG;
     if (!grads->dev || !weights->dev) return WS_ERR_INVALID_ARG;
-    if (grads->T != plan->T || weights->T != plan->T || grads->nsets != plan->R || weights->nsets != 1)
+    if (grads->T != plan->T || weights->T != plan->T || grads->nsets < 1 || weights->nsets != 1)
         return WS_ERR_INVALID_ARG;
     if ((grads->dtype != WS_F32 && grads->dtype != WS_BF16) || (weights->dtype != WS_F32 && weights->dtype != WS_BF16))
         return WS_ERR_DTYPE;

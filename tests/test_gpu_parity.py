@@ -500,3 +500,26 @@ def test_step_can_be_captured_in_a_cuda_graph():
     assert torch.equal(pw, ew) and torch.equal(pm, em) and torch.equal(pv, ev)
     for a, b in zip(outs, expect):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb"])
+@pytest.mark.parametrize("groups,M", [(2, 4), (5, 2), (3, 1)])
+def test_partial_sharding_more_gradient_copies_than_shards(opt, groups, M):
+    # Section 5.2: groups of replicas shard M ways each; shard j sums all groups*M copies
+    K = groups * M
+    wl, w, m, v, g = _model(SHAPES, K, seed=K)
+    plan = B.Plan(SHAPES, M, 32)
+    oplan = O.Plan(wl.numels, M, 32)
+    h = _hyper(opt)
+    ow, om, ov, _ = _oracle_unsharded(opt, h, w, m, v, g)          # plain definition over all K copies
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    assert len(pg) == K and plan.R == M
+    fw, fm, fv = pw.clone(), pm.clone(), pv.clone()
+    ws = torch.zeros(max(16, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv if opt != "sgdm" else None, B.make_hyper(opt, h), None, ws)
+    n = 3 if opt != "sgdm" else 2
+    _compare_state(oplan, opt, [pw, pm, pv][:n], [ow, om, ov][:n], TOL_LAMB if opt == "lamb" else TOL_FP32)
+    outs = [torch.zeros_like(x) for x in w]
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), fw, fm, fv if opt != "sgdm" else None,
+                      B.make_hyper(opt, h), B.TensorTable(plan, [outs]), ws)
+    assert torch.equal(fw, pw) and torch.equal(fm, pm)

@@ -469,3 +469,22 @@ def test_empty_tensors_are_inert():
     flat = O.pack(outs[0][0], [np.arange(n, dtype=np.float32) + 1 for n in numel_a])
     back = O.unpack(outs[0][0], flat)
     assert [b.size for b in back] == numel_a and (back[2] == np.arange(333) + 1).all()
+
+
+@pytest.mark.parametrize("groups,M", [(2, 4), (4, 2), (3, 1), (1, 5)])
+def test_partial_sharding_equals_unsharded(groups, M):
+    # Section 5.2: N groups of M replicas, each group shards M ways; the cross-group all-reduce
+    # adds the groups' partial shards -> shard j holds the sum of all N*M gradient copies
+    numel = [9, 64, 333, 2048]
+    K = groups * M
+    rng = np.random.default_rng(K)
+    hs, _ = _hyper("adam")
+    w, m, v, g = _rand_model(rng, numel, K)
+    p = O.Plan(numel, M, 8)
+    pw, pm, pv = O.pack(p, w), O.pack(p, m), O.pack(p, v)
+    O.sharded_update(hs, p, [O.pack(p, gk) for gk in g], pw, pm, pv)
+    O.update_unsharded(hs, g, w, m, v)
+    for a, b in zip(w, O.unpack(p, pw)):
+        assert a.tobytes() == b.tobytes()
+    for a, b in zip(v, O.unpack(p, pv)):
+        assert a.tobytes() == b.tobytes()
