@@ -31,20 +31,24 @@
  * used here are: momentum-SGD with L2 decay added to the gradient
  * (m' = mu m + g + wd w; w' = w - lr m'), Adam with bias correction and eps
  * outside the root, LAMB = Adam direction plus decoupled decay, scaled per
- * tensor by ||w|| / ||u|| (1 when either norm is zero).
+ * tensor by ||w|| / ||u|| (1 when either norm is zero).  LARS (the optimizer
+ * of the paper's ResNet-50 runs, Table 1; formula from the LARS paper it cites):
+ * local rate lambda = eta ||w|| / (||g|| + beta ||w||) per tensor (1 when either
+ * norm is zero), v' = mu v + lr lambda (g + beta w), w' = w - v'.
  */
 #include <math.h>
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
 
-enum { WSO_SGDM = 0, WSO_ADAM = 1, WSO_LAMB = 2 };
+enum { WSO_SGDM = 0, WSO_ADAM = 1, WSO_LAMB = 2, WSO_LARS = 3 };
 enum { WSO_F32 = 0, WSO_BF16 = 1 };
 
 typedef struct {
     int32_t opt;
     double lr, beta1, beta2, eps, weight_decay, momentum, grad_scale;
     int64_t step; /* 1-based index of the update being applied */
+    double trust_coeff; /* LARS eta */
 } wso_hyper;
 
 /* ---------------------------------------------------------------- bf16 -- */
@@ -329,6 +333,96 @@ void wso_shard_reduce(int32_t T, const int64_t *numel, const int64_t *piece, con
             }
             out[off[t] + q] = (float)g;
         }
+}
+
+/* ------------------------------------------------------------------ LARS -- */
+
+static double lars_rate(const wso_hyper *h, double a /* sum w^2 */, double b /* sum g^2 */) {
+    if (!(a > 0.0 && b > 0.0)) return 1.0;
+    return h->trust_coeff * sqrt(a) / (sqrt(b) + h->weight_decay * sqrt(a));
+}
+
+/* Unsharded LARS on one whole tensor: all-reduce (sum) the K gradient copies, take the norms
+ * of the weight and of the summed gradient over the whole tensor, then the momentum step with
+ * the tensor's local rate.  m is the momentum buffer v of the LARS paper.  In place. */
+void wso_lars_tensor(const wso_hyper *h, int64_t n, int32_t K, const void *const *grads,
+                     int32_t g_dtype, float *w, float *m, double *rate) {
+    double *g = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    double a = 0.0, b = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        double s = 0.0;
+        for (int32_t k = 0; k < K; ++k) s += load_grad(grads[k], g_dtype, i);
+        g[i] = s * h->grad_scale;
+        a += (double)w[i] * (double)w[i];
+        b += g[i] * g[i];
+    }
+    double lam = lars_rate(h, a, b);
+    if (rate) *rate = lam;
+    for (int64_t i = 0; i < n; ++i) {
+        double wd = (double)w[i];
+        double vn = h->momentum * (double)m[i] + h->lr * lam * (g[i] + h->weight_decay * wd);
+        m[i] = (float)vn;
+        w[i] = (float)(wd - vn);
+    }
+    free(g);
+}
+
+/* Sharded LARS, step by step (same buffers and conventions as wso_sharded_update): per shard,
+ * reduce the K copies of the slice with pads masked by location and take per-(shard, tensor)
+ * partial sums of w^2 and g^2; combine the partials over shards in ascending r (the scalar
+ * all-reduce of Section 4.1); then every shard applies the step with its tensors' rates. */
+void wso_lars_sharded(const wso_hyper *h, int32_t T, const int64_t *numel, const int64_t *piece,
+                      const int64_t *off, int64_t S, int32_t R, int32_t K,
+                      const void *const *gpacked, int32_t g_dtype, float *w, float *m,
+                      void *gathered, int32_t out_dtype, double *rate) {
+    double *g = (double *)calloc((size_t)R * (size_t)S + 1, sizeof(double));
+    double *part = (double *)calloc((size_t)R * (size_t)T * 2 + 1, sizeof(double));
+    for (int32_t r = 0; r < R; ++r)
+        for (int32_t t = 0; t < T; ++t) {
+            double pa = 0.0, pb = 0.0;
+            for (int64_t q = 0; q < piece[t]; ++q) {
+                int64_t j = (int64_t)r * S + off[t] + q;
+                if ((int64_t)r * piece[t] + q >= numel[t]) continue;   /* pad: identity */
+                double s = 0.0;
+                for (int32_t k = 0; k < K; ++k) s += load_grad(gpacked[k], g_dtype, j);
+                g[j] = s * h->grad_scale;
+                pa += (double)w[j] * (double)w[j];
+                pb += g[j] * g[j];
+            }
+            part[((size_t)r * T + t) * 2 + 0] = pa;
+            part[((size_t)r * T + t) * 2 + 1] = pb;
+        }
+    for (int32_t t = 0; t < T; ++t) {
+        double a = 0.0, b = 0.0;
+        for (int32_t r = 0; r < R; ++r) {
+            a += part[((size_t)r * T + t) * 2 + 0];
+            b += part[((size_t)r * T + t) * 2 + 1];
+        }
+        double lam = lars_rate(h, a, b);
+        if (rate) rate[t] = lam;
+        for (int32_t r = 0; r < R; ++r)
+            for (int64_t q = 0; q < piece[t]; ++q) {
+                int64_t j = (int64_t)r * S + off[t] + q;
+                if ((int64_t)r * piece[t] + q >= numel[t]) {
+                    w[j] = 0.0f;
+                    m[j] = 0.0f;
+                    continue;
+                }
+                double wd = (double)w[j];
+                double vn = h->momentum * (double)m[j] + h->lr * lam * (g[j] + h->weight_decay * wd);
+                m[j] = (float)vn;
+                w[j] = (float)(wd - vn);
+            }
+    }
+    if (gathered) {
+        int64_t G = (int64_t)R * S;
+        if (out_dtype == WSO_BF16)
+            for (int64_t j = 0; j < G; ++j) ((uint16_t *)gathered)[j] = wso_f32_to_bf16(w[j]);
+        else
+            memcpy(gathered, w, sizeof(float) * (size_t)G);
+    }
+    free(g);
+    free(part);
 }
 
 int32_t wso_num_threads(void) {

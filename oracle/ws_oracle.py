@@ -20,9 +20,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ws_oracle.c")
 _SO = os.path.join(_HERE, "libws_oracle.so")
 
-SGDM, ADAM, LAMB = 0, 1, 2
+SGDM, ADAM, LAMB, LARS = 0, 1, 2, 3
 F32, BF16 = 0, 1
-OPT_CODE = {"sgdm": SGDM, "adam": ADAM, "lamb": LAMB}
+OPT_CODE = {"sgdm": SGDM, "adam": ADAM, "lamb": LAMB, "lars": LARS}
 
 
 def build(force: bool = False) -> str:
@@ -38,14 +38,15 @@ def build(force: bool = False) -> str:
 class Hyper(C.Structure):
     _fields_ = [("opt", C.c_int32), ("lr", C.c_double), ("beta1", C.c_double),
                 ("beta2", C.c_double), ("eps", C.c_double), ("weight_decay", C.c_double),
-                ("momentum", C.c_double), ("grad_scale", C.c_double), ("step", C.c_int64)]
+                ("momentum", C.c_double), ("grad_scale", C.c_double), ("step", C.c_int64),
+                ("trust_coeff", C.c_double)]
 
 
 def make_hyper(opt, hyper: dict) -> Hyper:
     code = OPT_CODE[opt] if isinstance(opt, str) else int(opt)
     return Hyper(code, hyper["lr"], hyper["beta1"], hyper["beta2"], hyper["eps"],
                  hyper["weight_decay"], hyper["momentum"], hyper["grad_scale"],
-                 int(hyper["step"]))
+                 int(hyper["step"]), float(hyper.get("trust_coeff", 0.001)))
 
 
 _lib = None
@@ -73,6 +74,13 @@ def lib():
                                          C.c_int64, C.c_int32, C.c_int32, vpp, C.c_int32, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
                                          C.POINTER(C.c_double), C.POINTER(C.c_double)]
+        L.wso_lars_tensor.restype = None
+        L.wso_lars_tensor.argtypes = [C.POINTER(Hyper), C.c_int64, C.c_int32, vpp, C.c_int32,
+                                      C.c_void_p, C.c_void_p, C.POINTER(C.c_double)]
+        L.wso_lars_sharded.restype = None
+        L.wso_lars_sharded.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p, C.c_int64,
+                                       C.c_int32, C.c_int32, vpp, C.c_int32, C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
         L.wso_shard_reduce.restype = None
         L.wso_shard_reduce.argtypes = [C.c_int32, i64p, i64p, i64p, C.c_int64, C.c_int32,
                                        C.c_int32, vpp, C.c_int32, C.c_double, C.c_void_p]
@@ -140,9 +148,14 @@ def unpack(plan: Plan, flat: np.ndarray) -> List[np.ndarray]:
 
 def update_tensor(h: Hyper, grads: Sequence[np.ndarray], w: np.ndarray, m: np.ndarray,
                   v: Optional[np.ndarray]) -> float:
-    """Unsharded definition on one whole tensor, in place; returns rho."""
+    """Unsharded definition on one whole tensor, in place; returns rho (LAMB trust ratio,
+    LARS local rate, 1 otherwise)."""
     rho = C.c_double(1.0)
     n = w.size
+    if h.opt == LARS:
+        lib().wso_lars_tensor(C.byref(h), n, len(grads), _ptrs(grads), _dtype_code(grads[0]),
+                              w.ctypes.data, m.ctypes.data, C.byref(rho))
+        return rho.value
     lib().wso_update_tensor(C.byref(h), n, len(grads), _ptrs(grads), _dtype_code(grads[0]),
                             w.ctypes.data, m.ctypes.data,
                             v.ctypes.data if v is not None else None, C.byref(rho))
@@ -165,6 +178,13 @@ def sharded_update(h: Hyper, plan: Plan, gpacked: Sequence[np.ndarray], w: np.nd
     gathered = None
     if out_dtype is not None:
         gathered = np.empty(plan.G, dtype=np.uint16 if out_dtype == BF16 else np.float32)
+    if h.opt == LARS:
+        lib().wso_lars_sharded(
+            C.byref(h), plan.T, _p(plan.numel), _p(plan.piece), _p(plan.off), plan.S, plan.R,
+            len(gpacked), _ptrs(gpacked), _dtype_code(gpacked[0]), w.ctypes.data, m.ctypes.data,
+            gathered.ctypes.data if gathered is not None else None,
+            out_dtype if out_dtype is not None else F32, rho.ctypes.data_as(C.POINTER(C.c_double)))
+        return gathered, rho, partials
     lib().wso_sharded_update(
         C.byref(h), plan.T, _p(plan.numel), _p(plan.piece), _p(plan.off), plan.S, plan.R,
         len(gpacked), _ptrs(gpacked), _dtype_code(gpacked[0]), w.ctypes.data, m.ctypes.data,

@@ -344,8 +344,9 @@ def _run_both(opt, R, A, numel, bf16=False, poison=False, out_dtype=None, seed=0
             else:
                 buf[~valid] = nanbits
     uw, um, uv = [x.copy() for x in w], [x.copy() for x in m], [x.copy() for x in v]
-    rho_u = O.update_unsharded(hs, g, uw, um, uv if opt != "sgdm" else None)
-    gathered, rho_s, partials = O.sharded_update(hs, p, pg, pw, pm, pv if opt != "sgdm" else None,
+    has_v = opt in ("adam", "lamb")
+    rho_u = O.update_unsharded(hs, g, uw, um, uv if has_v else None)
+    gathered, rho_s, partials = O.sharded_update(hs, p, pg, pw, pm, pv if has_v else None,
                                                  out_dtype)
     return p, (uw, um, uv, rho_u), (pw, pm, pv, gathered, rho_s, partials)
 
@@ -488,3 +489,90 @@ def test_partial_sharding_equals_unsharded(groups, M):
         assert a.tobytes() == b.tobytes()
     for a, b in zip(v, O.unpack(p, pv)):
         assert a.tobytes() == b.tobytes()
+
+
+# ----------------------------------------------------------------- LARS ----
+def _lars_hyper(**kw):
+    h = dict(lr=10.0, beta1=0.0, beta2=0.0, eps=0.0, weight_decay=5e-5, momentum=0.9, grad_scale=1.0,
+             step=1, trust_coeff=0.001)
+    h.update(kw)
+    return O.make_hyper("lars", h), h
+
+
+@pytest.mark.parametrize("K", [1, 8])
+def test_lars_from_torch_sgd_with_local_rate_and_numpy_norms(K):
+    # with lambda = eta ||w|| / (||g|| + beta ||w||) from library norms, one LARS step is one
+    # torch.optim.SGD step at lr*lambda whose momentum buffer is v / (lr*lambda)
+    rng = np.random.default_rng(K)
+    n = 2501
+    hs, h = _lars_hyper()
+    w, m, _, g = _rand_model(rng, [n], K, gstd=1e-3)
+    w0, v0 = w[0].astype(np.float64), m[0].astype(np.float64)
+    gsum = sum(gk[0].astype(np.float64) for gk in g)
+    lam = h["trust_coeff"] * np.linalg.norm(w0) / (np.linalg.norm(gsum) + h["weight_decay"] * np.linalg.norm(w0))
+    eff = h["lr"] * lam
+    p = torch.nn.Parameter(torch.tensor(w0))
+    opt = torch.optim.SGD([p], lr=eff, momentum=h["momentum"], weight_decay=h["weight_decay"])
+    opt.state[p]["momentum_buffer"] = torch.tensor(v0 / eff)
+    p.grad = torch.tensor(gsum)
+    opt.step()
+    rate = O.update_tensor(hs, [gk[0] for gk in g], w[0], m[0], None)
+    assert abs(rate - lam) / lam < 1e-12
+    np.testing.assert_allclose(w[0], p.detach().numpy(), rtol=2e-7, atol=1e-12)
+    np.testing.assert_allclose(m[0], eff * opt.state[p]["momentum_buffer"].numpy(), rtol=2e-7, atol=1e-14)
+
+
+def test_lars_closed_forms():
+    n = 400
+    rng = np.random.default_rng(5)
+    w0 = rng.normal(0, 0.02, n).astype(np.float32)
+    g = rng.normal(0, 1e-3, n).astype(np.float32)
+    # no decay, no momentum: the step length lr*eta*||w|| does not depend on the gradient's scale
+    hs, h = _lars_hyper(weight_decay=0.0, momentum=0.0)
+    outs = []
+    for scale in (1.0, 64.0):
+        w, m = w0.copy(), np.zeros(n, np.float32)
+        O.update_tensor(hs, [(g * scale).astype(np.float32)], w, m, None)
+        outs.append(w)
+        step = np.linalg.norm(w.astype(np.float64) - w0)
+        expect = h["lr"] * h["trust_coeff"] * np.linalg.norm(w0.astype(np.float64))
+        assert abs(step - expect) / expect < 1e-5
+    np.testing.assert_allclose(outs[0], outs[1], rtol=1e-6)
+    # constant tensors: lambda = eta c / (d + beta c)
+    hs, h = _lars_hyper()
+    c, d = 0.5, 0.25
+    w, m = np.full(n, c, np.float32), np.zeros(n, np.float32)
+    rate = O.update_tensor(hs, [np.full(n, d, np.float32)], w, m, None)
+    lam = 0.001 * c / (d + 5e-5 * c)
+    assert abs(rate - lam) < 1e-15
+    np.testing.assert_allclose(w, c - 10.0 * lam * (d + 5e-5 * c), rtol=1e-7)
+    # zero weight norm or zero gradient norm: local rate 1
+    w, m = np.zeros(n, np.float32), np.zeros(n, np.float32)
+    assert O.update_tensor(hs, [g], w, m, None) == 1.0
+    w, m = w0.copy(), np.zeros(n, np.float32)
+    assert O.update_tensor(hs, [np.zeros(n, np.float32)], w, m, None) == 1.0
+
+
+@pytest.mark.parametrize("R", [1, 3, 8, 64])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_sharded_lars_equals_unsharded_within_one_ulp(R, bf16):
+    numel = [1, 9, 64, 333, 2048, 5000]
+    p, (uw, um, _, rate_u), (pw, pm, _, gathered, rate_s, _) = _run_both(
+        "lars", R, 8, numel, bf16=bf16, out_dtype=O.BF16, seed=R, lr=10.0, momentum=0.9, weight_decay=5e-5,
+        trust_coeff=0.001)
+    np.testing.assert_allclose(rate_s, rate_u, rtol=1e-13)
+    for a, b in zip(uw, O.unpack(p, pw)):
+        assert (np.abs(a.astype(np.float64) - b) <= np.spacing(np.abs(a))).all()
+    for a, b in zip(um, O.unpack(p, pm)):
+        assert (np.abs(a.astype(np.float64) - b) <= np.spacing(np.abs(a))).all()
+    np.testing.assert_array_equal(gathered, O.f32_to_bf16_bits(pw))
+
+
+def test_lars_poisoned_pads_never_leak():
+    numel = [1, 9, 64, 333, 2050]
+    kw = dict(lr=10.0, momentum=0.9, weight_decay=5e-5, trust_coeff=0.001)
+    p, _, clean = _run_both("lars", 7, 32, numel, out_dtype=O.BF16, seed=1, **kw)
+    _, _, dirty = _run_both("lars", 7, 32, numel, out_dtype=O.BF16, seed=1, poison=True, **kw)
+    for i in (0, 1, 3):
+        assert clean[i].tobytes() == dirty[i].tobytes()
+    np.testing.assert_array_equal(clean[4], dirty[4])
