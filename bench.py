@@ -46,7 +46,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50",
-                    choices=["tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b"])
+                    choices=["tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b", "resnet50_lars"])
     ap.add_argument("--R", type=int, default=0, help="override the workload's replica count")
     ap.add_argument("--align", type=int, default=32)
     ap.add_argument("--tile", type=int, default=0, help="work-tile elements (0 = library default)")
@@ -72,10 +72,12 @@ def bytes_per_param(wl):
     and its slots once; write weight and slots once; plus the gathered copy when it is a
     separate bf16 buffer) and of one pack / unpack launch."""
     gb = 2 if str(wl.grad_dtype).endswith("bfloat16") else 4
-    slots = 1 if wl.opt == "sgdm" else 2
+    slots = 1 if wl.opt in ("sgdm", "lars") else 2
     upd = gb * wl.R + 4 * (1 + slots) * 2
     if wl.opt == "lamb":
         upd += 12          # plain two-pass: phase 2 reads w, m', v' again and rewrites w
+    if wl.opt == "lars":
+        upd += 12          # phase 1 reads w and stores the summed gradient; phase 2 reads it back
     out_b = 2 if str(wl.out_dtype).endswith("bfloat16") else 0
     # fused formatting: same reads and state writes, plus the weight tensors written directly
     fused = upd + (2 if out_b else 4)
@@ -182,7 +184,7 @@ def oracle_one_step(sub, plan, g, pw, pm, pv):
     t0 = time.perf_counter()
     pg = [O.pack(plan, gk) for gk in g]
     out_dt = O.BF16 if str(sub.out_dtype).endswith("bfloat16") else None
-    gathered, _, _ = O.sharded_update(hs, plan, pg, pw, pm, pv if sub.opt != "sgdm" else None, out_dt)
+    gathered, _, _ = O.sharded_update(hs, plan, pg, pw, pm, pv if sub.opt in ("adam", "lamb") else None, out_dt)
     O.unpack(plan, gathered if gathered is not None else pw)
     return time.perf_counter() - t0
 
@@ -324,7 +326,7 @@ def run_ours(args):
     pm, pv = torch.empty_like(pw), torch.empty_like(pw)
     for src, dst in ((w, pw), (m, pm), (v, pv)):
         B.ws_pack(plan, src, dst)
-    if wl.opt == "sgdm":
+    if wl.opt in ("sgdm", "lars"):
         pv = None
     del w, m, v
     g_arena = [torch.zeros(A_el, dtype=gdt, device=dev) for _ in range(R)]
@@ -457,9 +459,10 @@ def run_ours(args):
     except Exception:
         pass
     bpp = bytes_per_param(wl)
-    n_upd_launch = 3 if wl.opt == "lamb" else 1
+    n_upd_launch = 3 if wl.opt in ("lamb", "lars") else 1
     chunks = -(-T // 1024)
-    upd_name = ("update_kernel" if wl.opt != "lamb" else "update_kernel phase 1 + lamb_finalize_kernel + update_kernel phase 2")
+    upd_name = ("update_kernel" if n_upd_launch == 1 else
+                "update_kernel phase 1 + lamb_finalize_kernel + update_kernel phase 2")
 
     def kernel_rows(path):
         ph = res[path][1]

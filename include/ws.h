@@ -50,7 +50,7 @@ typedef enum {
 } ws_status;
 
 typedef enum { WS_F32 = 0, WS_BF16 = 1 } ws_dtype;
-typedef enum { WS_SGDM = 0, WS_ADAM = 1, WS_LAMB = 2 } ws_opt;
+typedef enum { WS_SGDM = 0, WS_ADAM = 1, WS_LAMB = 2, WS_LARS = 3 } ws_opt;
 
 #define WS_MAX_DIMS 8
 typedef struct {
@@ -161,12 +161,18 @@ typedef struct {
  *   WS_LAMB  m', v' as Adam; u = Adam direction + weight_decay w;
  *            rho_t = ||w_t|| / ||u_t|| over tensor t (1 if either norm is 0);
  *            w' = w - lr rho_t u
+ *   WS_LARS  (the optimizer of the paper's ResNet-50 runs, Table 1; formula of
+ *            the LARS paper it cites) per tensor t the local rate
+ *            lambda_t = trust_coeff ||w_t|| / (||g_t|| + weight_decay ||w_t||)
+ *            (1 if either norm is 0); m' = momentum m + lr lambda_t (g +
+ *            weight_decay w);  w' = w - m'
  * `step` is the 1-based index of the update being applied.  Derived constants
  * are formed in double on the host and narrowed to fp32 for the kernels. */
 typedef struct {
     ws_opt opt;
     double lr, beta1, beta2, eps, weight_decay, momentum, grad_scale;
     int64_t step;
+    double trust_coeff; /* WS_LARS only (eta) */
 } ws_hyper;
 
 /* Where the updated weights go in the all-gather output layout (Section 2.2;
@@ -187,7 +193,10 @@ typedef struct {
  *   (padding to 16 bytes)
  *   double norms[T][2]       squared norms (sum w^2, sum u^2) per tensor
  *   float  partials[R][tiles][2]   per-tile partial sums from phase 1
- * so a caller can read rho and the norms back for logging. */
+ * so a caller can read rho and the norms back for logging.  WS_LARS uses the
+ * same three arrays (rho holds the local rates, norms sum w^2 and sum g^2)
+ * followed, at the next 256-byte boundary, by
+ *   float  ghat[R][S]        the summed gradients kept from phase 1 for phase 2 */
 size_t ws_workspace_bytes(const ws_plan* plan, ws_opt opt);
 
 /* Fused reduce + optimizer update + gathered-layout write for shard r
@@ -195,9 +204,10 @@ size_t ws_workspace_bytes(const ws_plan* plan, ws_opt opt);
  * Reads the r-th slice of each of the R gradient buffers exactly once, w/m/v
  * once, writes w/m/v (and the gathered slot) once (Section 2.2: the update is
  * memory bound - read gradient, weight, auxiliaries; write weight,
- * auxiliaries).  With opt == WS_LAMB only r == -1 is accepted here (phase 1
- * over all shards, finalize, phase 2 over all shards): the trust ratio needs
- * every shard's partial norms before any shard can apply (Section 4.1). */
+ * auxiliaries).  With opt == WS_LAMB or WS_LARS only r == -1 is accepted here
+ * (phase 1 over all shards, finalize, phase 2 over all shards): the per-tensor
+ * ratio needs every shard's partial norms before any shard can apply
+ * (Section 4.1). */
 ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_grads* grads,
                           const ws_state* state, const ws_hyper* hyper, const ws_out* out,
                           void* workspace, size_t workspace_bytes, void* stream);

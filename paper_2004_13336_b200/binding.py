@@ -18,8 +18,8 @@ LIB_PATH = os.path.join(_PKG, "libws.so")
 
 WS_OK = 0
 WS_F32, WS_BF16 = 0, 1
-WS_SGDM, WS_ADAM, WS_LAMB = 0, 1, 2
-OPT_CODE = {"sgdm": WS_SGDM, "adam": WS_ADAM, "lamb": WS_LAMB}
+WS_SGDM, WS_ADAM, WS_LAMB, WS_LARS = 0, 1, 2, 3
+OPT_CODE = {"sgdm": WS_SGDM, "adam": WS_ADAM, "lamb": WS_LAMB, "lars": WS_LARS}
 WS_MAX_DIMS = 8
 
 
@@ -51,7 +51,7 @@ class ws_state(C.Structure):
 class ws_hyper(C.Structure):
     _fields_ = [("opt", C.c_int32), ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double),
                 ("eps", C.c_double), ("weight_decay", C.c_double), ("momentum", C.c_double),
-                ("grad_scale", C.c_double), ("step", C.c_int64)]
+                ("grad_scale", C.c_double), ("step", C.c_int64), ("trust_coeff", C.c_double)]
 
 
 class ws_out(C.Structure):
@@ -198,7 +198,8 @@ def _ptr_array(tensors):
 def make_hyper(opt, hyper: dict) -> ws_hyper:
     code = OPT_CODE[opt] if isinstance(opt, str) else int(opt)
     return ws_hyper(code, hyper["lr"], hyper["beta1"], hyper["beta2"], hyper["eps"],
-                    hyper["weight_decay"], hyper["momentum"], hyper["grad_scale"], int(hyper["step"]))
+                    hyper["weight_decay"], hyper["momentum"], hyper["grad_scale"], int(hyper["step"]),
+                    float(hyper.get("trust_coeff", 0.001)))
 
 
 class Plan:

@@ -55,7 +55,9 @@ struct WsLambWs {
     float* rho;        // [T]
     double* norms;     // [T][2]
     float2* partials;  // [R][ntiles]
-    size_t bytes;
+    size_t bytes;      // through the partials: what LAMB needs
+    float* ghat;       // LARS only: [R][S] summed gradients, 256-byte aligned after the partials
+    size_t bytes_lars; // through ghat: what LARS needs
 };
 WsLambWs ws_lamb_layout(const ws_plan* plan, void* workspace);
 

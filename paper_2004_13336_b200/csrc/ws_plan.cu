@@ -173,10 +173,15 @@ WsLambWs ws_lamb_layout(const ws_plan* p, void* workspace) {
     L.partials = (float2*)(b + o);
     o = round16(o + sizeof(float2) * (size_t)p->R * (size_t)p->ntiles);
     L.bytes = o;
+    o = (o + 255) & ~(size_t)255;
+    L.ghat = (float*)(b + o);
+    L.bytes_lars = o + sizeof(float) * (size_t)p->R * (size_t)p->S;
     return L;
 }
 
 extern "C" size_t ws_workspace_bytes(const ws_plan* p, ws_opt opt) {
-    if (!p || opt != WS_LAMB) return 0;
-    return ws_lamb_layout(p, nullptr).bytes;
+    if (!p) return 0;
+    if (opt == WS_LAMB) return ws_lamb_layout(p, nullptr).bytes;
+    if (opt == WS_LARS) return ws_lamb_layout(p, nullptr).bytes_lars;
+    return 0;
 }

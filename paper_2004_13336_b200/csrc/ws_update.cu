@@ -49,7 +49,12 @@
 namespace {
 
 constexpr int kBlock = 256;
-enum { K_SGDM = 0, K_ADAM = 1, K_LAMB1 = 2, K_LAMB2 = 3 };
+// Kernel flavours.  The norm-based optimizers run as two phases around a finalize step:
+// phase 1 (K_LAMB1, K_LARS1) reduces the gradients and leaves per-tile partial sums of the
+// two norms; phase 2 (K_LAMB2, K_LARS2) applies the step with the per-tensor ratio.
+enum { K_SGDM = 0, K_ADAM = 1, K_LAMB1 = 2, K_LAMB2 = 3, K_LARS1 = 4, K_LARS2 = 5 };
+__host__ __device__ constexpr bool is_phase1(int o) { return o == K_LAMB1 || o == K_LARS1; }
+__host__ __device__ constexpr bool is_phase2(int o) { return o == K_LAMB2 || o == K_LARS2; }
 enum { O_NONE = 0, O_F32 = 1, O_BF16 = 2 };
 
 template <int N>
@@ -72,8 +77,9 @@ struct UpdParams {
     void* gathered;         // base of the G-element gathered buffer, or null
     const void* const* gtab; // fused formatting: device table [T][R] of gradient tensor pointers
     void* const* wtab;       // fused formatting: device table [T] of weight tensor pointers (outputs)
-    float2* partials;       // LAMB: [R][ntiles]
-    const float* rho;       // LAMB phase 2: [T]
+    float2* partials;       // phase 1: [R][ntiles] partial sums of the two norms
+    const float* rho;       // phase 2: [T] trust ratio (LAMB) / local rate (LARS)
+    float* ghat;            // LARS: [R][S] summed gradients, written by phase 1, read by phase 2
     WsConsts c;
 };
 
@@ -242,6 +248,13 @@ __device__ __forceinline__ void update_elem(const WsConsts& c, float g, float& w
         const float gp = fmaf(c.wd, w, g);
         m = fmaf(c.mu, m, gp);
         w = fmaf(-c.lr, m, w);
+    } else if (OPT == K_LARS1) {          // norms of the weight and of the summed gradient
+        sw = fmaf(w, w, sw);
+        su = fmaf(g, g, su);
+    } else if (OPT == K_LARS2) {          // lr_rho = lr * local rate of this tensor
+        const float gp = fmaf(c.wd, w, g);
+        m = fmaf(c.mu, m, lr_rho * gp);
+        w = w - m;
     } else {
         if (OPT != K_LAMB2) {
             m = fmaf(c.beta1, m, c.omb1 * g);
@@ -291,8 +304,11 @@ __device__ __forceinline__ float block_sum(float x, float* smem /* kBlock/32 flo
 // hardware CTA scheduler walks the buffers front to back.
 template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED>
 __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_MINB8 : WS_TUNE_MINB) update_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp) {
-    constexpr bool HAS_V = (OPT != K_SGDM);
-    constexpr bool READS_G = (OPT != K_LAMB2);
+    constexpr bool HAS_V = (OPT == K_ADAM || OPT == K_LAMB1 || OPT == K_LAMB2);
+    constexpr bool READS_G = !is_phase2(OPT);     // phase 2 works from state (and the stored gradient sum)
+    constexpr bool READS_M = (OPT != K_LARS1);
+    constexpr bool WRITES_W = !is_phase1(OPT);    // phase 1 only zeroes the pads of w
+    constexpr bool WRITES_M = (OPT != K_LAMB2 && OPT != K_LARS1);
     constexpr bool LOOPK = (NP > RB);   // R may exceed one tree block: loop and compensate
     __shared__ float red[2][kBlock / 32];
     // fused formatting: this tile's R gradient tensor pointers, fetched once per work item (the
@@ -323,7 +339,7 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_
         }
         const int nvec = tl.len / VEC;
         float lr_rho = 0.f;
-        if (OPT == K_LAMB2) lr_rho = P.c.lr * P.rho[tl.seg];
+        if (is_phase2(OPT)) lr_rho = P.c.lr * P.rho[tl.seg];
         float sw = 0.f, su = 0.f;
 
         for (int q0 = 0; q0 < nvec; q0 += U * kBlock) {
@@ -344,8 +360,9 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_
             for (int u = 0; u < U; ++u) {
                 if (nv[u] > 0) {
                     wv[u] = load_f32<VEC>(P.w + sbase + e0[u]);
-                    mv[u] = load_f32<VEC>(P.m + sbase + e0[u]);
+                    if (READS_M) mv[u] = load_f32<VEC>(P.m + sbase + e0[u]);
                     if (HAS_V) vv[u] = load_f32<VEC>(P.v + sbase + e0[u]);
+                    if (OPT == K_LARS2) gv[u] = load_f32<VEC>(P.ghat + obase + e0[u]);   // summed gradient from phase 1
                 }
             }
             if (READS_G) {
@@ -400,17 +417,17 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_
 #pragma unroll
                 for (int j = 0; j < VEC; ++j) {
                     if (j < nv[u]) {
-                        update_elem<OPT>(P.c, gv[u].f[j] * P.c.gscale, wv[u].f[j], mv[u].f[j], vv[u].f[j], lr_rho, sw, su);
+                        if (OPT != K_LARS2) gv[u].f[j] *= P.c.gscale;     // (phase 1 stored it already scaled)
+                        update_elem<OPT>(P.c, gv[u].f[j], wv[u].f[j], mv[u].f[j], vv[u].f[j], lr_rho, sw, su);
                     } else {  // pad: identity for the sums, +0 for every output
-                        wv[u].f[j] = 0.f; mv[u].f[j] = 0.f; vv[u].f[j] = 0.f;
+                        wv[u].f[j] = 0.f; mv[u].f[j] = 0.f; vv[u].f[j] = 0.f; gv[u].f[j] = 0.f;
                     }
                 }
                 const long long so = sbase + e0[u];
-                if (OPT != K_LAMB1 || nv[u] < VEC) store_f32<VEC>(P.w + so, wv[u]);
-                if (OPT != K_LAMB2) {
-                    store_f32<VEC>(P.m + so, mv[u]);
-                    if (HAS_V) store_f32<VEC>(P.v + so, vv[u]);
-                }
+                if (WRITES_W || nv[u] < VEC) store_f32<VEC>(P.w + so, wv[u]);
+                if (WRITES_M) store_f32<VEC>(P.m + so, mv[u]);
+                if (HAS_V && OPT != K_LAMB2) store_f32<VEC>(P.v + so, vv[u]);
+                if (OPT == K_LARS1) store_f32<VEC>(P.ghat + obase + e0[u], gv[u]);   // keep the sum for phase 2
                 if constexpr (FUSED) {
                     if (OUT == O_F32) {
                         float* dst = reinterpret_cast<float*>(wt) + toff + e0[u];
@@ -428,7 +445,7 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_
                 }
             }
         }
-        if (OPT == K_LAMB1) {
+        if (is_phase1(OPT)) {
             const float a = block_sum(sw, red[0]);
             const float b = block_sum(su, red[1]);
             if (threadIdx.x == 0) P.partials[r * P.ntiles + ti] = make_float2(a, b);
@@ -439,8 +456,10 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_
 // Sum every shard's per-tile partials of tensor t in a fixed order, in double
 // (stands where the paper combines per-replica reduce results with one batched
 // scalar all-reduce, Section 4.1 / 5.2), then rho_t = sqrt(a)/sqrt(b).
+// With lars != 0 the ratio is the LARS local rate eta sqrt(a) / (sqrt(b) + beta sqrt(a)).
 __global__ void __launch_bounds__(kBlock) lamb_finalize_kernel(const WsSegTiles* segtiles, const float2* partials,
-                                                               long long ntiles, int R, float* rho, double* norms) {
+                                                               long long ntiles, int R, float* rho, double* norms,
+                                                               int lars, double eta, double beta) {
     __shared__ double sa[kBlock], sb[kBlock];
     const int t = blockIdx.x;
     const WsSegTiles st = segtiles[t];
@@ -467,7 +486,9 @@ __global__ void __launch_bounds__(kBlock) lamb_finalize_kernel(const WsSegTiles*
         b = sb[0];
         norms[2 * t] = a;
         norms[2 * t + 1] = b;
-        rho[t] = (a > 0.0 && b > 0.0) ? (float)(sqrt(a) / sqrt(b)) : 1.0f;
+        if (!(a > 0.0 && b > 0.0)) rho[t] = 1.0f;
+        else if (lars) rho[t] = (float)(eta * sqrt(a) / (sqrt(b) + beta * sqrt(a)));
+        else rho[t] = (float)(sqrt(a) / sqrt(b));
     }
 }
 
@@ -488,7 +509,7 @@ ws_status launch(const UpdParams& P, const void* const* gptrs, cudaStream_t st) 
 // small R, where the fp32 streams dominate.
 template <int OPT, bool GBF, int OUT, bool FUSED>
 ws_status launch_r(const UpdParams& P, const void* const* gptrs, bool wide_ok, cudaStream_t st) {
-    if constexpr (OPT == K_LAMB2) {
+    if constexpr (is_phase2(OPT)) {
         if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 1, 1, FUSED>(P, gptrs, st);
         return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 1, 1, FUSED>(P, gptrs, st);
     } else {
@@ -519,9 +540,10 @@ bool aligned32(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 31u) ==
 template <int OPT, bool GBF, bool FUSED>
 ws_status launch_o(const UpdParams& P, const void* const* gptrs, int out, bool wide, cudaStream_t st) {
     wide = wide && aligned32(P.w) && aligned32(P.m) && aligned32(P.v) && aligned32(P.gathered);
-    if (!FUSED && OPT != K_LAMB2)
+    if (!FUSED && !is_phase2(OPT))
         for (int k = 0; k < P.R && wide; ++k) wide = aligned32(gptrs[k]);
-    if constexpr (OPT == K_LAMB1) {
+    if (OPT == K_LARS1 || OPT == K_LARS2) wide = wide && aligned32(P.ghat);
+    if constexpr (is_phase1(OPT)) {
         return launch_r<OPT, GBF, O_NONE, FUSED>(P, gptrs, wide, st);
     } else {
         switch (out) {
@@ -540,6 +562,8 @@ ws_status launch_f(int opt, bool gbf, int out, const UpdParams& P, const void* c
         case K_SGDM: return gbf ? launch_o<K_SGDM, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_SGDM, false, FUSED>(P, gptrs, out, wide, st);
         case K_ADAM: return gbf ? launch_o<K_ADAM, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_ADAM, false, FUSED>(P, gptrs, out, wide, st);
         case K_LAMB1: return gbf ? launch_o<K_LAMB1, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_LAMB1, false, FUSED>(P, gptrs, out, wide, st);
+        case K_LARS1: return gbf ? launch_o<K_LARS1, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_LARS1, false, FUSED>(P, gptrs, out, wide, st);
+        case K_LARS2: return launch_o<K_LARS2, false, FUSED>(P, gptrs, out, wide, st);
         default: return launch_o<K_LAMB2, false, FUSED>(P, gptrs, out, wide, st);
     }
 }
@@ -573,13 +597,13 @@ ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state
     if (!p->d_tiles) return WS_ERR_NOT_UPLOADED;
     if (r < -1 || r >= p->R) return WS_ERR_INVALID_ARG;
     if (h->step < 1) return WS_ERR_INVALID_ARG;
-    const bool needs_v = (phase != K_SGDM);
+    const bool needs_v = (phase == K_ADAM || phase == K_LAMB1 || phase == K_LAMB2);
     if (!s->w || !s->m || (needs_v && !s->v)) return WS_ERR_INVALID_ARG;
     if (!ws_aligned16(s->w) || !ws_aligned16(s->m) || (needs_v && !ws_aligned16(s->v))) return WS_ERR_ALIGNMENT;
     gbf = false;
     P.gtab = nullptr;
     P.wtab = nullptr;
-    if (phase != K_LAMB2 && !fused) {
+    if (!is_phase2(phase) && !fused) {
         if (!g || !g->ptrs || g->R < 1) return WS_ERR_INVALID_ARG;
         if (g->dtype != WS_F32 && g->dtype != WS_BF16) return WS_ERR_DTYPE;
         if (g->slice_mode != 0 && g->slice_mode != 1) return WS_ERR_INVALID_ARG;
@@ -609,7 +633,7 @@ ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state
     P.r0 = (r < 0) ? 0 : r;
     P.nitems = (long long)nshards * p->ntiles;
     P.st_stride = (r < 0) ? p->S : 0;
-    if (g && phase != K_LAMB2 && !fused) {
+    if (g && !is_phase2(phase) && !fused) {
         // slice mode 0: pointer is the packed buffer; the launch starts at shard r0
         P.g_stride = (g->slice_mode == 0) ? p->S : 0;
     } else {
@@ -621,6 +645,7 @@ ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state
     P.gathered = (out_kind != O_NONE) ? out->gathered : nullptr;
     P.partials = nullptr;
     P.rho = nullptr;
+    P.ghat = nullptr;
     P.c = make_consts(h);
     return WS_OK;
 }
@@ -637,8 +662,8 @@ void offset_grad_ptrs(const ws_plan* p, int32_t r, const ws_grads* g, std::vecto
     }
 }
 
-ws_status check_ws(const ws_plan* p, void* workspace, size_t bytes) {
-    if (!workspace || bytes < ws_workspace_bytes(p, WS_LAMB)) return WS_ERR_WORKSPACE;
+ws_status check_ws(const ws_plan* p, void* workspace, size_t bytes, ws_opt opt = WS_LAMB) {
+    if (!workspace || bytes < ws_workspace_bytes(p, opt)) return WS_ERR_WORKSPACE;
     if (!ws_aligned16(workspace)) return WS_ERR_ALIGNMENT;
     return WS_OK;
 }
@@ -666,7 +691,7 @@ extern "C" ws_status ws_lamb_finalize(const ws_plan* plan, void* workspace, size
     if (s != WS_OK) return s;
     WsLambWs L = ws_lamb_layout(plan, workspace);
     lamb_finalize_kernel<<<plan->T, kBlock, 0, (cudaStream_t)stream>>>(plan->d_segtiles, L.partials, plan->ntiles,
-                                                                      plan->R, L.rho, L.norms);
+                                                                      plan->R, L.rho, L.norms, 0, 0.0, 0.0);
     return ws_check_launch("ws_lamb_finalize");
 }
 
@@ -692,6 +717,31 @@ extern "C" ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_gr
         if (s != WS_OK) return s;
         if ((s = ws_lamb_finalize(plan, workspace, workspace_bytes, stream)) != WS_OK) return s;
         return ws_lamb_apply(plan, -1, state, hyper, out, workspace, workspace_bytes, stream);
+    }
+    if (hyper->opt == WS_LARS) {
+        // LARS (the optimizer of the paper's ResNet-50 runs, Table 1): phase 1 reduces the gradients,
+        // keeps the sum in the workspace and leaves partial sums of ||w||^2 and ||g||^2; the finalize
+        // step forms each tensor's local rate; phase 2 applies the momentum step.
+        if (r != -1) return WS_ERR_INVALID_ARG;
+        UpdParams P;
+        int ok;
+        bool gbf;
+        ws_status s = prepare(plan, -1, grads, state, hyper, nullptr, K_LARS1, P, ok, gbf);
+        if (s != WS_OK) return s;
+        if ((s = check_ws(plan, workspace, workspace_bytes, WS_LARS)) != WS_OK) return s;
+        const WsLambWs L = ws_lamb_layout(plan, workspace);
+        P.partials = L.partials;
+        P.ghat = L.ghat;
+        std::vector<const void*> gp;
+        offset_grad_ptrs(plan, -1, grads, gp);
+        if ((s = launch_any(K_LARS1, gbf, O_NONE, P, gp.data(), (cudaStream_t)stream)) != WS_OK) return s;
+        lamb_finalize_kernel<<<plan->T, kBlock, 0, (cudaStream_t)stream>>>(
+            plan->d_segtiles, L.partials, plan->ntiles, plan->R, L.rho, L.norms, 1, hyper->trust_coeff, hyper->weight_decay);
+        if ((s = ws_check_launch("ws_shard_update(LARS finalize)")) != WS_OK) return s;
+        if ((s = prepare(plan, -1, nullptr, state, hyper, out, K_LARS2, P, ok, gbf)) != WS_OK) return s;
+        P.rho = L.rho;
+        P.ghat = L.ghat;
+        return launch_any(K_LARS2, false, ok, P, nullptr, (cudaStream_t)stream);
     }
     if (hyper->opt != WS_SGDM && hyper->opt != WS_ADAM) return WS_ERR_INVALID_ARG;
     const int phase = hyper->opt == WS_SGDM ? K_SGDM : K_ADAM;
@@ -754,21 +804,22 @@ ws_status fused_phase(const ws_plan* plan, int32_t r, const ws_tensor_table* gra
     if (s != WS_OK) return s;
     bool wide = true;
     int out_kind = O_NONE;
-    if (phase != K_LAMB2) {
+    if (!is_phase2(phase)) {
         P.gtab = (const void* const*)grads->dev;
         P.R = grads->nsets;
         gbf = grads->dtype == WS_BF16;
         wide = wide && (gbf || grads->min_align >= 32);
     }
-    if (phase != K_LAMB1) {
+    if (!is_phase1(phase)) {
         P.wtab = (void* const*)weights->dev;
         out_kind = weights->dtype == WS_F32 ? O_F32 : O_BF16;
         wide = wide && (weights->dtype == WS_BF16 || weights->min_align >= 32);
     }
-    if (phase == K_LAMB1 || phase == K_LAMB2) {
+    if (is_phase1(phase) || is_phase2(phase)) {
         WsLambWs L = ws_lamb_layout(plan, workspace);
         P.partials = L.partials;
         P.rho = L.rho;
+        P.ghat = L.ghat;
     }
     return launch_f<true>(phase, gbf, out_kind, P, nullptr, wide, st);
 }
@@ -792,6 +843,17 @@ extern "C" ws_status ws_fused_update(const ws_plan* plan, int32_t r, const ws_te
         if ((s = fused_phase(plan, -1, grads, state, hyper, weights, K_LAMB1, workspace, st)) != WS_OK) return s;
         if ((s = ws_lamb_finalize(plan, workspace, workspace_bytes, stream)) != WS_OK) return s;
         return fused_phase(plan, -1, grads, state, hyper, weights, K_LAMB2, workspace, st);
+    }
+    if (hyper->opt == WS_LARS) {
+        if (r != -1) return WS_ERR_INVALID_ARG;
+        ws_status s = check_ws(plan, workspace, workspace_bytes, WS_LARS);
+        if (s != WS_OK) return s;
+        if ((s = fused_phase(plan, -1, grads, state, hyper, weights, K_LARS1, workspace, st)) != WS_OK) return s;
+        const WsLambWs L = ws_lamb_layout(plan, workspace);
+        lamb_finalize_kernel<<<plan->T, kBlock, 0, st>>>(plan->d_segtiles, L.partials, plan->ntiles, plan->R, L.rho,
+                                                        L.norms, 1, hyper->trust_coeff, hyper->weight_decay);
+        if ((s = ws_check_launch("ws_fused_update(LARS finalize)")) != WS_OK) return s;
+        return fused_phase(plan, -1, grads, state, hyper, weights, K_LARS2, workspace, st);
     }
     if (hyper->opt != WS_SGDM && hyper->opt != WS_ADAM) return WS_ERR_INVALID_ARG;
     return fused_phase(plan, r, grads, state, hyper, weights, hyper->opt == WS_SGDM ? K_SGDM : K_ADAM, nullptr, st);

@@ -23,7 +23,7 @@ Shape = Tuple[int, ...]
 
 # optimizer codes shared by name only (values mirror the public C enum and the
 # oracle's enum; each side defines its own copy)
-SGDM, ADAM, LAMB = "sgdm", "adam", "lamb"
+SGDM, ADAM, LAMB, LARS = "sgdm", "adam", "lamb", "lars"
 
 
 @dataclass
@@ -59,7 +59,7 @@ class Workload:
 
 def _hyper(**kw) -> Dict[str, float]:
     h = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0,
-             momentum=0.0, grad_scale=1.0, step=10)
+             momentum=0.0, grad_scale=1.0, step=10, trust_coeff=0.001)
     h.update(kw)
     return h
 
@@ -147,6 +147,12 @@ def resnet50() -> Workload:
                     seed=2)
 
 
+def resnet50_lars() -> Workload:
+    """The ResNet-50 tensor set under LARS, the optimizer of the paper's ResNet-50 runs (Table 1)."""
+    return Workload("resnet50_lars", resnet50_shapes(), R=8, opt=LARS,
+                    hyper=_hyper(lr=10.0, momentum=0.9, weight_decay=5e-5, trust_coeff=0.001), seed=6)
+
+
 def transformer(R: int = 8) -> Workload:
     return Workload("transformer", transformer_shapes(), R=R, opt=ADAM,
                     hyper=_hyper(), seed=3, R_sweep=(1, 2, 8, 32, 128, 1024))
@@ -166,7 +172,7 @@ def decoder_1p5b() -> Workload:
 
 WORKLOADS = {
     "tiny": tiny, "resnet50": resnet50, "transformer": transformer,
-    "bert_large": bert_large, "decoder_1p5b": decoder_1p5b,
+    "bert_large": bert_large, "decoder_1p5b": decoder_1p5b, "resnet50_lars": resnet50_lars,
 }
 
 

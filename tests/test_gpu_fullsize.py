@@ -280,3 +280,31 @@ def test_bert_large_lamb_fused_equals_unfused():
     assert torch.equal(fw, pw) and torch.equal(fm, pm) and torch.equal(fv, pv)
     for a, b in zip(w, ref):
         assert torch.equal(a, b)
+
+
+def test_resnet50_lars_full_model_every_element():
+    """The ResNet-50 tensor set under LARS (the optimizer of the paper's ResNet-50 runs, Table 1), R=8,
+    through the fused route the benchmark times; every element and every local rate against the oracle."""
+    wl = W.resnet50_lars()
+    plan = B.Plan(wl.shapes, wl.R, A)
+    w, m, _ = W.make_state(wl, DEV)
+    g = W.make_grads(wl, DEV)
+    ow, om = [to_np(x) for x in w], [to_np(x) for x in m]
+    og = [[to_np(x) for x in gk] for gk in g]
+    orate = O.update_unsharded(O.make_hyper(wl.opt, wl.hyper), og, ow, om, None)
+    pw = torch.empty(plan.G, device=DEV)
+    pm = torch.empty_like(pw)
+    B.ws_pack(plan, w, pw)
+    B.ws_pack(plan, m, pm)
+    ws = torch.empty(plan.workspace_bytes("lars"), dtype=torch.uint8, device=DEV)
+    outs = [torch.empty_like(x) for x in w]
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), pw, pm, None, B.make_hyper(wl.opt, wl.hyper),
+                      B.TensorTable(plan, [outs]), ws)
+    outs_m = [torch.empty_like(x) for x in w]
+    B.ws_unpack(plan, pm, outs_m)
+    ew = max(err(to_np(a), b) for a, b in zip(outs, ow))
+    em = max(err(to_np(a), b) for a, b in zip(outs_m, om))
+    rate = B.lamb_ratios(plan, ws).cpu().numpy().astype(np.float64)
+    er = float(np.max(np.abs(rate - np.array(orate)) / np.array(orate)))
+    print(f"resnet50 LARS full: err w {ew:.2e} m {em:.2e} rate {er:.2e}")
+    assert ew <= TOL_LAMB and em <= TOL_LAMB and er <= TOL_LAMB

@@ -523,3 +523,70 @@ def test_partial_sharding_more_gradient_copies_than_shards(opt, groups, M):
     B.ws_fused_update(plan, -1, B.TensorTable(plan, g), fw, fm, fv if opt != "sgdm" else None,
                       B.make_hyper(opt, h), B.TensorTable(plan, [outs]), ws)
     assert torch.equal(fw, pw) and torch.equal(fm, pm)
+
+
+# ------------------------------------------------------------------- LARS ---
+def _lars_hyper(**kw):
+    return _hyper("sgdm", lr=10.0, momentum=0.9, weight_decay=5e-5, trust_coeff=0.001, **kw)
+
+
+@pytest.mark.parametrize("R", [1, 2, 3, 8, 16, 40])
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+def test_lars_matches_oracle_and_fused_equals_unfused(R, gdtype):
+    wl, w, m, v, g = _model(SHAPES, R, gdtype, seed=R + 7, gstd=1e-3)
+    plan = B.Plan(SHAPES, R, 32)
+    oplan = O.Plan(wl.numels, R, 32)
+    h = _lars_hyper()
+    ow, om, _, orate = _oracle_unsharded("lars", h, w, m, v, g)
+    pw, pm, _, pg = _pack_all(plan, w, m, v, g)
+    fw, fm = pw.clone(), pm.clone()
+    ws = torch.zeros(plan.workspace_bytes("lars"), dtype=torch.uint8, device=DEV)
+    gath = torch.full((plan.G,), 3.0, dtype=torch.bfloat16, device=DEV)
+    B.ws_shard_update(plan, -1, pg, pw, pm, None, B.make_hyper("lars", h), gath, ws)
+    # the local rate carries fp32 norm error (~1e-7), so w' and m' get the LAMB-class tolerance
+    _compare_state(oplan, "sgdm", [pw, pm], [ow, om], TOL_LAMB)
+    rate = B.lamb_ratios(plan, ws).cpu().numpy().astype(np.float64)
+    rel = np.abs(rate - np.array(orate)) / np.array(orate)
+    assert rel.max() <= TOL_LAMB, rel.max()
+    assert _pads_are_zero(oplan, pw) and _pads_are_zero(oplan, pm) and _pads_are_zero(oplan, gath)
+    assert torch.equal(gath, pw.to(torch.bfloat16))
+    outs = [torch.zeros(n, dtype=torch.bfloat16, device=DEV) for n in wl.numels]
+    ws2 = torch.zeros_like(ws)
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), fw, fm, None, B.make_hyper("lars", h),
+                      B.TensorTable(plan, [outs]), ws2)
+    assert torch.equal(fw, pw) and torch.equal(fm, pm)
+    ref = [torch.zeros_like(o) for o in outs]
+    B.ws_unpack(plan, gath, ref)
+    for a, b in zip(outs, ref):
+        assert torch.equal(a, b)
+
+
+def test_lars_poisoned_pads_and_error_codes():
+    import ctypes as C
+    R = 5
+    wl, w, m, v, g = _model(SHAPES, R, seed=12, gstd=1e-3)
+    plan = B.Plan(SHAPES, R, 32)
+    oplan = O.Plan(wl.numels, R, 32)
+    hy = B.make_hyper("lars", _lars_hyper())
+    valid = torch.from_numpy(O.pack(oplan, [np.ones(int(n), np.float32) for n in oplan.numel]) != 0).to(DEV)
+    res = []
+    for poison in (False, True):
+        pw, pm, _, pg = _pack_all(plan, w, m, v, g)
+        ws = torch.zeros(plan.workspace_bytes("lars"), dtype=torch.uint8, device=DEV)
+        if poison:
+            for b in [pw, pm] + pg:
+                b[~valid] = float("nan")
+            ws.view(torch.float32)[:] = float("nan")       # the workspace may hold anything on entry
+        B.ws_shard_update(plan, -1, pg, pw, pm, None, hy, None, ws)
+        res.append((pw, pm, B.lamb_ratios(plan, ws).clone()))
+    for a, b in zip(*res):
+        assert torch.equal(a, b)
+    # too small a workspace and a single-shard call are refused before any launch
+    pw, pm, _, pg = _pack_all(plan, w, m, v, g)
+    small = torch.zeros(plan.workspace_bytes("lamb"), dtype=torch.uint8, device=DEV)
+    with pytest.raises(B.WsError) as e:
+        B.ws_shard_update(plan, -1, pg, pw, pm, None, hy, None, small)
+    assert e.value.status == 4
+    with pytest.raises(B.WsError) as e:
+        B.ws_shard_update(plan, 0, pg, pw, pm, None, hy, None, torch.zeros(plan.workspace_bytes("lars"), dtype=torch.uint8, device=DEV))
+    assert e.value.status == 1
