@@ -590,3 +590,36 @@ def test_lars_poisoned_pads_and_error_codes():
     with pytest.raises(B.WsError) as e:
         B.ws_shard_update(plan, 0, pg, pw, pm, None, hy, None, torch.zeros(plan.workspace_bytes("lars"), dtype=torch.uint8, device=DEV))
     assert e.value.status == 1
+
+
+# ------------------------------------------------------- host-buffer step ---
+@pytest.mark.parametrize("opt,gdtype,odtype", [("sgdm", torch.float32, torch.float32),
+                                               ("adam", torch.bfloat16, torch.bfloat16),
+                                               ("lamb", torch.float32, torch.bfloat16)])
+def test_step_host_from_pinned_arenas_matches_oracle(opt, gdtype, odtype):
+    R = 3
+    wl, w, m, v, g = _model(SHAPES, R, gdtype, seed=31)
+    plan = B.Plan(SHAPES, R, 32)
+    h = _hyper(opt)
+    ow, _, _, _ = _oracle_unsharded(opt, h, w, m, v, g)
+    pw, pm, pv, _ = _pack_all(plan, w, m, v, [])
+    n_el, numels = plan.arena_elems, wl.numels
+    host_g = []
+    for gk in g:                                   # one pinned arena per replica, tensors back to back
+        a = torch.zeros(n_el, dtype=gdtype).pin_memory()
+        for dst, src in zip(plan.arena_views(a, numels), gk):
+            dst.copy_(src)
+        host_g.append(a)
+    host_w = torch.full((n_el,), 5.0, dtype=odtype).pin_memory()
+    stage = torch.empty(n_el, dtype=gdtype, device=DEV)
+    packed = [torch.empty(plan.G, dtype=gdtype, device=DEV) for _ in range(R)]
+    dev_w = torch.empty(n_el, dtype=odtype, device=DEV)
+    gathered = torch.empty(plan.G, dtype=odtype, device=DEV) if odtype != torch.float32 else None
+    ws = torch.zeros(max(16, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+    B.ws_step_host(plan, host_g, stage, packed, pw, pm, pv if opt != "sgdm" else None, B.make_hyper(opt, h),
+                   dev_w, host_w, gathered, ws)
+    torch.cuda.synchronize()
+    tol = TOL_BF16 if odtype == torch.bfloat16 else (TOL_LAMB if opt == "lamb" else TOL_FP32)
+    for got, ref in zip(plan.arena_views(host_w, numels), ow):
+        got = to_np(got)
+        assert err(bf16_to_f64(got) if odtype == torch.bfloat16 else got, ref) <= tol
