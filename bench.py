@@ -36,7 +36,10 @@ FALLBACK_HBM_GBS = 6650.0
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
 # captures summarised under profiles/, keyed by (workload, kernel); None = not captured.
-NCU_TRAFFIC_BYTES = {("resnet50", "fused"): 1.2987e9}   # profiles/fused_update_kernel_resnet50_sgdm_R8.md
+NCU_TRAFFIC_BYTES = {
+    ("resnet50", "fused"): 1.2987e9,        # profiles/fused_update_kernel_resnet50_sgdm_R8.md
+    ("decoder_1p5b", "fused"): 52.55e9,     # profiles/fused_update_kernel_bf16_transformer_R4.md, scaled by parameter count
+}
 
 
 def parse_args():
@@ -48,6 +51,10 @@ def parse_args():
     ap.add_argument("--workload", default="resnet50",
                     choices=["tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b", "resnet50_lars"])
     ap.add_argument("--R", type=int, default=0, help="override the workload's replica count")
+    ap.add_argument("--opt", default="", choices=["", "sgdm", "adam", "lamb", "lars"],
+                    help="override the workload's optimizer (profiling of small cases)")
+    ap.add_argument("--grad-dtype", default="", choices=["", "f32", "bf16"], help="override the gradient dtype")
+    ap.add_argument("--out-dtype", default="", choices=["", "f32", "bf16"], help="override the emitted weight dtype")
     ap.add_argument("--align", type=int, default=32)
     ap.add_argument("--tile", type=int, default=0, help="work-tile elements (0 = library default)")
     ap.add_argument("--path", default="both", choices=["both", "fused", "unfused"],
@@ -64,6 +71,18 @@ def get_workload(args):
     wl = W.WORKLOADS[args.workload]()
     if args.R:
         wl.R = args.R
+    if args.opt or args.grad_dtype or args.out_dtype:
+        import torch
+        dt = {"f32": torch.float32, "bf16": torch.bfloat16}
+        if args.opt and args.opt != wl.opt:
+            wl.opt = args.opt
+            wl.hyper = dict(W.WORKLOADS[{"sgdm": "resnet50", "adam": "transformer", "lamb": "bert_large",
+                                         "lars": "resnet50_lars"}[args.opt]]().hyper)
+        if args.grad_dtype:
+            wl.grad_dtype = dt[args.grad_dtype]
+        if args.out_dtype:
+            wl.out_dtype = dt[args.out_dtype]
+        wl.name += "*"          # not one of the named workloads any more
     return wl
 
 
