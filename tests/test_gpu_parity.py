@@ -623,3 +623,33 @@ def test_step_host_from_pinned_arenas_matches_oracle(opt, gdtype, odtype):
     for got, ref in zip(plan.arena_views(host_w, numels), ow):
         got = to_np(got)
         assert err(bf16_to_f64(got) if odtype == torch.bfloat16 else got, ref) <= tol
+
+
+def test_more_than_1024_tensors():
+    # tensor pointers travel in kernel parameters in chunks of 1024: a list longer than that
+    # takes several pack launches; the update and the fused route see one table
+    rng = np.random.default_rng(0)
+    shapes = [(int(n),) for n in rng.integers(1, 300, 1100)] + [(5000,), (3, 7)]
+    R = 3
+    wl, w, m, v, g = _model(shapes, R, seed=2)
+    plan = B.Plan(shapes, R, 8)
+    oplan = O.Plan(wl.numels, R, 8)
+    flat = torch.empty(plan.G, device=DEV)
+    B.ws_pack(plan, w, flat)
+    assert to_np(flat).tobytes() == O.pack(oplan, [to_np(x) for x in w]).tobytes()
+    back = [torch.zeros_like(x) for x in w]
+    B.ws_unpack(plan, flat, back)
+    for a, b in zip(back, w):
+        assert torch.equal(a, b)
+    h = _hyper("adam")
+    ow, om, ov, _ = _oracle_unsharded("adam", h, w, m, v, g)
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    fw, fm, fv = pw.clone(), pm.clone(), pv.clone()
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv, B.make_hyper("adam", h))
+    _compare_state(oplan, "adam", [pw, pm, pv], [ow, om, ov], TOL_FP32)
+    outs = [torch.zeros_like(x) for x in w]
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), fw, fm, fv, B.make_hyper("adam", h), B.TensorTable(plan, [outs]))
+    assert torch.equal(fw, pw)
+    B.ws_unpack(plan, pw, back)
+    for a, b in zip(outs, back):
+        assert torch.equal(a, b)
