@@ -307,13 +307,13 @@ def run_ours(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the sharded update has no CPU fallback")
-    if not ws_build.up_to_date():
-        if rank == 0:
-            ws_build.build()
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    if rank == 0 and not ws_build.up_to_date():
+        ws_build.build()                      # one rank builds; the others wait at the barrier
+    if world > 1:
         dist.barrier()
     B.lib()
 
