@@ -55,6 +55,8 @@ def parse_args():
                     help="override the workload's optimizer (profiling of small cases)")
     ap.add_argument("--grad-dtype", default="", choices=["", "f32", "bf16"], help="override the gradient dtype")
     ap.add_argument("--out-dtype", default="", choices=["", "f32", "bf16"], help="override the emitted weight dtype")
+    ap.add_argument("--shards", type=int, default=0,
+                    help="shard count of the plan when it differs from the replica count (partial sharding)")
     ap.add_argument("--align", type=int, default=32)
     ap.add_argument("--tile", type=int, default=0, help="work-tile elements (0 = library default)")
     ap.add_argument("--path", default="both", choices=["both", "fused", "unfused"],
@@ -259,7 +261,7 @@ def config_of(wl, args, extra=None, path="unfused"):
                       "update of all shards, weights written to the weight tensors"}
     c = {"workload": f"{wl.name}: {wl.T} tensors, {wl.N} params, R={wl.R} replicas, {wl.opt}, "
                      f"grads {str(wl.grad_dtype).split('.')[-1]}, gathered {str(wl.out_dtype).split('.')[-1]}",
-         "R": wl.R, "optimizer": wl.opt, "align_elems": args.align,
+         "R": wl.R, "shards": getattr(args, "shards", 0) or wl.R, "optimizer": wl.opt, "align_elems": args.align,
          "step": steps[path],
          "l2": "inputs exceed L2 (no flush)" if wl.N * 4 * (wl.R + 3) > 256e6 else "flush between steps"}
     if extra:
@@ -320,7 +322,11 @@ def run_ours(args):
     wl = get_workload(args)
     wl.seed = rank_seed(wl.seed, rank)        # every rank owns its own tensor set
     R, T, N = wl.R, wl.T, wl.N
-    plan = B.Plan(wl.shapes, R, args.align, args.tile, device=dev)
+    # partial sharding (Section 5.2): R gradient copies, but the update is sharded only `shards` ways
+    shards = args.shards or R
+    plan = B.Plan(wl.shapes, shards, args.align, args.tile, device=dev)
+    if shards != R:
+        args.no_e2e = True        # the host-buffer entry point takes one gradient arena per shard
     gdt, odt = wl.grad_dtype, wl.out_dtype
     gb = 2 if gdt == torch.bfloat16 else 4
     wb = 2 if odt == torch.bfloat16 else 4
