@@ -425,6 +425,111 @@ void wso_lars_sharded(const wso_hyper *h, int32_t T, const int64_t *numel, const
     free(part);
 }
 
+/* ------------------------------------------- concatenated (flat) layout -- */
+
+/* Section 5.2, "Batched communication operators": for a combined all-reduce the input tensors
+ * are concatenated in their full shapes and the internal shards are partitions of the
+ * concatenation, whatever tensor a boundary falls in.  As a sharding layout for the update:
+ * tensor t starts at cat[t] (each start rounded up to a multiple of A elements), the
+ * concatenation of length C = cat[T] is cut into R shards of S = A * ceil(ceil(C / R) / A)
+ * elements, and shard r is positions [r S, (r+1) S).  Returns S. */
+int64_t wso_plan_flat(const int64_t *numel, int32_t T, int32_t R, int32_t A, int64_t *cat) {
+    int64_t c = 0;
+    for (int32_t t = 0; t < T; ++t) {
+        cat[t] = c;
+        c = ((c + numel[t] + A - 1) / A) * A;
+    }
+    cat[T] = c;
+    int64_t per = (c + R - 1) / R;
+    return ((per + A - 1) / A) * A;
+}
+
+/* Sharded route over an explicit position map: tmap[p] is the tensor that owns position p of the
+ * [R][S] layout (or -1 for padding).  Per shard r: reduce the K gradient copies of the slice with
+ * pads masked by location, update the slice; for the norm-based optimizers take per-(shard, tensor)
+ * partial sums, combine them over shards in ascending r, then apply.  Same buffers, outputs and
+ * conventions as wso_sharded_update / wso_lars_sharded; serves any layout that has a map. */
+void wso_sharded_update_map(const wso_hyper *h, int32_t T, const int32_t *tmap, int64_t S, int32_t R,
+                            int32_t K, const void *const *gpacked, int32_t g_dtype, float *w, float *m,
+                            float *v, void *gathered, int32_t out_dtype, double *rho) {
+    bias_corr b = bias_of(h);
+    const int lamb = (h->opt == WSO_LAMB), lars = (h->opt == WSO_LARS);
+    const int64_t G = (int64_t)R * S;
+    double *u = (double *)calloc((size_t)G + 1, sizeof(double));       /* LAMB: u;  LARS: summed gradient */
+    double *part = (double *)calloc((size_t)R * (size_t)T * 2 + 1, sizeof(double));
+    for (int32_t r = 0; r < R; ++r)
+        for (int64_t q = 0; q < S; ++q) {
+            const int64_t j = (int64_t)r * S + q;
+            const int32_t t = tmap[j];
+            if (t < 0) {                                              /* pad */
+                w[j] = 0.0f;
+                m[j] = 0.0f;
+                if (v) v[j] = 0.0f;
+                continue;
+            }
+            double g = 0.0;
+            for (int32_t k = 0; k < K; ++k) g += load_grad(gpacked[k], g_dtype, j);
+            g *= h->grad_scale;
+            double wd = (double)w[j], md = (double)m[j];
+            double *pa = &part[((size_t)r * T + t) * 2];
+            if (h->opt == WSO_SGDM) {
+                sgdm_elem(h, g, &wd, &md);
+                w[j] = (float)wd;
+                m[j] = (float)md;
+            } else if (lars) {
+                u[j] = g;
+                pa[0] += wd * wd;
+                pa[1] += g * g;
+            } else {
+                double vd = (double)v[j];
+                double dir = adam_moments(h, b, g, &md, &vd);
+                v[j] = (float)vd;
+                m[j] = (float)md;
+                if (lamb) {
+                    u[j] = dir + h->weight_decay * wd;
+                    pa[0] += wd * wd;
+                    pa[1] += u[j] * u[j];
+                } else {
+                    w[j] = (float)(wd - h->lr * dir);
+                }
+            }
+        }
+    double *ratio = (double *)calloc((size_t)T + 1, sizeof(double));
+    for (int32_t t = 0; t < T; ++t) {
+        double a = 0.0, bb = 0.0;
+        for (int32_t r = 0; r < R; ++r) {
+            a += part[((size_t)r * T + t) * 2 + 0];
+            bb += part[((size_t)r * T + t) * 2 + 1];
+        }
+        ratio[t] = 1.0;
+        if (lamb) ratio[t] = (a > 0.0 && bb > 0.0) ? sqrt(a) / sqrt(bb) : 1.0;
+        if (lars) ratio[t] = lars_rate(h, a, bb);
+        if (rho) rho[t] = ratio[t];
+    }
+    if (lamb || lars)
+        for (int64_t j = 0; j < G; ++j) {
+            const int32_t t = tmap[j];
+            if (t < 0) continue;
+            const double wd = (double)w[j];
+            if (lamb) {
+                w[j] = (float)(wd - h->lr * ratio[t] * u[j]);
+            } else {
+                const double vn = h->momentum * (double)m[j] + h->lr * ratio[t] * (u[j] + h->weight_decay * wd);
+                m[j] = (float)vn;
+                w[j] = (float)(wd - vn);
+            }
+        }
+    if (gathered) {
+        if (out_dtype == WSO_BF16)
+            for (int64_t j = 0; j < G; ++j) ((uint16_t *)gathered)[j] = wso_f32_to_bf16(w[j]);
+        else
+            memcpy(gathered, w, sizeof(float) * (size_t)G);
+    }
+    free(ratio);
+    free(u);
+    free(part);
+}
+
 int32_t wso_num_threads(void) {
 #ifdef _OPENMP
     extern int omp_get_max_threads(void);

@@ -81,6 +81,12 @@ def lib():
         L.wso_lars_sharded.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p, C.c_int64,
                                        C.c_int32, C.c_int32, vpp, C.c_int32, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
+        L.wso_plan_flat.restype = C.c_int64
+        L.wso_plan_flat.argtypes = [i64p, C.c_int32, C.c_int32, C.c_int32, i64p]
+        L.wso_sharded_update_map.restype = None
+        L.wso_sharded_update_map.argtypes = [C.POINTER(Hyper), C.c_int32, C.POINTER(C.c_int32), C.c_int64,
+                                             C.c_int32, C.c_int32, vpp, C.c_int32, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
         L.wso_shard_reduce.restype = None
         L.wso_shard_reduce.argtypes = [C.c_int32, i64p, i64p, i64p, C.c_int64, C.c_int32,
                                        C.c_int32, vpp, C.c_int32, C.c_double, C.c_void_p]
@@ -217,3 +223,51 @@ def bf16_bits_to_f64(x: np.ndarray) -> np.ndarray:
 
 def num_threads() -> int:
     return int(lib().wso_num_threads())
+
+
+class FlatPlan:
+    """Concatenated layout (Section 5.2): tensors back to back (starts rounded up to A), the
+    concatenation cut into R equal shards wherever the boundaries fall."""
+
+    def __init__(self, numel: Sequence[int], R: int, A: int):
+        self.numel = _i64(numel)
+        self.T, self.R, self.A = len(self.numel), int(R), int(A)
+        self.cat = np.zeros(self.T + 1, dtype=np.int64)
+        self.S = int(lib().wso_plan_flat(_p(self.numel), self.T, self.R, self.A, _p(self.cat)))
+        self.G = self.R * self.S
+        self.N = int(self.numel.sum())
+
+    def tensor_map(self) -> np.ndarray:
+        """Owner tensor of every position of the [R][S] layout, -1 for padding."""
+        tmap = np.full(self.G, -1, dtype=np.int32)
+        for t in range(self.T):
+            tmap[self.cat[t]:self.cat[t] + self.numel[t]] = t
+        return tmap
+
+
+def pack_flat(plan: FlatPlan, tensors: Sequence[np.ndarray]) -> np.ndarray:
+    dt = tensors[0].dtype if len(tensors) else np.float32
+    flat = np.zeros(plan.G, dtype=dt)                      # pads are all-zero bits
+    for t, x in enumerate(tensors):
+        flat[plan.cat[t]:plan.cat[t] + plan.numel[t]] = x  # position = start of the tensor + index
+    return flat
+
+
+def unpack_flat(plan: FlatPlan, flat: np.ndarray) -> List[np.ndarray]:
+    return [flat[plan.cat[t]:plan.cat[t] + plan.numel[t]].copy() for t in range(plan.T)]
+
+
+def sharded_update_flat(h: Hyper, plan: FlatPlan, gpacked: Sequence[np.ndarray], w: np.ndarray, m: np.ndarray,
+                        v: Optional[np.ndarray], out_dtype: Optional[int] = None):
+    """Sharded route on the concatenated layout, in place.  Returns (gathered or None, rho[T])."""
+    rho = np.ones(plan.T, dtype=np.float64)
+    gathered = None
+    if out_dtype is not None:
+        gathered = np.empty(plan.G, dtype=np.uint16 if out_dtype == BF16 else np.float32)
+    tmap = plan.tensor_map()
+    lib().wso_sharded_update_map(
+        C.byref(h), plan.T, tmap.ctypes.data_as(C.POINTER(C.c_int32)), plan.S, plan.R, len(gpacked),
+        _ptrs(gpacked), _dtype_code(gpacked[0]), w.ctypes.data, m.ctypes.data,
+        v.ctypes.data if v is not None else None, gathered.ctypes.data if gathered is not None else None,
+        out_dtype if out_dtype is not None else F32, rho.ctypes.data_as(C.POINTER(C.c_double)))
+    return gathered, rho

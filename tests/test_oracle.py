@@ -576,3 +576,72 @@ def test_lars_poisoned_pads_never_leak():
     for i in (0, 1, 3):
         assert clean[i].tobytes() == dirty[i].tobytes()
     np.testing.assert_array_equal(clean[4], dirty[4])
+
+
+# ------------------------------------------- concatenated (flat) layout ----
+@pytest.mark.parametrize("R", [1, 3, 8, 64, 1024])
+@pytest.mark.parametrize("A", [8, 32])
+def test_flat_plan_partitions_the_concatenation(R, A):
+    numel = [1, 5, 8, 9, 63, 64, 65, 130, 0, 4099]
+    p = O.FlatPlan(numel, R, A)
+    assert p.cat[0] == 0 and (p.cat % A == 0).all()
+    assert (np.diff(p.cat) >= p.numel).all() and (np.diff(p.cat) - p.numel < A).all()   # only alignment gaps
+    assert p.S % A == 0 and p.G >= p.cat[-1] and p.G - p.cat[-1] < R * A                # and a short tail
+    tmap = p.tensor_map()
+    assert int((tmap >= 0).sum()) == sum(numel)
+    for t, n in enumerate(numel):                       # every element has exactly one position, in order
+        assert (np.nonzero(tmap == t)[0] == p.cat[t] + np.arange(n)).all()
+    # never more padding than the per-tensor layout
+    assert p.G <= O.Plan(numel, R, A).G
+
+
+def test_flat_layout_has_almost_no_padding_at_1024_shards():
+    wl = W.transformer(1024)
+    flat, per = O.FlatPlan(wl.numels, 1024, 32), O.Plan(wl.numels, 1024, 32)
+    assert flat.G - wl.N < 40000 and per.G - wl.N > 2_000_000
+
+
+@pytest.mark.parametrize("R", [1, 2, 3, 7, 16])
+@pytest.mark.parametrize("dtype", [np.float32, np.uint16])
+def test_flat_pack_unpack_identity(R, dtype):
+    rng = np.random.default_rng(R)
+    numel = [1, 2, 13, 127, 128, 1031, 4096]
+    p = O.FlatPlan(numel, R, 8)
+    bits = np.uint32 if dtype == np.float32 else np.uint16
+    tensors = [rng.integers(1, np.iinfo(bits).max, n, dtype=np.uint64).astype(bits).view(dtype) for n in numel]
+    flat = O.pack_flat(p, tensors)
+    for a, b in zip(tensors, O.unpack_flat(p, flat)):
+        assert a.tobytes() == b.tobytes()
+    assert int((flat.view(bits) == 0).sum()) == p.G - p.N
+
+
+@pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb", "lars"])
+@pytest.mark.parametrize("R", [1, 3, 8, 64])
+def test_flat_sharded_equals_unsharded(opt, R):
+    numel = [1, 9, 64, 333, 2048, 5000]
+    rng = np.random.default_rng(R)
+    kw = dict(momentum=0.9, weight_decay=5e-5 if opt in ("sgdm", "lars") else (0.01 if opt == "lamb" else 0.0),
+              eps=1e-6 if opt == "lamb" else 1e-8, lr=10.0 if opt == "lars" else 1e-3)
+    hs, _ = _hyper(opt, **kw)
+    w, m, v, g = _rand_model(rng, numel, R, gstd=1e-3)
+    has_v = opt in ("adam", "lamb")
+    p = O.FlatPlan(numel, R, 8)
+    pw, pm, pv = O.pack_flat(p, w), O.pack_flat(p, m), O.pack_flat(p, v)
+    valid = p.tensor_map() >= 0
+    for buf in (pw, pm, pv):
+        buf[~valid] = np.float32(np.nan)                     # pads may hold anything on entry
+    pg = [O.pack_flat(p, gk) for gk in g]
+    for buf in pg:
+        buf[~valid] = np.float32(np.nan)
+    gathered, rho_s = O.sharded_update_flat(hs, p, pg, pw, pm, pv if has_v else None, O.BF16)
+    rho_u = O.update_unsharded(hs, g, w, m, v if has_v else None)
+    np.testing.assert_allclose(rho_s, rho_u, rtol=1e-13)
+    exact = opt in ("sgdm", "adam")
+    for ref, got in ((w, O.unpack_flat(p, pw)), (m, O.unpack_flat(p, pm))):
+        for a, b in zip(ref, got):
+            if exact:
+                assert a.tobytes() == b.tobytes()
+            else:
+                assert (np.abs(a.astype(np.float64) - b) <= np.spacing(np.abs(a))).all()
+    assert (pw.view(np.uint32)[~valid] == 0).all() and (pm.view(np.uint32)[~valid] == 0).all()
+    np.testing.assert_array_equal(gathered, O.f32_to_bf16_bits(pw))
