@@ -57,6 +57,8 @@ def parse_args():
     ap.add_argument("--out-dtype", default="", choices=["", "f32", "bf16"], help="override the emitted weight dtype")
     ap.add_argument("--shards", type=int, default=0,
                     help="shard count of the plan when it differs from the replica count (partial sharding)")
+    ap.add_argument("--layout", default="per_tensor", choices=["per_tensor", "concat"],
+                    help="per_tensor: one piece of every tensor per shard; concat: the concatenation cut into R shards")
     ap.add_argument("--align", type=int, default=32)
     ap.add_argument("--tile", type=int, default=0, help="work-tile elements (0 = library default)")
     ap.add_argument("--path", default="both", choices=["both", "fused", "unfused"],
@@ -262,6 +264,7 @@ def config_of(wl, args, extra=None, path="unfused"):
     c = {"workload": f"{wl.name}: {wl.T} tensors, {wl.N} params, R={wl.R} replicas, {wl.opt}, "
                      f"grads {str(wl.grad_dtype).split('.')[-1]}, gathered {str(wl.out_dtype).split('.')[-1]}",
          "R": wl.R, "shards": getattr(args, "shards", 0) or wl.R, "optimizer": wl.opt, "align_elems": args.align,
+         "layout": getattr(args, "layout", "per_tensor"),
          "step": steps[path],
          "l2": "inputs exceed L2 (no flush)" if wl.N * 4 * (wl.R + 3) > 256e6 else "flush between steps"}
     if extra:
@@ -324,7 +327,7 @@ def run_ours(args):
     R, T, N = wl.R, wl.T, wl.N
     # partial sharding (Section 5.2): R gradient copies, but the update is sharded only `shards` ways
     shards = args.shards or R
-    plan = B.Plan(wl.shapes, shards, args.align, args.tile, device=dev)
+    plan = B.Plan(wl.shapes, shards, args.align, args.tile, device=dev, layout=args.layout)
     if shards != R:
         args.no_e2e = True        # the host-buffer entry point takes one gradient arena per shard
     gdt, odt = wl.grad_dtype, wl.out_dtype

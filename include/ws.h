@@ -85,6 +85,25 @@ ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int32_t R, int3
                          int32_t tile_elems, ws_plan** out);
 void ws_plan_destroy(ws_plan* plan);
 
+/* Second layout policy (Section 5.2, "Batched communication operators": for a
+ * combined all-reduce the input tensors are concatenated in their full shapes
+ * and the internal shards are partitions of the concatenation, not bound to
+ * any tensor's own sharding).  WS_LAYOUT_CONCAT lays the tensors back to back
+ * (each start rounded up to A elements), cuts the concatenation of length C
+ * into R shards of S = A ceil(ceil(C / R) / A) elements wherever the
+ * boundaries fall, and so pads at most A-1 elements per tensor plus a tail
+ * shorter than R A - against up to R A per tensor for the per-tensor layout,
+ * which is what makes tiny shards expensive at large R.  A tensor may span
+ * several shards or share a shard with many others; every call of this
+ * library accepts plans of either layout.  In ws_plan_segments `piece` is 0
+ * and `shard_off` is the tensor's start inside the concatenation;
+ * ws_plan_num_tiles counts the tiles of all shards.  ws_plan_create is
+ * ws_plan_create_layout with WS_LAYOUT_PER_TENSOR. */
+typedef enum { WS_LAYOUT_PER_TENSOR = 0, WS_LAYOUT_CONCAT = 1 } ws_layout;
+ws_status ws_plan_create_layout(const ws_tensor_desc* descs, int32_t T, int32_t R, int32_t align_elems,
+                                int32_t tile_elems, ws_layout layout, ws_plan** out);
+int32_t ws_plan_layout(const ws_plan* plan);
+
 int32_t ws_plan_num_tensors(const ws_plan* plan); /* T */
 int32_t ws_plan_num_shards(const ws_plan* plan);  /* R */
 int32_t ws_plan_align(const ws_plan* plan);       /* A */
@@ -193,6 +212,7 @@ typedef struct {
  *   (padding to 16 bytes)
  *   double norms[T][2]       squared norms (sum w^2, sum u^2) per tensor
  *   float  partials[R][tiles][2]   per-tile partial sums from phase 1
+ *                                  ([tiles][2] for the concatenated layout)
  * so a caller can read rho and the norms back for logging.  WS_LARS uses the
  * same three arrays (rho holds the local rates, norms sum w^2 and sum g^2)
  * followed, at the next 256-byte boundary, by

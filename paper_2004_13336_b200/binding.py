@@ -20,6 +20,8 @@ WS_OK = 0
 WS_F32, WS_BF16 = 0, 1
 WS_SGDM, WS_ADAM, WS_LAMB, WS_LARS = 0, 1, 2, 3
 OPT_CODE = {"sgdm": WS_SGDM, "adam": WS_ADAM, "lamb": WS_LAMB, "lars": WS_LARS}
+WS_LAYOUT_PER_TENSOR, WS_LAYOUT_CONCAT = 0, 1
+LAYOUT_CODE = {"per_tensor": WS_LAYOUT_PER_TENSOR, "concat": WS_LAYOUT_CONCAT}
 WS_MAX_DIMS = 8
 
 
@@ -77,6 +79,7 @@ EXPORTS = [
     "ws_last_cuda_error", "ws_plan_arena_elems", "ws_plan_arena_offsets", "ws_step_host",
     "ws_static_scratch_bytes", "ws_lamb_update_static_scratch",
     "ws_tensor_table_bytes", "ws_tensor_table_upload", "ws_fused_update",
+    "ws_plan_create_layout", "ws_plan_layout",
 ]
 
 _lib = None
@@ -96,6 +99,11 @@ def lib() -> C.CDLL:
     L.ws_plan_create.restype = C.c_int
     L.ws_plan_create.argtypes = [C.POINTER(ws_tensor_desc), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                  C.POINTER(vp)]
+    L.ws_plan_create_layout.restype = C.c_int
+    L.ws_plan_create_layout.argtypes = [C.POINTER(ws_tensor_desc), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                        C.c_int, C.POINTER(vp)]
+    L.ws_plan_layout.restype = C.c_int32
+    L.ws_plan_layout.argtypes = [vp]
     L.ws_plan_destroy.restype = None
     L.ws_plan_destroy.argtypes = [vp]
     for name, rt in (("ws_plan_num_tensors", C.c_int32), ("ws_plan_num_shards", C.c_int32),
@@ -206,7 +214,7 @@ class Plan:
     """Owns a ws_plan and the device buffer that holds its tables."""
 
     def __init__(self, shapes: Sequence[Sequence[int]], R: int, align_elems: int = 32, tile_elems: int = 0,
-                 device: Optional[torch.device] = None, upload: bool = True):
+                 device: Optional[torch.device] = None, upload: bool = True, layout: str = "per_tensor"):
         T = len(shapes)
         descs = (ws_tensor_desc * max(1, T))()
         for i, s in enumerate(shapes):
@@ -217,7 +225,9 @@ class Plan:
             for j, d in enumerate(s):
                 descs[i].dims[j] = d
         self._h = C.c_void_p()
-        _check(lib().ws_plan_create(descs, T, R, align_elems, tile_elems, C.byref(self._h)), "ws_plan_create")
+        self.layout = layout
+        _check(lib().ws_plan_create_layout(descs, T, R, align_elems, tile_elems, LAYOUT_CODE[layout],
+                                           C.byref(self._h)), "ws_plan_create_layout")
         L = lib()
         self.T, self.R, self.A = L.ws_plan_num_tensors(self._h), L.ws_plan_num_shards(self._h), L.ws_plan_align(self._h)
         self.S, self.N = L.ws_plan_shard_elems(self._h), L.ws_plan_valid_elems(self._h)

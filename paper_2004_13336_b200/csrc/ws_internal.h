@@ -14,6 +14,8 @@
 //   shard position of element e of the tile : pos + e
 //   index of that element in tensor `seg`    : r*piece + poff + e      (shard r)
 //   it exists in the tensor iff              : e < vt - r*piece
+// Per-tensor layout: one tile list serves every shard r.  Concatenated layout: every shard
+// has its own tiles (`shard` says which), piece is 0 and poff / vt are absolute.
 struct __align__(16) WsTile {
     long long pos;    // start inside a shard, multiple of 8
     long long vt;     // numel - poff: valid elements from the tile start in shard 0
@@ -21,7 +23,8 @@ struct __align__(16) WsTile {
     long long poff;   // pos - off_t: start inside the piece
     int len;          // elements in the tile, multiple of 8, <= tile_elems
     int seg;          // tensor index t
-    int pad0, pad1;
+    int shard;        // concatenated layout only: the shard this tile lies in
+    int pad1;
 };
 static_assert(sizeof(WsTile) == 48, "WsTile is read as three 16-byte words");
 
@@ -33,7 +36,10 @@ struct WsSegTiles {
 
 struct ws_plan {
     int T = 0, R = 0, A = 0, K = 0;
-    long long S = 0, N = 0, ntiles = 0;
+    int layout = 0;                           // ws_layout
+    long long S = 0, N = 0;
+    long long ntiles = 0;                     // per-tensor layout: tiles per shard; concatenated: all tiles
+    std::vector<long long> shard_tile_begin;  // concatenated layout: [R+1] first tile of every shard
     std::vector<ws_segment> segs;
     std::vector<WsTile> tiles;
     std::vector<WsSegTiles> segtiles;

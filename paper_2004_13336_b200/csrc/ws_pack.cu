@@ -5,7 +5,8 @@
 // all-zero bits (Section 4.1: the pad is fused into the slice).
 //
 // Work item = (shard r, tile).  A tile is moved as 16-byte vectors; the one
-// vector that straddles n_t is moved element by element.
+// vector that straddles n_t is moved element by element.  In the concatenated
+// layout every shard has its own tiles and a tile names its shard.
 #include "ws_internal.h"
 
 namespace {
@@ -24,6 +25,7 @@ struct PackParams {
     long long nitems;     // R * ntl
     long long S;
     int seg_lo;           // tensor index of PtrChunk::p[0]
+    int concat;           // concatenated layout: every tile names its own shard
 };
 
 __device__ __forceinline__ uint4 ld_stream(const uint4* p) { return __ldcs(p); }
@@ -35,8 +37,9 @@ __global__ void __launch_bounds__(kBlock) pack_kernel(PackParams P, const __grid
                                                       char* __restrict__ flat) {
     constexpr int EPV = 16 / EB;  // elements per 16-byte vector
     for (long long item = blockIdx.x; item < P.nitems; item += gridDim.x) {
-        const long long r = item / P.ntl;
+        long long r = P.concat ? 0 : item / P.ntl;
         const WsTile tl = P.tiles[P.tile_lo + (item - r * P.ntl)];
+        if (P.concat) r = tl.shard;
         char* tensor = (char*)tab.p[tl.seg - P.seg_lo];
         const long long src0 = r * tl.piece + tl.poff;      // element index in the tensor
         long long nv = tl.vt - r * tl.piece;                // valid elements in this tile
@@ -95,7 +98,8 @@ ws_status run(const ws_plan* p, void* const* tensor_ptrs, ws_dtype dtype, void* 
         P.tile_lo = p->segtiles[seg_lo].tile_begin;
         const long long tile_hi = (long long)p->segtiles[seg_hi - 1].tile_begin + p->segtiles[seg_hi - 1].tile_count;
         P.ntl = tile_hi - P.tile_lo;
-        P.nitems = P.ntl * p->R;
+        P.concat = (p->layout == WS_LAYOUT_CONCAT);
+        P.nitems = P.concat ? P.ntl : P.ntl * p->R;
         P.S = p->S;
         P.seg_lo = seg_lo;
         long long grid = P.nitems;   // one CTA per (shard, tile): the CTA scheduler walks the buffers in order

@@ -43,9 +43,17 @@ extern "C" const char* ws_status_string(ws_status s) {
 
 extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int32_t R,
                                     int32_t align_elems, int32_t tile_elems, ws_plan** out) {
+    return ws_plan_create_layout(descs, T, R, align_elems, tile_elems, WS_LAYOUT_PER_TENSOR, out);
+}
+
+extern "C" int32_t ws_plan_layout(const ws_plan* p) { return p ? p->layout : 0; }
+
+extern "C" ws_status ws_plan_create_layout(const ws_tensor_desc* descs, int32_t T, int32_t R, int32_t align_elems,
+                                           int32_t tile_elems, ws_layout layout, ws_plan** out) {
     if (!out) return WS_ERR_INVALID_ARG;
     *out = nullptr;
     if (!descs || T < 1 || R < 1) return WS_ERR_INVALID_ARG;
+    if (layout != WS_LAYOUT_PER_TENSOR && layout != WS_LAYOUT_CONCAT) return WS_ERR_INVALID_ARG;
     if (align_elems < 8 || (align_elems & (align_elems - 1)) != 0) return WS_ERR_INVALID_ARG;
     if (tile_elems == 0) {
         // Default: the largest tile that still leaves >= 20000 work items for an all-shard
@@ -74,10 +82,71 @@ extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int3
     p->R = R;
     p->A = align_elems;
     p->K = tile_elems;
+    p->layout = layout;
     try {
         p->segs.resize(T);
         p->segtiles.resize(T);
         long long off = 0;
+        for (int t = 0; layout == WS_LAYOUT_CONCAT && t < T; ++t) {
+            // Concatenated layout (Section 5.2): tensors back to back, each start rounded up to A.
+            const ws_tensor_desc& d = descs[t];
+            if (d.ndim < 0 || d.ndim > WS_MAX_DIMS) { delete p; return WS_ERR_INVALID_ARG; }
+            long long n = 1;
+            for (int i = 0; i < d.ndim; ++i) {
+                if (d.dims[i] < 0 || (d.dims[i] > 0 && n > (1LL << 46) / d.dims[i])) { delete p; return WS_ERR_INVALID_ARG; }
+                n *= d.dims[i];
+            }
+            p->segs[t].numel = n;
+            p->segs[t].piece = 0;
+            p->segs[t].shard_off = off;          // start inside the concatenation
+            p->N += n;
+            p->arena_off.push_back(p->arena_elems);
+            p->arena_elems += (n + 7) / 8 * 8;
+            off = (off + n + align_elems - 1) / align_elems * align_elems;
+        }
+        if (layout == WS_LAYOUT_CONCAT) {
+            const long long C = off;
+            const long long per = (C + R - 1) / R;
+            p->S = (per + align_elems - 1) / align_elems * align_elems;
+            const long long G = p->S * R;
+            // region of tensor t: from its start to the next tensor's start (the alignment gap
+            // belongs to it as padding); the last region runs to the end of the last shard
+            int t = 0;
+            p->shard_tile_begin.assign(R + 1, 0);
+            for (int k = 0; k < T; ++k) { p->segtiles[k].tile_begin = 0; p->segtiles[k].tile_count = 0; }
+            std::vector<char> seen(T, 0);
+            for (int r = 0; r < R; ++r) {
+                p->shard_tile_begin[r] = (long long)p->tiles.size();
+                long long pos = (long long)r * p->S;            // global position
+                const long long end = pos + p->S;
+                while (pos < end) {
+                    // tensor whose region holds `pos`
+                    while (t < T - 1 && p->segs[t + 1].shard_off <= pos) ++t;
+                    const long long reg_end = (t < T - 1) ? p->segs[t + 1].shard_off : G;
+                    long long stop = reg_end < end ? reg_end : end;
+                    long long len = stop - pos;
+                    if (len > tile_elems) len = tile_elems;
+                    WsTile tl;
+                    memset(&tl, 0, sizeof(tl));
+                    tl.pos = pos - (long long)r * p->S;
+                    tl.poff = pos - p->segs[t].shard_off;
+                    tl.vt = p->segs[t].numel - tl.poff;
+                    tl.piece = 0;
+                    tl.len = (int)len;
+                    tl.seg = t;
+                    tl.shard = r;
+                    if ((long long)p->tiles.size() >= 0x7fffffffLL) { delete p; return WS_ERR_TOO_LARGE; }
+                    if (!seen[t]) { seen[t] = 1; p->segtiles[t].tile_begin = (int)p->tiles.size(); }
+                    p->segtiles[t].tile_count += 1;
+                    p->tiles.push_back(tl);
+                    pos += len;
+                }
+            }
+            p->shard_tile_begin[R] = (long long)p->tiles.size();
+            p->ntiles = (long long)p->tiles.size();
+            *out = p;
+            return WS_OK;
+        }
         for (int t = 0; t < T; ++t) {
             const ws_tensor_desc& d = descs[t];
             if (d.ndim < 0 || d.ndim > WS_MAX_DIMS) { delete p; return WS_ERR_INVALID_ARG; }
@@ -171,7 +240,7 @@ WsLambWs ws_lamb_layout(const ws_plan* p, void* workspace) {
     L.norms = (double*)(b + o);
     o = round16(o + sizeof(double) * 2 * (size_t)p->T);
     L.partials = (float2*)(b + o);
-    o = round16(o + sizeof(float2) * (size_t)p->R * (size_t)p->ntiles);
+    o = round16(o + sizeof(float2) * (size_t)(p->layout == WS_LAYOUT_CONCAT ? 1 : p->R) * (size_t)p->ntiles);
     L.bytes = o;
     o = (o + 255) & ~(size_t)255;
     L.ghat = (float*)(b + o);

@@ -71,6 +71,8 @@ struct UpdParams {
     long long st_stride;    // per-shard element stride inside w/m/v (S for [R][S] state, 0 for one shard)
     int R;
     int r0;                 // first shard of this launch
+    int concat;             // concatenated layout: tiles [tile_lo, tile_lo + nitems), each names its shard
+    long long tile_lo;
     float* w;
     float* m;
     float* v;
@@ -316,10 +318,11 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_
     __shared__ const void* sgp[(FUSED && READS_G) ? NP : 1];
 
     for (long long item = blockIdx.x; item < P.nitems; item += gridDim.x) {
-        const long long rs = item / P.ntiles;              // shard index inside this launch
-        const long long ti = item - rs * P.ntiles;
-        const long long r = P.r0 + rs;
+        long long rs = P.concat ? 0 : item / P.ntiles;     // shard index inside this launch
+        const long long ti = P.concat ? P.tile_lo + item : item - rs * P.ntiles;
         const WsTile tl = P.tiles[ti];
+        if (P.concat) rs = tl.shard - P.r0;
+        const long long r = P.r0 + rs;
         long long nvl = tl.vt - r * tl.piece;              // valid elements in this tile for shard r
         const int nvalid = nvl < 0 ? 0 : (nvl > tl.len ? tl.len : (int)nvl);
         const long long gbase = rs * P.g_stride + tl.pos;  // into each gradient buffer
@@ -448,7 +451,7 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_
         if (is_phase1(OPT)) {
             const float a = block_sum(sw, red[0]);
             const float b = block_sum(su, red[1]);
-            if (threadIdx.x == 0) P.partials[r * P.ntiles + ti] = make_float2(a, b);
+            if (threadIdx.x == 0) P.partials[P.concat ? ti : r * P.ntiles + ti] = make_float2(a, b);
         }
     }
 }
@@ -460,6 +463,7 @@ __global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_
 __global__ void __launch_bounds__(kBlock) lamb_finalize_kernel(const WsSegTiles* segtiles, const float2* partials,
                                                                long long ntiles, int R, float* rho, double* norms,
                                                                int lars, double eta, double beta) {
+    // R == 1 with the concatenated layout: a tensor's tiles of all shards are one contiguous run
     __shared__ double sa[kBlock], sb[kBlock];
     const int t = blockIdx.x;
     const WsSegTiles st = segtiles[t];
@@ -632,6 +636,12 @@ ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state
     const int nshards = (r < 0) ? p->R : 1;
     P.r0 = (r < 0) ? 0 : r;
     P.nitems = (long long)nshards * p->ntiles;
+    P.concat = (p->layout == WS_LAYOUT_CONCAT);
+    P.tile_lo = 0;
+    if (P.concat) {
+        P.tile_lo = (r < 0) ? 0 : p->shard_tile_begin[r];
+        P.nitems = (r < 0) ? p->ntiles : p->shard_tile_begin[r + 1] - p->shard_tile_begin[r];
+    }
     P.st_stride = (r < 0) ? p->S : 0;
     if (g && !is_phase2(phase) && !fused) {
         // slice mode 0: pointer is the packed buffer; the launch starts at shard r0
@@ -662,6 +672,10 @@ void offset_grad_ptrs(const ws_plan* p, int32_t r, const ws_grads* g, std::vecto
     }
 }
 
+// How many strided repetitions of a tensor's tile run the finalize step sums: R (one run per
+// shard, ntiles apart) for the per-tensor layout, 1 for the concatenated layout.
+int finalize_reps(const ws_plan* p) { return p->layout == WS_LAYOUT_CONCAT ? 1 : p->R; }
+
 ws_status check_ws(const ws_plan* p, void* workspace, size_t bytes, ws_opt opt = WS_LAMB) {
     if (!workspace || bytes < ws_workspace_bytes(p, opt)) return WS_ERR_WORKSPACE;
     if (!ws_aligned16(workspace)) return WS_ERR_ALIGNMENT;
@@ -691,7 +705,7 @@ extern "C" ws_status ws_lamb_finalize(const ws_plan* plan, void* workspace, size
     if (s != WS_OK) return s;
     WsLambWs L = ws_lamb_layout(plan, workspace);
     lamb_finalize_kernel<<<plan->T, kBlock, 0, (cudaStream_t)stream>>>(plan->d_segtiles, L.partials, plan->ntiles,
-                                                                      plan->R, L.rho, L.norms, 0, 0.0, 0.0);
+                                                                      finalize_reps(plan), L.rho, L.norms, 0, 0.0, 0.0);
     return ws_check_launch("ws_lamb_finalize");
 }
 
@@ -736,7 +750,7 @@ extern "C" ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_gr
         offset_grad_ptrs(plan, -1, grads, gp);
         if ((s = launch_any(K_LARS1, gbf, O_NONE, P, gp.data(), (cudaStream_t)stream)) != WS_OK) return s;
         lamb_finalize_kernel<<<plan->T, kBlock, 0, (cudaStream_t)stream>>>(
-            plan->d_segtiles, L.partials, plan->ntiles, plan->R, L.rho, L.norms, 1, hyper->trust_coeff, hyper->weight_decay);
+            plan->d_segtiles, L.partials, plan->ntiles, finalize_reps(plan), L.rho, L.norms, 1, hyper->trust_coeff, hyper->weight_decay);
         if ((s = ws_check_launch("ws_shard_update(LARS finalize)")) != WS_OK) return s;
         if ((s = prepare(plan, -1, nullptr, state, hyper, out, K_LARS2, P, ok, gbf)) != WS_OK) return s;
         P.rho = L.rho;
@@ -850,7 +864,7 @@ extern "C" ws_status ws_fused_update(const ws_plan* plan, int32_t r, const ws_te
         if (s != WS_OK) return s;
         if ((s = fused_phase(plan, -1, grads, state, hyper, weights, K_LARS1, workspace, st)) != WS_OK) return s;
         const WsLambWs L = ws_lamb_layout(plan, workspace);
-        lamb_finalize_kernel<<<plan->T, kBlock, 0, st>>>(plan->d_segtiles, L.partials, plan->ntiles, plan->R, L.rho,
+        lamb_finalize_kernel<<<plan->T, kBlock, 0, st>>>(plan->d_segtiles, L.partials, plan->ntiles, finalize_reps(plan), L.rho,
                                                         L.norms, 1, hyper->trust_coeff, hyper->weight_decay);
         if ((s = ws_check_launch("ws_fused_update(LARS finalize)")) != WS_OK) return s;
         return fused_phase(plan, -1, grads, state, hyper, weights, K_LARS2, workspace, st);

@@ -34,17 +34,23 @@ def _gather(t, idx_dev):
     return to_np(t[idx_dev])
 
 
-def _run_sampled(wl, samples_per_tensor=1500, path="unfused"):
+def _run_sampled(wl, samples_per_tensor=1500, path="unfused", layout="per_tensor"):
     """Elementwise optimizers: full-size GPU step, oracle on sampled elements.
     path "unfused": ws_pack of every gradient list, ws_shard_update, ws_unpack;
     path "fused":   ws_fused_update straight from the gradient lists into weight tensors
                     (the configuration the benchmark reports)."""
     torch.cuda.empty_cache()
     rng = np.random.default_rng(wl.seed)
-    plan = B.Plan(wl.shapes, wl.R, A)
-    oplan = O.Plan(wl.numels, wl.R, A)
+    plan = B.Plan(wl.shapes, wl.R, A, layout=layout)
+    if layout == "concat":
+        oplan = O.FlatPlan(wl.numels, wl.R, A)
+        # shard boundaries fall inside tensors: sample both sides of the first one in each tensor
+        piece = [max(1, int(oplan.S - (oplan.cat[t] % oplan.S))) for t in range(wl.T)]
+    else:
+        oplan = O.Plan(wl.numels, wl.R, A)
+        piece = [int(p) for p in oplan.piece]
     assert (plan.S, plan.N) == (oplan.S, oplan.N)
-    idx = [_sample_indices(n, int(p), wl.R, rng, samples_per_tensor) for n, p in zip(wl.numels, oplan.piece)]
+    idx = [_sample_indices(n, p, wl.R, rng, samples_per_tensor) for n, p in zip(wl.numels, piece)]
     idx_dev = [torch.from_numpy(i).to(DEV) for i in idx]
     w, m, v = W.make_state(wl, DEV)
     sw, sm, sv = ([_gather(x, i) for x, i in zip(lst, idx_dev)] for lst in (w, m, v))
@@ -156,6 +162,13 @@ def test_transformer_adam_R128_sampled(path):
 @pytest.mark.parametrize("path", ["unfused", "fused"])
 def test_decoder_1p5b_bf16_grads_bf16_gathered_sampled(path):
     _run_sampled(W.decoder_1p5b(), samples_per_tensor=500, path=path)
+
+
+@pytest.mark.parametrize("path", ["unfused", "fused"])
+@pytest.mark.parametrize("R", [8, 32])
+def test_transformer_concat_layout_sampled(R, path):
+    """The concatenated layout (Section 5.2) at full size: shards cut tensors wherever they fall."""
+    _run_sampled(W.transformer(R), path=path, layout="concat")
 
 
 def test_resnet50_fused_path_sampled():

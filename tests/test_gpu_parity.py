@@ -653,3 +653,85 @@ def test_more_than_1024_tensors():
     B.ws_unpack(plan, pw, back)
     for a, b in zip(outs, back):
         assert torch.equal(a, b)
+
+
+# ------------------------------------------- concatenated layout (Section 5.2) ---
+CONCAT_SHAPES = SHAPES + [(0,), (77,)]
+
+
+@pytest.mark.parametrize("R", [1, 2, 3, 7, 16, 64, 1024])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_concat_pack_unpack_bit_exact(R, dtype):
+    numel = [int(np.prod(s)) for s in CONCAT_SHAPES]
+    plan = B.Plan(CONCAT_SHAPES, R, 32, layout="concat")
+    oplan = O.FlatPlan(numel, R, 32)
+    assert (plan.S, plan.G) == (oplan.S, oplan.G)
+    gen = torch.Generator(device=DEV).manual_seed(R)
+    tensors = [torch.randn(n, device=DEV, generator=gen).to(dtype) for n in numel]
+    big, flat = _guarded(plan.G, dtype, 7.0)
+    B.ws_pack(plan, tensors, flat)
+    assert to_np(flat).tobytes() == O.pack_flat(oplan, [to_np(t) for t in tensors]).tobytes()
+    assert _guards_intact(big, plan.G, 7.0)
+    outs = [_guarded(n, dtype, 7.0) for n in numel]
+    B.ws_unpack(plan, flat, [o[1] for o in outs])
+    for (bg, o), t, n in zip(outs, tensors, numel):
+        assert torch.equal(o, t) and _guards_intact(bg, n, 7.0)
+
+
+@pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb", "lars"])
+@pytest.mark.parametrize("R", [1, 3, 8, 40])
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+def test_concat_update_matches_oracle_on_both_routes(opt, R, gdtype):
+    wl, w, m, v, g = _model(CONCAT_SHAPES, R, gdtype, seed=R + 3, gstd=1e-3)
+    plan = B.Plan(CONCAT_SHAPES, R, 32, layout="concat")
+    oplan = O.FlatPlan(wl.numels, R, 32)
+    h = _lars_hyper() if opt == "lars" else _hyper(opt)
+    has_v = opt in ("adam", "lamb")
+    ow, om, ov, orho = _oracle_unsharded(opt, h, w, m, v, g)
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    valid = torch.from_numpy(oplan.tensor_map() >= 0).to(DEV)
+    for b in [pw, pm, pv] + pg:                      # pads may hold anything on entry
+        b[~valid] = float("nan")
+    fw, fm, fv = pw.clone(), pm.clone(), pv.clone()
+    ws = torch.zeros(max(16, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+    gath = torch.full((plan.G,), 3.0, dtype=torch.bfloat16, device=DEV)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv if has_v else None, B.make_hyper(opt, h), gath, ws)
+    tol = TOL_LAMB if opt in ("lamb", "lars") else TOL_FP32
+    for name, buf, ref in (("w", pw, ow), ("m", pm, om), ("v", pv, ov)):
+        if name == "v" and not has_v:
+            continue
+        for t, (a, b) in enumerate(zip(O.unpack_flat(oplan, to_np(buf)), ref)):
+            assert err(a, b) <= (TOL_FP32 if name == "v" else tol), f"{name}[{t}]"
+        assert (to_np(buf).view(np.uint32)[~valid.cpu().numpy()] == 0).all()
+    assert torch.equal(gath, pw.to(torch.bfloat16))
+    if opt in ("lamb", "lars"):
+        rho = B.lamb_ratios(plan, ws).cpu().numpy().astype(np.float64)
+        assert (np.abs(rho - np.array(orho)) / np.array(orho)).max() <= TOL_LAMB
+    # formatting fused in: same state bit for bit, weights equal to the unpacked gathered buffer
+    outs = [torch.zeros(n, dtype=torch.bfloat16, device=DEV) for n in wl.numels]
+    ws2 = torch.zeros_like(ws)
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), fw, fm, fv if has_v else None, B.make_hyper(opt, h),
+                      B.TensorTable(plan, [outs]), ws2)
+    assert torch.equal(fw, pw) and torch.equal(fm, pm)
+    ref = [torch.zeros_like(o) for o in outs]
+    B.ws_unpack(plan, gath, ref)
+    for a, b in zip(outs, ref):
+        assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("slice_mode", [0, 1])
+def test_concat_shard_by_shard_equals_all_shards(slice_mode):
+    R = 6
+    wl, w, m, v, g = _model(CONCAT_SHAPES, R, seed=8)
+    plan = B.Plan(CONCAT_SHAPES, R, 32, layout="concat")
+    h = B.make_hyper("adam", _hyper("adam"))
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    aw, am, av = pw.clone(), pm.clone(), pv.clone()
+    ga, gb = torch.zeros(plan.G, device=DEV), torch.zeros(plan.G, device=DEV)
+    B.ws_shard_update(plan, -1, pg, aw, am, av, h, ga)
+    S = plan.S
+    for r in range(R):
+        sl = slice(r * S, (r + 1) * S)
+        gr = [b[sl] for b in pg] if slice_mode == 1 else pg
+        B.ws_shard_update(plan, r, gr, pw[sl], pm[sl], pv[sl], h, gb, slice_mode=slice_mode)
+    assert torch.equal(aw, pw) and torch.equal(am, pm) and torch.equal(av, pv) and torch.equal(ga, gb)
