@@ -327,8 +327,10 @@ def test_argument_errors_are_status_codes():
     assert call(2, g, s) == 1 and call(-2, g, s) == 1                       # r out of range
     bad = B.ws_state(buf.data_ptr() + 4, buf.data_ptr(), buf.data_ptr())
     assert call(0, g, bad) == 2                                              # misaligned
-    g3 = B.ws_grads(C.cast(ptrs, C.POINTER(C.c_void_p)), 3, 0, 0)
-    assert call(0, g3, s) == 1                                               # R mismatch
+    g0 = B.ws_grads(C.cast(ptrs, C.POINTER(C.c_void_p)), 0, 0, 0)
+    assert call(0, g0, s) == 1                                               # no gradient copies
+    gbig = B.ws_grads(C.cast(ptrs, C.POINTER(C.c_void_p)), 1025, 0, 0)
+    assert call(0, gbig, s) in (1, 7)                                        # more copies than the limit
     g1 = B.ws_grads(C.cast(ptrs, C.POINTER(C.c_void_p)), 2, 0, 1)
     assert call(-1, g1, s) == 1                                              # slice mode needs one shard
     gd = B.ws_grads(C.cast(ptrs, C.POINTER(C.c_void_p)), 2, 7, 0)
