@@ -42,6 +42,9 @@
 #ifndef WS_TUNE_U8
 #define WS_TUNE_U8 1
 #endif
+#ifndef WS_TUNE_RBL
+#define WS_TUNE_RBL 16   // gradients per tree block when R > 32
+#endif
 #ifndef WS_TUNE_U4
 #define WS_TUNE_U4 1     // 128-bit accesses per thread per pass
 #endif
@@ -305,7 +308,7 @@ __device__ __forceinline__ float block_sum(float x, float* smem /* kBlock/32 flo
 // One CTA handles one (shard, tile) work item; the grid is the item count, so the
 // hardware CTA scheduler walks the buffers front to back.
 template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED>
-__global__ void __launch_bounds__(kBlock, (VEC == 8 && GBF && !FUSED) ? WS_TUNE_MINB8 : WS_TUNE_MINB) update_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp) {
+__global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8) ? WS_TUNE_MINB8 : WS_TUNE_MINB) update_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp) {
     constexpr bool HAS_V = (OPT == K_ADAM || OPT == K_LAMB1 || OPT == K_LAMB2);
     constexpr bool READS_G = !is_phase2(OPT);     // phase 2 works from state (and the stored gradient sum)
     constexpr bool READS_M = (OPT != K_LARS1);
@@ -533,7 +536,8 @@ ws_status launch_r(const UpdParams& P, const void* const* gptrs, bool wide_ok, c
             if constexpr (GBF) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 8, 32, FUSED>(P, gptrs, st);
             return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 8, 32, FUSED>(P, gptrs, st);
         }
-        if (P.R <= 1024) return launch<OPT, GBF, OUT, 4, 1, 8, 1024, FUSED>(P, gptrs, st);
+        // many replicas make small shards and few CTAs: more loads in flight per thread
+        if (P.R <= 1024) return launch<OPT, GBF, OUT, 4, 1, WS_TUNE_RBL, 1024, FUSED>(P, gptrs, st);
         return WS_ERR_TOO_LARGE;
     }
 }
