@@ -737,3 +737,39 @@ def test_concat_shard_by_shard_equals_all_shards(slice_mode):
         gr = [b[sl] for b in pg] if slice_mode == 1 else pg
         B.ws_shard_update(plan, r, gr, pw[sl], pm[sl], pv[sl], h, gb, slice_mode=slice_mode)
     assert torch.equal(aw, pw) and torch.equal(am, pm) and torch.equal(av, pv) and torch.equal(ga, gb)
+
+
+def test_tiny_workload_against_stored_oracle_values():
+    # config "tiny": CPU-drawn inputs, GPU update (both routes), compared with the values the oracle
+    # wrote to tests/golden/tiny_adam_expected.txt
+    import os
+    wl = W.tiny()
+    w, m, v = W.make_state(wl, "cpu")
+    g = W.make_grads(wl, "cpu")
+    w, m, v = ([x.to(DEV) for x in lst] for lst in (w, m, v))
+    g = [[x.to(DEV) for x in gk] for gk in g]
+    plan = B.Plan(wl.shapes, wl.R, 32)
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    fw, fm, fv = pw.clone(), pm.clone(), pv.clone()
+    hy = B.make_hyper(wl.opt, wl.hyper)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv, hy)
+    outs = [torch.zeros_like(x) for x in w]
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), fw, fm, fv, hy, B.TensorTable(plan, [outs]))
+    assert torch.equal(fw, pw) and torch.equal(fm, pm) and torch.equal(fv, pv)
+    rows = {}
+    with open(os.path.join(os.path.dirname(__file__), "golden", "tiny_adam_expected.txt")) as f:
+        for line in f:
+            if not line.startswith("#"):
+                p = line.split()
+                rows[(p[0], int(p[1]))] = (int(p[2]), float(p[3]), float(p[4]), [float.fromhex(h) for h in p[5:9]])
+    for name, buf in (("w", pw), ("m", pm), ("v", pv)):
+        got = [torch.zeros_like(x) for x in w]
+        B.ws_unpack(plan, buf, got)
+        for t, x in enumerate(got):
+            x = to_np(x).astype(np.float64)
+            n, s, s2, picks = rows[(name, t)]
+            rms = np.sqrt(s2 / n)
+            assert x.size == n
+            assert abs(np.sum(x * x) - s2) <= 4e-6 * s2
+            for i, ref in zip((0, n // 3, 2 * n // 3, n - 1), picks):
+                assert abs(x[i] - ref) <= TOL_FP32 * max(abs(ref), rms), (name, t, i)

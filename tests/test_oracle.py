@@ -645,3 +645,34 @@ def test_flat_sharded_equals_unsharded(opt, R):
                 assert (np.abs(a.astype(np.float64) - b) <= np.spacing(np.abs(a))).all()
     assert (pw.view(np.uint32)[~valid] == 0).all() and (pm.view(np.uint32)[~valid] == 0).all()
     np.testing.assert_array_equal(gathered, O.f32_to_bf16_bits(pw))
+
+
+def _tiny_expected():
+    rows = {}
+    with open(os.path.join(GOLDEN, "tiny_adam_expected.txt")) as f:
+        for line in f:
+            if line.startswith("#"):
+                continue
+            p = line.split()
+            rows[(p[0], int(p[1]))] = (int(p[2]), float(p[3]), float(p[4]), [float.fromhex(h) for h in p[5:9]])
+    return rows
+
+
+def test_oracle_reproduces_the_stored_tiny_result():
+    # regression pin: values written by tests/golden/make_tiny_expected.py (oracle only)
+    wl = W.tiny()
+    w, m, v = [[x.numpy() for x in lst] for lst in W.make_state(wl, "cpu")]
+    g = [[x.numpy() for x in gk] for gk in W.make_grads(wl, "cpu")]
+    O.update_unsharded(O.make_hyper(wl.opt, wl.hyper), g, w, m, v)
+    rows = _tiny_expected()
+    for name, lst in (("w", w), ("m", m), ("v", v)):
+        for t, x in enumerate(lst):
+            n, s, s2, picks = rows[(name, t)]
+            assert x.size == n
+            # (a relative tolerance, not bit equality: the CPU random generator's vector maths may
+            # differ in the last bit between processor generations)
+            rms = np.sqrt(s2 / n)
+            assert abs(float((x.astype(np.float64) ** 2).sum()) - s2) <= 1e-6 * s2
+            assert abs(float(x.astype(np.float64).sum()) - s) <= 1e-6 * rms * n
+            for i, ref in zip((0, n // 3, 2 * n // 3, n - 1), picks):
+                assert abs(float(x[i]) - ref) <= 1e-6 * max(abs(ref), rms)
