@@ -773,3 +773,51 @@ def test_tiny_workload_against_stored_oracle_values():
             assert abs(np.sum(x * x) - s2) <= 4e-6 * s2
             for i, ref in zip((0, n // 3, 2 * n // 3, n - 1), picks):
                 assert abs(x[i] - ref) <= TOL_FP32 * max(abs(ref), rms), (name, t, i)
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_randomised_configurations_on_both_routes(case):
+    """Random tensor lists, shard and copy counts, alignments, tile sizes, dtypes, optimizers and
+    layouts: the separate-kernel route against the oracle's plain definition, the fused route
+    bit-equal to the separate-kernel route."""
+    rng = np.random.default_rng(1000 + case)
+    T = int(rng.integers(1, 14))
+    numel = [int(x) for x in rng.choice([0, 1, 5, 8, 33, 250, 1023, 2048, 4100, 9001, 30011], T)]
+    if sum(numel) == 0:
+        numel[0] = 17
+    shapes = [(n,) for n in numel]
+    M = int(rng.choice([1, 2, 3, 4, 7, 8, 12, 40]))
+    K = M * int(rng.choice([1, 1, 2]))                     # sometimes more copies than shards
+    A = int(rng.choice([8, 32, 128]))
+    tile = int(rng.choice([0, 1024, 2048]))
+    opt = str(rng.choice(["sgdm", "adam", "lamb", "lars"]))
+    gdtype = torch.bfloat16 if rng.integers(2) else torch.float32
+    odtype = torch.bfloat16 if rng.integers(2) else torch.float32
+    layout = "concat" if rng.integers(2) else "per_tensor"
+    wl, w, m, v, g = _model(shapes, K, gdtype, seed=case, gstd=1e-3)
+    plan = B.Plan(shapes, M, A, tile, layout=layout)
+    h = _lars_hyper() if opt == "lars" else _hyper(opt)
+    has_v = opt in ("adam", "lamb")
+    ow, om, ov, _ = _oracle_unsharded(opt, h, w, m, v, g)
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    fw, fm, fv = pw.clone(), pm.clone(), pv.clone()
+    ws = torch.zeros(max(16, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+    gath = torch.zeros(plan.G, dtype=odtype, device=DEV)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv if has_v else None, B.make_hyper(opt, h), gath, ws)
+    tol = TOL_LAMB if opt in ("lamb", "lars") else TOL_FP32
+    for name, buf, ref in (("w", pw, ow), ("m", pm, om), ("v", pv, ov)):
+        if name == "v" and not has_v:
+            continue
+        got = [torch.zeros_like(x) for x in w]
+        B.ws_unpack(plan, buf, got)
+        for t, (a, b) in enumerate(zip(got, ref)):
+            assert err(to_np(a), b) <= (TOL_FP32 if name == "v" else tol), (name, t)
+    outs = [torch.full((n,), 9.0, dtype=odtype, device=DEV) for n in numel]
+    ws2 = torch.zeros_like(ws)
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), fw, fm, fv if has_v else None, B.make_hyper(opt, h),
+                      B.TensorTable(plan, [outs]), ws2)
+    assert torch.equal(fw, pw) and torch.equal(fm, pm) and (not has_v or torch.equal(fv, pv))
+    ref = [torch.zeros_like(o) for o in outs]
+    B.ws_unpack(plan, gath, ref)
+    for a, b in zip(outs, ref):
+        assert torch.equal(a, b)

@@ -125,3 +125,27 @@ def test_calls_fail_cleanly_before_upload():
     assert L.ws_shard_update(None, 0, C.byref(g), C.byref(s), C.byref(hy), None, None, 0, None) == 1
     assert plan.workspace_bytes("adam") == 0 and plan.workspace_bytes("sgdm") == 0
     assert plan.workspace_bytes("lamb") >= 4 * 1 + 16 * 1 + 8 * 2 * plan.ntiles
+
+
+def test_planner_fuzz_against_oracle():
+    # random tensor lists, shard counts, alignments, tile sizes and both layouts: the host planner and
+    # the oracle's planners must agree on every offset, and the tiles must cover every shard exactly
+    rng = np.random.default_rng(2004)
+    for case in range(120):
+        T = int(rng.integers(1, 40))
+        numel = [int(x) for x in rng.choice([0, 1, 2, 7, 8, 31, 32, 33, 255, 1000, 4097, 70001], T)]
+        R = int(rng.choice([1, 2, 3, 5, 8, 16, 33, 128, 1024]))
+        A = int(rng.choice([8, 16, 32, 64, 256]))
+        tile = int(rng.choice([0, 1024, 2048, 4096]))
+        shapes = [(n,) for n in numel]
+        per = B.Plan(shapes, R, A, tile, upload=False)
+        ref = O.Plan(numel, R, A)
+        assert (per.S, per.N) == (ref.S, ref.N)
+        assert [(s.piece, s.shard_off) for s in per.segments()] == list(zip(ref.piece.tolist(), ref.off.tolist()))
+        cat = B.Plan(shapes, R, A, tile, upload=False, layout="concat")
+        fref = O.FlatPlan(numel, R, A)
+        assert (cat.S, cat.N) == (fref.S, fref.N)
+        assert [s.shard_off for s in cat.segments()] == fref.cat[:-1].tolist()
+        assert cat.G <= per.G
+        k = tile or 8192
+        assert cat.ntiles >= R * (-(-cat.S // k)) if cat.S else cat.ntiles == 0
