@@ -67,6 +67,8 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-large", action="store_true",
+                    help="skip the short fused-route runs of the large workloads that are appended to the line")
     return ap.parse_args()
 
 
@@ -543,6 +545,10 @@ def run_ours(args):
         from oracle import ws_oracle as O
         O.build()
         line["cpu_baseline"] = cpu_baseline(wl, args.align)
+    if world == 1 and not args.no_large and args.workload == "resnet50" and not (args.R or args.opt):
+        del pw, pm, pv, g_arena, g_views, w_arena, w_views, pg, gathered, gtab, wtab
+        torch.cuda.empty_cache()
+        line["large_workloads"] = large_workload_rows(args)
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
@@ -604,6 +610,26 @@ def run_shard_window(args, wl, plan, dev, world, rank):
         "gpu_launches": K * len(window), "e2e": None,
     }
     print(json.dumps(line))
+
+
+def large_workload_rows(args):
+    """Short fused-route runs of the large model-shaped workloads (each in its own process so that its
+    memory is returned), summarised next to the headline workload."""
+    rows = []
+    for name, extra in (("transformer", ["--R", "8"]), ("bert_large", []), ("decoder_1p5b", [])):
+        cmd = [sys.executable, os.path.abspath(__file__), "--workload", name, *extra, "--path", "fused", "--steps", "30",
+               "--warmup", "5", "--no-e2e", "--no-cpu-baseline", "--no-large", "--align", str(args.align)]
+        try:
+            r = subprocess.run(cmd, capture_output=True, text=True, timeout=600)
+            j = json.loads(r.stdout.strip().splitlines()[-1])
+            rf = j["roofline"]
+            rows.append({"workload": j["config"]["workload"], "value": j["value"], "unit": UNIT,
+                         "ms_per_step": j["ms_per_step"], "gpu_launches_per_step": j["gpu_launches"] // j["steps"],
+                         "achieved_gbs": rf["achieved"], "frac_of_measured_peak": rf["frac"],
+                         "frac_of_nominal_8TBs": rf["frac_of_nominal_8TBs"], "clocks": j["clocks"]})
+        except Exception as e:      # a failed side run must not lose the headline line
+            rows.append({"workload": name, "error": str(e)[:200]})
+    return rows
 
 
 def main():
