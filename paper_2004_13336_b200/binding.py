@@ -371,13 +371,15 @@ class TensorTable:
     """Device-resident table of tensor pointers for ws_fused_update: `sets` is a list of
     tensor lists (R gradient lists, or one weight list).  Keeps the device buffer alive."""
 
-    def __init__(self, plan: Plan, sets: Sequence[Sequence[torch.Tensor]]):
+    def __init__(self, plan: Plan, sets: Sequence[Sequence[torch.Tensor]], device=None):
         nsets = len(sets)
         flat = [t for s in sets for t in s]
         assert len(flat) == nsets * plan.T
         self.sets = [list(s) for s in sets]
         nbytes = lib().ws_tensor_table_bytes(plan.handle, nsets)
-        self.dev_buf = torch.empty(nbytes, dtype=torch.uint8, device=flat[0].device)
+        if device is None:      # the table itself always lives on the GPU
+            device = flat[0].device if flat[0].is_cuda else plan.dev_buf.device
+        self.dev_buf = torch.empty(nbytes, dtype=torch.uint8, device=device)
         self.c = ws_tensor_table()
         _check(lib().ws_tensor_table_upload(plan.handle, _ptr_array(flat), nsets, _dtype_code(flat[0].dtype),
                                             self.dev_buf.data_ptr(), nbytes, _stream(), C.byref(self.c)),
