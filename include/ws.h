@@ -272,6 +272,10 @@ ws_status ws_lamb_apply(const ws_plan* plan, int32_t r, const ws_state* state,
  *   together with the device buffer, while it is in use.  Every tensor pointer
  *   must be 16-byte aligned; 32-byte alignment of all of them lets the kernels
  *   use 256-bit accesses.
+ * The tensors may live in any memory the device can address, pinned host
+ * memory included: the kernel then pulls the gradients over PCIe itself and
+ * writes the weights back the same way, with no staging copy (the table
+ * itself must be in device memory).
  * ws_fused_update arguments: `grads` is a table of R sets (the R replicas'
  * gradient lists), `weights` a table of one set (the weight tensors that
  * receive the result), `state` as for ws_shard_update (r >= 0: one shard;
