@@ -165,7 +165,7 @@ typedef struct {
  * (Section 2.2: auxiliary variables stay sharded across iterations).
  * With r >= 0 each pointer is the S-element shard r.  With r == -1 each is
  * the shard-major [R][S] buffer of all shards.  Updated in place; pads are
- * written +0.  v is unused (may be NULL) for WS_SGDM. */
+ * written +0.  v is unused (may be NULL) for WS_SGDM and WS_LARS. */
 typedef struct {
     void* w;
     void* m;

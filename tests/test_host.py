@@ -149,3 +149,17 @@ def test_planner_fuzz_against_oracle():
         assert cat.G <= per.G
         k = tile or 8192
         assert cat.ntiles >= R * (-(-cat.S // k)) if cat.S else cat.ntiles == 0
+
+
+def test_header_is_plain_c_and_links_from_c(tmp_path):
+    """include/ws.h compiles as strict C99 and a C program linked against libws.so can plan
+    (host-only entry points; the paper's worked sharding numbers are checked inside it)."""
+    import subprocess
+    exe = tmp_path / "abi_host_check"
+    src = os.path.join(ROOT, "tests", "c", "abi_host_check.c")
+    cmd = ["gcc", "-std=c99", "-Wall", "-Wextra", "-Werror", "-pedantic", "-I", os.path.join(ROOT, "include"),
+           src, "-o", str(exe), "-L", os.path.dirname(B.LIB_PATH), "-lws", f"-Wl,-rpath,{os.path.dirname(B.LIB_PATH)}"]
+    subprocess.run(cmd, check=True)
+    r = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert r.returncode == 0, r.stdout + r.stderr
+    assert "piece 73728" in r.stdout and "piece 9216" in r.stdout
