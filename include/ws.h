@@ -293,6 +293,11 @@ size_t ws_tensor_table_bytes(const ws_plan* plan, int32_t nsets);
 ws_status ws_tensor_table_upload(const ws_plan* plan, const void* const* ptrs, int32_t nsets,
                                  ws_dtype dtype, void* dev_buf, size_t bytes, void* stream,
                                  ws_tensor_table* out);
+/* ws_pack of every set of a tensor table in ONE launch: set k goes to flats[k] (host array of
+ * table->nsets device pointers, G elements of the table's dtype each).  Same result as nsets calls
+ * of ws_pack; meant for the R gradient lists of a step on the separate-kernel route. */
+ws_status ws_pack_sets(const ws_plan* plan, const ws_tensor_table* table, void* const* flats,
+                       void* stream);
 ws_status ws_fused_update(const ws_plan* plan, int32_t r, const ws_tensor_table* grads,
                           const ws_state* state, const ws_hyper* hyper,
                           const ws_tensor_table* weights, void* workspace, size_t workspace_bytes,

@@ -79,7 +79,7 @@ EXPORTS = [
     "ws_last_cuda_error", "ws_plan_arena_elems", "ws_plan_arena_offsets", "ws_step_host",
     "ws_static_scratch_bytes", "ws_lamb_update_static_scratch",
     "ws_tensor_table_bytes", "ws_tensor_table_upload", "ws_fused_update",
-    "ws_plan_create_layout", "ws_plan_layout",
+    "ws_plan_create_layout", "ws_plan_layout", "ws_pack_sets",
 ]
 
 _lib = None
@@ -150,6 +150,8 @@ def lib() -> C.CDLL:
     L.ws_tensor_table_upload.restype = C.c_int
     L.ws_tensor_table_upload.argtypes = [vp, vpp, C.c_int32, C.c_int, vp, C.c_size_t, vp,
                                          C.POINTER(ws_tensor_table)]
+    L.ws_pack_sets.restype = C.c_int
+    L.ws_pack_sets.argtypes = [vp, C.POINTER(ws_tensor_table), vpp, vp]
     L.ws_fused_update.restype = C.c_int
     L.ws_fused_update.argtypes = [vp, C.c_int32, C.POINTER(ws_tensor_table), C.POINTER(ws_state),
                                   C.POINTER(ws_hyper), C.POINTER(ws_tensor_table), vp, C.c_size_t, vp]
@@ -393,3 +395,8 @@ def ws_fused_update(plan: Plan, r: int, grads: TensorTable, w, m, v, hyper: ws_h
                                  workspace.data_ptr() if workspace is not None else None,
                                  workspace.numel() * workspace.element_size() if workspace is not None else 0,
                                  _stream()), "ws_fused_update")
+
+
+def ws_pack_sets(plan: Plan, table: TensorTable, flats):
+    """All sets of a tensor table packed in one launch (set k -> flats[k])."""
+    _check(lib().ws_pack_sets(plan.handle, C.byref(table.c), _ptr_array(flats), _stream()), "ws_pack_sets")

@@ -77,6 +77,50 @@ __global__ void __launch_bounds__(kBlock) pack_kernel(PackParams P, const __grid
     }
 }
 
+// All gradient lists of a step in one launch: set k's tensors (found through the device table
+// [T][nsets]) go to flats.p[k].  Work items are set-major, so each set is walked front to back.
+struct FlatPtrs {
+    void* p[kPtrChunk];
+};
+
+template <int EB>
+__global__ void __launch_bounds__(kBlock) pack_sets_kernel(PackParams P, const void* const* __restrict__ table, int nsets,
+                                                           const __grid_constant__ FlatPtrs flats) {
+    constexpr int EPV = 16 / EB;
+    const long long total = P.nitems * nsets;
+    for (long long gi = blockIdx.x; gi < total; gi += gridDim.x) {
+        const int k = (int)(gi / P.nitems);
+        const long long item = gi - (long long)k * P.nitems;
+        long long r = P.concat ? 0 : item / P.ntl;
+        const WsTile tl = P.tiles[item - r * P.ntl];
+        if (P.concat) r = tl.shard;
+        const char* tn = (const char*)table[(long long)tl.seg * nsets + k] + (r * tl.piece + tl.poff) * EB;
+        long long nv = tl.vt - r * tl.piece;
+        nv = nv < 0 ? 0 : (nv > tl.len ? (long long)tl.len : nv);
+        char* fl = (char*)flats.p[k] + (r * P.S + tl.pos) * EB;
+        const int nvec = tl.len / EPV;
+        for (int i = threadIdx.x; i < nvec; i += kBlock) {
+            const long long e0 = (long long)i * EPV;
+            if (e0 + EPV <= nv) {
+                st_stream((uint4*)(fl) + i, ld_stream((const uint4*)(tn) + i));
+            } else if (e0 >= nv) {
+                st_stream((uint4*)(fl) + i, make_uint4(0, 0, 0, 0));
+            } else {
+                const int kk = (int)(nv - e0);
+                if (EB == 4) {
+                    unsigned int* f = (unsigned int*)fl + e0;
+                    const unsigned int* t = (const unsigned int*)tn + e0;
+                    for (int j = 0; j < EPV; ++j) f[j] = j < kk ? t[j] : 0u;
+                } else {
+                    unsigned short* f = (unsigned short*)fl + e0;
+                    const unsigned short* t = (const unsigned short*)tn + e0;
+                    for (int j = 0; j < EPV; ++j) f[j] = j < kk ? t[j] : (unsigned short)0;
+                }
+            }
+        }
+    }
+}
+
 template <bool PACK>
 ws_status run(const ws_plan* p, void* const* tensor_ptrs, ws_dtype dtype, void* flat, void* stream) {
     if (!p || !tensor_ptrs || !flat) return WS_ERR_INVALID_ARG;
@@ -123,4 +167,34 @@ extern "C" ws_status ws_pack(const ws_plan* plan, const void* const* tensor_ptrs
 extern "C" ws_status ws_unpack(const ws_plan* plan, const void* flat, ws_dtype dtype, void* const* tensor_ptrs,
                                void* stream) {
     return run<false>(plan, tensor_ptrs, dtype, (void*)flat, stream);
+}
+
+extern "C" ws_status ws_pack_sets(const ws_plan* p, const ws_tensor_table* table, void* const* flats, void* stream) {
+    if (!p || !table || !table->dev || !flats) return WS_ERR_INVALID_ARG;
+    if (!p->d_tiles) return WS_ERR_NOT_UPLOADED;
+    if (table->T != p->T || table->nsets < 1 || table->nsets > kPtrChunk) return WS_ERR_INVALID_ARG;
+    if (table->dtype != WS_F32 && table->dtype != WS_BF16) return WS_ERR_DTYPE;
+    FlatPtrs fp;
+    for (int k = 0; k < table->nsets; ++k) {
+        if (!flats[k]) return WS_ERR_INVALID_ARG;
+        if (!ws_aligned16(flats[k])) return WS_ERR_ALIGNMENT;
+        fp.p[k] = flats[k];
+    }
+    PackParams P;
+    P.tiles = p->d_tiles;
+    P.tile_lo = 0;
+    P.ntl = p->ntiles;
+    P.concat = (p->layout == WS_LAYOUT_CONCAT);
+    P.nitems = P.concat ? P.ntl : P.ntl * p->R;
+    P.S = p->S;
+    P.seg_lo = 0;
+    long long grid = P.nitems * table->nsets;
+    if (grid < 1) return WS_OK;
+    if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (table->dtype == WS_F32)
+        pack_sets_kernel<4><<<(unsigned)grid, kBlock, 0, st>>>(P, (const void* const*)table->dev, table->nsets, fp);
+    else
+        pack_sets_kernel<2><<<(unsigned)grid, kBlock, 0, st>>>(P, (const void* const*)table->dev, table->nsets, fp);
+    return ws_check_launch("ws_pack_sets");
 }

@@ -821,3 +821,20 @@ def test_randomised_configurations_on_both_routes(case):
     B.ws_unpack(plan, gath, ref)
     for a, b in zip(outs, ref):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("layout", ["per_tensor", "concat"])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_pack_sets_equals_pack_per_set(layout, dtype):
+    R = 5
+    wl, w, m, v, g = _model(SHAPES, R, dtype, seed=13)
+    plan = B.Plan(SHAPES, R, 32, layout=layout)
+    one = []
+    for gk in g:
+        b = torch.empty(plan.G, dtype=dtype, device=DEV)
+        B.ws_pack(plan, gk, b)
+        one.append(b)
+    many = [torch.full((plan.G,), 3.0, dtype=dtype, device=DEV) for _ in range(R)]
+    B.ws_pack_sets(plan, B.TensorTable(plan, g), many)
+    for a, b in zip(one, many):
+        assert torch.equal(a, b)
