@@ -135,7 +135,7 @@ ws_status run(const ws_plan* p, void* const* tensor_ptrs, ws_dtype dtype, void* 
     cudaStream_t st = (cudaStream_t)stream;
     for (int seg_lo = 0; seg_lo < p->T; seg_lo += kPtrChunk) {
         const int seg_hi = seg_lo + kPtrChunk < p->T ? seg_lo + kPtrChunk : p->T;
-        PtrChunk tab;
+        PtrChunk tab = {};
         for (int t = seg_lo; t < seg_hi; ++t) tab.p[t - seg_lo] = tensor_ptrs[t];
         PackParams P;
         P.tiles = p->d_tiles;
@@ -174,7 +174,7 @@ extern "C" ws_status ws_pack_sets(const ws_plan* p, const ws_tensor_table* table
     if (!p->d_tiles) return WS_ERR_NOT_UPLOADED;
     if (table->T != p->T || table->nsets < 1 || table->nsets > kPtrChunk) return WS_ERR_INVALID_ARG;
     if (table->dtype != WS_F32 && table->dtype != WS_BF16) return WS_ERR_DTYPE;
-    FlatPtrs fp;
+    FlatPtrs fp = {};
     for (int k = 0; k < table->nsets; ++k) {
         if (!flats[k]) return WS_ERR_INVALID_ARG;
         if (!ws_aligned16(flats[k])) return WS_ERR_ALIGNMENT;
