@@ -838,3 +838,31 @@ def test_pack_sets_equals_pack_per_set(layout, dtype):
     B.ws_pack_sets(plan, B.TensorTable(plan, g), many)
     for a, b in zip(one, many):
         assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("opt", ["lamb", "lars"])
+def test_zero_norm_tensors_get_ratio_one(opt):
+    # the degenerate cases of the norm-based optimizers: an all-zero weight tensor and a tensor
+    # whose update direction (LAMB) or gradient (LARS) is all zero
+    shapes = [(300, 7), (5000,), (64,), (2100,)]
+    R = 3
+    wl, w, m, v, g = _model(shapes, R, seed=21, gstd=1e-3)
+    w[1].zero_()                                   # zero weight norm
+    for gk in g:
+        gk[3].zero_()                              # zero gradient ...
+    m[3].zero_()
+    v[3].zero_()                                   # ... and zero moments
+    h = _lars_hyper() if opt == "lars" else _hyper("lamb", weight_decay=0.0)
+    plan = B.Plan(shapes, R, 32)
+    oplan = O.Plan(wl.numels, R, 32)
+    ow, om, ov, orho = _oracle_unsharded(opt, h, w, m, v, g)
+    assert orho[1] == 1.0 and orho[3] == 1.0
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    ws = torch.zeros(plan.workspace_bytes(opt), dtype=torch.uint8, device=DEV)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv if opt == "lamb" else None, B.make_hyper(opt, h), None, ws)
+    rho = B.lamb_ratios(plan, ws).cpu().numpy()
+    assert rho[1] == 1.0 and rho[3] == 1.0
+    _compare_state(oplan, "sgdm", [pw, pm], [ow, om], TOL_LAMB)
+    if opt == "lamb":                              # (LARS still applies its weight decay at rate 1)
+        got = O.unpack(oplan, to_np(pw))
+        assert (got[3] == to_np(w[3])).all()       # nothing to apply: weights unchanged bit for bit
