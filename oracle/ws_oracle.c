@@ -35,6 +35,16 @@
  * of the paper's ResNet-50 runs, Table 1; formula from the LARS paper it cites):
  * local rate lambda = eta ||w|| / (||g|| + beta ||w||) per tensor (1 when either
  * norm is zero), v' = mu v + lr lambda (g + beta w), w' = w - v'.
+ * Adafactor (the paper's second example of an optimizer with reduce operators, Section 4.1;
+ * formula from the Adafactor paper it cites, the variant with factored second moments,
+ * update clipping, relative step size, increasing decay and no momentum): for a
+ * rows x cols matrix with summed gradient G and beta = 1 - t^-c,
+ *   Rv' = beta Rv + (1-beta) rowsum(G^2 + eps1),  Cv' = beta Cv + (1-beta) colsum(G^2 + eps1),
+ *   V = Rv' Cv'^T / sum(Rv'),  U = G / sqrt(V),  U^ = U / max(1, RMS(U)/d),
+ *   w' = w - max(eps2, RMS(w)) min(lr, 1/sqrt(t)) U^;
+ * a vector keeps the full v' = beta v + (1-beta)(g^2 + eps1) and uses V = v'.  A tensor of
+ * more than two dimensions is the matrix of its last dimension (columns) against all the
+ * leading ones together (rows).
  */
 #include <math.h>
 #include <stdint.h>
@@ -49,6 +59,7 @@ typedef struct {
     double lr, beta1, beta2, eps, weight_decay, momentum, grad_scale;
     int64_t step; /* 1-based index of the update being applied */
     double trust_coeff; /* LARS eta */
+    double eps2, clip_threshold, decay_exponent; /* Adafactor: eps_2, d, c of beta2_t = 1 - t^-c */
 } wso_hyper;
 
 /* ---------------------------------------------------------------- bf16 -- */
@@ -528,6 +539,164 @@ void wso_sharded_update_map(const wso_hyper *h, int32_t T, const int32_t *tmap, 
     free(ratio);
     free(u);
     free(part);
+}
+
+/* ------------------------------------------------------------- Adafactor -- */
+
+static double af_decay(const wso_hyper *h) { return 1.0 - pow((double)h->step, -h->decay_exponent); }
+
+static double af_rho(const wso_hyper *h) {
+    double r = 1.0 / sqrt((double)h->step);
+    return h->lr < r ? h->lr : r;
+}
+
+/* Unsharded Adafactor on one whole tensor, seen as rows x cols (cols == 0: a vector of `rows`
+ * elements, not factored).  All-reduce (sum) the K gradient copies first.  vr: rows floats
+ * (the vector's full second moment when cols == 0), vc: cols floats.  In place.
+ * info (may be NULL): [0] step size alpha, [1] RMS(U), [2] sum(Rv'). */
+void wso_adafactor_tensor(const wso_hyper *h, int64_t rows, int64_t cols, int32_t K,
+                          const void *const *grads, int32_t g_dtype, float *w, float *vr, float *vc,
+                          double *info) {
+    const int64_t n = cols > 0 ? rows * cols : rows;
+    double *g = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    double *u = (double *)malloc(sizeof(double) * (size_t)(n > 0 ? n : 1));
+    const double beta = af_decay(h);
+    double sw = 0.0;
+    for (int64_t i = 0; i < n; ++i) {
+        double s = 0.0;
+        for (int32_t k = 0; k < K; ++k) s += load_grad(grads[k], g_dtype, i);
+        g[i] = s * h->grad_scale;
+        sw += (double)w[i] * (double)w[i];
+    }
+    double sum_r = 0.0;
+    if (cols > 0) {
+        double *rv = (double *)malloc(sizeof(double) * (size_t)rows);
+        double *cv = (double *)malloc(sizeof(double) * (size_t)cols);
+        for (int64_t i = 0; i < rows; ++i) {
+            double s = 0.0;
+            for (int64_t j = 0; j < cols; ++j) s += g[i * cols + j] * g[i * cols + j] + h->eps;
+            rv[i] = beta * (double)vr[i] + (1.0 - beta) * s;
+            vr[i] = (float)rv[i];
+            sum_r += rv[i];
+        }
+        for (int64_t j = 0; j < cols; ++j) {
+            double s = 0.0;
+            for (int64_t i = 0; i < rows; ++i) s += g[i * cols + j] * g[i * cols + j] + h->eps;
+            cv[j] = beta * (double)vc[j] + (1.0 - beta) * s;
+            vc[j] = (float)cv[j];
+        }
+        for (int64_t i = 0; i < rows; ++i)
+            for (int64_t j = 0; j < cols; ++j) u[i * cols + j] = g[i * cols + j] / sqrt(rv[i] * cv[j] / sum_r);
+        free(rv);
+        free(cv);
+    } else {
+        for (int64_t i = 0; i < n; ++i) {
+            double v = beta * (double)vr[i] + (1.0 - beta) * (g[i] * g[i] + h->eps);
+            vr[i] = (float)v;
+            u[i] = g[i] / sqrt(v);
+        }
+    }
+    double su = 0.0;
+    for (int64_t i = 0; i < n; ++i) su += u[i] * u[i];
+    const double rms_u = n > 0 ? sqrt(su / (double)n) : 0.0;
+    const double rms_w = n > 0 ? sqrt(sw / (double)n) : 0.0;
+    const double clip = rms_u / h->clip_threshold > 1.0 ? rms_u / h->clip_threshold : 1.0;
+    const double alpha = (h->eps2 > rms_w ? h->eps2 : rms_w) * af_rho(h);
+    for (int64_t i = 0; i < n; ++i) w[i] = (float)((double)w[i] - alpha * (u[i] / clip));
+    if (info) { info[0] = alpha; info[1] = rms_u; info[2] = sum_r; }
+    free(g);
+    free(u);
+}
+
+/* Sharded Adafactor, step by step on packed [R][S] buffers (conventions of wso_sharded_update;
+ * K gradient copies).  The row and column reduces collapse a dimension that the sharding cuts,
+ * so (Section 4.1, "Non-elementwise operators") every shard masks its pads by location, reduces
+ * what it holds, and the per-shard results are combined over the shards (ascending r): here the
+ * row sums, the column sums, sum w^2 and later sum U^2 of every tensor.  Tensor t is
+ * rows[t] x cols[t] (cols 0: vector); its factored state starts at fstate[foff[t]]: rows[t]
+ * floats then cols[t] floats.  info: T x 3 doubles as in wso_adafactor_tensor, or NULL. */
+void wso_adafactor_sharded(const wso_hyper *h, int32_t T, const int64_t *numel, const int64_t *piece,
+                           const int64_t *off, int64_t S, int32_t R, int32_t K,
+                           const void *const *gpacked, int32_t g_dtype, const int64_t *rows,
+                           const int64_t *cols, const int64_t *foff, float *w, float *fstate,
+                           void *gathered, int32_t out_dtype, double *info) {
+    const int64_t G = (int64_t)R * S;
+    const double beta = af_decay(h);
+    double *g = (double *)calloc((size_t)G + 1, sizeof(double));
+    double *u = (double *)calloc((size_t)G + 1, sizeof(double));
+    for (int32_t t = 0; t < T; ++t) {
+        const int64_t n = numel[t], nr = rows[t], nc = cols[t];
+        const int64_t nstate = nc > 0 ? nr + nc : nr;
+        float *vr = fstate + foff[t], *vc = vr + nr;
+        /* per-shard partial reduce results: [R][nstate] sums of g^2 + eps1, [R] sums of w^2 */
+        double *part = (double *)calloc((size_t)R * (size_t)(nstate > 0 ? nstate : 1), sizeof(double));
+        double *pw = (double *)calloc((size_t)R, sizeof(double));
+        for (int32_t r = 0; r < R; ++r)
+            for (int64_t q = 0; q < piece[t]; ++q) {
+                const int64_t e = (int64_t)r * piece[t] + q;        /* location in the full tensor */
+                const int64_t j = (int64_t)r * S + off[t] + q;
+                if (e >= n) continue;                                /* pad: identity of the sum */
+                double s = 0.0;
+                for (int32_t k = 0; k < K; ++k) s += load_grad(gpacked[k], g_dtype, j);
+                g[j] = s * h->grad_scale;
+                const double x = g[j] * g[j] + h->eps;
+                if (nc > 0) {
+                    part[(size_t)r * nstate + (size_t)(e / nc)] += x;
+                    part[(size_t)r * nstate + (size_t)(nr + e % nc)] += x;
+                } else {
+                    part[(size_t)r * nstate + (size_t)e] += x;
+                }
+                pw[r] += (double)w[j] * (double)w[j];
+            }
+        /* combine over shards, then the moving averages */
+        double *st = (double *)calloc((size_t)(nstate > 0 ? nstate : 1), sizeof(double));
+        double sw = 0.0, sum_r = 0.0;
+        for (int32_t r = 0; r < R; ++r) sw += pw[r];
+        for (int64_t i = 0; i < nstate; ++i) {
+            double s = 0.0;
+            for (int32_t r = 0; r < R; ++r) s += part[(size_t)r * nstate + (size_t)i];
+            st[i] = beta * (double)vr[i] + (1.0 - beta) * s;
+            vr[i] = (float)st[i];
+            if (nc > 0 && i < nr) sum_r += st[i];
+        }
+        (void)vc;
+        /* the update direction on every shard and its partial sum of squares */
+        double su = 0.0;
+        for (int32_t r = 0; r < R; ++r) {
+            double p = 0.0;
+            for (int64_t q = 0; q < piece[t]; ++q) {
+                const int64_t e = (int64_t)r * piece[t] + q;
+                const int64_t j = (int64_t)r * S + off[t] + q;
+                if (e >= n) continue;
+                const double V = nc > 0 ? st[e / nc] * st[nr + e % nc] / sum_r : st[e];
+                u[j] = g[j] / sqrt(V);
+                p += u[j] * u[j];
+            }
+            su += p;
+        }
+        const double rms_u = n > 0 ? sqrt(su / (double)n) : 0.0;
+        const double rms_w = n > 0 ? sqrt(sw / (double)n) : 0.0;
+        const double clip = rms_u / h->clip_threshold > 1.0 ? rms_u / h->clip_threshold : 1.0;
+        const double alpha = (h->eps2 > rms_w ? h->eps2 : rms_w) * af_rho(h);
+        for (int32_t r = 0; r < R; ++r)
+            for (int64_t q = 0; q < piece[t]; ++q) {
+                const int64_t e = (int64_t)r * piece[t] + q;
+                const int64_t j = (int64_t)r * S + off[t] + q;
+                w[j] = e < n ? (float)((double)w[j] - alpha * (u[j] / clip)) : 0.0f;
+            }
+        if (info) { info[3 * t] = alpha; info[3 * t + 1] = rms_u; info[3 * t + 2] = sum_r; }
+        free(part);
+        free(pw);
+        free(st);
+    }
+    if (gathered) {
+        if (out_dtype == WSO_BF16)
+            for (int64_t j = 0; j < G; ++j) ((uint16_t *)gathered)[j] = wso_f32_to_bf16(w[j]);
+        else
+            memcpy(gathered, w, sizeof(float) * (size_t)G);
+    }
+    free(g);
+    free(u);
 }
 
 int32_t wso_num_threads(void) {

@@ -20,9 +20,9 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "ws_oracle.c")
 _SO = os.path.join(_HERE, "libws_oracle.so")
 
-SGDM, ADAM, LAMB, LARS = 0, 1, 2, 3
+SGDM, ADAM, LAMB, LARS, ADAFACTOR = 0, 1, 2, 3, 4
 F32, BF16 = 0, 1
-OPT_CODE = {"sgdm": SGDM, "adam": ADAM, "lamb": LAMB, "lars": LARS}
+OPT_CODE = {"sgdm": SGDM, "adam": ADAM, "lamb": LAMB, "lars": LARS, "adafactor": ADAFACTOR}
 
 
 def build(force: bool = False) -> str:
@@ -39,14 +39,17 @@ class Hyper(C.Structure):
     _fields_ = [("opt", C.c_int32), ("lr", C.c_double), ("beta1", C.c_double),
                 ("beta2", C.c_double), ("eps", C.c_double), ("weight_decay", C.c_double),
                 ("momentum", C.c_double), ("grad_scale", C.c_double), ("step", C.c_int64),
-                ("trust_coeff", C.c_double)]
+                ("trust_coeff", C.c_double), ("eps2", C.c_double), ("clip_threshold", C.c_double),
+                ("decay_exponent", C.c_double)]
 
 
 def make_hyper(opt, hyper: dict) -> Hyper:
     code = OPT_CODE[opt] if isinstance(opt, str) else int(opt)
     return Hyper(code, hyper["lr"], hyper["beta1"], hyper["beta2"], hyper["eps"],
                  hyper["weight_decay"], hyper["momentum"], hyper["grad_scale"],
-                 int(hyper["step"]), float(hyper.get("trust_coeff", 0.001)))
+                 int(hyper["step"]), float(hyper.get("trust_coeff", 0.001)),
+                 float(hyper.get("eps2", 1e-3)), float(hyper.get("clip_threshold", 1.0)),
+                 float(hyper.get("decay_exponent", 0.8)))
 
 
 _lib = None
@@ -81,6 +84,14 @@ def lib():
         L.wso_lars_sharded.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p, C.c_int64,
                                        C.c_int32, C.c_int32, vpp, C.c_int32, C.c_void_p, C.c_void_p,
                                        C.c_void_p, C.c_int32, C.POINTER(C.c_double)]
+        L.wso_adafactor_tensor.restype = None
+        L.wso_adafactor_tensor.argtypes = [C.POINTER(Hyper), C.c_int64, C.c_int64, C.c_int32, vpp, C.c_int32,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_double)]
+        L.wso_adafactor_sharded.restype = None
+        L.wso_adafactor_sharded.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p, C.c_int64,
+                                            C.c_int32, C.c_int32, vpp, C.c_int32, i64p, i64p, i64p,
+                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32,
+                                            C.POINTER(C.c_double)]
         L.wso_plan_flat.restype = C.c_int64
         L.wso_plan_flat.argtypes = [i64p, C.c_int32, C.c_int32, C.c_int32, i64p]
         L.wso_sharded_update_map.restype = None
@@ -200,6 +211,55 @@ def sharded_update(h: Hyper, plan: Plan, gpacked: Sequence[np.ndarray], w: np.nd
         rho.ctypes.data_as(C.POINTER(C.c_double)),
         partials.ctypes.data_as(C.POINTER(C.c_double)))
     return gathered, rho, partials
+
+
+def factor_shapes(shapes):
+    """Adafactor's view of each tensor: (rows, cols) with cols the last dimension and rows all the
+    leading ones together; a vector (or scalar) is (numel, 0) and keeps a full second moment.
+    Returns int64 arrays rows, cols, foff (start of each tensor's factored state) and the total."""
+    rows, cols, foff, tot = [], [], [], 0
+    for s in shapes:
+        s = tuple(int(d) for d in s)
+        n = int(np.prod(s)) if len(s) else 1
+        if len(s) >= 2 and n > 0:
+            rows.append(n // s[-1]); cols.append(s[-1])
+        else:
+            rows.append(n); cols.append(0)
+        foff.append(tot)
+        tot += rows[-1] + cols[-1]
+    return _i64(rows), _i64(cols), _i64(foff), tot
+
+
+def adafactor_tensor(h: Hyper, grads: Sequence[np.ndarray], w: np.ndarray, vr: np.ndarray,
+                     vc: Optional[np.ndarray]):
+    """One whole tensor, unsharded.  w is (rows, cols) or 1-D; vr/vc fp32, in place.
+    Returns (alpha, rms_u, sum_vr)."""
+    if w.ndim >= 2:
+        cols = w.shape[-1]; rows = w.size // cols
+    else:
+        rows, cols = w.size, 0
+    info = (C.c_double * 3)()
+    lib().wso_adafactor_tensor(C.byref(h), rows, cols, len(grads), _ptrs(grads), _dtype_code(grads[0]),
+                               w.ctypes.data, vr.ctypes.data, vc.ctypes.data if vc is not None else None, info)
+    return tuple(info)
+
+
+def adafactor_sharded(h: Hyper, plan: Plan, shapes, gpacked: Sequence[np.ndarray], w: np.ndarray,
+                      fstate: np.ndarray, out_dtype: Optional[int] = None):
+    """Sharded route on packed [R][S] buffers; fstate is the concatenated factored state
+    (factor_shapes).  In place.  Returns (gathered or None, info[T][3])."""
+    rows, cols, foff, tot = factor_shapes(shapes)
+    assert fstate.size == tot and fstate.dtype == np.float32
+    info = np.zeros((plan.T, 3), dtype=np.float64)
+    gathered = None
+    if out_dtype is not None:
+        gathered = np.empty(plan.G, dtype=np.uint16 if out_dtype == BF16 else np.float32)
+    lib().wso_adafactor_sharded(
+        C.byref(h), plan.T, _p(plan.numel), _p(plan.piece), _p(plan.off), plan.S, plan.R,
+        len(gpacked), _ptrs(gpacked), _dtype_code(gpacked[0]), _p(rows), _p(cols), _p(foff),
+        w.ctypes.data, fstate.ctypes.data, gathered.ctypes.data if gathered is not None else None,
+        out_dtype if out_dtype is not None else F32, info.ctypes.data_as(C.POINTER(C.c_double)))
+    return gathered, info
 
 
 def shard_reduce(plan: Plan, r: int, gpacked: Sequence[np.ndarray], grad_scale: float = 1.0):
