@@ -50,7 +50,7 @@ typedef enum {
 } ws_status;
 
 typedef enum { WS_F32 = 0, WS_BF16 = 1 } ws_dtype;
-typedef enum { WS_SGDM = 0, WS_ADAM = 1, WS_LAMB = 2, WS_LARS = 3 } ws_opt;
+typedef enum { WS_SGDM = 0, WS_ADAM = 1, WS_LAMB = 2, WS_LARS = 3, WS_ADAFACTOR = 4 } ws_opt;
 
 #define WS_MAX_DIMS 8
 typedef struct {
@@ -165,7 +165,10 @@ typedef struct {
  * (Section 2.2: auxiliary variables stay sharded across iterations).
  * With r >= 0 each pointer is the S-element shard r.  With r == -1 each is
  * the shard-major [R][S] buffer of all shards.  Updated in place; pads are
- * written +0.  v is unused (may be NULL) for WS_SGDM and WS_LARS. */
+ * written +0.  v is unused (may be NULL) for WS_SGDM and WS_LARS.
+ * With WS_ADAFACTOR m is unused (may be NULL) and v is the factored second
+ * moment of every tensor, ws_plan_factored_elems() floats laid out as
+ * ws_plan_factored_layout() says; it is small and is not sharded. */
 typedef struct {
     void* w;
     void* m;
@@ -185,6 +188,20 @@ typedef struct {
  *            lambda_t = trust_coeff ||w_t|| / (||g_t|| + weight_decay ||w_t||)
  *            (1 if either norm is 0); m' = momentum m + lr lambda_t (g +
  *            weight_decay w);  w' = w - m'
+ *   WS_ADAFACTOR (the paper's other example of an optimizer with reduce
+ *            operators, Section 4.1; formula of the Adafactor paper it cites:
+ *            factored second moments, update clipping, relative step size,
+ *            no momentum).  Tensor t is a rows x cols matrix, cols its last
+ *            dimension and rows all leading ones together; with
+ *            beta = 1 - step^-decay_exponent:
+ *            Rv' = beta Rv + (1-beta) rowsum(g^2 + eps);
+ *            Cv' = beta Cv + (1-beta) colsum(g^2 + eps);
+ *            V = Rv' Cv'^T / sum(Rv');  U = g / sqrt(V);
+ *            w' = w - max(eps2, RMS(w_t)) min(lr, 1/sqrt(step))
+ *                     U / max(1, RMS(U_t) / clip_threshold).
+ *            A tensor of fewer than two dimensions keeps the full
+ *            v' = beta v + (1-beta)(g^2 + eps) and uses V = v'.
+ *            weight_decay must be 0.
  * `step` is the 1-based index of the update being applied.  Derived constants
  * are formed in double on the host and narrowed to fp32 for the kernels. */
 typedef struct {
@@ -192,6 +209,7 @@ typedef struct {
     double lr, beta1, beta2, eps, weight_decay, momentum, grad_scale;
     int64_t step;
     double trust_coeff; /* WS_LARS only (eta) */
+    double eps2, clip_threshold, decay_exponent; /* WS_ADAFACTOR only (1e-3, 1.0, 0.8 in its paper) */
 } ws_hyper;
 
 /* Where the updated weights go in the all-gather output layout (Section 2.2;
@@ -206,6 +224,17 @@ typedef struct {
     ws_dtype dtype;
 } ws_out;
 
+/* Adafactor's view of the plan's tensors (Section 4.1 names it as an optimizer
+ * whose reduces collapse some dimensions and pass others through).  Tensor t of
+ * two or more dimensions holds rows_t + cols_t floats of factored state (row
+ * accumulator, then column accumulator); a tensor of fewer dimensions holds
+ * numel_t floats.  ws_plan_factored_elems is the total F;
+ * ws_plan_factored_layout fills layout[3 t + 0..2] = {offset of tensor t's
+ * state in floats, rows_t, cols_t} with rows_t = numel_t, cols_t = 0 for the
+ * unfactored ones.  layout is a host array of 3 T entries.  Host only. */
+int64_t ws_plan_factored_elems(const ws_plan* plan);
+ws_status ws_plan_factored_layout(const ws_plan* plan, int64_t* layout);
+
 /* Bytes of caller-provided scratch (device, 16-byte aligned) the update needs:
  * 0 for WS_SGDM / WS_ADAM.  For WS_LAMB it holds, in this order:
  *   float  rho[T]            trust ratios written by ws_lamb_finalize
@@ -216,7 +245,13 @@ typedef struct {
  * so a caller can read rho and the norms back for logging.  WS_LARS uses the
  * same three arrays (rho holds the local rates, norms sum w^2 and sum g^2)
  * followed, at the next 256-byte boundary, by
- *   float  ghat[R][S]        the summed gradients kept from phase 1 for phase 2 */
+ *   float  ghat[R][S]        the summed gradients kept from phase 1 for phase 2
+ * WS_ADAFACTOR uses all four (rho holds the applied step size alpha_t / max(1,
+ * RMS(U_t)/d), norms sum w^2 and sum U^2) followed by
+ *   float  acc[F]            this step's row / column sums of g^2 + eps
+ *   float  fac[F]            1/sqrt factors of V for the two elementwise passes
+ *   float  alpha[T]          max(eps2, RMS(w_t)) min(lr, 1/sqrt(step))
+ * with F = ws_plan_factored_elems(). */
 size_t ws_workspace_bytes(const ws_plan* plan, ws_opt opt);
 
 /* Fused reduce + optimizer update + gathered-layout write for shard r
@@ -227,7 +262,16 @@ size_t ws_workspace_bytes(const ws_plan* plan, ws_opt opt);
  * auxiliaries).  With opt == WS_LAMB or WS_LARS only r == -1 is accepted here
  * (phase 1 over all shards, finalize, phase 2 over all shards): the per-tensor
  * ratio needs every shard's partial norms before any shard can apply
- * (Section 4.1). */
+ * (Section 4.1).
+ * WS_ADAFACTOR (r == -1 only) runs three passes: (1) reduce the gradients, keep
+ * the sum, and add every tile's partial row sums and column sums of g^2 + eps
+ * (pads masked by location) into acc - the sharding cuts rows and columns, so
+ * this stands where the paper combines the shards' partial reduce results with
+ * an all-reduce (Section 4.1, "Non-elementwise operators"); a finalize step
+ * forms Rv', Cv' and the step size; (2) sum U^2 per tensor; a second finalize
+ * forms the clipping; (3) apply.  The row and column sums use floating-point
+ * atomic adds, so Rv', Cv' and everything after them can differ in the last
+ * bits between runs. */
 ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_grads* grads,
                           const ws_state* state, const ws_hyper* hyper, const ws_out* out,
                           void* workspace, size_t workspace_bytes, void* stream);

@@ -19,7 +19,8 @@ LIB_PATH = os.path.join(_PKG, "libws.so")
 WS_OK = 0
 WS_F32, WS_BF16 = 0, 1
 WS_SGDM, WS_ADAM, WS_LAMB, WS_LARS = 0, 1, 2, 3
-OPT_CODE = {"sgdm": WS_SGDM, "adam": WS_ADAM, "lamb": WS_LAMB, "lars": WS_LARS}
+WS_ADAFACTOR = 4
+OPT_CODE = {"sgdm": WS_SGDM, "adam": WS_ADAM, "lamb": WS_LAMB, "lars": WS_LARS, "adafactor": WS_ADAFACTOR}
 WS_LAYOUT_PER_TENSOR, WS_LAYOUT_CONCAT = 0, 1
 LAYOUT_CODE = {"per_tensor": WS_LAYOUT_PER_TENSOR, "concat": WS_LAYOUT_CONCAT}
 WS_MAX_DIMS = 8
@@ -53,7 +54,8 @@ class ws_state(C.Structure):
 class ws_hyper(C.Structure):
     _fields_ = [("opt", C.c_int32), ("lr", C.c_double), ("beta1", C.c_double), ("beta2", C.c_double),
                 ("eps", C.c_double), ("weight_decay", C.c_double), ("momentum", C.c_double),
-                ("grad_scale", C.c_double), ("step", C.c_int64), ("trust_coeff", C.c_double)]
+                ("grad_scale", C.c_double), ("step", C.c_int64), ("trust_coeff", C.c_double),
+                ("eps2", C.c_double), ("clip_threshold", C.c_double), ("decay_exponent", C.c_double)]
 
 
 class ws_out(C.Structure):
@@ -80,6 +82,7 @@ EXPORTS = [
     "ws_static_scratch_bytes", "ws_lamb_update_static_scratch",
     "ws_tensor_table_bytes", "ws_tensor_table_upload", "ws_fused_update",
     "ws_plan_create_layout", "ws_plan_layout", "ws_pack_sets",
+    "ws_plan_factored_elems", "ws_plan_factored_layout",
 ]
 
 _lib = None
@@ -135,6 +138,10 @@ def lib() -> C.CDLL:
                                 C.POINTER(ws_out), vp, C.c_size_t, vp]
     L.ws_plan_arena_elems.restype = C.c_int64
     L.ws_plan_arena_elems.argtypes = [vp]
+    L.ws_plan_factored_elems.restype = C.c_int64
+    L.ws_plan_factored_elems.argtypes = [vp]
+    L.ws_plan_factored_layout.restype = C.c_int
+    L.ws_plan_factored_layout.argtypes = [vp, C.POINTER(C.c_int64)]
     L.ws_plan_arena_offsets.restype = C.c_int
     L.ws_plan_arena_offsets.argtypes = [vp, C.POINTER(C.POINTER(C.c_int64)), C.POINTER(C.c_int32)]
     L.ws_step_host.restype = C.c_int
@@ -209,7 +216,8 @@ def make_hyper(opt, hyper: dict) -> ws_hyper:
     code = OPT_CODE[opt] if isinstance(opt, str) else int(opt)
     return ws_hyper(code, hyper["lr"], hyper["beta1"], hyper["beta2"], hyper["eps"],
                     hyper["weight_decay"], hyper["momentum"], hyper["grad_scale"], int(hyper["step"]),
-                    float(hyper.get("trust_coeff", 0.001)))
+                    float(hyper.get("trust_coeff", 0.001)), float(hyper.get("eps2", 1e-3)),
+                    float(hyper.get("clip_threshold", 1.0)), float(hyper.get("decay_exponent", 0.8)))
 
 
 class Plan:
@@ -266,6 +274,17 @@ class Plan:
         """Per-tensor views of a tensor arena (host or device)."""
         return [arena[o:o + n] for o, n in zip(self.arena_offsets(), numels)]
 
+    @property
+    def factored_elems(self) -> int:
+        """Floats of Adafactor's factored second-moment state for all tensors."""
+        return lib().ws_plan_factored_elems(self._h)
+
+    def factored_layout(self):
+        """Per tensor (offset, rows, cols) of its factored state; cols == 0: unfactored, rows = numel."""
+        buf = (C.c_int64 * (3 * max(1, self.T)))()
+        _check(lib().ws_plan_factored_layout(self._h, buf), "ws_plan_factored_layout")
+        return [(buf[3 * t], buf[3 * t + 1], buf[3 * t + 2]) for t in range(self.T)]
+
     def workspace_bytes(self, opt) -> int:
         code = OPT_CODE[opt] if isinstance(opt, str) else int(opt)
         return lib().ws_workspace_bytes(self._h, code)
@@ -297,7 +316,7 @@ def _grads(gbufs: Sequence[torch.Tensor], slice_mode: int):
 
 
 def _state(w, m, v):
-    return ws_state(w.data_ptr(), m.data_ptr(), v.data_ptr() if v is not None else None)
+    return ws_state(w.data_ptr(), m.data_ptr() if m is not None else None, v.data_ptr() if v is not None else None)
 
 
 def _out(gathered):

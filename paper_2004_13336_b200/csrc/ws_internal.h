@@ -34,6 +34,16 @@ struct WsSegTiles {
     int tile_count;
 };
 
+// Adafactor's view of a tensor: foff = start of its factored state (floats); nrow row
+// accumulators (0 for an unfactored tensor) followed by ncol column accumulators (the full
+// second moment for an unfactored tensor, which is handled as a single row).
+struct WsSegAf {
+    long long foff;
+    long long nrow;
+    long long ncol;
+    long long numel;
+};
+
 struct ws_plan {
     int T = 0, R = 0, A = 0, K = 0;
     int layout = 0;                           // ws_layout
@@ -49,6 +59,9 @@ struct ws_plan {
     // device copies (caller-owned memory, set by ws_plan_upload)
     const WsTile* d_tiles = nullptr;
     const WsSegTiles* d_segtiles = nullptr;
+    std::vector<WsSegAf> segaf;
+    long long F = 0;                          // total factored-state floats
+    const WsSegAf* d_segaf = nullptr;
 };
 
 // Optimizer constants narrowed to fp32 for the kernels.
@@ -64,6 +77,10 @@ struct WsLambWs {
     size_t bytes;      // through the partials: what LAMB needs
     float* ghat;       // LARS only: [R][S] summed gradients, 256-byte aligned after the partials
     size_t bytes_lars; // through ghat: what LARS needs
+    float* acc;        // Adafactor: [F] this step's row / column sums
+    float* fac;        // Adafactor: [F] 1/sqrt factors of V
+    float* alpha;      // Adafactor: [T] step sizes
+    size_t bytes_af;   // through alpha: what Adafactor needs
 };
 WsLambWs ws_lamb_layout(const ws_plan* plan, void* workspace);
 

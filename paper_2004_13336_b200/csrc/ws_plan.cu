@@ -41,6 +41,30 @@ extern "C" const char* ws_status_string(ws_status s) {
     return "unknown status";
 }
 
+// Adafactor's matrix view of every tensor: columns = last dimension, rows = all leading
+// dimensions together; fewer than two dimensions: one row, no row accumulator.
+static void ws_matrix_views(ws_plan* p, const ws_tensor_desc* descs) {
+    p->segaf.resize(p->T);
+    long long foff = 0;
+    for (int t = 0; t < p->T; ++t) {
+        const ws_tensor_desc& d = descs[t];
+        const long long n = p->segs[t].numel;
+        WsSegAf a;
+        a.foff = foff;
+        a.numel = n;
+        if (d.ndim >= 2 && n > 0) {
+            a.ncol = d.dims[d.ndim - 1];
+            a.nrow = n / a.ncol;
+        } else {
+            a.nrow = 0;
+            a.ncol = n;
+        }
+        foff += a.nrow + a.ncol;
+        p->segaf[t] = a;
+    }
+    p->F = foff;
+}
+
 extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int32_t R,
                                     int32_t align_elems, int32_t tile_elems, ws_plan** out) {
     return ws_plan_create_layout(descs, T, R, align_elems, tile_elems, WS_LAYOUT_PER_TENSOR, out);
@@ -144,6 +168,7 @@ extern "C" ws_status ws_plan_create_layout(const ws_tensor_desc* descs, int32_t 
             }
             p->shard_tile_begin[R] = (long long)p->tiles.size();
             p->ntiles = (long long)p->tiles.size();
+            ws_matrix_views(p, descs);
             *out = p;
             return WS_OK;
         }
@@ -184,6 +209,7 @@ extern "C" ws_status ws_plan_create_layout(const ws_tensor_desc* descs, int32_t 
         }
         p->S = off;
         p->ntiles = (long long)p->tiles.size();
+        ws_matrix_views(p, descs);
     } catch (...) {
         delete p;
         return WS_ERR_INVALID_ARG;
@@ -211,7 +237,21 @@ static size_t round16(size_t x) { return (x + 15) & ~(size_t)15; }
 
 extern "C" size_t ws_plan_device_bytes(const ws_plan* p) {
     if (!p) return 0;
-    return round16(p->tiles.size() * sizeof(WsTile)) + round16(p->segtiles.size() * sizeof(WsSegTiles));
+    return round16(p->tiles.size() * sizeof(WsTile)) + round16(p->segtiles.size() * sizeof(WsSegTiles)) +
+           round16(p->segaf.size() * sizeof(WsSegAf));
+}
+
+extern "C" int64_t ws_plan_factored_elems(const ws_plan* p) { return p ? p->F : 0; }
+
+extern "C" ws_status ws_plan_factored_layout(const ws_plan* p, int64_t* layout) {
+    if (!p || !layout) return WS_ERR_INVALID_ARG;
+    for (int t = 0; t < p->T; ++t) {
+        const WsSegAf& a = p->segaf[t];
+        layout[3 * t] = a.foff;
+        layout[3 * t + 1] = a.nrow > 0 ? a.nrow : a.ncol;
+        layout[3 * t + 2] = a.nrow > 0 ? a.ncol : 0;
+    }
+    return WS_OK;
 }
 
 extern "C" ws_status ws_plan_upload(ws_plan* p, void* dev_buf, size_t bytes, void* stream) {
@@ -226,8 +266,12 @@ extern "C" ws_status ws_plan_upload(ws_plan* p, void* dev_buf, size_t bytes, voi
     e = cudaMemcpyAsync(base + round16(tb), p->segtiles.data(), p->segtiles.size() * sizeof(WsSegTiles),
                         cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return ws_cuda_fail(e, "ws_plan_upload(segments)");
+    const size_t ab = round16(tb) + round16(p->segtiles.size() * sizeof(WsSegTiles));
+    e = cudaMemcpyAsync(base + ab, p->segaf.data(), p->segaf.size() * sizeof(WsSegAf), cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return ws_cuda_fail(e, "ws_plan_upload(matrix views)");
     p->d_tiles = (const WsTile*)base;
     p->d_segtiles = (const WsSegTiles*)(base + round16(tb));
+    p->d_segaf = (const WsSegAf*)(base + ab);
     return WS_OK;
 }
 
@@ -245,6 +289,13 @@ WsLambWs ws_lamb_layout(const ws_plan* p, void* workspace) {
     o = (o + 255) & ~(size_t)255;
     L.ghat = (float*)(b + o);
     L.bytes_lars = o + sizeof(float) * (size_t)p->R * (size_t)p->S;
+    o = (L.bytes_lars + 255) & ~(size_t)255;
+    L.acc = (float*)(b + o);
+    o = (o + sizeof(float) * (size_t)p->F + 255) & ~(size_t)255;
+    L.fac = (float*)(b + o);
+    o = (o + sizeof(float) * (size_t)p->F + 255) & ~(size_t)255;
+    L.alpha = (float*)(b + o);
+    L.bytes_af = o + sizeof(float) * (size_t)p->T;
     return L;
 }
 
@@ -252,5 +303,6 @@ extern "C" size_t ws_workspace_bytes(const ws_plan* p, ws_opt opt) {
     if (!p) return 0;
     if (opt == WS_LAMB) return ws_lamb_layout(p, nullptr).bytes;
     if (opt == WS_LARS) return ws_lamb_layout(p, nullptr).bytes_lars;
+    if (opt == WS_ADAFACTOR) return ws_lamb_layout(p, nullptr).bytes_af;
     return 0;
 }

@@ -55,9 +55,18 @@ constexpr int kBlock = 256;
 // Kernel flavours.  The norm-based optimizers run as two phases around a finalize step:
 // phase 1 (K_LAMB1, K_LARS1) reduces the gradients and leaves per-tile partial sums of the
 // two norms; phase 2 (K_LAMB2, K_LARS2) applies the step with the per-tensor ratio.
-enum { K_SGDM = 0, K_ADAM = 1, K_LAMB1 = 2, K_LAMB2 = 3, K_LARS1 = 4, K_LARS2 = 5 };
-__host__ __device__ constexpr bool is_phase1(int o) { return o == K_LAMB1 || o == K_LARS1; }
-__host__ __device__ constexpr bool is_phase2(int o) { return o == K_LAMB2 || o == K_LARS2; }
+// Adafactor runs as three passes around two finalize steps: K_AF1 reduces the gradients, keeps
+// the sum and accumulates row / column sums of g^2 + eps1; K_AF2 sums U^2 per tensor; K_AF3 applies.
+enum { K_SGDM = 0, K_ADAM = 1, K_LAMB1 = 2, K_LAMB2 = 3, K_LARS1 = 4, K_LARS2 = 5, K_AF1 = 6, K_AF2 = 7, K_AF3 = 8 };
+__host__ __device__ constexpr bool is_af(int o) { return o == K_AF1 || o == K_AF2 || o == K_AF3; }
+// phase 1: reduces the gradient lists and leaves partial sums, no weight step
+__host__ __device__ constexpr bool is_phase1(int o) { return o == K_LAMB1 || o == K_LARS1 || o == K_AF1; }
+// phase 2: does not read the gradient lists (works from state and the stored gradient sum)
+__host__ __device__ constexpr bool is_phase2(int o) { return o == K_LAMB2 || o == K_LARS2 || o == K_AF2 || o == K_AF3; }
+__host__ __device__ constexpr bool writes_weights(int o) { return !is_phase1(o) && o != K_AF2; }
+__host__ __device__ constexpr bool leaves_partials(int o) { return is_phase1(o) || o == K_AF2; }
+constexpr int kAfRows = 2048;   // shared-memory row accumulators of one tile (Adafactor pass 1)
+constexpr int kAfCols = 4096;   // shared-memory column accumulators
 enum { O_NONE = 0, O_F32 = 1, O_BF16 = 2 };
 
 template <int N>
@@ -84,7 +93,10 @@ struct UpdParams {
     void* const* wtab;       // fused formatting: device table [T] of weight tensor pointers (outputs)
     float2* partials;       // phase 1: [R][ntiles] partial sums of the two norms
     const float* rho;       // phase 2: [T] trust ratio (LAMB) / local rate (LARS)
-    float* ghat;            // LARS: [R][S] summed gradients, written by phase 1, read by phase 2
+    float* ghat;            // LARS, Adafactor: [R][S] summed gradients, written by phase 1, read afterwards
+    const WsSegAf* segaf;   // Adafactor: [T] matrix view of every tensor
+    float* af_acc;          // Adafactor pass 1: [F] row / column sums of g^2 + eps1 (atomic adds)
+    const float* af_fac;    // Adafactor passes 2, 3: [F] 1/sqrt factors of V
     WsConsts c;
 };
 
@@ -311,14 +323,20 @@ template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED
 __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8) ? WS_TUNE_MINB8 : WS_TUNE_MINB) update_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp) {
     constexpr bool HAS_V = (OPT == K_ADAM || OPT == K_LAMB1 || OPT == K_LAMB2);
     constexpr bool READS_G = !is_phase2(OPT);     // phase 2 works from state (and the stored gradient sum)
-    constexpr bool READS_M = (OPT != K_LARS1);
-    constexpr bool WRITES_W = !is_phase1(OPT);    // phase 1 only zeroes the pads of w
-    constexpr bool WRITES_M = (OPT != K_LAMB2 && OPT != K_LARS1);
+    constexpr bool READS_W = (OPT != K_AF2);
+    constexpr bool READS_M = (OPT != K_LARS1 && !is_af(OPT));
+    constexpr bool READS_GHAT = (OPT == K_LARS2 || OPT == K_AF2 || OPT == K_AF3);
+    constexpr bool WRITES_W = writes_weights(OPT);   // phase 1 only zeroes the pads of w
+    constexpr bool WRITES_M = (OPT != K_LAMB2 && OPT != K_LARS1 && !is_af(OPT));
+    constexpr bool WRITES_GHAT = (OPT == K_LARS1 || OPT == K_AF1);
     constexpr bool LOOPK = (NP > RB);   // R may exceed one tree block: loop and compensate
     __shared__ float red[2][kBlock / 32];
     // fused formatting: this tile's R gradient tensor pointers, fetched once per work item (the
     // streaming data would push the table's lines out of L1 between passes)
     __shared__ const void* sgp[(FUSED && READS_G) ? NP : 1];
+    // Adafactor pass 1: this tile's partial row sums and column sums
+    __shared__ float srow[OPT == K_AF1 ? kAfRows : 1];
+    __shared__ float scol[OPT == K_AF1 ? kAfCols : 1];
 
     for (long long item = blockIdx.x; item < P.nitems; item += gridDim.x) {
         long long rs = P.concat ? 0 : item / P.ntiles;     // shard index inside this launch
@@ -345,8 +363,36 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
         }
         const int nvec = tl.len / VEC;
         float lr_rho = 0.f;
-        if (is_phase2(OPT)) lr_rho = P.c.lr * P.rho[tl.seg];
+        if (OPT == K_LAMB2 || OPT == K_LARS2) lr_rho = P.c.lr * P.rho[tl.seg];
+        if (OPT == K_AF3) lr_rho = P.rho[tl.seg];         // alpha_t / max(1, RMS(U_t)/d)
         float sw = 0.f, su = 0.f;
+        // Adafactor: where the tile starts inside its tensor's rows x cols matrix
+        WsSegAf af;
+        long long row0 = 0, c0 = 0;
+        int nrows_tile = 0;
+        bool rowsum = false, bigcol = false, rows_sm = false, cols_sm = false;
+        if constexpr (is_af(OPT)) {
+            af = P.segaf[tl.seg];
+            rowsum = af.nrow > 0;                          // unfactored tensors are one row
+            if (af.ncol > 0) {
+                row0 = toff / af.ncol;
+                c0 = toff - row0 * af.ncol;
+            }
+            bigcol = af.ncol >= tl.len;                    // the tile touches at most two rows
+            if constexpr (OPT == K_AF1) {
+                if (rowsum && nvalid > 0) {
+                    const long long nr = (c0 + nvalid - 1) / af.ncol + 1;
+                    rows_sm = nr <= kAfRows;
+                    cols_sm = af.ncol <= kAfCols;
+                    nrows_tile = rows_sm ? (int)nr : 0;
+                    __syncthreads();                       // the previous item's flush is done
+                    for (int k = threadIdx.x; k < nrows_tile; k += kBlock) srow[k] = 0.f;
+                    if (cols_sm)
+                        for (int k = threadIdx.x; k < (int)af.ncol; k += kBlock) scol[k] = 0.f;
+                    __syncthreads();
+                }
+            }
+        }
 
         for (int q0 = 0; q0 < nvec; q0 += U * kBlock) {
             int e0[U];
@@ -365,10 +411,10 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 if (nv[u] > 0) {
-                    wv[u] = load_f32<VEC>(P.w + sbase + e0[u]);
+                    if (READS_W) wv[u] = load_f32<VEC>(P.w + sbase + e0[u]);
                     if (READS_M) mv[u] = load_f32<VEC>(P.m + sbase + e0[u]);
                     if (HAS_V) vv[u] = load_f32<VEC>(P.v + sbase + e0[u]);
-                    if (OPT == K_LARS2) gv[u] = load_f32<VEC>(P.ghat + obase + e0[u]);   // summed gradient from phase 1
+                    if (READS_GHAT) gv[u] = load_f32<VEC>(P.ghat + obase + e0[u]);   // summed gradient from phase 1
                 }
             }
             if (READS_G) {
@@ -417,24 +463,125 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
                     }
                 }
             }
+            if constexpr (OPT == K_AF1) {
+                // g^2 + eps1 of every valid element goes to its row and to its column.  A thread's
+                // elements are consecutive, so they form one run per row; when a whole warp sits in
+                // one row (the usual case) the runs are combined by shuffles before the one add.
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const bool has = nv[u] > 0;
+                    long long col = c0 + e0[u];
+                    unsigned rl = 0;
+                    if (bigcol) {
+                        if (col >= af.ncol) { rl = 1; col -= af.ncol; }
+                    } else {
+                        rl = (unsigned)col / (unsigned)af.ncol;
+                        col = (unsigned)col - rl * (unsigned)af.ncol;
+                    }
+                    unsigned cur = rl;
+                    bool simple = true;
+                    float racc = 0.f;
+                    if (has) {
+                        float* gcol = P.af_acc + af.foff + af.nrow;
+#pragma unroll
+                        for (int j = 0; j < VEC; ++j) {
+                            if (j < nv[u]) {
+                                const float g = gv[u].f[j] * P.c.gscale;
+                                gv[u].f[j] = g;
+                                sw = fmaf(wv[u].f[j], wv[u].f[j], sw);
+                                const float x = fmaf(g, g, P.c.eps);
+                                if (!rowsum) {
+                                    gcol[col] = x;                 // unfactored: every element has its own slot
+                                } else {
+                                    if (cols_sm) atomicAdd(&scol[col], x);
+                                    else atomicAdd(&gcol[col], x);
+                                    if (rl != cur) {
+                                        if (rows_sm) atomicAdd(&srow[cur], racc);
+                                        else atomicAdd(&P.af_acc[af.foff + row0 + cur], racc);
+                                        racc = 0.f;
+                                        cur = rl;
+                                        simple = false;
+                                    }
+                                    racc += x;
+                                }
+                                if (++col == af.ncol) { col = 0; ++rl; }
+                            }
+                        }
+                    }
+                    if (rowsum) {   // uniform over the CTA
+                        const unsigned act = __ballot_sync(0xffffffffu, has);
+                        if (act) {
+                            const int lead = __ffs(act) - 1;
+                            const unsigned lead_row = __shfl_sync(0xffffffffu, cur, lead);
+                            const bool uni = __all_sync(0xffffffffu, !has || (simple && cur == lead_row));
+                            if (uni) {
+                                float tsum = has ? racc : 0.f;
+#pragma unroll
+                                for (int o = 16; o > 0; o >>= 1) tsum += __shfl_xor_sync(0xffffffffu, tsum, o);
+                                if ((int)(threadIdx.x & 31) == lead) {
+                                    if (rows_sm) atomicAdd(&srow[lead_row], tsum);
+                                    else atomicAdd(&P.af_acc[af.foff + row0 + lead_row], tsum);
+                                }
+                            } else if (has) {
+                                if (rows_sm) atomicAdd(&srow[cur], racc);
+                                else atomicAdd(&P.af_acc[af.foff + row0 + cur], racc);
+                            }
+                        }
+                    }
+                }
+            }
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 if (nv[u] < 0) continue;
+                if constexpr (OPT == K_AF2 || OPT == K_AF3) {
+                    // U = g / sqrt(V) with V = Rv' Cv'^T / sum(Rv'): the finalize step left
+                    // sqrt(sum(Rv') / Rv'_i) and 1 / sqrt(Cv'_j), so U = g * fr_i * fc_j
+                    long long col = c0 + e0[u];
+                    unsigned rl = 0;
+                    if (bigcol) {
+                        if (col >= af.ncol) { rl = 1; col -= af.ncol; }
+                    } else {
+                        rl = (unsigned)col / (unsigned)af.ncol;
+                        col = (unsigned)col - rl * (unsigned)af.ncol;
+                    }
+                    const float* frp = P.af_fac + af.foff + row0;
+                    const float* fcp = P.af_fac + af.foff + af.nrow;
+                    float fr = 1.f;
+                    if (rowsum && nv[u] > 0) fr = __ldg(frp + rl);
 #pragma unroll
-                for (int j = 0; j < VEC; ++j) {
-                    if (j < nv[u]) {
-                        if (OPT != K_LARS2) gv[u].f[j] *= P.c.gscale;     // (phase 1 stored it already scaled)
-                        update_elem<OPT>(P.c, gv[u].f[j], wv[u].f[j], mv[u].f[j], vv[u].f[j], lr_rho, sw, su);
-                    } else {  // pad: identity for the sums, +0 for every output
-                        wv[u].f[j] = 0.f; mv[u].f[j] = 0.f; vv[u].f[j] = 0.f; gv[u].f[j] = 0.f;
+                    for (int j = 0; j < VEC; ++j) {
+                        if (j < nv[u]) {
+                            const float uu = (gv[u].f[j] * fr) * __ldg(fcp + col);
+                            if (OPT == K_AF2) su = fmaf(uu, uu, su);
+                            else wv[u].f[j] = fmaf(-lr_rho, uu, wv[u].f[j]);
+                            if (++col == af.ncol) {
+                                col = 0;
+                                ++rl;
+                                if (rowsum && j + 1 < nv[u]) fr = __ldg(frp + rl);
+                            }
+                        } else {
+                            wv[u].f[j] = 0.f;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < VEC; ++j) {
+                        if (j < nv[u]) {
+                            if (READS_G && OPT != K_AF1) gv[u].f[j] *= P.c.gscale;     // (phase 1 stored it already scaled)
+                            if (OPT != K_AF1) update_elem<OPT>(P.c, gv[u].f[j], wv[u].f[j], mv[u].f[j], vv[u].f[j], lr_rho, sw, su);
+                        } else {  // pad: identity for the sums, +0 for every output
+                            wv[u].f[j] = 0.f; mv[u].f[j] = 0.f; vv[u].f[j] = 0.f; gv[u].f[j] = 0.f;
+                        }
                     }
                 }
                 const long long so = sbase + e0[u];
-                if (WRITES_W || nv[u] < VEC) store_f32<VEC>(P.w + so, wv[u]);
+                if (WRITES_W || (READS_W && nv[u] < VEC)) store_f32<VEC>(P.w + so, wv[u]);
                 if (WRITES_M) store_f32<VEC>(P.m + so, mv[u]);
                 if (HAS_V && OPT != K_LAMB2) store_f32<VEC>(P.v + so, vv[u]);
-                if (OPT == K_LARS1) store_f32<VEC>(P.ghat + obase + e0[u], gv[u]);   // keep the sum for phase 2
-                if constexpr (FUSED) {
+                if (WRITES_GHAT) store_f32<VEC>(P.ghat + obase + e0[u], gv[u]);   // keep the sum for the later passes
+                if constexpr (!WRITES_W) {
+                    // no weight output in this pass
+                } else if constexpr (FUSED) {
                     if (OUT == O_F32) {
                         float* dst = reinterpret_cast<float*>(wt) + toff + e0[u];
                         if (nv[u] == VEC) store_f32<VEC>(dst, wv[u]);
@@ -451,7 +598,23 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
                 }
             }
         }
-        if (is_phase1(OPT)) {
+        if constexpr (OPT == K_AF1) {
+            // the tile's sums join the tensor's (this add of partial reduce results across tiles
+            // and shards stands where the paper combines them with an all-reduce, Section 4.1)
+            if (rowsum && nvalid > 0) {
+                __syncthreads();
+                for (int k = threadIdx.x; k < nrows_tile; k += kBlock) atomicAdd(&P.af_acc[af.foff + row0 + k], srow[k]);
+                if (cols_sm) {
+                    const int ncov = nvalid < af.ncol ? nvalid : (int)af.ncol;
+                    for (int k = threadIdx.x; k < ncov; k += kBlock) {
+                        long long col = c0 + k;
+                        if (col >= af.ncol) col -= af.ncol;
+                        atomicAdd(&P.af_acc[af.foff + af.nrow + col], scol[col]);
+                    }
+                }
+            }
+        }
+        if (leaves_partials(OPT)) {
             const float a = block_sum(sw, red[0]);
             const float b = block_sum(su, red[1]);
             if (threadIdx.x == 0) P.partials[P.concat ? ti : r * P.ntiles + ti] = make_float2(a, b);
@@ -463,15 +626,14 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
 // (stands where the paper combines per-replica reduce results with one batched
 // scalar all-reduce, Section 4.1 / 5.2), then rho_t = sqrt(a)/sqrt(b).
 // With lars != 0 the ratio is the LARS local rate eta sqrt(a) / (sqrt(b) + beta sqrt(a)).
-__global__ void __launch_bounds__(kBlock) lamb_finalize_kernel(const WsSegTiles* segtiles, const float2* partials,
-                                                               long long ntiles, int R, float* rho, double* norms,
-                                                               int lars, double eta, double beta) {
-    // R == 1 with the concatenated layout: a tensor's tiles of all shards are one contiguous run
+// Sums tensor t's per-tile partials over all shards in a fixed order, in double; the totals
+// are valid in thread 0.
+__device__ __forceinline__ void sum_partials(const WsSegTiles st, const float2* partials, long long ntiles, int R,
+                                             double& a, double& b) {
     __shared__ double sa[kBlock], sb[kBlock];
-    const int t = blockIdx.x;
-    const WsSegTiles st = segtiles[t];
     const long long n = (long long)R * st.tile_count;
-    double a = 0.0, b = 0.0;
+    a = 0.0;
+    b = 0.0;
     for (long long i = threadIdx.x; i < n; i += kBlock) {
         const long long r = i / st.tile_count, k = i - r * st.tile_count;
         const float2 p = partials[r * ntiles + st.tile_begin + k];
@@ -488,14 +650,83 @@ __global__ void __launch_bounds__(kBlock) lamb_finalize_kernel(const WsSegTiles*
         }
         __syncthreads();
     }
+    a = sa[0];
+    b = sb[0];
+}
+
+__global__ void __launch_bounds__(kBlock) lamb_finalize_kernel(const WsSegTiles* segtiles, const float2* partials,
+                                                               long long ntiles, int R, float* rho, double* norms,
+                                                               int lars, double eta, double beta) {
+    // R == 1 with the concatenated layout: a tensor's tiles of all shards are one contiguous run
+    const int t = blockIdx.x;
+    double a, b;
+    sum_partials(segtiles[t], partials, ntiles, R, a, b);
     if (threadIdx.x == 0) {
-        a = sa[0];
-        b = sb[0];
         norms[2 * t] = a;
         norms[2 * t + 1] = b;
         if (!(a > 0.0 && b > 0.0)) rho[t] = 1.0f;
         else if (lars) rho[t] = (float)(eta * sqrt(a) / (sqrt(b) + beta * sqrt(a)));
         else rho[t] = (float)(sqrt(a) / sqrt(b));
+    }
+}
+
+// Adafactor, after pass 1 (one block per tensor): the moving averages of the row and column sums,
+// Rv' = beta Rv + (1-beta) acc, the factors the elementwise passes multiply by
+// (sqrt(sum(Rv') / Rv'_i) per row, 1/sqrt(Cv'_j) per column; 1/sqrt(v'_i) for an unfactored tensor),
+// and the step size alpha_t = max(eps2, RMS(w_t)) * rho_step from pass 1's partial sums of w^2.
+__global__ void __launch_bounds__(kBlock) af_finalize_moments_kernel(const WsSegTiles* segtiles, const WsSegAf* segaf,
+                                                                     const float2* partials, long long ntiles, int R,
+                                                                     float* state, const float* acc, float* fac,
+                                                                     float* alpha, double* norms, double beta,
+                                                                     double eps2, double rho_step) {
+    __shared__ double srs[kBlock];
+    const int t = blockIdx.x;
+    const WsSegAf a = segaf[t];
+    double sw, unused;
+    sum_partials(segtiles[t], partials, ntiles, R, sw, unused);
+    if (threadIdx.x == 0) {
+        const double rms_w = a.numel > 0 ? sqrt(sw / (double)a.numel) : 0.0;
+        alpha[t] = (float)((eps2 > rms_w ? eps2 : rms_w) * rho_step);
+        norms[2 * t] = sw;
+    }
+    float* vr = state + a.foff;
+    float* vc = vr + a.nrow;
+    double rs = 0.0;
+    for (long long i = threadIdx.x; i < a.nrow; i += kBlock) {
+        const double v = beta * (double)vr[i] + (1.0 - beta) * (double)acc[a.foff + i];
+        vr[i] = (float)v;
+        rs += v;
+    }
+    srs[threadIdx.x] = rs;
+    __syncthreads();
+    for (int s = kBlock / 2; s > 0; s >>= 1) {
+        if (threadIdx.x < s) srs[threadIdx.x] += srs[threadIdx.x + s];
+        __syncthreads();
+    }
+    rs = srs[0];
+    for (long long i = threadIdx.x; i < a.nrow; i += kBlock) fac[a.foff + i] = (float)sqrt(rs / (double)vr[i]);
+    for (long long j = threadIdx.x; j < a.ncol; j += kBlock) {
+        const double v = beta * (double)vc[j] + (1.0 - beta) * (double)acc[a.foff + a.nrow + j];
+        vc[j] = (float)v;
+        fac[a.foff + a.nrow + j] = (float)(1.0 / sqrt(v));
+    }
+}
+
+// Adafactor, after pass 2: RMS(U_t) from the partial sums of U^2, then the applied step size
+// rho[t] = alpha_t / max(1, RMS(U_t) / d).
+__global__ void __launch_bounds__(kBlock) af_finalize_clip_kernel(const WsSegTiles* segtiles, const WsSegAf* segaf,
+                                                                  const float2* partials, long long ntiles, int R,
+                                                                  const float* alpha, float* rho, double* norms,
+                                                                  double d) {
+    const int t = blockIdx.x;
+    double unused, su;
+    sum_partials(segtiles[t], partials, ntiles, R, unused, su);
+    if (threadIdx.x == 0) {
+        const long long n = segaf[t].numel;
+        const double rms_u = n > 0 ? sqrt(su / (double)n) : 0.0;
+        const double clip = rms_u / d > 1.0 ? rms_u / d : 1.0;
+        norms[2 * t + 1] = su;
+        rho[t] = (float)((double)alpha[t] / clip);
     }
 }
 
@@ -550,8 +781,10 @@ ws_status launch_o(const UpdParams& P, const void* const* gptrs, int out, bool w
     wide = wide && aligned32(P.w) && aligned32(P.m) && aligned32(P.v) && aligned32(P.gathered);
     if (!FUSED && !is_phase2(OPT))
         for (int k = 0; k < P.R && wide; ++k) wide = aligned32(gptrs[k]);
-    if (OPT == K_LARS1 || OPT == K_LARS2) wide = wide && aligned32(P.ghat);
-    if constexpr (is_phase1(OPT)) {
+    if (OPT == K_LARS1 || OPT == K_LARS2 || is_af(OPT)) wide = wide && aligned32(P.ghat);
+    if constexpr (OPT == K_AF2) {
+        return launch_r<OPT, false, O_NONE, false>(P, gptrs, wide, st);   // touches no tensor list and no output
+    } else if constexpr (is_phase1(OPT)) {
         return launch_r<OPT, GBF, O_NONE, FUSED>(P, gptrs, wide, st);
     } else {
         switch (out) {
@@ -572,6 +805,9 @@ ws_status launch_f(int opt, bool gbf, int out, const UpdParams& P, const void* c
         case K_LAMB1: return gbf ? launch_o<K_LAMB1, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_LAMB1, false, FUSED>(P, gptrs, out, wide, st);
         case K_LARS1: return gbf ? launch_o<K_LARS1, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_LARS1, false, FUSED>(P, gptrs, out, wide, st);
         case K_LARS2: return launch_o<K_LARS2, false, FUSED>(P, gptrs, out, wide, st);
+        case K_AF1: return gbf ? launch_o<K_AF1, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_AF1, false, FUSED>(P, gptrs, out, wide, st);
+        case K_AF2: return launch_o<K_AF2, false, false>(P, gptrs, out, wide, st);
+        case K_AF3: return launch_o<K_AF3, false, FUSED>(P, gptrs, out, wide, st);
         default: return launch_o<K_LAMB2, false, FUSED>(P, gptrs, out, wide, st);
     }
 }
@@ -606,8 +842,9 @@ ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state
     if (r < -1 || r >= p->R) return WS_ERR_INVALID_ARG;
     if (h->step < 1) return WS_ERR_INVALID_ARG;
     const bool needs_v = (phase == K_ADAM || phase == K_LAMB1 || phase == K_LAMB2);
-    if (!s->w || !s->m || (needs_v && !s->v)) return WS_ERR_INVALID_ARG;
-    if (!ws_aligned16(s->w) || !ws_aligned16(s->m) || (needs_v && !ws_aligned16(s->v))) return WS_ERR_ALIGNMENT;
+    const bool needs_m = !is_af(phase);
+    if (!s->w || (needs_m && !s->m) || (needs_v && !s->v)) return WS_ERR_INVALID_ARG;
+    if (!ws_aligned16(s->w) || (needs_m && !ws_aligned16(s->m)) || (needs_v && !ws_aligned16(s->v))) return WS_ERR_ALIGNMENT;
     gbf = false;
     P.gtab = nullptr;
     P.wtab = nullptr;
@@ -654,8 +891,11 @@ ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state
         P.g_stride = 0;
     }
     P.w = (float*)s->w;
-    P.m = (float*)s->m;
-    P.v = (float*)s->v;
+    P.m = needs_m ? (float*)s->m : nullptr;
+    P.v = needs_v ? (float*)s->v : nullptr;
+    P.segaf = p->d_segaf;
+    P.af_acc = nullptr;
+    P.af_fac = nullptr;
     P.gathered = (out_kind != O_NONE) ? out->gathered : nullptr;
     P.partials = nullptr;
     P.rho = nullptr;
@@ -725,10 +965,18 @@ extern "C" ws_status ws_lamb_apply(const ws_plan* plan, int32_t r, const ws_stat
     return launch_any(K_LAMB2, false, ok, P, nullptr, (cudaStream_t)stream);
 }
 
+namespace {
+ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_tensor_table* gtab,
+                    const ws_state* state, const ws_hyper* hyper, const ws_out* out, const ws_tensor_table* wtab,
+                    void* workspace, size_t workspace_bytes, cudaStream_t st);
+}
+
 extern "C" ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_state* state,
                                      const ws_hyper* hyper, const ws_out* out, void* workspace,
                                      size_t workspace_bytes, void* stream) {
     if (!hyper) return WS_ERR_INVALID_ARG;
+    if (hyper->opt == WS_ADAFACTOR)
+        return af_update(plan, r, grads, nullptr, state, hyper, out, nullptr, workspace, workspace_bytes, (cudaStream_t)stream);
     if (hyper->opt == WS_LAMB) {
         if (r != -1) return WS_ERR_INVALID_ARG;
         ws_status s = ws_lamb_partial(plan, -1, grads, state, hyper, workspace, workspace_bytes, stream);
@@ -838,8 +1086,75 @@ ws_status fused_phase(const ws_plan* plan, int32_t r, const ws_tensor_table* gra
         P.partials = L.partials;
         P.rho = L.rho;
         P.ghat = L.ghat;
+        if (is_af(phase)) {
+            P.af_acc = L.acc;
+            P.af_fac = L.fac;
+        }
     }
     return launch_f<true>(phase, gbf, out_kind, P, nullptr, wide, st);
+}
+
+// Adafactor, all shards: zero the row / column sums, pass 1 (reduce, keep the sum, partial row and
+// column sums), moments + step size, pass 2 (sum U^2), clipping, pass 3 (apply).  Either the
+// packed-buffer arguments (grads, out) or the tensor tables (gtab, wtab) are given.
+ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_tensor_table* gtab,
+                    const ws_state* state, const ws_hyper* hyper, const ws_out* out, const ws_tensor_table* wtab,
+                    void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (!plan || !state || !hyper) return WS_ERR_INVALID_ARG;
+    if (!plan->d_tiles) return WS_ERR_NOT_UPLOADED;
+    if (r != -1) return WS_ERR_INVALID_ARG;
+    if (hyper->weight_decay != 0.0 || !(hyper->clip_threshold > 0.0) || !(hyper->decay_exponent > 0.0) ||
+        !(hyper->eps >= 0.0) || !(hyper->eps2 >= 0.0) || hyper->step < 1)
+        return WS_ERR_INVALID_ARG;
+    if (!state->v) return WS_ERR_INVALID_ARG;
+    if (!ws_aligned16(state->v)) return WS_ERR_ALIGNMENT;
+    ws_status s = check_ws(plan, workspace, workspace_bytes, WS_ADAFACTOR);
+    if (s != WS_OK) return s;
+    const WsLambWs L = ws_lamb_layout(plan, workspace);
+    const bool fused = gtab != nullptr;
+    const double beta = 1.0 - pow((double)hyper->step, -hyper->decay_exponent);
+    const double inv_sqrt_t = 1.0 / sqrt((double)hyper->step);
+    const double rho_step = hyper->lr < inv_sqrt_t ? hyper->lr : inv_sqrt_t;
+    const int reps = finalize_reps(plan);
+
+    if (plan->F > 0) {
+        cudaError_t e = cudaMemsetAsync(L.acc, 0, sizeof(float) * (size_t)plan->F, st);
+        if (e != cudaSuccess) return ws_cuda_fail(e, "adafactor(clear sums)");
+    }
+    UpdParams P;
+    int ok;
+    bool gbf;
+    if (fused) {
+        if ((s = fused_phase(plan, -1, gtab, state, hyper, wtab, K_AF1, workspace, st)) != WS_OK) return s;
+    } else {
+        if ((s = prepare(plan, -1, grads, state, hyper, nullptr, K_AF1, P, ok, gbf)) != WS_OK) return s;
+        P.partials = L.partials;
+        P.ghat = L.ghat;
+        P.af_acc = L.acc;
+        std::vector<const void*> gp;
+        offset_grad_ptrs(plan, -1, grads, gp);
+        if ((s = launch_any(K_AF1, gbf, O_NONE, P, gp.data(), st)) != WS_OK) return s;
+    }
+    af_finalize_moments_kernel<<<plan->T, kBlock, 0, st>>>(plan->d_segtiles, plan->d_segaf, L.partials, plan->ntiles, reps,
+                                                          (float*)state->v, L.acc, L.fac, L.alpha, L.norms, beta,
+                                                          hyper->eps2, rho_step);
+    if ((s = ws_check_launch("adafactor(moments)")) != WS_OK) return s;
+
+    if ((s = prepare(plan, -1, nullptr, state, hyper, nullptr, K_AF2, P, ok, gbf)) != WS_OK) return s;
+    P.partials = L.partials;
+    P.ghat = L.ghat;
+    P.af_fac = L.fac;
+    if ((s = launch_any(K_AF2, false, O_NONE, P, nullptr, st)) != WS_OK) return s;
+    af_finalize_clip_kernel<<<plan->T, kBlock, 0, st>>>(plan->d_segtiles, plan->d_segaf, L.partials, plan->ntiles, reps,
+                                                       L.alpha, L.rho, L.norms, hyper->clip_threshold);
+    if ((s = ws_check_launch("adafactor(clipping)")) != WS_OK) return s;
+
+    if (fused) return fused_phase(plan, -1, gtab, state, hyper, wtab, K_AF3, workspace, st);
+    if ((s = prepare(plan, -1, nullptr, state, hyper, out, K_AF3, P, ok, gbf)) != WS_OK) return s;
+    P.rho = L.rho;
+    P.ghat = L.ghat;
+    P.af_fac = L.fac;
+    return launch_any(K_AF3, false, ok, P, nullptr, st);
 }
 
 }  // namespace
@@ -854,6 +1169,8 @@ extern "C" ws_status ws_fused_update(const ws_plan* plan, int32_t r, const ws_te
     if ((grads->dtype != WS_F32 && grads->dtype != WS_BF16) || (weights->dtype != WS_F32 && weights->dtype != WS_BF16))
         return WS_ERR_DTYPE;
     cudaStream_t st = (cudaStream_t)stream;
+    if (hyper->opt == WS_ADAFACTOR)
+        return af_update(plan, r, nullptr, grads, state, hyper, nullptr, weights, workspace, workspace_bytes, st);
     if (hyper->opt == WS_LAMB) {
         if (r != -1) return WS_ERR_INVALID_ARG;
         ws_status s = check_ws(plan, workspace, workspace_bytes);

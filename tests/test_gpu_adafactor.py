@@ -1,0 +1,222 @@
+"""GPU parity for Adafactor (the optimizer with row / column reduces that the sharding cuts,
+Section 4.1): the CUDA library through its C ABI against the CPU oracle's whole-tensor
+definition on the same seeded inputs.  Tolerances: 1e-5 under the per-tensor error metric for
+the weights (they pass through fp32 row / column sums, as LAMB's pass through fp32 norms),
+1e-5 relative for the factored state and the per-tensor scalars, 1e-2 for bf16 outputs."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import ws_oracle as O
+from paper_2004_13336_b200 import binding as B
+from paper_2004_13336_b200 import workloads as W
+from tests._util import TOL_BF16, TOL_LAMB, bf16_to_f64, err, to_np
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+# matrices with rows longer and shorter than a tile, single rows and columns, 3-D and 4-D tensors,
+# vectors (unfactored), tiny and prime sizes
+SHAPES = [(1,), (7,), (3, 3, 16, 32), (64, 128), (1031,), (5, 1, 9), (4099, 3), (300, 301), (32,), (20011,),
+          (2, 9001), (1, 4500), (4500, 1), (6, 5000)]
+
+
+def _hyper(**kw):
+    h = dict(lr=1e-2, beta1=0.0, beta2=0.0, eps=1e-30, weight_decay=0.0, momentum=0.0, grad_scale=1.0, step=10,
+             eps2=1e-3, clip_threshold=1.0, decay_exponent=0.8)
+    h.update(kw)
+    return h
+
+
+def _setup(shapes, R, gdtype=torch.float32, seed=0, gstd=1e-2, A=32, tile=0, layout="per_tensor", K=None):
+    wl = W.Workload("t", list(shapes), R=K or R, opt="adam", hyper={}, grad_dtype=gdtype, grad_std=gstd, seed=seed)
+    w, _, _ = W.make_state(wl, DEV)
+    g = W.make_grads(wl, DEV)
+    plan = B.Plan(shapes, R, A, tile, layout=layout)
+    gen = torch.Generator(device="cpu").manual_seed(seed + 99)
+    f0 = (torch.rand(plan.factored_elems, generator=gen) * 1e-3 + 1e-6).to(DEV)
+    return wl, plan, w, g, f0
+
+
+def _oracle(shapes, h, w, g, f0):
+    hs = O.make_hyper("adafactor", h)
+    rows, cols, foff, tot = O.factor_shapes(shapes)
+    assert tot == f0.numel()
+    f = to_np(f0)
+    ow = [to_np(x).reshape(s) for x, s in zip(w, shapes)]
+    og = [[to_np(x) for x in gk] for gk in g]
+    info = []
+    for t in range(len(shapes)):
+        vr = f[foff[t]:foff[t] + rows[t]]
+        vc = f[foff[t] + rows[t]:foff[t] + rows[t] + cols[t]] if cols[t] else None
+        info.append(O.adafactor_tensor(hs, [gk[t] for gk in og], ow[t], vr, vc))
+    return ow, f, np.array(info)
+
+
+def _pack(plan, lists):
+    out = []
+    for l in lists:
+        b = torch.empty(plan.G, dtype=l[0].dtype, device=DEV)
+        B.ws_pack(plan, l, b)
+        out.append(b)
+    return out
+
+
+def _check(plan, shapes, pw, fs, ws, ow, of, oinfo, tol=TOL_LAMB, d=1.0):
+    got = [torch.empty(int(np.prod(s)), dtype=torch.float32, device=DEV) for s in shapes]
+    B.ws_unpack(plan, pw, got)
+    for t, (a, b) in enumerate(zip(got, ow)):
+        e = err(to_np(a), b)
+        assert e <= tol, f"w[{t}] {shapes[t]} err {e:.3e}"
+    # the factored state per tensor under the same metric: an entry fed by a single element whose R
+    # gradient copies cancel carries that fp32 sum's error, far above its own size
+    gs = to_np(fs)
+    for t, (off, rows, cols) in enumerate(plan.factored_layout()):
+        e = err(gs[off:off + rows + cols], of[off:off + rows + cols])
+        assert e <= tol, f"state[{t}] {shapes[t]} err {e:.3e}"
+    T = plan.T
+    coef = ws[:4 * T].view(torch.float32).cpu().numpy().astype(np.float64)
+    clip = np.maximum(1.0, oinfo[:, 1] / d)
+    np.testing.assert_allclose(coef, oinfo[:, 0] / clip, rtol=1e-5)
+
+
+@pytest.mark.parametrize("R", [1, 2, 3, 8, 16, 40])
+@pytest.mark.parametrize("gdtype", [torch.float32, torch.bfloat16])
+def test_adafactor_matches_oracle_and_fused_equals_unfused(R, gdtype):
+    wl, plan, w, g, f0 = _setup(SHAPES, R, gdtype, seed=R + 3)
+    h = _hyper()
+    ow, of, oinfo = _oracle(SHAPES, h, w, g, f0)
+    pw, = _pack(plan, [w])
+    pg = _pack(plan, g)
+    fs = f0.clone()
+    ws = torch.zeros(plan.workspace_bytes("adafactor"), dtype=torch.uint8, device=DEV)
+    gath = torch.full((plan.G,), 3.0, dtype=torch.bfloat16, device=DEV)
+    B.ws_shard_update(plan, -1, pg, pw, None, fs, B.make_hyper("adafactor", h), gath, ws)
+    _check(plan, SHAPES, pw, fs, ws, ow, of, oinfo)
+    assert torch.equal(gath, pw.to(torch.bfloat16))
+    oplan = O.Plan(wl.numels, R, 32)
+    valid = torch.from_numpy(O.pack(oplan, [np.ones(int(n), np.float32) for n in oplan.numel]) != 0).to(DEV)
+    assert bool((pw[~valid].view(torch.int32) == 0).all()) and bool((gath[~valid].view(torch.int16) == 0).all())
+    # formatting fused in: gradients read from the tensor lists, weights written to the tensors
+    fw, = _pack(plan, [w])
+    ff = f0.clone()
+    outs = [torch.zeros(n, dtype=torch.float32, device=DEV) for n in wl.numels]
+    ws2 = torch.full_like(ws, 0xFF)                       # the workspace may hold anything on entry
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), fw, None, ff, B.make_hyper("adafactor", h),
+                      B.TensorTable(plan, [outs]), ws2)
+    _check(plan, SHAPES, fw, ff, ws2, ow, of, oinfo)
+    got = [torch.empty_like(o) for o in outs]
+    B.ws_unpack(plan, fw, got)
+    for a, b in zip(outs, got):
+        assert torch.equal(a, b)
+
+
+@pytest.mark.parametrize("tile", [1024, 4096, 16384])
+@pytest.mark.parametrize("layout", ["per_tensor", "concat"])
+def test_tile_sizes_and_layouts(tile, layout):
+    R = 5
+    wl, plan, w, g, f0 = _setup(SHAPES, R, seed=21, tile=tile, layout=layout, A=8)
+    h = _hyper(step=3, clip_threshold=0.5)
+    ow, of, oinfo = _oracle(SHAPES, h, w, g, f0)
+    pw, = _pack(plan, [w])
+    fs = f0.clone()
+    ws = torch.zeros(plan.workspace_bytes("adafactor"), dtype=torch.uint8, device=DEV)
+    outs = [torch.zeros(n, dtype=torch.bfloat16, device=DEV) for n in wl.numels]
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), pw, None, fs, B.make_hyper("adafactor", h),
+                      B.TensorTable(plan, [outs]), ws)
+    _check(plan, SHAPES, pw, fs, ws, ow, of, oinfo, d=0.5)
+    for t, (a, b) in enumerate(zip(outs, ow)):
+        assert err(bf16_to_f64(to_np(a)), b) <= TOL_BF16, t
+
+
+def test_first_step_without_history_and_grad_scale():
+    # step 1: beta = 0, the old state is ignored entirely (even NaN-free garbage); mean of 4 copies
+    R = 4
+    wl, plan, w, g, f0 = _setup(SHAPES, R, seed=5)
+    h = _hyper(step=1, grad_scale=0.25, lr=0.5)
+    ow, of, oinfo = _oracle(SHAPES, h, w, g, f0)
+    pw, = _pack(plan, [w])
+    fs = f0.clone()
+    ws = torch.zeros(plan.workspace_bytes("adafactor"), dtype=torch.uint8, device=DEV)
+    B.ws_shard_update(plan, -1, _pack(plan, g), pw, None, fs, B.make_hyper("adafactor", h), None, ws)
+    _check(plan, SHAPES, pw, fs, ws, ow, of, oinfo)
+
+
+def test_partial_sharding_more_copies_than_shards():
+    # 3 groups x 2 shards: 6 gradient copies into a 2-shard plan
+    wl, plan, w, g, f0 = _setup(SHAPES, 2, seed=8, K=6)
+    h = _hyper()
+    ow, of, oinfo = _oracle(SHAPES, h, w, g, f0)
+    pw, = _pack(plan, [w])
+    fs = f0.clone()
+    ws = torch.zeros(plan.workspace_bytes("adafactor"), dtype=torch.uint8, device=DEV)
+    B.ws_shard_update(plan, -1, _pack(plan, g), pw, None, fs, B.make_hyper("adafactor", h), None, ws)
+    _check(plan, SHAPES, pw, fs, ws, ow, of, oinfo)
+
+
+def test_three_consecutive_steps_track_the_oracle():
+    R = 3
+    wl, plan, w, g, f0 = _setup(SHAPES, R, seed=13)
+    pw, = _pack(plan, [w])
+    fs = f0.clone()
+    ws = torch.zeros(plan.workspace_bytes("adafactor"), dtype=torch.uint8, device=DEV)
+    ow = [to_np(x) for x in w]
+    of = f0.clone()
+    for it in range(3):
+        wl.seed = 100 + it
+        g = W.make_grads(wl, DEV)
+        h = _hyper(step=5 + it)
+        # oracle continues from its own previous result
+        wt = [torch.from_numpy(np.ascontiguousarray(a).ravel()).to(DEV) for a in ow]
+        ow, off, oinfo = _oracle(SHAPES, h, wt, g, of)
+        of = torch.from_numpy(off).to(DEV)
+        B.ws_shard_update(plan, -1, _pack(plan, g), pw, None, fs, B.make_hyper("adafactor", h), None, ws)
+    _check(plan, SHAPES, pw, fs, ws, ow, to_np(of), oinfo, tol=3 * TOL_LAMB)
+
+
+def test_poisoned_pads_and_dirty_workspace_change_nothing():
+    R = 7
+    wl, plan, w, g, f0 = _setup(SHAPES, R, seed=12)
+    oplan = O.Plan(wl.numels, R, 32)
+    valid = torch.from_numpy(O.pack(oplan, [np.ones(int(n), np.float32) for n in oplan.numel]) != 0).to(DEV)
+    hy = B.make_hyper("adafactor", _hyper())
+    h = _hyper()
+    ow, of, oinfo = _oracle(SHAPES, h, w, g, f0)
+    pw, = _pack(plan, [w])
+    pg = _pack(plan, g)
+    fs = f0.clone()
+    ws = torch.zeros(plan.workspace_bytes("adafactor"), dtype=torch.uint8, device=DEV)
+    for b in [pw] + pg:
+        b[~valid] = float("nan")
+    ws.view(torch.float32)[:] = float("nan")
+    B.ws_shard_update(plan, -1, pg, pw, None, fs, hy, None, ws)
+    _check(plan, SHAPES, pw, fs, ws, ow, of, oinfo)
+    assert bool((pw[~valid].view(torch.int32) == 0).all())
+
+
+def test_argument_errors():
+    R = 2
+    wl, plan, w, g, f0 = _setup(SHAPES[:4], R, seed=1)
+    pw, = _pack(plan, [w])
+    pg = _pack(plan, g)
+    ws = torch.zeros(plan.workspace_bytes("adafactor"), dtype=torch.uint8, device=DEV)
+    ok = B.make_hyper("adafactor", _hyper())
+    for bad, status in ((dict(weight_decay=0.1), 1), (dict(clip_threshold=0.0), 1), (dict(decay_exponent=0.0), 1)):
+        with pytest.raises(B.WsError) as e:
+            B.ws_shard_update(plan, -1, pg, pw, None, f0, B.make_hyper("adafactor", _hyper(**bad)), None, ws)
+        assert e.value.status == status
+    with pytest.raises(B.WsError) as e:
+        B.ws_shard_update(plan, 0, pg, pw, None, f0, ok, None, ws)             # single shard: refused
+    assert e.value.status == 1
+    with pytest.raises(B.WsError) as e:
+        B.ws_shard_update(plan, -1, pg, pw, None, None, ok, None, ws)          # no factored state
+    assert e.value.status == 1
+    small = torch.zeros(plan.workspace_bytes("lars"), dtype=torch.uint8, device=DEV)
+    with pytest.raises(B.WsError) as e:
+        B.ws_shard_update(plan, -1, pg, pw, None, f0, ok, None, small)
+    assert e.value.status == 4
+    lay = plan.factored_layout()
+    rows, cols, foff, tot = O.factor_shapes(SHAPES[:4])
+    assert [tuple(x) for x in lay] == list(zip(foff.tolist(), rows.tolist(), cols.tolist())) and plan.factored_elems == tot

@@ -163,3 +163,13 @@ def test_header_is_plain_c_and_links_from_c(tmp_path):
     r = subprocess.run([str(exe)], capture_output=True, text=True)
     assert r.returncode == 0, r.stdout + r.stderr
     assert "piece 73728" in r.stdout and "piece 9216" in r.stdout
+
+
+def test_factored_layout_matches_oracle_view():
+    # Adafactor's matrix view of every tensor (rows = leading dimensions together, cols = last one)
+    shapes = [(5, 7), (0,), (3, 0, 4), (100,), (2, 3, 4, 5), (1,), (9, 1), (1, 9)]
+    plan = B.Plan(shapes, 4, 8, upload=False)
+    rows, cols, foff, tot = O.factor_shapes(shapes)
+    assert plan.factored_elems == tot == 12 + 0 + 0 + 100 + 29 + 1 + 10 + 10
+    assert plan.factored_layout() == list(zip(foff.tolist(), rows.tolist(), cols.tolist()))
+    assert plan.workspace_bytes("adafactor") >= plan.workspace_bytes("lars") + 8 * tot + 4 * plan.T
