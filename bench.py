@@ -49,9 +49,10 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=20)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet50",
-                    choices=["tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b", "resnet50_lars"])
+                    choices=["tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b", "resnet50_lars",
+                             "transformer_adafactor"])
     ap.add_argument("--R", type=int, default=0, help="override the workload's replica count")
-    ap.add_argument("--opt", default="", choices=["", "sgdm", "adam", "lamb", "lars"],
+    ap.add_argument("--opt", default="", choices=["", "sgdm", "adam", "lamb", "lars", "adafactor"],
                     help="override the workload's optimizer (profiling of small cases)")
     ap.add_argument("--grad-dtype", default="", choices=["", "f32", "bf16"], help="override the gradient dtype")
     ap.add_argument("--out-dtype", default="", choices=["", "f32", "bf16"], help="override the emitted weight dtype")
@@ -83,7 +84,7 @@ def get_workload(args):
         if args.opt and args.opt != wl.opt:
             wl.opt = args.opt
             wl.hyper = dict(W.WORKLOADS[{"sgdm": "resnet50", "adam": "transformer", "lamb": "bert_large",
-                                         "lars": "resnet50_lars"}[args.opt]]().hyper)
+                                         "lars": "resnet50_lars", "adafactor": "transformer_adafactor"}[args.opt]]().hyper)
         if args.grad_dtype:
             wl.grad_dtype = dt[args.grad_dtype]
         if args.out_dtype:
@@ -97,12 +98,14 @@ def bytes_per_param(wl):
     and its slots once; write weight and slots once; plus the gathered copy when it is a
     separate bf16 buffer) and of one pack / unpack launch."""
     gb = 2 if str(wl.grad_dtype).endswith("bfloat16") else 4
-    slots = 1 if wl.opt in ("sgdm", "lars") else 2
+    slots = {"sgdm": 1, "lars": 1, "adafactor": 0}.get(wl.opt, 2)
     upd = gb * wl.R + 4 * (1 + slots) * 2
     if wl.opt == "lamb":
         upd += 12          # plain two-pass: phase 2 reads w, m', v' again and rewrites w
     if wl.opt == "lars":
         upd += 12          # phase 1 reads w and stores the summed gradient; phase 2 reads it back
+    if wl.opt == "adafactor":
+        upd += 16          # pass 1 stores the summed gradient, passes 2 and 3 read it back, pass 3 reads w again
     out_b = 2 if str(wl.out_dtype).endswith("bfloat16") else 0
     # fused formatting: same reads and state writes, plus the weight tensors written directly
     fused = upd + (2 if out_b else 4)
@@ -199,6 +202,8 @@ def oracle_step_inputs(wl, stride, align):
     w, m, v = ([np_(x) for x in lst] for lst in (w, m, v))
     g = [[np_(x) for x in gk] for gk in g]
     pw, pm, pv = O.pack(plan, w), O.pack(plan, m), O.pack(plan, v)
+    if sub.opt == "adafactor":      # no momentum; the second slot is the factored state
+        pm, pv = None, W.make_factored_state(sub, O.factor_shapes(sub.shapes)[3], "cpu").numpy()
     return sub, plan, g, pw, pm, pv
 
 
@@ -209,7 +214,10 @@ def oracle_one_step(sub, plan, g, pw, pm, pv):
     t0 = time.perf_counter()
     pg = [O.pack(plan, gk) for gk in g]
     out_dt = O.BF16 if str(sub.out_dtype).endswith("bfloat16") else None
-    gathered, _, _ = O.sharded_update(hs, plan, pg, pw, pm, pv if sub.opt in ("adam", "lamb") else None, out_dt)
+    if sub.opt == "adafactor":
+        gathered, _ = O.adafactor_sharded(hs, plan, sub.shapes, pg, pw, pv, out_dt)
+    else:
+        gathered, _, _ = O.sharded_update(hs, plan, pg, pw, pm, pv if sub.opt in ("adam", "lamb") else None, out_dt)
     O.unpack(plan, gathered if gathered is not None else pw)
     return time.perf_counter() - t0
 
@@ -358,6 +366,8 @@ def run_ours(args):
         B.ws_pack(plan, src, dst)
     if wl.opt in ("sgdm", "lars"):
         pv = None
+    if wl.opt == "adafactor":
+        pm, pv = None, W.make_factored_state(wl, plan.factored_elems, dev)
     del w, m, v
     g_arena = [torch.zeros(A_el, dtype=gdt, device=dev) for _ in range(R)]
     g_views = [B.PtrList(plan.arena_views(a, numels)) for a in g_arena]
@@ -513,9 +523,11 @@ def run_ours(args):
     except Exception:
         pass
     bpp = bytes_per_param(wl)
-    n_upd_launch = 3 if wl.opt in ("lamb", "lars") else 1
+    n_upd_launch = {"lamb": 3, "lars": 3, "adafactor": 6}.get(wl.opt, 1)
     chunks = -(-T // 1024)
     upd_name = ("update_kernel" if n_upd_launch == 1 else
+                "update_kernel pass 1 + af_moments_kernel + af_factors_kernel + pass 2 + af_finalize_clip_kernel + pass 3"
+                if n_upd_launch == 6 else
                 "update_kernel phase 1 + lamb_finalize_kernel + update_kernel phase 2")
 
     def kernel_rows(path):

@@ -248,10 +248,12 @@ ws_status ws_plan_factored_layout(const ws_plan* plan, int64_t* layout);
  *   float  ghat[R][S]        the summed gradients kept from phase 1 for phase 2
  * WS_ADAFACTOR uses all four (rho holds the applied step size alpha_t / max(1,
  * RMS(U_t)/d), norms sum w^2 and sum U^2) followed by
- *   float  acc[F]            this step's row / column sums of g^2 + eps
- *   float  fac[F]            1/sqrt factors of V for the two elementwise passes
+ *   float  acc[F']           this step's row / column sums of g^2 + eps
+ *   double rsum[T]           sum of the new row accumulators per tensor
+ *   float  fac[F']           1/sqrt factors of V for the two elementwise passes
  *   float  alpha[T]          max(eps2, RMS(w_t)) min(lr, 1/sqrt(step))
- * with F = ws_plan_factored_elems(). */
+ * where F' is F = ws_plan_factored_elems() with every tensor's row part and
+ * column part padded to a multiple of 8 floats. */
 size_t ws_workspace_bytes(const ws_plan* plan, ws_opt opt);
 
 /* Fused reduce + optimizer update + gathered-layout write for shard r

@@ -42,6 +42,18 @@ struct WsSegAf {
     long long nrow;
     long long ncol;
     long long numel;
+    // the workspace arrays (this step's sums, the 1/sqrt factors) use a padded layout so that a
+    // thread's run of columns can be moved as one vector: row part and column part each start on
+    // a multiple of 8 floats
+    long long irow;
+    long long icol;
+};
+
+// The finalize steps walk the factored state in chunks of at most 1024 entries (one CTA each).
+struct WsAfChunk {
+    long long begin;   // first entry inside tensor seg's state (0 .. nrow + ncol)
+    int count;
+    int seg;
 };
 
 struct ws_plan {
@@ -60,8 +72,11 @@ struct ws_plan {
     const WsTile* d_tiles = nullptr;
     const WsSegTiles* d_segtiles = nullptr;
     std::vector<WsSegAf> segaf;
+    std::vector<WsAfChunk> afchunks;
     long long F = 0;                          // total factored-state floats
+    long long Fi = 0;                         // floats of the padded workspace layout
     const WsSegAf* d_segaf = nullptr;
+    const WsAfChunk* d_afchunks = nullptr;
 };
 
 // Optimizer constants narrowed to fp32 for the kernels.
@@ -77,8 +92,10 @@ struct WsLambWs {
     size_t bytes;      // through the partials: what LAMB needs
     float* ghat;       // LARS only: [R][S] summed gradients, 256-byte aligned after the partials
     size_t bytes_lars; // through ghat: what LARS needs
-    float* acc;        // Adafactor: [F] this step's row / column sums
-    float* fac;        // Adafactor: [F] 1/sqrt factors of V
+    float* acc;        // Adafactor: [Fi] this step's row / column sums (padded layout)
+    double* rsum;      // Adafactor: [T] sum of the new row accumulators, directly after acc
+    size_t acc_bytes;  // acc and rsum together: cleared at the start of every step
+    float* fac;        // Adafactor: [Fi] 1/sqrt factors of V (padded layout)
     float* alpha;      // Adafactor: [T] step sizes
     size_t bytes_af;   // through alpha: what Adafactor needs
 };

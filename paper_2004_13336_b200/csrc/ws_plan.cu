@@ -45,7 +45,8 @@ extern "C" const char* ws_status_string(ws_status s) {
 // dimensions together; fewer than two dimensions: one row, no row accumulator.
 static void ws_matrix_views(ws_plan* p, const ws_tensor_desc* descs) {
     p->segaf.resize(p->T);
-    long long foff = 0;
+    p->afchunks.clear();
+    long long foff = 0, ioff = 0;
     for (int t = 0; t < p->T; ++t) {
         const ws_tensor_desc& d = descs[t];
         const long long n = p->segs[t].numel;
@@ -60,9 +61,21 @@ static void ws_matrix_views(ws_plan* p, const ws_tensor_desc* descs) {
             a.ncol = n;
         }
         foff += a.nrow + a.ncol;
+        a.irow = ioff;
+        ioff += (a.nrow + 7) / 8 * 8;
+        a.icol = ioff;
+        ioff += (a.ncol + 7) / 8 * 8;
         p->segaf[t] = a;
+        for (long long b = 0; b < a.nrow + a.ncol; b += 1024) {
+            WsAfChunk c;
+            c.begin = b;
+            c.count = (int)((a.nrow + a.ncol - b) < 1024 ? (a.nrow + a.ncol - b) : 1024);
+            c.seg = t;
+            p->afchunks.push_back(c);
+        }
     }
     p->F = foff;
+    p->Fi = ioff;
 }
 
 extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int32_t R,
@@ -238,7 +251,7 @@ static size_t round16(size_t x) { return (x + 15) & ~(size_t)15; }
 extern "C" size_t ws_plan_device_bytes(const ws_plan* p) {
     if (!p) return 0;
     return round16(p->tiles.size() * sizeof(WsTile)) + round16(p->segtiles.size() * sizeof(WsSegTiles)) +
-           round16(p->segaf.size() * sizeof(WsSegAf));
+           round16(p->segaf.size() * sizeof(WsSegAf)) + round16(p->afchunks.size() * sizeof(WsAfChunk));
 }
 
 extern "C" int64_t ws_plan_factored_elems(const ws_plan* p) { return p ? p->F : 0; }
@@ -272,6 +285,12 @@ extern "C" ws_status ws_plan_upload(ws_plan* p, void* dev_buf, size_t bytes, voi
     p->d_tiles = (const WsTile*)base;
     p->d_segtiles = (const WsSegTiles*)(base + round16(tb));
     p->d_segaf = (const WsSegAf*)(base + ab);
+    const size_t cb = ab + round16(p->segaf.size() * sizeof(WsSegAf));
+    if (!p->afchunks.empty()) {
+        e = cudaMemcpyAsync(base + cb, p->afchunks.data(), p->afchunks.size() * sizeof(WsAfChunk), cudaMemcpyHostToDevice, st);
+        if (e != cudaSuccess) return ws_cuda_fail(e, "ws_plan_upload(state chunks)");
+    }
+    p->d_afchunks = (const WsAfChunk*)(base + cb);
     return WS_OK;
 }
 
@@ -291,9 +310,14 @@ WsLambWs ws_lamb_layout(const ws_plan* p, void* workspace) {
     L.bytes_lars = o + sizeof(float) * (size_t)p->R * (size_t)p->S;
     o = (L.bytes_lars + 255) & ~(size_t)255;
     L.acc = (float*)(b + o);
-    o = (o + sizeof(float) * (size_t)p->F + 255) & ~(size_t)255;
+    const size_t acc0 = o;
+    o = (o + sizeof(float) * (size_t)p->Fi + 15) & ~(size_t)15;
+    L.rsum = (double*)(b + o);
+    o += sizeof(double) * (size_t)p->T;
+    L.acc_bytes = o - acc0;
+    o = (o + 255) & ~(size_t)255;
     L.fac = (float*)(b + o);
-    o = (o + sizeof(float) * (size_t)p->F + 255) & ~(size_t)255;
+    o = (o + sizeof(float) * (size_t)p->Fi + 255) & ~(size_t)255;
     L.alpha = (float*)(b + o);
     L.bytes_af = o + sizeof(float) * (size_t)p->T;
     return L;

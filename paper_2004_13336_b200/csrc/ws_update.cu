@@ -65,8 +65,6 @@ __host__ __device__ constexpr bool is_phase1(int o) { return o == K_LAMB1 || o =
 __host__ __device__ constexpr bool is_phase2(int o) { return o == K_LAMB2 || o == K_LARS2 || o == K_AF2 || o == K_AF3; }
 __host__ __device__ constexpr bool writes_weights(int o) { return !is_phase1(o) && o != K_AF2; }
 __host__ __device__ constexpr bool leaves_partials(int o) { return is_phase1(o) || o == K_AF2; }
-constexpr int kAfRows = 2048;   // shared-memory row accumulators of one tile (Adafactor pass 1)
-constexpr int kAfCols = 4096;   // shared-memory column accumulators
 enum { O_NONE = 0, O_F32 = 1, O_BF16 = 2 };
 
 template <int N>
@@ -310,6 +308,17 @@ __device__ __forceinline__ float block_sum(float x, float* smem /* kBlock/32 flo
     return t;  // valid in thread 0
 }
 
+// Adds VEC consecutive floats to global memory with vector reductions (one or two
+// red.global.add.v4.f32; p is 16-byte aligned).  Floating-point reductions on global memory are
+// native at the L2; on shared memory they would be compare-and-swap loops.
+template <int VEC>
+__device__ __forceinline__ void red_add_vec(float* p, const float* x) {
+#pragma unroll
+    for (int j = 0; j < VEC; j += 4)
+        asm volatile("red.global.add.v4.f32 [%0], {%1,%2,%3,%4};"
+                     :: "l"(p + j), "f"(x[j]), "f"(x[j + 1]), "f"(x[j + 2]), "f"(x[j + 3]) : "memory");
+}
+
 // ---------------------------------------------------------------- kernel ---
 // OPT: optimizer / phase.  GBF: gradients are bf16.  OUT: gathered dtype.
 // VEC: elements per thread access.  U: accesses per thread per pass.
@@ -334,9 +343,6 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
     // fused formatting: this tile's R gradient tensor pointers, fetched once per work item (the
     // streaming data would push the table's lines out of L1 between passes)
     __shared__ const void* sgp[(FUSED && READS_G) ? NP : 1];
-    // Adafactor pass 1: this tile's partial row sums and column sums
-    __shared__ float srow[OPT == K_AF1 ? kAfRows : 1];
-    __shared__ float scol[OPT == K_AF1 ? kAfCols : 1];
 
     for (long long item = blockIdx.x; item < P.nitems; item += gridDim.x) {
         long long rs = P.concat ? 0 : item / P.ntiles;     // shard index inside this launch
@@ -369,8 +375,7 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
         // Adafactor: where the tile starts inside its tensor's rows x cols matrix
         WsSegAf af;
         long long row0 = 0, c0 = 0;
-        int nrows_tile = 0;
-        bool rowsum = false, bigcol = false, rows_sm = false, cols_sm = false;
+        bool rowsum = false, bigcol = false;
         if constexpr (is_af(OPT)) {
             af = P.segaf[tl.seg];
             rowsum = af.nrow > 0;                          // unfactored tensors are one row
@@ -379,29 +384,41 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
                 c0 = toff - row0 * af.ncol;
             }
             bigcol = af.ncol >= tl.len;                    // the tile touches at most two rows
-            if constexpr (OPT == K_AF1) {
-                if (rowsum && nvalid > 0) {
-                    const long long nr = (c0 + nvalid - 1) / af.ncol + 1;
-                    rows_sm = nr <= kAfRows;
-                    cols_sm = af.ncol <= kAfCols;
-                    nrows_tile = rows_sm ? (int)nr : 0;
-                    __syncthreads();                       // the previous item's flush is done
-                    for (int k = threadIdx.x; k < nrows_tile; k += kBlock) srow[k] = 0.f;
-                    if (cols_sm)
-                        for (int k = threadIdx.x; k < (int)af.ncol; k += kBlock) scol[k] = 0.f;
-                    __syncthreads();
-                }
-            }
         }
+        // When the row length is a multiple of VEC a vector never straddles rows and starts on a
+        // multiple of VEC (colrun).  Pass 1 then adds a vector's g^2 + eps1 to the column sums with
+        // one vector reduction; when the row length also divides the CTA's stride, a thread meets the
+        // same VEC columns on every pass (and no other thread of the CTA does), keeps their sums in
+        // registers and adds them once per tile (stationary).
+        const bool colrun = is_af(OPT) && af.ncol % VEC == 0;
+        const bool stationary = colrun && (kBlock * VEC * U) % af.ncol == 0;
+        float cacc[OPT == K_AF1 ? VEC : 1];
+        long long cbase = -1;
+#pragma unroll
+        for (int j = 0; j < (OPT == K_AF1 ? VEC : 1); ++j) cacc[j] = 0.f;
 
         for (int q0 = 0; q0 < nvec; q0 += U * kBlock) {
             int e0[U];
             int nv[U];
             Fv<VEC> wv[U], mv[U], vv[U], gv[U], gc[U];
+            unsigned rl0[is_af(OPT) ? U : 1];      // Adafactor: row (relative to the tile's first) and
+            long long col0[is_af(OPT) ? U : 1];    // column of each vector's first element
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 const int q = q0 + u * kBlock + threadIdx.x;
                 e0[u] = q * VEC;
+                if constexpr (is_af(OPT)) {
+                    long long col = c0 + q * VEC;
+                    unsigned rl = 0;
+                    if (bigcol) {
+                        if (col >= af.ncol) { rl = 1; col -= af.ncol; }
+                    } else if (q < nvec) {
+                        rl = (unsigned)col / (unsigned)af.ncol;
+                        col = (unsigned)col - rl * (unsigned)af.ncol;
+                    }
+                    rl0[u] = rl;
+                    col0[u] = col;
+                }
                 const int left = nvalid - e0[u];
                 nv[u] = q < nvec ? (left < 0 ? 0 : (left > VEC ? VEC : left)) : -1;  // -1: nothing here
 #pragma unroll
@@ -470,41 +487,60 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
 #pragma unroll
                 for (int u = 0; u < U; ++u) {
                     const bool has = nv[u] > 0;
-                    long long col = c0 + e0[u];
-                    unsigned rl = 0;
-                    if (bigcol) {
-                        if (col >= af.ncol) { rl = 1; col -= af.ncol; }
-                    } else {
-                        rl = (unsigned)col / (unsigned)af.ncol;
-                        col = (unsigned)col - rl * (unsigned)af.ncol;
-                    }
+                    long long col = col0[u];
+                    unsigned rl = rl0[u];
                     unsigned cur = rl;
                     bool simple = true;
                     float racc = 0.f;
                     if (has) {
-                        float* gcol = P.af_acc + af.foff + af.nrow;
+                        float* gcol = P.af_acc + af.icol;
+                        float xs[VEC];
 #pragma unroll
                         for (int j = 0; j < VEC; ++j) {
+                            xs[j] = 0.f;
                             if (j < nv[u]) {
                                 const float g = gv[u].f[j] * P.c.gscale;
                                 gv[u].f[j] = g;
                                 sw = fmaf(wv[u].f[j], wv[u].f[j], sw);
-                                const float x = fmaf(g, g, P.c.eps);
-                                if (!rowsum) {
-                                    gcol[col] = x;                 // unfactored: every element has its own slot
+                                xs[j] = fmaf(g, g, P.c.eps);
+                            }
+                        }
+                        if (colrun) {
+                            // the whole vector lies in one row, on VEC aligned columns
+                            if (!rowsum) {
+                                // unfactored: every element has its own slot
+#pragma unroll
+                                for (int j = 0; j < VEC; j += 4)
+                                    *reinterpret_cast<float4*>(gcol + col + j) = make_float4(xs[j], xs[j + 1], xs[j + 2], xs[j + 3]);
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < VEC; ++j) racc += xs[j];
+                                if (stationary) {
+                                    cbase = col;
+#pragma unroll
+                                    for (int j = 0; j < VEC; ++j) cacc[j] += xs[j];
                                 } else {
-                                    if (cols_sm) atomicAdd(&scol[col], x);
-                                    else atomicAdd(&gcol[col], x);
-                                    if (rl != cur) {
-                                        if (rows_sm) atomicAdd(&srow[cur], racc);
-                                        else atomicAdd(&P.af_acc[af.foff + row0 + cur], racc);
-                                        racc = 0.f;
-                                        cur = rl;
-                                        simple = false;
-                                    }
-                                    racc += x;
+                                    red_add_vec<VEC>(gcol + col, xs);
                                 }
-                                if (++col == af.ncol) { col = 0; ++rl; }
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < VEC; ++j) {
+                                if (j < nv[u]) {
+                                    if (!rowsum) {
+                                        gcol[col] = xs[j];
+                                    } else {
+                                        atomicAdd(&gcol[col], xs[j]);
+                                        if (rl != cur) {
+                                            atomicAdd(&P.af_acc[af.irow + row0 + cur], racc);
+                                            racc = 0.f;
+                                            cur = rl;
+                                            simple = false;
+                                        }
+                                        racc += xs[j];
+                                    }
+                                    if (++col == af.ncol) { col = 0; ++rl; }
+                                }
                             }
                         }
                     }
@@ -518,13 +554,9 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
                                 float tsum = has ? racc : 0.f;
 #pragma unroll
                                 for (int o = 16; o > 0; o >>= 1) tsum += __shfl_xor_sync(0xffffffffu, tsum, o);
-                                if ((int)(threadIdx.x & 31) == lead) {
-                                    if (rows_sm) atomicAdd(&srow[lead_row], tsum);
-                                    else atomicAdd(&P.af_acc[af.foff + row0 + lead_row], tsum);
-                                }
+                                if ((int)(threadIdx.x & 31) == lead) atomicAdd(&P.af_acc[af.irow + row0 + lead_row], tsum);
                             } else if (has) {
-                                if (rows_sm) atomicAdd(&srow[cur], racc);
-                                else atomicAdd(&P.af_acc[af.foff + row0 + cur], racc);
+                                atomicAdd(&P.af_acc[af.irow + row0 + cur], racc);
                             }
                         }
                     }
@@ -536,31 +568,45 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
                 if constexpr (OPT == K_AF2 || OPT == K_AF3) {
                     // U = g / sqrt(V) with V = Rv' Cv'^T / sum(Rv'): the finalize step left
                     // sqrt(sum(Rv') / Rv'_i) and 1 / sqrt(Cv'_j), so U = g * fr_i * fc_j
-                    long long col = c0 + e0[u];
-                    unsigned rl = 0;
-                    if (bigcol) {
-                        if (col >= af.ncol) { rl = 1; col -= af.ncol; }
-                    } else {
-                        rl = (unsigned)col / (unsigned)af.ncol;
-                        col = (unsigned)col - rl * (unsigned)af.ncol;
-                    }
-                    const float* frp = P.af_fac + af.foff + row0;
-                    const float* fcp = P.af_fac + af.foff + af.nrow;
+                    long long col = col0[u];
+                    unsigned rl = rl0[u];
+                    const float* frp = P.af_fac + af.irow + row0;
+                    const float* fcp = P.af_fac + af.icol;
                     float fr = 1.f;
                     if (rowsum && nv[u] > 0) fr = __ldg(frp + rl);
+                    if (colrun && nv[u] > 0) {
+                        // the vector lies in one row and its column factors are one aligned vector
+                        float fc[VEC];
 #pragma unroll
-                    for (int j = 0; j < VEC; ++j) {
-                        if (j < nv[u]) {
-                            const float uu = (gv[u].f[j] * fr) * __ldg(fcp + col);
-                            if (OPT == K_AF2) su = fmaf(uu, uu, su);
-                            else wv[u].f[j] = fmaf(-lr_rho, uu, wv[u].f[j]);
-                            if (++col == af.ncol) {
-                                col = 0;
-                                ++rl;
-                                if (rowsum && j + 1 < nv[u]) fr = __ldg(frp + rl);
+                        for (int j4 = 0; j4 < VEC; j4 += 4) {
+                            const float4 t4 = __ldg(reinterpret_cast<const float4*>(fcp + col + j4));
+                            fc[j4] = t4.x; fc[j4 + 1] = t4.y; fc[j4 + 2] = t4.z; fc[j4 + 3] = t4.w;
+                        }
+#pragma unroll
+                        for (int j = 0; j < VEC; ++j) {
+                            if (j < nv[u]) {
+                                const float uu = (gv[u].f[j] * fr) * fc[j];
+                                if (OPT == K_AF2) su = fmaf(uu, uu, su);
+                                else wv[u].f[j] = fmaf(-lr_rho, uu, wv[u].f[j]);
+                            } else {
+                                wv[u].f[j] = 0.f;
                             }
-                        } else {
-                            wv[u].f[j] = 0.f;
+                        }
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < VEC; ++j) {
+                            if (j < nv[u]) {
+                                const float uu = (gv[u].f[j] * fr) * __ldg(fcp + col);
+                                if (OPT == K_AF2) su = fmaf(uu, uu, su);
+                                else wv[u].f[j] = fmaf(-lr_rho, uu, wv[u].f[j]);
+                                if (++col == af.ncol) {
+                                    col = 0;
+                                    ++rl;
+                                    if (rowsum && j + 1 < nv[u]) fr = __ldg(frp + rl);
+                                }
+                            } else {
+                                wv[u].f[j] = 0.f;
+                            }
                         }
                     }
                 } else {
@@ -599,25 +645,18 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
             }
         }
         if constexpr (OPT == K_AF1) {
-            // the tile's sums join the tensor's (this add of partial reduce results across tiles
-            // and shards stands where the paper combines them with an all-reduce, Section 4.1)
-            if (rowsum && nvalid > 0) {
-                __syncthreads();
-                for (int k = threadIdx.x; k < nrows_tile; k += kBlock) atomicAdd(&P.af_acc[af.foff + row0 + k], srow[k]);
-                if (cols_sm) {
-                    const int ncov = nvalid < af.ncol ? nvalid : (int)af.ncol;
-                    for (int k = threadIdx.x; k < ncov; k += kBlock) {
-                        long long col = c0 + k;
-                        if (col >= af.ncol) col -= af.ncol;
-                        atomicAdd(&P.af_acc[af.foff + af.nrow + col], scol[col]);
-                    }
-                }
-            }
+            // (these adds of partial reduce results across tiles and shards stand where the paper
+            // combines them with an all-reduce, Section 4.1)
+            if (cbase >= 0) red_add_vec<VEC>(P.af_acc + af.icol + cbase, cacc);
         }
         if (leaves_partials(OPT)) {
             const float a = block_sum(sw, red[0]);
             const float b = block_sum(su, red[1]);
-            if (threadIdx.x == 0) P.partials[P.concat ? ti : r * P.ntiles + ti] = make_float2(a, b);
+            if (threadIdx.x == 0) {
+                float2* dst = P.partials + (P.concat ? ti : r * P.ntiles + ti);
+                if (OPT == K_AF2) dst->y = b;          // pass 1's sum of w^2 stays in .x
+                else *dst = make_float2(a, b);
+            }
         }
     }
 }
@@ -670,63 +709,68 @@ __global__ void __launch_bounds__(kBlock) lamb_finalize_kernel(const WsSegTiles*
     }
 }
 
-// Adafactor, after pass 1 (one block per tensor): the moving averages of the row and column sums,
-// Rv' = beta Rv + (1-beta) acc, the factors the elementwise passes multiply by
-// (sqrt(sum(Rv') / Rv'_i) per row, 1/sqrt(Cv'_j) per column; 1/sqrt(v'_i) for an unfactored tensor),
-// and the step size alpha_t = max(eps2, RMS(w_t)) * rho_step from pass 1's partial sums of w^2.
-__global__ void __launch_bounds__(kBlock) af_finalize_moments_kernel(const WsSegTiles* segtiles, const WsSegAf* segaf,
-                                                                     const float2* partials, long long ntiles, int R,
-                                                                     float* state, const float* acc, float* fac,
-                                                                     float* alpha, double* norms, double beta,
-                                                                     double eps2, double rho_step) {
+// Adafactor, after pass 1, one CTA per chunk of at most 1024 state entries: the moving averages
+// Rv' = beta Rv + (1-beta) acc (rows, then columns; the full v' for an unfactored tensor), and the
+// sum of the tensor's new row accumulators (double atomic adds into rsum[t], cleared with acc).
+__global__ void __launch_bounds__(kBlock) af_moments_kernel(const WsAfChunk* chunks, const WsSegAf* segaf, float* state,
+                                                            const float* acc, double* rsum, double beta) {
     __shared__ double srs[kBlock];
-    const int t = blockIdx.x;
-    const WsSegAf a = segaf[t];
-    double sw, unused;
-    sum_partials(segtiles[t], partials, ntiles, R, sw, unused);
-    if (threadIdx.x == 0) {
-        const double rms_w = a.numel > 0 ? sqrt(sw / (double)a.numel) : 0.0;
-        alpha[t] = (float)((eps2 > rms_w ? eps2 : rms_w) * rho_step);
-        norms[2 * t] = sw;
-    }
-    float* vr = state + a.foff;
-    float* vc = vr + a.nrow;
+    const WsAfChunk ch = chunks[blockIdx.x];
+    const WsSegAf a = segaf[ch.seg];
     double rs = 0.0;
-    for (long long i = threadIdx.x; i < a.nrow; i += kBlock) {
-        const double v = beta * (double)vr[i] + (1.0 - beta) * (double)acc[a.foff + i];
-        vr[i] = (float)v;
-        rs += v;
+    for (int i = threadIdx.x; i < ch.count; i += kBlock) {
+        const long long e = ch.begin + i;
+        const bool isrow = e < a.nrow;
+        const long long k = isrow ? a.irow + e : a.icol + (e - a.nrow);
+        const double v = beta * (double)state[a.foff + e] + (1.0 - beta) * (double)acc[k];
+        state[a.foff + e] = (float)v;
+        if (isrow) rs += v;
     }
+    if (ch.begin >= a.nrow) return;     // a chunk of columns only (uniform over the CTA)
     srs[threadIdx.x] = rs;
     __syncthreads();
     for (int s = kBlock / 2; s > 0; s >>= 1) {
         if (threadIdx.x < s) srs[threadIdx.x] += srs[threadIdx.x + s];
         __syncthreads();
     }
-    rs = srs[0];
-    for (long long i = threadIdx.x; i < a.nrow; i += kBlock) fac[a.foff + i] = (float)sqrt(rs / (double)vr[i]);
-    for (long long j = threadIdx.x; j < a.ncol; j += kBlock) {
-        const double v = beta * (double)vc[j] + (1.0 - beta) * (double)acc[a.foff + a.nrow + j];
-        vc[j] = (float)v;
-        fac[a.foff + a.nrow + j] = (float)(1.0 / sqrt(v));
+    if (threadIdx.x == 0) atomicAdd(&rsum[ch.seg], srs[0]);
+}
+
+// ... then the factors the elementwise passes multiply by: sqrt(sum(Rv') / Rv'_i) per row,
+// 1/sqrt(Cv'_j) per column (1/sqrt(v'_i) for an unfactored tensor), so that U = g * fr_i * fc_j.
+__global__ void __launch_bounds__(kBlock) af_factors_kernel(const WsAfChunk* chunks, const WsSegAf* segaf,
+                                                            const float* state, const double* rsum, float* fac) {
+    const WsAfChunk ch = chunks[blockIdx.x];
+    const WsSegAf a = segaf[ch.seg];
+    const double rs = rsum[ch.seg];
+    for (int i = threadIdx.x; i < ch.count; i += kBlock) {
+        const long long e = ch.begin + i;
+        const double v = (double)state[a.foff + e];
+        if (e < a.nrow) fac[a.irow + e] = (float)sqrt(rs / v);
+        else fac[a.icol + (e - a.nrow)] = (float)(1.0 / sqrt(v));
     }
 }
 
-// Adafactor, after pass 2: RMS(U_t) from the partial sums of U^2, then the applied step size
-// rho[t] = alpha_t / max(1, RMS(U_t) / d).
+// Adafactor, after pass 2 (one CTA per tensor): the step size alpha_t = max(eps2, RMS(w_t)) *
+// rho_step from pass 1's partial sums of w^2, RMS(U_t) from pass 2's partial sums of U^2, and
+// the applied step size rho[t] = alpha_t / max(1, RMS(U_t) / d).
 __global__ void __launch_bounds__(kBlock) af_finalize_clip_kernel(const WsSegTiles* segtiles, const WsSegAf* segaf,
                                                                   const float2* partials, long long ntiles, int R,
-                                                                  const float* alpha, float* rho, double* norms,
-                                                                  double d) {
+                                                                  float* alpha, float* rho, double* norms, double eps2,
+                                                                  double rho_step, double d) {
     const int t = blockIdx.x;
-    double unused, su;
-    sum_partials(segtiles[t], partials, ntiles, R, unused, su);
+    double sw, su;
+    sum_partials(segtiles[t], partials, ntiles, R, sw, su);
     if (threadIdx.x == 0) {
         const long long n = segaf[t].numel;
+        const double rms_w = n > 0 ? sqrt(sw / (double)n) : 0.0;
         const double rms_u = n > 0 ? sqrt(su / (double)n) : 0.0;
+        const double al = (eps2 > rms_w ? eps2 : rms_w) * rho_step;
         const double clip = rms_u / d > 1.0 ? rms_u / d : 1.0;
+        norms[2 * t] = sw;
         norms[2 * t + 1] = su;
-        rho[t] = (float)((double)alpha[t] / clip);
+        alpha[t] = (float)al;
+        rho[t] = (float)(al / clip);
     }
 }
 
@@ -748,8 +792,11 @@ ws_status launch(const UpdParams& P, const void* const* gptrs, cudaStream_t st) 
 template <int OPT, bool GBF, int OUT, bool FUSED>
 ws_status launch_r(const UpdParams& P, const void* const* gptrs, bool wide_ok, cudaStream_t st) {
     if constexpr (is_phase2(OPT)) {
-        if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 1, 1, FUSED>(P, gptrs, st);
-        return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 1, 1, FUSED>(P, gptrs, st);
+        // Adafactor's later passes stream one (pass 2) or two (pass 3) arrays: more vectors per thread
+        // keep enough bytes in flight
+        constexpr int UA = OPT == K_AF2 ? 4 : (OPT == K_AF3 ? 2 : 1);
+        if (wide_ok) return launch<OPT, GBF, OUT, 8, UA, 1, 1, FUSED>(P, gptrs, st);
+        return launch<OPT, GBF, OUT, 4, UA * WS_TUNE_U4, 1, 1, FUSED>(P, gptrs, st);
     } else {
         if (P.R <= 2) {
             if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 2, 2, FUSED>(P, gptrs, st);
@@ -1117,10 +1164,8 @@ ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const
     const double rho_step = hyper->lr < inv_sqrt_t ? hyper->lr : inv_sqrt_t;
     const int reps = finalize_reps(plan);
 
-    if (plan->F > 0) {
-        cudaError_t e = cudaMemsetAsync(L.acc, 0, sizeof(float) * (size_t)plan->F, st);
-        if (e != cudaSuccess) return ws_cuda_fail(e, "adafactor(clear sums)");
-    }
+    cudaError_t e = cudaMemsetAsync(L.acc, 0, L.acc_bytes, st);
+    if (e != cudaSuccess) return ws_cuda_fail(e, "adafactor(clear sums)");
     UpdParams P;
     int ok;
     bool gbf;
@@ -1135,10 +1180,13 @@ ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const
         offset_grad_ptrs(plan, -1, grads, gp);
         if ((s = launch_any(K_AF1, gbf, O_NONE, P, gp.data(), st)) != WS_OK) return s;
     }
-    af_finalize_moments_kernel<<<plan->T, kBlock, 0, st>>>(plan->d_segtiles, plan->d_segaf, L.partials, plan->ntiles, reps,
-                                                          (float*)state->v, L.acc, L.fac, L.alpha, L.norms, beta,
-                                                          hyper->eps2, rho_step);
-    if ((s = ws_check_launch("adafactor(moments)")) != WS_OK) return s;
+    const unsigned nchunks = (unsigned)plan->afchunks.size();
+    if (nchunks > 0) {
+        af_moments_kernel<<<nchunks, kBlock, 0, st>>>(plan->d_afchunks, plan->d_segaf, (float*)state->v, L.acc, L.rsum, beta);
+        if ((s = ws_check_launch("adafactor(moments)")) != WS_OK) return s;
+        af_factors_kernel<<<nchunks, kBlock, 0, st>>>(plan->d_afchunks, plan->d_segaf, (const float*)state->v, L.rsum, L.fac);
+        if ((s = ws_check_launch("adafactor(factors)")) != WS_OK) return s;
+    }
 
     if ((s = prepare(plan, -1, nullptr, state, hyper, nullptr, K_AF2, P, ok, gbf)) != WS_OK) return s;
     P.partials = L.partials;
@@ -1146,7 +1194,8 @@ ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const
     P.af_fac = L.fac;
     if ((s = launch_any(K_AF2, false, O_NONE, P, nullptr, st)) != WS_OK) return s;
     af_finalize_clip_kernel<<<plan->T, kBlock, 0, st>>>(plan->d_segtiles, plan->d_segaf, L.partials, plan->ntiles, reps,
-                                                       L.alpha, L.rho, L.norms, hyper->clip_threshold);
+                                                       L.alpha, L.rho, L.norms, hyper->eps2, rho_step,
+                                                       hyper->clip_threshold);
     if ((s = ws_check_launch("adafactor(clipping)")) != WS_OK) return s;
 
     if (fused) return fused_phase(plan, -1, gtab, state, hyper, wtab, K_AF3, workspace, st);

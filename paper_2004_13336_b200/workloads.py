@@ -23,7 +23,7 @@ Shape = Tuple[int, ...]
 
 # optimizer codes shared by name only (values mirror the public C enum and the
 # oracle's enum; each side defines its own copy)
-SGDM, ADAM, LAMB, LARS = "sgdm", "adam", "lamb", "lars"
+SGDM, ADAM, LAMB, LARS, ADAFACTOR = "sgdm", "adam", "lamb", "lars", "adafactor"
 
 
 @dataclass
@@ -158,6 +158,13 @@ def transformer(R: int = 8) -> Workload:
                     hyper=_hyper(), seed=3, R_sweep=(1, 2, 8, 32, 128, 1024))
 
 
+def transformer_adafactor(R: int = 8) -> Workload:
+    """The Transformer tensor set under Adafactor, the optimizer the paper names (with LARS) for its
+    reduce operators (Section 4.1): factored second moments, clipping at 1, relative step size."""
+    return Workload("transformer_adafactor", transformer_shapes(), R=R, opt=ADAFACTOR,
+                    hyper=_hyper(lr=1e-2, eps=1e-30, eps2=1e-3, clip_threshold=1.0, decay_exponent=0.8), seed=7)
+
+
 def bert_large() -> Workload:
     return Workload("bert_large", bert_large_shapes(), R=16, opt=LAMB,
                     hyper=_hyper(eps=1e-6, weight_decay=0.01), seed=4)
@@ -173,6 +180,7 @@ def decoder_1p5b() -> Workload:
 WORKLOADS = {
     "tiny": tiny, "resnet50": resnet50, "transformer": transformer,
     "bert_large": bert_large, "decoder_1p5b": decoder_1p5b, "resnet50_lars": resnet50_lars,
+    "transformer_adafactor": transformer_adafactor,
 }
 
 
@@ -190,7 +198,7 @@ def scaled_down(wl: Workload, max_dim: int) -> Workload:
 # --------------------------------------------------------------------------
 # seeded generators (no method arithmetic)
 # --------------------------------------------------------------------------
-_ROLE = {"w": 1, "m": 2, "v": 3, "g": 4}
+_ROLE = {"w": 1, "m": 2, "v": 3, "g": 4, "f": 5}
 
 
 def _gen(device, seed: int, role: str, k: int) -> torch.Generator:
@@ -213,6 +221,13 @@ def make_state(wl: Workload, device="cpu"):
     m = [_normal(n, wl.m_std, gm, device) for n in wl.numels]
     v = [_normal(n, wl.v_std, gv, device).abs_() for n in wl.numels]
     return w, m, v
+
+
+def make_factored_state(wl: Workload, n: int, device="cpu") -> torch.Tensor:
+    """Adafactor's row / column accumulators (n floats for the whole model): uniform in
+    [1e-6, 1e-3], the size of sums of squared gradients a few steps into training."""
+    gen = _gen(device, wl.seed, "f", 0)
+    return torch.empty(n, dtype=torch.float32, device=device).uniform_(1e-6, 1e-3, generator=gen)
 
 
 def make_grads_one(wl: Workload, k: int, device="cpu", numels=None) -> List[torch.Tensor]:
