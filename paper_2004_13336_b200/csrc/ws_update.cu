@@ -48,6 +48,15 @@
 #ifndef WS_TUNE_U4
 #define WS_TUNE_U4 1     // 128-bit accesses per thread per pass
 #endif
+#ifndef WS_TUNE_UAF2
+#define WS_TUNE_UAF2 2   // ... in Adafactor's pass 1 with up to 2 / up to 4 / more gradient copies
+#endif
+#ifndef WS_TUNE_UAF4
+#define WS_TUNE_UAF4 2
+#endif
+#ifndef WS_TUNE_UAF8
+#define WS_TUNE_UAF8 1
+#endif
 
 namespace {
 
@@ -392,6 +401,25 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
         // registers and adds them once per tile (stationary).
         const bool colrun = is_af(OPT) && af.ncol % VEC == 0;
         const bool stationary = colrun && (kBlock * VEC * U) % af.ncol == 0;
+        // the thread's first vector starts at column run_col of row run_rl (relative to the tile's first
+        // row); consecutive vectors of a thread lie kBlock * VEC elements apart = sub_rl rows and
+        // sub_col columns, so rows and columns advance without a division per vector
+        long long run_col = 0, sub_col = 0;
+        unsigned run_rl = 0, sub_rl = 0;
+        if constexpr (is_af(OPT)) {
+            run_col = c0 + (long long)threadIdx.x * VEC;
+            sub_col = kBlock * VEC;
+            if (bigcol) {
+                if (run_col >= af.ncol) { run_rl = 1; run_col -= af.ncol; }
+            } else {
+                run_rl = (unsigned)run_col / (unsigned)af.ncol;
+                run_col = (unsigned)run_col - run_rl * (unsigned)af.ncol;
+            }
+            if (af.ncol <= kBlock * VEC) {
+                sub_rl = (unsigned)(kBlock * VEC) / (unsigned)af.ncol;
+                sub_col = (unsigned)(kBlock * VEC) - sub_rl * (unsigned)af.ncol;
+            }
+        }
         float cacc[OPT == K_AF1 ? VEC : 1];
         long long cbase = -1;
 #pragma unroll
@@ -408,16 +436,12 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
                 const int q = q0 + u * kBlock + threadIdx.x;
                 e0[u] = q * VEC;
                 if constexpr (is_af(OPT)) {
-                    long long col = c0 + q * VEC;
-                    unsigned rl = 0;
-                    if (bigcol) {
-                        if (col >= af.ncol) { rl = 1; col -= af.ncol; }
-                    } else if (q < nvec) {
-                        rl = (unsigned)col / (unsigned)af.ncol;
-                        col = (unsigned)col - rl * (unsigned)af.ncol;
-                    }
-                    rl0[u] = rl;
-                    col0[u] = col;
+                    // this vector's row and column, then on to the thread's next vector
+                    rl0[u] = run_rl;
+                    col0[u] = run_col;
+                    run_col += sub_col;
+                    run_rl += sub_rl;
+                    if (run_col >= af.ncol) { run_col -= af.ncol; ++run_rl; }
                 }
                 const int left = nvalid - e0[u];
                 nv[u] = q < nvec ? (left < 0 ? 0 : (left > VEC ? VEC : left)) : -1;  // -1: nothing here
@@ -650,8 +674,9 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
             if (cbase >= 0) red_add_vec<VEC>(P.af_acc + af.icol + cbase, cacc);
         }
         if (leaves_partials(OPT)) {
-            const float a = block_sum(sw, red[0]);
-            const float b = block_sum(su, red[1]);
+            // (Adafactor's passes leave one sum each)
+            const float a = OPT == K_AF2 ? 0.f : block_sum(sw, red[0]);
+            const float b = OPT == K_AF1 ? 0.f : block_sum(su, red[1]);
             if (threadIdx.x == 0) {
                 float2* dst = P.partials + (P.concat ? ti : r * P.ntiles + ti);
                 if (OPT == K_AF2) dst->y = b;          // pass 1's sum of w^2 stays in .x
@@ -792,26 +817,23 @@ ws_status launch(const UpdParams& P, const void* const* gptrs, cudaStream_t st) 
 template <int OPT, bool GBF, int OUT, bool FUSED>
 ws_status launch_r(const UpdParams& P, const void* const* gptrs, bool wide_ok, cudaStream_t st) {
     if constexpr (is_phase2(OPT)) {
-        // Adafactor's later passes stream one (pass 2) or two (pass 3) arrays: more vectors per thread
-        // keep enough bytes in flight
-        constexpr int UA = OPT == K_AF2 ? 4 : (OPT == K_AF3 ? 2 : 1);
-        if (wide_ok) return launch<OPT, GBF, OUT, 8, UA, 1, 1, FUSED>(P, gptrs, st);
-        return launch<OPT, GBF, OUT, 4, UA * WS_TUNE_U4, 1, 1, FUSED>(P, gptrs, st);
+        if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 1, 1, FUSED>(P, gptrs, st);
+        return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 1, 1, FUSED>(P, gptrs, st);
     } else {
         if (P.R <= 2) {
-            if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 2, 2, FUSED>(P, gptrs, st);
-            return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 2, 2, FUSED>(P, gptrs, st);
+            if constexpr (OPT != K_AF1) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 2, 2, FUSED>(P, gptrs, st);
+            return launch<OPT, GBF, OUT, 4, OPT == K_AF1 ? WS_TUNE_UAF2 : WS_TUNE_U4, 2, 2, FUSED>(P, gptrs, st);
         }
         if (P.R <= 4) {
-            if constexpr (GBF) if (wide_ok) return launch<OPT, GBF, OUT, 8, WS_TUNE_U8, 4, 4, FUSED>(P, gptrs, st);
-            return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 4, 4, FUSED>(P, gptrs, st);
+            if constexpr (GBF && OPT != K_AF1) if (wide_ok) return launch<OPT, GBF, OUT, 8, WS_TUNE_U8, 4, 4, FUSED>(P, gptrs, st);
+            return launch<OPT, GBF, OUT, 4, OPT == K_AF1 ? WS_TUNE_UAF4 : WS_TUNE_U4, 4, 4, FUSED>(P, gptrs, st);
         }
         if (P.R <= 8) {
-            if constexpr (GBF) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 8, 8, FUSED>(P, gptrs, st);
-            return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 8, 8, FUSED>(P, gptrs, st);
+            if constexpr (GBF && OPT != K_AF1) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 8, 8, FUSED>(P, gptrs, st);
+            return launch<OPT, GBF, OUT, 4, OPT == K_AF1 ? WS_TUNE_UAF8 : WS_TUNE_U4, 8, 8, FUSED>(P, gptrs, st);
         }
         if (P.R <= 32) {
-            if constexpr (GBF) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 8, 32, FUSED>(P, gptrs, st);
+            if constexpr (GBF && OPT != K_AF1) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 8, 32, FUSED>(P, gptrs, st);
             return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 8, 32, FUSED>(P, gptrs, st);
         }
         // many replicas make small shards and few CTAs: more loads in flight per thread
@@ -829,6 +851,7 @@ ws_status launch_o(const UpdParams& P, const void* const* gptrs, int out, bool w
     if (!FUSED && !is_phase2(OPT))
         for (int k = 0; k < P.R && wide; ++k) wide = aligned32(gptrs[k]);
     if (OPT == K_LARS1 || OPT == K_LARS2 || is_af(OPT)) wide = wide && aligned32(P.ghat);
+    if (OPT == K_AF1) wide = false;   // pass 1 is instruction-heavy: 128-bit vectors measured faster at every R
     if constexpr (OPT == K_AF2) {
         return launch_r<OPT, false, O_NONE, false>(P, gptrs, wide, st);   // touches no tensor list and no output
     } else if constexpr (is_phase1(OPT)) {
