@@ -652,7 +652,8 @@ def large_workload_rows(args):
     """Short fused-route runs of the large model-shaped workloads (each in its own process so that its
     memory is returned), summarised next to the headline workload."""
     rows = []
-    for name, extra in (("transformer", ["--R", "8"]), ("bert_large", []), ("decoder_1p5b", [])):
+    for name, extra in (("transformer", ["--R", "8"]), ("bert_large", []), ("decoder_1p5b", []),
+                        ("transformer_adafactor", [])):
         cmd = [sys.executable, os.path.abspath(__file__), "--workload", name, *extra, "--path", "fused", "--steps", "30",
                "--warmup", "5", "--no-e2e", "--no-cpu-baseline", "--no-large", "--align", str(args.align)]
         try:

@@ -389,8 +389,14 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
             af = P.segaf[tl.seg];
             rowsum = af.nrow > 0;                          // unfactored tensors are one row
             if (af.ncol > 0) {
-                row0 = toff / af.ncol;
-                c0 = toff - row0 * af.ncol;
+                if ((((unsigned long long)toff | (unsigned long long)af.ncol) >> 32) == 0) {
+                    const unsigned q32 = (unsigned)toff / (unsigned)af.ncol;   // the usual case: no 64-bit division
+                    row0 = q32;
+                    c0 = (unsigned)toff - q32 * (unsigned)af.ncol;
+                } else {
+                    row0 = toff / af.ncol;
+                    c0 = toff - row0 * af.ncol;
+                }
             }
             bigcol = af.ncol >= tl.len;                    // the tile touches at most two rows
         }

@@ -321,3 +321,53 @@ def test_resnet50_lars_full_model_every_element():
     er = float(np.max(np.abs(rate - np.array(orate)) / np.array(orate)))
     print(f"resnet50 LARS full: err w {ew:.2e} m {em:.2e} rate {er:.2e}")
     assert ew <= TOL_LAMB and em <= TOL_LAMB and er <= TOL_LAMB
+
+
+def test_transformer_adafactor_whole_tensors():
+    """The Transformer tensor set under Adafactor (the paper's example, with LARS, of an optimizer whose
+    reduces the sharding cuts, Section 4.1), R=8, full size, through the fused route the benchmark
+    times.  The oracle recomputes whole tensors (row and column sums span all shards): the embedding,
+    the first and last layers with their vectors, one of each matrix shape."""
+    wl = W.transformer_adafactor()
+    torch.cuda.empty_cache()
+    plan = B.Plan(wl.shapes, wl.R, A)
+    hy = B.make_hyper(wl.opt, wl.hyper)
+    hs = O.make_hyper(wl.opt, wl.hyper)
+    chosen = sorted(set([0] + list(range(1, 12)) + list(range(wl.T - 14, wl.T))))
+    w, _, _ = W.make_state(wl, DEV)
+    f0 = W.make_factored_state(wl, plan.factored_elems, DEV)
+    lay = plan.factored_layout()
+    rows_, cols_, foff_, tot = O.factor_shapes(wl.shapes)
+    assert tot == plan.factored_elems and [x[0] for x in lay] == foff_.tolist()
+    ref_w = {t: to_np(w[t]).reshape(wl.shapes[t]) for t in chosen}
+    ref_f = to_np(f0)
+    pw = torch.empty(plan.G, device=DEV)
+    B.ws_pack(plan, w, pw)
+    g = []
+    og = {t: [] for t in chosen}
+    for k in range(wl.R):
+        gk = W.make_grads_one(wl, k, DEV)
+        for t in chosen:
+            og[t].append(to_np(gk[t]))
+        g.append(gk)
+    ws = torch.empty(plan.workspace_bytes("adafactor"), dtype=torch.uint8, device=DEV)
+    outs = [torch.empty_like(x) for x in w]
+    fs = f0.clone()
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), pw, None, fs, hy, B.TensorTable(plan, [outs]), ws)
+    coef = ws[:4 * plan.T].view(torch.float32).cpu().numpy().astype(np.float64)
+    got_f = to_np(fs)
+    worst_w = worst_f = worst_c = 0.0
+    for t in chosen:
+        off, nr, nc = lay[t]
+        vr = ref_f[off:off + nr]
+        vc = ref_f[off + nr:off + nr + nc] if nc else None
+        alpha, rms_u, _ = O.adafactor_tensor(hs, og[t], ref_w[t], vr, vc)
+        worst_c = max(worst_c, abs(coef[t] - alpha / max(1.0, rms_u)) / (alpha / max(1.0, rms_u)))
+        worst_w = max(worst_w, err(to_np(outs[t]), ref_w[t]))
+        worst_f = max(worst_f, err(got_f[off:off + nr + nc], ref_f[off:off + nr + nc]))
+    print(f"transformer Adafactor: err w {worst_w:.2e} factored state {worst_f:.2e} step size {worst_c:.2e}")
+    assert worst_w <= TOL_LAMB and worst_f <= TOL_LAMB and worst_c <= TOL_LAMB
+    # the sharded weight state and the weight tensors hold the same values
+    B.ws_unpack(plan, pw, w)
+    for t in chosen:
+        assert torch.equal(w[t], outs[t])
