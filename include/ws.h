@@ -256,6 +256,16 @@ ws_status ws_plan_factored_layout(const ws_plan* plan, int64_t* layout);
  * column part padded to a multiple of 8 floats. */
 size_t ws_workspace_bytes(const ws_plan* plan, ws_opt opt);
 
+/* Where the per-tile partial sums live inside the workspace: byte offset of
+ * partials[0] and the bytes of one shard's row (per-tensor layout: tiles * 8).
+ * A multi-GPU caller that runs ws_lamb_partial for its own shard r on every
+ * rank exchanges row r with the other ranks (an all-gather of rows, or an
+ * all-reduce over rows that are zero elsewhere: the combination of per-replica
+ * reduce results of Section 4.1) before every rank calls ws_lamb_finalize.
+ * Host only.  WS_ERR_INVALID_ARG for the concatenated layout, whose shards own
+ * different numbers of tiles. */
+ws_status ws_workspace_partials(const ws_plan* plan, size_t* offset_bytes, size_t* row_bytes);
+
 /* Fused reduce + optimizer update + gathered-layout write for shard r
  * (0 <= r < R), or for all R shards in one launch when r == -1.
  * Reads the r-th slice of each of the R gradient buffers exactly once, w/m/v

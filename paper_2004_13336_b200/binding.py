@@ -82,7 +82,7 @@ EXPORTS = [
     "ws_static_scratch_bytes", "ws_lamb_update_static_scratch",
     "ws_tensor_table_bytes", "ws_tensor_table_upload", "ws_fused_update",
     "ws_plan_create_layout", "ws_plan_layout", "ws_pack_sets",
-    "ws_plan_factored_elems", "ws_plan_factored_layout",
+    "ws_plan_factored_elems", "ws_plan_factored_layout", "ws_workspace_partials",
 ]
 
 _lib = None
@@ -138,6 +138,8 @@ def lib() -> C.CDLL:
                                 C.POINTER(ws_out), vp, C.c_size_t, vp]
     L.ws_plan_arena_elems.restype = C.c_int64
     L.ws_plan_arena_elems.argtypes = [vp]
+    L.ws_workspace_partials.restype = C.c_int
+    L.ws_workspace_partials.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     L.ws_plan_factored_elems.restype = C.c_int64
     L.ws_plan_factored_elems.argtypes = [vp]
     L.ws_plan_factored_layout.restype = C.c_int
@@ -354,6 +356,13 @@ def ws_lamb_apply(plan: Plan, r: int, w, m, v, hyper: ws_hyper, workspace: torch
     _check(lib().ws_lamb_apply(plan.handle, r, C.byref(s), C.byref(hyper),
                                C.byref(o) if o is not None else None, workspace.data_ptr(),
                                workspace.numel() * workspace.element_size(), _stream()), "ws_lamb_apply")
+
+
+def lamb_partials(plan: Plan, workspace: torch.Tensor) -> torch.Tensor:
+    """The [R][tiles * 2] float view of the per-tile partial sums inside a LAMB workspace."""
+    off, row = C.c_size_t(), C.c_size_t()
+    _check(lib().ws_workspace_partials(plan.handle, C.byref(off), C.byref(row)), "ws_workspace_partials")
+    return workspace[off.value: off.value + plan.R * row.value].view(torch.float32).view(plan.R, row.value // 4)
 
 
 def lamb_ratios(plan: Plan, workspace: torch.Tensor) -> torch.Tensor:

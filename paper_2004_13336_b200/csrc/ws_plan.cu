@@ -323,6 +323,14 @@ WsLambWs ws_lamb_layout(const ws_plan* p, void* workspace) {
     return L;
 }
 
+extern "C" ws_status ws_workspace_partials(const ws_plan* p, size_t* offset_bytes, size_t* row_bytes) {
+    if (!p || !offset_bytes || !row_bytes || p->layout != WS_LAYOUT_PER_TENSOR) return WS_ERR_INVALID_ARG;
+    const WsLambWs L = ws_lamb_layout(p, nullptr);
+    *offset_bytes = (size_t)((char*)L.partials - (char*)nullptr);
+    *row_bytes = sizeof(float2) * (size_t)p->ntiles;
+    return WS_OK;
+}
+
 extern "C" size_t ws_workspace_bytes(const ws_plan* p, ws_opt opt) {
     if (!p) return 0;
     if (opt == WS_LAMB) return ws_lamb_layout(p, nullptr).bytes;

@@ -1,0 +1,66 @@
+"""The multi-replica route of Section 2.2 (pack, NCCL reduce-scatter, update of the own shard
+from the receive buffer, NCCL all-gather, unpack) on the GPU.  A run has one GPU, so the
+process group has one rank: the collectives are real NCCL calls on a world of one and the
+kernels run exactly as rank r of R would run them (single shard, slice_mode 1, LAMB in its
+three per-shard phases with the partial sums exchanged).  Ranks > 1 are covered on CPU
+(tests/test_collective_cpu.py)."""
+import socket
+
+import numpy as np
+import pytest
+import torch
+import torch.distributed as dist
+
+from oracle import ws_oracle as O
+from paper_2004_13336_b200 import workloads as W
+from paper_2004_13336_b200.collective import ShardedUpdate
+from tests._util import TOL_BF16, TOL_FP32, TOL_LAMB, bf16_to_f64, err, to_np
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+SHAPES = [(1,), (7,), (3, 3, 16, 32), (64, 128), (1031,), (5, 1, 9), (4099, 3), (300, 301)]
+
+
+@pytest.fixture(scope="module")
+def world_of_one():
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    torch.cuda.set_device(0)
+    dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1)
+    yield
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("opt,out_dtype,gdtype", [("sgdm", torch.float32, torch.float32),
+                                                  ("adam", torch.bfloat16, torch.bfloat16),
+                                                  ("lamb", torch.float32, torch.float32),
+                                                  ("lamb", torch.bfloat16, torch.float32)])
+def test_one_rank_group_matches_the_oracle(world_of_one, opt, out_dtype, gdtype):
+    wl = W.Workload("t", list(SHAPES), R=1, opt=opt, hyper={}, grad_dtype=gdtype, grad_std=1e-2, seed=23)
+    w, m, v = W.make_state(wl, DEV)
+    g = W.make_grads(wl, DEV)[0]
+    hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-6, weight_decay=0.01 if opt != "adam" else 0.0,
+                 momentum=0.9, grad_scale=1.0, step=4)
+    su = ShardedUpdate(SHAPES, opt, hyper, out_dtype=out_dtype, grad_dtype=gdtype, device=DEV)
+    su.load_state(w, m, v)
+    outs = [torch.zeros(n, dtype=out_dtype, device=DEV) for n in wl.numels]
+    for step in (4, 5):                       # two steps: the sharded slots carry over
+        hyper["step"] = step
+        su.step(g, outs, step=step)
+    torch.cuda.synchronize()
+    ow, om, ov = [to_np(x) for x in w], [to_np(x) for x in m], [to_np(x) for x in v]
+    og = [to_np(x) for x in g]
+    for step in (4, 5):
+        hyper["step"] = step
+        O.update_unsharded(O.make_hyper(opt, hyper), [og], ow, om, ov if opt != "sgdm" else None)
+    tol = TOL_LAMB if opt == "lamb" else 2 * TOL_FP32
+    for t, (a, b) in enumerate(zip(outs, ow)):
+        if out_dtype == torch.bfloat16:
+            assert err(bf16_to_f64(to_np(a)), b) <= TOL_BF16, t
+        else:
+            assert err(to_np(a), b) <= tol, t
+    m_full = [torch.zeros(n, device=DEV) for n in wl.numels]
+    su.gather_slot(su.m, m_full)
+    for t, (a, b) in enumerate(zip(m_full, om)):
+        assert err(to_np(a), b) <= tol, t
