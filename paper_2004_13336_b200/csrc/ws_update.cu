@@ -48,6 +48,12 @@
 #ifndef WS_TUNE_U4
 #define WS_TUNE_U4 1     // 128-bit accesses per thread per pass
 #endif
+#ifndef WS_TUNE_AF2_UNROLL
+#define WS_TUNE_AF2_UNROLL 2
+#endif
+#ifndef WS_TUNE_AF2_CTAS
+#define WS_TUNE_AF2_CTAS 4   // CTAs per SM of Adafactor's pass 2 (a persistent grid)
+#endif
 #ifndef WS_TUNE_UAF2
 #define WS_TUNE_UAF2 2   // ... in Adafactor's pass 1 with up to 2 / up to 4 / more gradient copies
 #endif
@@ -61,11 +67,13 @@
 namespace {
 
 constexpr int kBlock = 256;
+constexpr int kAf2Unroll = WS_TUNE_AF2_UNROLL;
 // Kernel flavours.  The norm-based optimizers run as two phases around a finalize step:
 // phase 1 (K_LAMB1, K_LARS1) reduces the gradients and leaves per-tile partial sums of the
 // two norms; phase 2 (K_LAMB2, K_LARS2) applies the step with the per-tensor ratio.
 // Adafactor runs as three passes around two finalize steps: K_AF1 reduces the gradients, keeps
-// the sum and accumulates row / column sums of g^2 + eps1; K_AF2 sums U^2 per tensor; K_AF3 applies.
+// the sum and accumulates row / column sums of g^2 + eps1; K_AF2 sums U^2 per tensor (a kernel of its
+// own, af_sumsq_kernel; the id only names the pass to the argument checks); K_AF3 applies.
 enum { K_SGDM = 0, K_ADAM = 1, K_LAMB1 = 2, K_LAMB2 = 3, K_LARS1 = 4, K_LARS2 = 5, K_AF1 = 6, K_AF2 = 7, K_AF3 = 8 };
 __host__ __device__ constexpr bool is_af(int o) { return o == K_AF1 || o == K_AF2 || o == K_AF3; }
 // phase 1: reduces the gradient lists and leaves partial sums, no weight step
@@ -341,9 +349,9 @@ template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED
 __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8) ? WS_TUNE_MINB8 : WS_TUNE_MINB) update_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp) {
     constexpr bool HAS_V = (OPT == K_ADAM || OPT == K_LAMB1 || OPT == K_LAMB2);
     constexpr bool READS_G = !is_phase2(OPT);     // phase 2 works from state (and the stored gradient sum)
-    constexpr bool READS_W = (OPT != K_AF2);
+    constexpr bool READS_W = true;
     constexpr bool READS_M = (OPT != K_LARS1 && !is_af(OPT));
-    constexpr bool READS_GHAT = (OPT == K_LARS2 || OPT == K_AF2 || OPT == K_AF3);
+    constexpr bool READS_GHAT = (OPT == K_LARS2 || OPT == K_AF3);
     constexpr bool WRITES_W = writes_weights(OPT);   // phase 1 only zeroes the pads of w
     constexpr bool WRITES_M = (OPT != K_LAMB2 && OPT != K_LARS1 && !is_af(OPT));
     constexpr bool WRITES_GHAT = (OPT == K_LARS1 || OPT == K_AF1);
@@ -595,7 +603,7 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 if (nv[u] < 0) continue;
-                if constexpr (OPT == K_AF2 || OPT == K_AF3) {
+                if constexpr (OPT == K_AF3) {
                     // U = g / sqrt(V) with V = Rv' Cv'^T / sum(Rv'): the finalize step left
                     // sqrt(sum(Rv') / Rv'_i) and 1 / sqrt(Cv'_j), so U = g * fr_i * fc_j
                     long long col = col0[u];
@@ -616,8 +624,7 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
                         for (int j = 0; j < VEC; ++j) {
                             if (j < nv[u]) {
                                 const float uu = (gv[u].f[j] * fr) * fc[j];
-                                if (OPT == K_AF2) su = fmaf(uu, uu, su);
-                                else wv[u].f[j] = fmaf(-lr_rho, uu, wv[u].f[j]);
+                                wv[u].f[j] = fmaf(-lr_rho, uu, wv[u].f[j]);
                             } else {
                                 wv[u].f[j] = 0.f;
                             }
@@ -627,8 +634,7 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
                         for (int j = 0; j < VEC; ++j) {
                             if (j < nv[u]) {
                                 const float uu = (gv[u].f[j] * fr) * __ldg(fcp + col);
-                                if (OPT == K_AF2) su = fmaf(uu, uu, su);
-                                else wv[u].f[j] = fmaf(-lr_rho, uu, wv[u].f[j]);
+                                wv[u].f[j] = fmaf(-lr_rho, uu, wv[u].f[j]);
                                 if (++col == af.ncol) {
                                     col = 0;
                                     ++rl;
@@ -681,12 +687,11 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
         }
         if (leaves_partials(OPT)) {
             // (Adafactor's passes leave one sum each)
-            const float a = OPT == K_AF2 ? 0.f : block_sum(sw, red[0]);
+            const float a = block_sum(sw, red[0]);
             const float b = OPT == K_AF1 ? 0.f : block_sum(su, red[1]);
             if (threadIdx.x == 0) {
                 float2* dst = P.partials + (P.concat ? ti : r * P.ntiles + ti);
-                if (OPT == K_AF2) dst->y = b;          // pass 1's sum of w^2 stays in .x
-                else *dst = make_float2(a, b);
+                *dst = make_float2(a, b);      // (Adafactor's pass 1: b = 0, pass 2 adds its sum there)
             }
         }
     }
@@ -805,6 +810,117 @@ __global__ void __launch_bounds__(kBlock) af_finalize_clip_kernel(const WsSegTil
     }
 }
 
+// Adafactor pass 2 on its own: sum of U^2 per tile, U = g * fr_i * fc_j, from the stored gradient
+// sum and the factors.  It reads 4 bytes per parameter and nothing else, so a CTA that handled
+// one tile would spend most of its life waiting for the tile descriptor, then the matrix view,
+// then the row factor; here a CTA walks many tiles and fetches the next tile's descriptor and
+// matrix view while it works on the current one.
+__global__ void __launch_bounds__(kBlock, WS_TUNE_AF2_CTAS) af_sumsq_kernel(const UpdParams P) {
+    long long item = blockIdx.x;
+    if (item >= P.nitems) return;
+    auto tile_of = [&](long long it, long long& rs) {
+        rs = P.concat ? 0 : it / P.ntiles;
+        return P.concat ? P.tile_lo + it : it - rs * P.ntiles;
+    };
+    long long rs, ti = tile_of(item, rs);
+    WsTile tl = P.tiles[ti];
+    WsSegAf af = P.segaf[tl.seg];
+    while (true) {
+        const long long nxt = item + gridDim.x;
+        const bool more = nxt < P.nitems;
+        long long rs_n = 0, ti_n = 0;
+        WsTile tn = tl;
+        if (more) {
+            ti_n = tile_of(nxt, rs_n);
+            tn = P.tiles[ti_n];                        // in flight during this tile's work
+        }
+        if (P.concat) rs = tl.shard - P.r0;
+        const long long r = P.r0 + rs;
+        const long long nvl = tl.vt - r * tl.piece;
+        const int nvalid = nvl < 0 ? 0 : (nvl > tl.len ? tl.len : (int)nvl);
+        const float* g = P.ghat + r * P.S + tl.pos;
+        const long long toff = r * tl.piece + tl.poff;
+        long long row0 = 0, c0 = 0;
+        if (af.ncol > 0) {
+            if ((((unsigned long long)toff | (unsigned long long)af.ncol) >> 32) == 0) {
+                const unsigned q32 = (unsigned)toff / (unsigned)af.ncol;
+                row0 = q32;
+                c0 = (unsigned)toff - q32 * (unsigned)af.ncol;
+            } else {
+                row0 = toff / af.ncol;
+                c0 = toff - row0 * af.ncol;
+            }
+        }
+        const bool rowsum = af.nrow > 0;
+        const float* frp = P.af_fac + af.irow + row0;
+        const float* fcp = P.af_fac + af.icol;
+        float su = 0.f;
+        if (af.ncol % 8 == 0 && af.ncol < (1LL << 30)) {
+            // a vector of 8 never straddles rows; rows and columns advance by a fixed step per vector
+            const unsigned ncol = (unsigned)af.ncol;
+            unsigned col = (unsigned)c0 + 8u * threadIdx.x, rl = 0;
+            if (col >= ncol) { rl = col / ncol; col -= rl * ncol; }
+            unsigned sub_col = 8 * kBlock, sub_rl = 0;
+            if (ncol <= 8 * kBlock) { sub_rl = (8 * kBlock) / ncol; sub_col = 8 * kBlock - sub_rl * ncol; }
+            const int nfull = nvalid / 8;
+            int q = threadIdx.x;
+            // a row length that divides the CTA's stride: the thread's 8 column factors never change
+            const bool stationary = sub_col == 0;
+            float4 fa = make_float4(0.f, 0.f, 0.f, 0.f), fb = fa;
+            if (stationary && q < nfull) {
+                fa = __ldg(reinterpret_cast<const float4*>(fcp + col));
+                fb = __ldg(reinterpret_cast<const float4*>(fcp + col + 4));
+            }
+#pragma unroll kAf2Unroll
+            for (; q < nfull; q += kBlock) {
+                const Fv<8> gv = load_f32<8>(g + 8 * q);
+                if (!stationary) {
+                    fa = __ldg(reinterpret_cast<const float4*>(fcp + col));
+                    fb = __ldg(reinterpret_cast<const float4*>(fcp + col + 4));
+                }
+                const float fr = rowsum ? __ldg(frp + rl) : 1.f;
+                float t = 0.f, x;
+                x = gv.f[0] * fa.x; t = fmaf(x, x, t);
+                x = gv.f[1] * fa.y; t = fmaf(x, x, t);
+                x = gv.f[2] * fa.z; t = fmaf(x, x, t);
+                x = gv.f[3] * fa.w; t = fmaf(x, x, t);
+                x = gv.f[4] * fb.x; t = fmaf(x, x, t);
+                x = gv.f[5] * fb.y; t = fmaf(x, x, t);
+                x = gv.f[6] * fb.z; t = fmaf(x, x, t);
+                x = gv.f[7] * fb.w; t = fmaf(x, x, t);
+                su = fmaf(t, fr * fr, su);
+                col += sub_col;
+                rl += sub_rl;
+                if (col >= ncol) { col -= ncol; ++rl; }
+            }
+            if (q == nfull && (nvalid & 7)) {          // the one ragged vector of the tile
+                const float fr = rowsum ? __ldg(frp + rl) : 1.f;
+                for (int j = 0; j < (nvalid & 7); ++j) {
+                    const float u = g[8 * q + j] * fr * __ldg(fcp + col + j);
+                    su = fmaf(u, u, su);
+                }
+            }
+        } else {
+            for (int e = threadIdx.x; e < nvalid; e += kBlock) {
+                const long long c = c0 + e;
+                const long long rl = c / af.ncol;
+                const float fr = rowsum ? __ldg(frp + rl) : 1.f;
+                const float u = __ldcs(g + e) * fr * __ldg(fcp + (c - rl * af.ncol));
+                su = fmaf(u, u, su);
+            }
+        }
+        WsSegAf an = af;
+        if (more) an = P.segaf[tn.seg];                // the next descriptor arrived long ago
+        // no CTA-wide barrier at the end of a tile (it would drain the CTA's loads once per tile): every
+        // warp adds its own sum to the tile's slot, which pass 1 left at zero
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) su += __shfl_xor_sync(0xffffffffu, su, o);
+        if ((threadIdx.x & 31) == 0) atomicAdd(&P.partials[P.concat ? ti : r * P.ntiles + ti].y, su);
+        if (!more) break;
+        item = nxt; rs = rs_n; ti = ti_n; tl = tn; af = an;
+    }
+}
+
 // -------------------------------------------------------------- dispatch ---
 template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED>
 ws_status launch(const UpdParams& P, const void* const* gptrs, cudaStream_t st) {
@@ -858,9 +974,7 @@ ws_status launch_o(const UpdParams& P, const void* const* gptrs, int out, bool w
         for (int k = 0; k < P.R && wide; ++k) wide = aligned32(gptrs[k]);
     if (OPT == K_LARS1 || OPT == K_LARS2 || is_af(OPT)) wide = wide && aligned32(P.ghat);
     if (OPT == K_AF1) wide = false;   // pass 1 is instruction-heavy: 128-bit vectors measured faster at every R
-    if constexpr (OPT == K_AF2) {
-        return launch_r<OPT, false, O_NONE, false>(P, gptrs, wide, st);   // touches no tensor list and no output
-    } else if constexpr (is_phase1(OPT)) {
+    if constexpr (is_phase1(OPT)) {
         return launch_r<OPT, GBF, O_NONE, FUSED>(P, gptrs, wide, st);
     } else {
         switch (out) {
@@ -882,7 +996,6 @@ ws_status launch_f(int opt, bool gbf, int out, const UpdParams& P, const void* c
         case K_LARS1: return gbf ? launch_o<K_LARS1, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_LARS1, false, FUSED>(P, gptrs, out, wide, st);
         case K_LARS2: return launch_o<K_LARS2, false, FUSED>(P, gptrs, out, wide, st);
         case K_AF1: return gbf ? launch_o<K_AF1, true, FUSED>(P, gptrs, out, wide, st) : launch_o<K_AF1, false, FUSED>(P, gptrs, out, wide, st);
-        case K_AF2: return launch_o<K_AF2, false, false>(P, gptrs, out, wide, st);
         case K_AF3: return launch_o<K_AF3, false, FUSED>(P, gptrs, out, wide, st);
         default: return launch_o<K_LAMB2, false, FUSED>(P, gptrs, out, wide, st);
     }
@@ -1221,7 +1334,14 @@ ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const
     P.partials = L.partials;
     P.ghat = L.ghat;
     P.af_fac = L.fac;
-    if ((s = launch_any(K_AF2, false, O_NONE, P, nullptr, st)) != WS_OK) return s;
+    if (P.nitems > 0) {
+        int dev = 0, sms = 148;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const long long cap = (long long)sms * WS_TUNE_AF2_CTAS;
+        af_sumsq_kernel<<<(unsigned)(P.nitems < cap ? P.nitems : cap), kBlock, 0, st>>>(P);
+        if ((s = ws_check_launch("adafactor(pass 2)")) != WS_OK) return s;
+    }
     af_finalize_clip_kernel<<<plan->T, kBlock, 0, st>>>(plan->d_segtiles, plan->d_segaf, L.partials, plan->ntiles, reps,
                                                        L.alpha, L.rho, L.norms, hyper->eps2, rho_step,
                                                        hyper->clip_threshold);
