@@ -309,20 +309,28 @@ __device__ __forceinline__ void update_elem(const WsConsts& c, float g, float& w
     }
 }
 
-__device__ __forceinline__ float block_sum(float x, float* smem /* kBlock/32 floats */) {
+// Sums two values over the CTA at once (one pair of barriers for both); the totals are valid in
+// thread 0.  The order of the additions is fixed, so the result is run-to-run bit-stable.
+__device__ __forceinline__ float2 block_sum2(float x, float y, float2* smem /* kBlock/32 entries */) {
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xffffffffu, x, o);
+    for (int o = 16; o > 0; o >>= 1) {
+        x += __shfl_xor_sync(0xffffffffu, x, o);
+        y += __shfl_xor_sync(0xffffffffu, y, o);
+    }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     __syncthreads();
-    if (lane == 0) smem[warp] = x;
+    if (lane == 0) smem[warp] = make_float2(x, y);
     __syncthreads();
-    float t = 0.f;
+    float2 t = make_float2(0.f, 0.f);
     if (threadIdx.x < 32) {
-        t = lane < kBlock / 32 ? smem[lane] : 0.f;
+        if (lane < kBlock / 32) t = smem[lane];
 #pragma unroll
-        for (int o = 4; o > 0; o >>= 1) t += __shfl_xor_sync(0xffffffffu, t, o);
+        for (int o = 4; o > 0; o >>= 1) {
+            t.x += __shfl_xor_sync(0xffffffffu, t.x, o);
+            t.y += __shfl_xor_sync(0xffffffffu, t.y, o);
+        }
     }
-    return t;  // valid in thread 0
+    return t;
 }
 
 // Adds VEC consecutive floats to global memory with vector reductions (one or two
@@ -356,7 +364,7 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
     constexpr bool WRITES_M = (OPT != K_LAMB2 && OPT != K_LARS1 && !is_af(OPT));
     constexpr bool WRITES_GHAT = (OPT == K_LARS1 || OPT == K_AF1);
     constexpr bool LOOPK = (NP > RB);   // R may exceed one tree block: loop and compensate
-    __shared__ float red[2][kBlock / 32];
+    __shared__ float2 red[kBlock / 32];
     // fused formatting: this tile's R gradient tensor pointers, fetched once per work item (the
     // streaming data would push the table's lines out of L1 between passes)
     __shared__ const void* sgp[(FUSED && READS_G) ? NP : 1];
@@ -687,8 +695,8 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
         }
         if (leaves_partials(OPT)) {
             // (Adafactor's passes leave one sum each)
-            const float a = block_sum(sw, red[0]);
-            const float b = OPT == K_AF1 ? 0.f : block_sum(su, red[1]);
+            const float2 ab = block_sum2(sw, su, red);
+            const float a = ab.x, b = ab.y;
             if (threadIdx.x == 0) {
                 float2* dst = P.partials + (P.concat ? ti : r * P.ntiles + ti);
                 *dst = make_float2(a, b);      // (Adafactor's pass 1: b = 0, pass 2 adds its sum there)
