@@ -93,6 +93,15 @@ def get_workload(args):
     return wl
 
 
+def measured_peak():
+    """(GB/s, source): the measured device copy bandwidth of this machine, else the stated fallback."""
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
 def bytes_per_param(wl):
     """Algorithmic bytes per valid parameter of the fused update (read R gradients, the weight
     and its slots once; write weight and slots once; plus the gathered copy when it is a
@@ -441,7 +450,10 @@ def run_ours(args):
             total_ms = sum(e[0].elapsed_time(e[nev - 1]) for e in evs)
         phase_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / K for i in range(nev - 1)]
         total_ms = reduce_max(total_ms, dev)
-        return total_ms / K, phase_ms, (t0, t1)
+        per_step = sorted(e[0].elapsed_time(e[nev - 1]) for e in evs)      # each step's own launches
+        stats = {"median": per_step[len(per_step) // 2], "min": per_step[0], "max": per_step[-1],
+                 "mean_back_to_back": total_ms / K}
+        return total_ms / K, phase_ms, (t0, t1), stats
 
     sampler = ClockSampler(local)
     if rank == 0:
@@ -452,8 +464,32 @@ def run_ours(args):
     if run_fused:
         res["fused"] = time_path(step_fused, 2)
     primary = "fused" if run_fused else "unfused"
-    ms_per_step, _, window = res[primary]
+    ms_per_step, _, window, step_stats = res[primary]
     value = job_value(N, world, ms_per_step)
+
+    # ---- one replica's work: ws_shard_update for a single shard r (reads slice r of the R packed buffers)
+    single = None
+    if run_unfused and wl.opt in ("sgdm", "adam") and args.layout == "per_tensor":
+        r_mid, S_ = R // 2, plan.S
+        sl = slice(r_mid * S_, (r_mid + 1) * S_)
+        valid = sum(min(max(sg.numel - r_mid * sg.piece, 0), sg.piece) for sg in plan.segments())
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+        times = []
+        for i in range(5 + 30):
+            if flush is not None:
+                flush.zero_()
+            ev[0].record()
+            B.ws_shard_update(plan, r_mid, pg, pw[sl], pm[sl], pv[sl] if pv is not None else None, hy, gathered, ws)
+            ev[1].record()
+            torch.cuda.synchronize()
+            if i >= 5:
+                times.append(ev[0].elapsed_time(ev[1]))
+        times.sort()
+        med = times[len(times) // 2]
+        single = {"call": f"ws_shard_update(r={r_mid}) alone, one launch", "valid_params": valid,
+                  "ms_median": med, "ms_min": times[0], "value": valid / (med * 1e-3), "unit": UNIT,
+                  "achieved_gbs": valid * bytes_per_param(wl)["update"] / (med * 1e-3) / 1e9}
+        single["frac"] = single["achieved_gbs"] / measured_peak()[0]
 
     # ---- end to end through the host-buffer entry point
     e2e = None
@@ -516,12 +552,7 @@ def run_ours(args):
         return
 
     # ---- per-kernel rates and the roofline of the dominant kernel
-    peak, peak_src = FALLBACK_HBM_GBS, "fallback"
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-            peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured"
-    except Exception:
-        pass
+    peak, peak_src = measured_peak()
     bpp = bytes_per_param(wl)
     n_upd_launch = {"lamb": 3, "lars": 3, "adafactor": 6}.get(wl.opt, 1)
     chunks = -(-T // 1024)
@@ -566,13 +597,17 @@ def run_ours(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": config_of(wl, args, path=primary), "roofline": roofline, "kernels": kernels, "clocks": clocks,
         "gpu_launches": K * sum(kz["launches_per_step"] for kz in kernels),
+        "step_ms": step_stats,
     }
     if "unfused" in res and primary != "unfused":
         rows = kernel_rows("unfused")
         line["unfused_path"] = {
             "step": "ws_pack_sets (R gradient lists) + ws_shard_update(all shards) + ws_unpack as separate kernels",
             "value": world * N / (res["unfused"][0] * 1e-3), "unit": UNIT, "ms_per_step": res["unfused"][0],
-            "kernels": rows, "gpu_launches": K * sum(kz["launches_per_step"] for kz in rows)}
+            "kernels": rows, "gpu_launches": K * sum(kz["launches_per_step"] for kz in rows),
+            "step_ms": res["unfused"][3]}
+        if single is not None:
+            line["unfused_path"]["single_shard"] = single
     if unfused_skipped:
         line["unfused_path"] = {"skipped": unfused_skipped}
     if e2e is not None:
@@ -623,12 +658,7 @@ def run_shard_window(args, wl, plan, dev, world, rank):
     mean_ms = reduce_max(float(np.mean(per_shard)), dev)
     if rank != 0:
         return
-    peak, peak_src = FALLBACK_HBM_GBS, "fallback"
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
-            peak, peak_src = float(json.load(f)["hbm_gbs"]), "measured"
-    except Exception:
-        pass
+    peak, peak_src = measured_peak()
     bpp = bytes_per_param(wl)["update"]
     gbs = (N / R) * bpp / (mean_ms * 1e-3) / 1e9
     line = {
