@@ -306,6 +306,24 @@ ws_status ws_lamb_apply(const ws_plan* plan, int32_t r, const ws_state* state,
                         const ws_hyper* hyper, const ws_out* out, void* workspace,
                         size_t workspace_bytes, void* stream);
 
+/* LARS shard by shard, the same three steps (the paper ran ResNet-50 with LARS
+ * on real replicas, Table 1): phase 1 for shard r reduces the gradients, keeps
+ * the sum in ghat slot r of the workspace and leaves per-tile partial sums of
+ * w^2 and g^2; ws_lars_finalize (after phase 1 of ALL shards, with every
+ * shard's partial rows present in the workspace - ws_workspace_partials) forms
+ * the local rates lambda_t from hyper->trust_coeff and hyper->weight_decay;
+ * phase 2 for shard r applies the momentum step and writes the gathered slot.
+ * The workspace has ws_workspace_bytes(plan, WS_LARS) bytes.  hyper->opt must
+ * be WS_LARS. */
+ws_status ws_lars_partial(const ws_plan* plan, int32_t r, const ws_grads* grads,
+                          const ws_state* state, const ws_hyper* hyper, void* workspace,
+                          size_t workspace_bytes, void* stream);
+ws_status ws_lars_finalize(const ws_plan* plan, const ws_hyper* hyper, void* workspace,
+                           size_t workspace_bytes, void* stream);
+ws_status ws_lars_apply(const ws_plan* plan, int32_t r, const ws_state* state,
+                        const ws_hyper* hyper, const ws_out* out, void* workspace,
+                        size_t workspace_bytes, void* stream);
+
 /* ------------------------------------- formatting fused into the update ---
  * Section 5.1: padding the gradient before the reduce-scatter costs every
  * replica a read and a write of the full data, so the paper fuses the

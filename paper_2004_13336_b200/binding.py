@@ -83,6 +83,7 @@ EXPORTS = [
     "ws_tensor_table_bytes", "ws_tensor_table_upload", "ws_fused_update",
     "ws_plan_create_layout", "ws_plan_layout", "ws_pack_sets",
     "ws_plan_factored_elems", "ws_plan_factored_layout", "ws_workspace_partials",
+    "ws_lars_partial", "ws_lars_finalize", "ws_lars_apply",
 ]
 
 _lib = None
@@ -138,6 +139,14 @@ def lib() -> C.CDLL:
                                 C.POINTER(ws_out), vp, C.c_size_t, vp]
     L.ws_plan_arena_elems.restype = C.c_int64
     L.ws_plan_arena_elems.argtypes = [vp]
+    L.ws_lars_partial.restype = C.c_int
+    L.ws_lars_partial.argtypes = [vp, C.c_int32, C.POINTER(ws_grads), C.POINTER(ws_state), C.POINTER(ws_hyper),
+                                  vp, C.c_size_t, vp]
+    L.ws_lars_finalize.restype = C.c_int
+    L.ws_lars_finalize.argtypes = [vp, C.POINTER(ws_hyper), vp, C.c_size_t, vp]
+    L.ws_lars_apply.restype = C.c_int
+    L.ws_lars_apply.argtypes = [vp, C.c_int32, C.POINTER(ws_state), C.POINTER(ws_hyper), C.POINTER(ws_out),
+                                vp, C.c_size_t, vp]
     L.ws_workspace_partials.restype = C.c_int
     L.ws_workspace_partials.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     L.ws_plan_factored_elems.restype = C.c_int64
@@ -356,6 +365,25 @@ def ws_lamb_apply(plan: Plan, r: int, w, m, v, hyper: ws_hyper, workspace: torch
     _check(lib().ws_lamb_apply(plan.handle, r, C.byref(s), C.byref(hyper),
                                C.byref(o) if o is not None else None, workspace.data_ptr(),
                                workspace.numel() * workspace.element_size(), _stream()), "ws_lamb_apply")
+
+
+def ws_lars_partial(plan: Plan, r: int, gbufs, w, m, hyper: ws_hyper, workspace: torch.Tensor, slice_mode: int = 0):
+    g, s = _grads(gbufs, slice_mode), _state(w, m, None)
+    _check(lib().ws_lars_partial(plan.handle, r, C.byref(g), C.byref(s), C.byref(hyper), workspace.data_ptr(),
+                                 workspace.numel() * workspace.element_size(), _stream()), "ws_lars_partial")
+
+
+def ws_lars_finalize(plan: Plan, hyper: ws_hyper, workspace: torch.Tensor):
+    _check(lib().ws_lars_finalize(plan.handle, C.byref(hyper), workspace.data_ptr(),
+                                  workspace.numel() * workspace.element_size(), _stream()), "ws_lars_finalize")
+
+
+def ws_lars_apply(plan: Plan, r: int, w, m, hyper: ws_hyper, workspace: torch.Tensor,
+                  gathered: Optional[torch.Tensor] = None):
+    s, o = _state(w, m, None), _out(gathered)
+    _check(lib().ws_lars_apply(plan.handle, r, C.byref(s), C.byref(hyper), C.byref(o) if o is not None else None,
+                               workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
+           "ws_lars_apply")
 
 
 def lamb_partials(plan: Plan, workspace: torch.Tensor) -> torch.Tensor:

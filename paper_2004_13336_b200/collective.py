@@ -3,8 +3,8 @@
 shard-major layout, a reduce-scatter leaves replica r the summed shard r, replica r updates
 its 1/R of the weights and of the optimizer slots (which stay sharded between steps), and an
 all-gather of the updated shards rebuilds the full weights - in bfloat16 when asked, while
-the update stays fp32 (Section 4.2).  LAMB adds the combination of the replicas' partial
-norm sums between its two phases (Section 4.1, "Non-elementwise operators").
+the update stays fp32 (Section 4.2).  LAMB and LARS add the combination of the replicas'
+partial norm sums between their two phases (Section 4.1, "Non-elementwise operators").
 
 This module is plumbing only: the collectives are ``torch.distributed`` calls (NCCL on GPUs)
 and every arithmetic step is a call into the C-ABI library through ``binding``.  The receive
@@ -13,9 +13,9 @@ gradient copy), and the kernel writes slot r of the gathered buffer, which is th
 own input and output layout, so no extra copy sits between a collective and a kernel.
 
 ``ops`` names the module that supplies ``Plan``, ``ws_pack``, ``ws_unpack``,
-``ws_shard_update``, ``ws_lamb_partial``, ``ws_lamb_finalize``, ``ws_lamb_apply``,
-``lamb_partials`` and ``make_hyper``; it is the CUDA binding unless a test passes a stand-in
-to run the choreography on CPU ranks.
+``ws_shard_update``, ``ws_lamb_partial / _finalize / _apply``, ``ws_lars_partial / _finalize /
+_apply``, ``lamb_partials`` and ``make_hyper``; it is the CUDA binding unless a test passes a
+stand-in to run the choreography on CPU ranks.
 """
 from __future__ import annotations
 
@@ -34,8 +34,8 @@ class ShardedUpdate:
                  align_elems: int = 32, device=None, group=None, ops=None):
         if ops is None:
             from . import binding as ops      # fails loudly without the built CUDA library
-        if opt not in ("sgdm", "adam", "lamb"):
-            raise ValueError("shard-by-shard updates exist for sgdm, adam and lamb")
+        if opt not in ("sgdm", "adam", "lamb", "lars"):
+            raise ValueError("shard-by-shard updates exist for sgdm, adam, lamb and lars")
         self.ops, self.opt, self.hyper_dict, self.group = ops, opt, dict(hyper), group
         self.rank, self.world = dist.get_rank(group), dist.get_world_size(group)
         self.device = torch.device(device) if device is not None else torch.device("cuda", torch.cuda.current_device())
@@ -47,8 +47,8 @@ class ShardedUpdate:
         self.recv = torch.empty(S, dtype=grad_dtype, device=self.device)      # ... and output
         self.gathered = torch.zeros(G, dtype=out_dtype, device=self.device)   # all-gather buffer
         self.workspace = None
-        if opt == "lamb":
-            self.workspace = torch.zeros(max(16, self.plan.workspace_bytes("lamb")), dtype=torch.uint8,
+        if opt in ("lamb", "lars"):
+            self.workspace = torch.zeros(max(16, self.plan.workspace_bytes(opt)), dtype=torch.uint8,
                                          device=self.device)
 
     # -- sharding program (Section 4.2): every replica starts from the same full state -----
@@ -81,6 +81,12 @@ class ShardedUpdate:
             dist.all_gather_into_tensor(rows.view(-1), rows[r], group=self.group)
             ops.ws_lamb_finalize(plan, self.workspace)                          # same sums, same order, every rank
             ops.ws_lamb_apply(plan, r, self.w, self.m, self.v, hy, self.workspace, self.gathered)
+        elif self.opt == "lars":
+            ops.ws_lars_partial(plan, r, [self.recv], self.w, self.m, hy, self.workspace, slice_mode=1)
+            rows = ops.lamb_partials(plan, self.workspace)
+            dist.all_gather_into_tensor(rows.view(-1), rows[r], group=self.group)
+            ops.ws_lars_finalize(plan, hy, self.workspace)
+            ops.ws_lars_apply(plan, r, self.w, self.m, hy, self.workspace, self.gathered)
         else:
             ops.ws_shard_update(plan, r, [self.recv], self.w, self.m, self.v if self.opt == "adam" else None,
                                 hy, self.gathered, None, slice_mode=1)

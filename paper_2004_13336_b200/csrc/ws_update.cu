@@ -1162,6 +1162,51 @@ extern "C" ws_status ws_lamb_apply(const ws_plan* plan, int32_t r, const ws_stat
     return launch_any(K_LAMB2, false, ok, P, nullptr, (cudaStream_t)stream);
 }
 
+extern "C" ws_status ws_lars_partial(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_state* state,
+                                     const ws_hyper* hyper, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!hyper || hyper->opt != WS_LARS) return WS_ERR_INVALID_ARG;
+    UpdParams P;
+    int ok;
+    bool gbf;
+    ws_status s = prepare(plan, r, grads, state, hyper, nullptr, K_LARS1, P, ok, gbf);
+    if (s != WS_OK) return s;
+    if ((s = check_ws(plan, workspace, workspace_bytes, WS_LARS)) != WS_OK) return s;
+    const WsLambWs L = ws_lamb_layout(plan, workspace);
+    P.partials = L.partials;
+    P.ghat = L.ghat;
+    std::vector<const void*> gp;
+    offset_grad_ptrs(plan, r, grads, gp);
+    return launch_any(K_LARS1, gbf, O_NONE, P, gp.data(), (cudaStream_t)stream);
+}
+
+extern "C" ws_status ws_lars_finalize(const ws_plan* plan, const ws_hyper* hyper, void* workspace,
+                                      size_t workspace_bytes, void* stream) {
+    if (!plan || !hyper || hyper->opt != WS_LARS) return WS_ERR_INVALID_ARG;
+    if (!plan->d_tiles) return WS_ERR_NOT_UPLOADED;
+    ws_status s = check_ws(plan, workspace, workspace_bytes, WS_LARS);
+    if (s != WS_OK) return s;
+    const WsLambWs L = ws_lamb_layout(plan, workspace);
+    lamb_finalize_kernel<<<plan->T, kBlock, 0, (cudaStream_t)stream>>>(plan->d_segtiles, L.partials, plan->ntiles,
+                                                                      finalize_reps(plan), L.rho, L.norms, 1,
+                                                                      hyper->trust_coeff, hyper->weight_decay);
+    return ws_check_launch("ws_lars_finalize");
+}
+
+extern "C" ws_status ws_lars_apply(const ws_plan* plan, int32_t r, const ws_state* state, const ws_hyper* hyper,
+                                   const ws_out* out, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!hyper || hyper->opt != WS_LARS) return WS_ERR_INVALID_ARG;
+    UpdParams P;
+    int ok;
+    bool gbf;
+    ws_status s = prepare(plan, r, nullptr, state, hyper, out, K_LARS2, P, ok, gbf);
+    if (s != WS_OK) return s;
+    if ((s = check_ws(plan, workspace, workspace_bytes, WS_LARS)) != WS_OK) return s;
+    const WsLambWs L = ws_lamb_layout(plan, workspace);
+    P.rho = L.rho;
+    P.ghat = L.ghat;
+    return launch_any(K_LARS2, false, ok, P, nullptr, (cudaStream_t)stream);
+}
+
 namespace {
 ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_tensor_table* gtab,
                     const ws_state* state, const ws_hyper* hyper, const ws_out* out, const ws_tensor_table* wtab,
@@ -1186,25 +1231,10 @@ extern "C" ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_gr
         // keeps the sum in the workspace and leaves partial sums of ||w||^2 and ||g||^2; the finalize
         // step forms each tensor's local rate; phase 2 applies the momentum step.
         if (r != -1) return WS_ERR_INVALID_ARG;
-        UpdParams P;
-        int ok;
-        bool gbf;
-        ws_status s = prepare(plan, -1, grads, state, hyper, nullptr, K_LARS1, P, ok, gbf);
+        ws_status s = ws_lars_partial(plan, -1, grads, state, hyper, workspace, workspace_bytes, stream);
         if (s != WS_OK) return s;
-        if ((s = check_ws(plan, workspace, workspace_bytes, WS_LARS)) != WS_OK) return s;
-        const WsLambWs L = ws_lamb_layout(plan, workspace);
-        P.partials = L.partials;
-        P.ghat = L.ghat;
-        std::vector<const void*> gp;
-        offset_grad_ptrs(plan, -1, grads, gp);
-        if ((s = launch_any(K_LARS1, gbf, O_NONE, P, gp.data(), (cudaStream_t)stream)) != WS_OK) return s;
-        lamb_finalize_kernel<<<plan->T, kBlock, 0, (cudaStream_t)stream>>>(
-            plan->d_segtiles, L.partials, plan->ntiles, finalize_reps(plan), L.rho, L.norms, 1, hyper->trust_coeff, hyper->weight_decay);
-        if ((s = ws_check_launch("ws_shard_update(LARS finalize)")) != WS_OK) return s;
-        if ((s = prepare(plan, -1, nullptr, state, hyper, out, K_LARS2, P, ok, gbf)) != WS_OK) return s;
-        P.rho = L.rho;
-        P.ghat = L.ghat;
-        return launch_any(K_LARS2, false, ok, P, nullptr, (cudaStream_t)stream);
+        if ((s = ws_lars_finalize(plan, hyper, workspace, workspace_bytes, stream)) != WS_OK) return s;
+        return ws_lars_apply(plan, -1, state, hyper, out, workspace, workspace_bytes, stream);
     }
     if (hyper->opt != WS_SGDM && hyper->opt != WS_ADAM) return WS_ERR_INVALID_ARG;
     const int phase = hyper->opt == WS_SGDM ? K_SGDM : K_ADAM;

@@ -35,13 +35,16 @@ def world_of_one():
 @pytest.mark.parametrize("opt,out_dtype,gdtype", [("sgdm", torch.float32, torch.float32),
                                                   ("adam", torch.bfloat16, torch.bfloat16),
                                                   ("lamb", torch.float32, torch.float32),
-                                                  ("lamb", torch.bfloat16, torch.float32)])
+                                                  ("lamb", torch.bfloat16, torch.float32),
+                                                  ("lars", torch.float32, torch.float32)])
 def test_one_rank_group_matches_the_oracle(world_of_one, opt, out_dtype, gdtype):
     wl = W.Workload("t", list(SHAPES), R=1, opt=opt, hyper={}, grad_dtype=gdtype, grad_std=1e-2, seed=23)
     w, m, v = W.make_state(wl, DEV)
     g = W.make_grads(wl, DEV)[0]
     hyper = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-6, weight_decay=0.01 if opt != "adam" else 0.0,
                  momentum=0.9, grad_scale=1.0, step=4)
+    if opt == "lars":
+        hyper.update(lr=10.0, weight_decay=5e-5, trust_coeff=0.001)
     su = ShardedUpdate(SHAPES, opt, hyper, out_dtype=out_dtype, grad_dtype=gdtype, device=DEV)
     su.load_state(w, m, v)
     outs = [torch.zeros(n, dtype=out_dtype, device=DEV) for n in wl.numels]
@@ -53,8 +56,8 @@ def test_one_rank_group_matches_the_oracle(world_of_one, opt, out_dtype, gdtype)
     og = [to_np(x) for x in g]
     for step in (4, 5):
         hyper["step"] = step
-        O.update_unsharded(O.make_hyper(opt, hyper), [og], ow, om, ov if opt != "sgdm" else None)
-    tol = TOL_LAMB if opt == "lamb" else 2 * TOL_FP32
+        O.update_unsharded(O.make_hyper(opt, hyper), [og], ow, om, ov if opt in ("adam", "lamb") else None)
+    tol = TOL_LAMB if opt in ("lamb", "lars") else 2 * TOL_FP32
     for t, (a, b) in enumerate(zip(outs, ow)):
         if out_dtype == torch.bfloat16:
             assert err(bf16_to_f64(to_np(a)), b) <= TOL_BF16, t

@@ -563,6 +563,34 @@ def test_lars_matches_oracle_and_fused_equals_unfused(R, gdtype):
         assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("R", [1, 3, 8])
+def test_lars_shard_by_shard_phases(R):
+    # what R replicas would run (phase 1 per shard, finalize, phase 2 per shard) equals the all-shard call
+    wl, w, m, v, g = _model(SHAPES, R, seed=16, gstd=1e-3)
+    plan = B.Plan(SHAPES, R, 32)
+    h = B.make_hyper("lars", _lars_hyper())
+    pw, pm, _, pg = _pack_all(plan, w, m, v, g)
+    aw, am = pw.clone(), pm.clone()
+    wsa = torch.zeros(plan.workspace_bytes("lars"), dtype=torch.uint8, device=DEV)
+    wsb = torch.zeros_like(wsa)
+    ga = torch.zeros(plan.G, dtype=torch.bfloat16, device=DEV)
+    gb = torch.zeros_like(ga)
+    B.ws_shard_update(plan, -1, pg, aw, am, None, h, ga, wsa)
+    S = plan.S
+    for r in range(R):
+        sl = slice(r * S, (r + 1) * S)
+        B.ws_lars_partial(plan, r, pg, pw[sl], pm[sl], h, wsb)
+    B.ws_lars_finalize(plan, h, wsb)
+    for r in range(R):
+        sl = slice(r * S, (r + 1) * S)
+        B.ws_lars_apply(plan, r, pw[sl], pm[sl], h, wsb, gb)
+    assert torch.equal(wsa, wsb)
+    assert torch.equal(aw, pw) and torch.equal(am, pm) and torch.equal(ga, gb)
+    with pytest.raises(B.WsError) as e:           # the LARS calls refuse another optimizer's hyper-parameters
+        B.ws_lars_finalize(plan, B.make_hyper("lamb", _hyper("lamb")), wsb)
+    assert e.value.status == 1
+
+
 def test_lars_poisoned_pads_and_error_codes():
     import ctypes as C
     R = 5
