@@ -353,8 +353,19 @@ ws_status ws_lars_apply(const ws_plan* plan, int32_t r, const ws_state* state,
  * ws_fused_update arguments: `grads` is a table of R sets (the R replicas'
  * gradient lists), `weights` a table of one set (the weight tensors that
  * receive the result), `state` as for ws_shard_update (r >= 0: one shard;
- * r == -1: all shards, the only form accepted for WS_LAMB), `workspace` as for
- * ws_shard_update. */
+ * r == -1: all shards, the only form accepted for WS_LAMB, WS_LARS and
+ * WS_ADAFACTOR), `workspace` as for ws_shard_update.
+ * With WS_SGDM and WS_ADAM `weights` may hold up to grads->nsets sets: the
+ * kernel then writes the updated weights into every set.  This is the form
+ * for real replicas whose tensors are mapped into one another's address space
+ * (CUDA IPC or symmetric memory; the caller fills the tables with the peers'
+ * addresses): replica r calls ws_fused_update(plan, r, ...) with the R
+ * replicas' gradient lists and the R replicas' weight lists, so the one kernel
+ * pulls its slice of every peer's gradients (the reduce-scatter), updates its
+ * shard, and stores the new weights into every peer's tensors (the
+ * all-gather) - Section 5.1's fusion of the formatting into both collectives,
+ * with plain peer loads and stores.  The caller orders the kernels of
+ * different replicas (gradients complete before, weights read after). */
 typedef struct {
     void* dev;        /* device table, layout [T][nsets] */
     int32_t nsets;

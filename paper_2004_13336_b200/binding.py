@@ -443,6 +443,24 @@ class TensorTable:
                                             self.dev_buf.data_ptr(), nbytes, _stream(), C.byref(self.c)),
                "ws_tensor_table_upload")
 
+    @classmethod
+    def from_pointers(cls, plan: Plan, ptr_sets: Sequence[Sequence[int]], dtype: torch.dtype, device):
+        """The same table from raw device addresses (sets of T integers) - for tensors that live in
+        another process's memory mapped into this one (CUDA IPC, symmetric memory).  The caller keeps
+        the mappings alive."""
+        self = cls.__new__(cls)
+        nsets = len(ptr_sets)
+        flat = [int(p) for s in ptr_sets for p in s]
+        assert len(flat) == nsets * plan.T
+        self.sets = None
+        nbytes = lib().ws_tensor_table_bytes(plan.handle, nsets)
+        self.dev_buf = torch.empty(nbytes, dtype=torch.uint8, device=device)
+        self.c = ws_tensor_table()
+        arr = (C.c_void_p * max(1, len(flat)))(*flat)
+        _check(lib().ws_tensor_table_upload(plan.handle, arr, nsets, _dtype_code(dtype), self.dev_buf.data_ptr(),
+                                            nbytes, _stream(), C.byref(self.c)), "ws_tensor_table_upload")
+        return self
+
 
 def ws_fused_update(plan: Plan, r: int, grads: TensorTable, w, m, v, hyper: ws_hyper, weights: TensorTable,
                     workspace: Optional[torch.Tensor] = None):

@@ -92,3 +92,67 @@ class ShardedUpdate:
                                 hy, self.gathered, None, slice_mode=1)
         dist.all_gather_into_tensor(self.gathered, self.gathered[r * S:(r + 1) * S], group=self.group)
         ops.ws_unpack(plan, self.gathered, weights_out)                         # reverse formatting
+
+
+class PeerShardedUpdate:
+    """The same step as ONE kernel per replica over peer-mapped tensors (Section 5.1: the formatting
+    fused into the reduce-scatter and into the all-gather).  Every replica keeps its gradient tensors
+    and its weight tensors in a symmetric-memory arena that all replicas of the NVLink domain map;
+    replica r's ``ws_fused_update(plan, r, ...)`` reads its slice of every replica's gradients with
+    plain peer loads, updates shard r, and stores the new weights into every replica's weight tensors
+    with plain peer stores.  No packed buffer, no receive buffer, no gathered buffer exist.  Two
+    stream-ordered NCCL barriers bracket the kernel: every replica's gradients are complete before any
+    kernel reads them, and every replica's shard has landed before the weights are used.
+
+    ``grads`` / ``weights``: this replica's tensors (views into the arenas) - the backward pass leaves
+    its gradients in ``grads``, the forward pass reads ``weights``.  Elementwise optimizers only.
+    Not run on more than one GPU so far."""
+
+    def __init__(self, shapes: Sequence[Sequence[int]], opt: str, hyper: Dict[str, float],
+                 out_dtype: torch.dtype = torch.float32, grad_dtype: torch.dtype = torch.float32,
+                 align_elems: int = 32, device=None, group=None):
+        import torch.distributed._symmetric_memory as symm
+        from . import binding as B
+        if opt not in ("sgdm", "adam"):
+            raise ValueError("one-kernel replica updates exist for sgdm and adam")
+        self.B, self.opt, self.hyper_dict = B, opt, dict(hyper)
+        self.group = group if group is not None else dist.group.WORLD
+        self.rank, self.world = dist.get_rank(group), dist.get_world_size(group)
+        self.device = torch.device(device) if device is not None else torch.device("cuda", torch.cuda.current_device())
+        self.plan = B.Plan(shapes, self.world, align_elems, device=self.device)
+        numels = [int(torch.Size(s).numel()) for s in shapes]
+        n_el, offs = self.plan.arena_elems, self.plan.arena_offsets()
+        self.grad_arena = symm.empty(n_el, dtype=grad_dtype, device=self.device)
+        self.weight_arena = symm.empty(n_el, dtype=out_dtype, device=self.device)
+        hg = symm.rendezvous(self.grad_arena, self.group)
+        hw = symm.rendezvous(self.weight_arena, self.group)
+        self._handles = (hg, hw)          # keep the peer mappings alive
+        eg, ew = self.grad_arena.element_size(), self.weight_arena.element_size()
+        self.gtab = B.TensorTable.from_pointers(
+            self.plan, [[int(hg.buffer_ptrs[k]) + o * eg for o in offs] for k in range(self.world)], grad_dtype, self.device)
+        self.wtab = B.TensorTable.from_pointers(
+            self.plan, [[int(hw.buffer_ptrs[k]) + o * ew for o in offs] for k in range(self.world)], out_dtype, self.device)
+        self.grads = self.plan.arena_views(self.grad_arena, numels)
+        self.weights = self.plan.arena_views(self.weight_arena, numels)
+        z = dict(dtype=torch.float32, device=self.device)
+        S = self.plan.S
+        self.w, self.m, self.v = torch.zeros(S, **z), torch.zeros(S, **z), torch.zeros(S, **z)
+        self._token = torch.zeros(1, **z)
+
+    def load_state(self, w: Sequence[torch.Tensor], m: Sequence[torch.Tensor], v: Sequence[torch.Tensor]):
+        S, r = self.plan.S, self.rank
+        full = torch.empty(self.plan.G, dtype=torch.float32, device=self.device)
+        for src, dst in ((w, self.w), (m, self.m), (v, self.v)):
+            self.B.ws_pack(self.plan, src, full)
+            dst.copy_(full[r * S:(r + 1) * S])
+        for dst, src in zip(self.weights, w):
+            dst.copy_(src.reshape(-1))
+
+    def step(self, step: Optional[int] = None):
+        if step is not None:
+            self.hyper_dict["step"] = step
+        hy = self.B.make_hyper(self.opt, self.hyper_dict)
+        dist.all_reduce(self._token, group=self.group)     # all replicas' gradients are in place
+        self.B.ws_fused_update(self.plan, self.rank, self.gtab, self.w, self.m,
+                               self.v if self.opt == "adam" else None, hy, self.wtab, None)
+        dist.all_reduce(self._token, group=self.group)     # all shards have been stored into these weights

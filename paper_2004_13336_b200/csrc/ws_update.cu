@@ -105,7 +105,8 @@ struct UpdParams {
     float* v;
     void* gathered;         // base of the G-element gathered buffer, or null
     const void* const* gtab; // fused formatting: device table [T][R] of gradient tensor pointers
-    void* const* wtab;       // fused formatting: device table [T] of weight tensor pointers (outputs)
+    void* const* wtab;       // fused formatting: device table [T][nw] of weight tensor pointers (outputs)
+    int nw;                  // number of weight lists written (1, or one per replica)
     float2* partials;       // phase 1: [R][ntiles] partial sums of the two norms
     const float* rho;       // phase 2: [T] trust ratio (LAMB) / local rate (LARS)
     float* ghat;            // LARS, Adafactor: [R][S] summed gradients, written by phase 1, read afterwards
@@ -368,6 +369,9 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
     // fused formatting: this tile's R gradient tensor pointers, fetched once per work item (the
     // streaming data would push the table's lines out of L1 between passes)
     __shared__ const void* sgp[(FUSED && READS_G) ? NP : 1];
+    // ... and, when the updated weights go to several weight lists (one per replica: the all-gather
+    // of Section 2.2 written straight into every replica's tensors), the tile's further output pointers
+    __shared__ void* swp[(FUSED && READS_G && writes_weights(OPT)) ? NP : 1];
 
     for (long long item = blockIdx.x; item < P.nitems; item += gridDim.x) {
         long long rs = P.concat ? 0 : item / P.ntiles;     // shard index inside this launch
@@ -384,11 +388,15 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
         const void* const* gt = nullptr;
         char* wt = nullptr;
         if constexpr (FUSED) {
-            if (OUT != O_NONE) wt = reinterpret_cast<char*>(P.wtab[tl.seg]);
+            if (OUT != O_NONE) wt = reinterpret_cast<char*>(P.wtab[(long long)tl.seg * P.nw]);
             if constexpr (READS_G) {
                 gt = P.gtab + (long long)tl.seg * P.R;
                 __syncthreads();   // the previous item's readers are done with sgp
                 for (int k = threadIdx.x; k < P.R; k += kBlock) sgp[k] = gt[k];
+                if constexpr (writes_weights(OPT)) {
+                    if (OUT != O_NONE)
+                        for (int k = threadIdx.x; k < P.nw; k += kBlock) swp[k] = P.wtab[(long long)tl.seg * P.nw + k];
+                }
                 __syncthreads();
             }
         }
@@ -680,6 +688,19 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
                         unsigned short* dst = reinterpret_cast<unsigned short*>(wt) + toff + e0[u];
                         if (nv[u] == VEC) store_bf16<VEC>(dst, wv[u]);
                         else store_bf16_partial<VEC>(dst, wv[u], nv[u]);
+                    }
+                    if constexpr (READS_G) {
+                        for (int k = 1; k < P.nw; ++k) {      // the other replicas' weight tensors
+                            if (OUT == O_F32) {
+                                float* dst = reinterpret_cast<float*>(swp[k]) + toff + e0[u];
+                                if (nv[u] == VEC) store_f32<VEC>(dst, wv[u]);
+                                else store_f32_partial<VEC>(dst, wv[u], nv[u]);
+                            } else if (OUT == O_BF16) {
+                                unsigned short* dst = reinterpret_cast<unsigned short*>(swp[k]) + toff + e0[u];
+                                if (nv[u] == VEC) store_bf16<VEC>(dst, wv[u]);
+                                else store_bf16_partial<VEC>(dst, wv[u], nv[u]);
+                            }
+                        }
                     }
                 } else if (OUT == O_F32) {
                     store_f32<VEC>(reinterpret_cast<float*>(P.gathered) + obase + e0[u], wv[u]);
@@ -1045,6 +1066,7 @@ ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state
     gbf = false;
     P.gtab = nullptr;
     P.wtab = nullptr;
+    P.nw = 1;
     if (!is_phase2(phase) && !fused) {
         if (!g || !g->ptrs || g->R < 1) return WS_ERR_INVALID_ARG;
         if (g->dtype != WS_F32 && g->dtype != WS_BF16) return WS_ERR_DTYPE;
@@ -1305,6 +1327,7 @@ ws_status fused_phase(const ws_plan* plan, int32_t r, const ws_tensor_table* gra
     }
     if (!is_phase1(phase)) {
         P.wtab = (void* const*)weights->dev;
+        P.nw = weights->nsets;
         out_kind = weights->dtype == WS_F32 ? O_F32 : O_BF16;
         wide = wide && (weights->dtype == WS_BF16 || weights->min_align >= 32);
     }
@@ -1400,7 +1423,10 @@ extern "C" ws_status ws_fused_update(const ws_plan* plan, int32_t r, const ws_te
                                      size_t workspace_bytes, void* stream) {
     if (!plan || !grads || !weights || !hyper || !state) return WS_ERR_INVALID_ARG;
     if (!grads->dev || !weights->dev) return WS_ERR_INVALID_ARG;
-    if (grads->T != plan->T || weights->T != plan->T || grads->nsets < 1 || weights->nsets != 1)
+    if (grads->T != plan->T || weights->T != plan->T || grads->nsets < 1 || weights->nsets < 1) return WS_ERR_INVALID_ARG;
+    // several weight lists (every replica's tensors written by the one kernel) only where one kernel both
+    // reads the gradient lists and writes the weights, and never more lists than gradient sets
+    if (weights->nsets > 1 && ((hyper->opt != WS_SGDM && hyper->opt != WS_ADAM) || weights->nsets > grads->nsets))
         return WS_ERR_INVALID_ARG;
     if ((grads->dtype != WS_F32 && grads->dtype != WS_BF16) || (weights->dtype != WS_F32 && weights->dtype != WS_BF16))
         return WS_ERR_DTYPE;

@@ -67,3 +67,32 @@ def test_one_rank_group_matches_the_oracle(world_of_one, opt, out_dtype, gdtype)
     su.gather_slot(su.m, m_full)
     for t, (a, b) in enumerate(zip(m_full, om)):
         assert err(to_np(a), b) <= tol, t
+
+
+@pytest.mark.parametrize("opt,out_dtype,gdtype", [("sgdm", torch.float32, torch.float32),
+                                                  ("adam", torch.bfloat16, torch.bfloat16)])
+def test_one_kernel_route_over_symmetric_memory(world_of_one, opt, out_dtype, gdtype):
+    """The peer-mapped route on a world of one: the arenas are symmetric memory, the tables hold
+    the addresses the rendezvous returned, one kernel does the whole step."""
+    from paper_2004_13336_b200.collective import PeerShardedUpdate
+    wl = W.Workload("t", list(SHAPES), R=1, opt=opt, hyper={}, grad_dtype=gdtype, grad_std=1e-2, seed=29)
+    w, m, v = W.make_state(wl, DEV)
+    g = W.make_grads(wl, DEV)[0]
+    hyper = dict(lr=1e-2, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=5e-5 if opt == "sgdm" else 0.0,
+                 momentum=0.9, grad_scale=1.0, step=2)
+    try:
+        pu = PeerShardedUpdate(SHAPES, opt, hyper, out_dtype=out_dtype, grad_dtype=gdtype, device=DEV)
+    except (RuntimeError, NotImplementedError) as e:      # no symmetric-memory support in this environment
+        pytest.skip(f"symmetric memory unavailable: {str(e)[:120]}")
+    pu.load_state(w, m, v)
+    for dst, src in zip(pu.grads, g):
+        dst.copy_(src)
+    pu.step()
+    torch.cuda.synchronize()
+    ow, om, ov = [to_np(x) for x in w], [to_np(x) for x in m], [to_np(x) for x in v]
+    O.update_unsharded(O.make_hyper(opt, hyper), [[to_np(x) for x in g]], ow, om, ov if opt == "adam" else None)
+    for t, (a, b) in enumerate(zip(pu.weights, ow)):
+        if out_dtype == torch.bfloat16:
+            assert err(bf16_to_f64(to_np(a)), b) <= TOL_BF16, t
+        else:
+            assert err(to_np(a), b) <= TOL_FP32, t

@@ -894,3 +894,45 @@ def test_zero_norm_tensors_get_ratio_one(opt):
     if opt == "lamb":                              # (LARS still applies its weight decay at rate 1)
         got = O.unpack(oplan, to_np(pw))
         assert (got[3] == to_np(w[3])).all()       # nothing to apply: weights unchanged bit for bit
+
+
+# ------------------------- one kernel per replica over every replica's tensors ---
+@pytest.mark.parametrize("opt,gdtype,odtype", [("sgdm", torch.float32, torch.float32),
+                                               ("adam", torch.bfloat16, torch.bfloat16),
+                                               ("adam", torch.float32, torch.float32)])
+@pytest.mark.parametrize("R", [2, 5, 8])
+def test_replica_kernels_over_all_replicas_tensors(opt, gdtype, odtype, R):
+    """What R replicas with peer-mapped tensors would run, emulated on one GPU by R independent
+    launches: replica r's single kernel reads its slice of all R gradient lists (the reduce-scatter),
+    updates shard r, and writes the new weights into all R replicas' weight lists (the all-gather).
+    Afterwards every replica's weight tensors hold the unsharded result."""
+    wl, w, m, v, g = _model(SHAPES, R, gdtype, seed=40 + R)
+    plan = B.Plan(SHAPES, R, 32)
+    oplan = O.Plan(wl.numels, R, 32)
+    h = _hyper(opt)
+    ow, om, ov, _ = _oracle_unsharded(opt, h, w, m, v, g)
+    pw, pm, pv, _ = _pack_all(plan, w, m, v, [])
+    fill = -7.0
+    bigs, lists = [], []
+    for k in range(R):                 # replica k's weight tensors, with guard zones
+        bl = [_guarded(n, odtype, fill) for n in wl.numels]
+        bigs.append([b for b, _ in bl])
+        lists.append([vw for _, vw in bl])
+    gtab = B.TensorTable(plan, g)
+    wtab = B.TensorTable(plan, lists)
+    hy = B.make_hyper(opt, h)
+    S = plan.S
+    for r in range(R):                 # independent launches: none waits for another
+        sl = slice(r * S, (r + 1) * S)
+        B.ws_fused_update(plan, r, gtab, pw[sl], pm[sl], pv[sl] if opt == "adam" else None, hy, wtab, None)
+    _compare_state(oplan, opt, [pw, pm, pv], [ow, om, ov], TOL_FP32)
+    ref = [torch.empty(n, dtype=odtype, device=DEV) for n in wl.numels]
+    B.ws_unpack(plan, pw.to(odtype) if odtype != torch.float32 else pw, ref)
+    for k in range(R):
+        for t, (a, b) in enumerate(zip(lists[k], ref)):
+            assert torch.equal(a, b), (k, t)
+            assert _guards_intact(bigs[k][t], wl.numels[t], fill), (k, t)
+    # more weight lists than gradient sets, or several lists under a two-phase optimizer: refused
+    with pytest.raises(B.WsError) as e:
+        B.ws_fused_update(plan, 0, B.TensorTable(plan, g[:1]), pw[:S], pm[:S], pv[:S], hy, wtab, None)
+    assert e.value.status == 1
