@@ -406,7 +406,7 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
         if (OPT == K_AF3) lr_rho = P.rho[tl.seg];         // alpha_t / max(1, RMS(U_t)/d)
         float sw = 0.f, su = 0.f;
         // Adafactor: where the tile starts inside its tensor's rows x cols matrix
-        WsSegAf af;
+        WsSegAf af = {};
         long long row0 = 0, c0 = 0;
         bool rowsum = false, bigcol = false;
         if constexpr (is_af(OPT)) {
