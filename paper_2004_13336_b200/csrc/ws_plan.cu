@@ -181,6 +181,11 @@ extern "C" ws_status ws_plan_create_layout(const ws_tensor_desc* descs, int32_t 
             }
             p->shard_tile_begin[R] = (long long)p->tiles.size();
             p->ntiles = (long long)p->tiles.size();
+            // a tensor without tiles (empty, and no padding region of its own) still names the place
+            // in the tile list where its tiles would be, so that a range of tensors maps to a range of tiles
+            for (int k = 0; k < T; ++k)
+                if (!seen[k])
+                    p->segtiles[k].tile_begin = k > 0 ? p->segtiles[k - 1].tile_begin + p->segtiles[k - 1].tile_count : 0;
             ws_matrix_views(p, descs);
             *out = p;
             return WS_OK;

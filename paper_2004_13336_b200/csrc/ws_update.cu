@@ -426,11 +426,11 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
         }
         // When the row length is a multiple of VEC a vector never straddles rows and starts on a
         // multiple of VEC (colrun).  Pass 1 then adds a vector's g^2 + eps1 to the column sums with
-        // one vector reduction; when the row length also divides the CTA's stride, a thread meets the
-        // same VEC columns on every pass (and no other thread of the CTA does), keeps their sums in
-        // registers and adds them once per tile (stationary).
+        // one vector reduction; when the row length also divides the distance between a thread's
+        // consecutive vectors, the thread meets the same VEC columns in every vector, keeps their sums
+        // in registers and adds them once per tile (stationary).
         const bool colrun = is_af(OPT) && af.ncol % VEC == 0;
-        const bool stationary = colrun && (kBlock * VEC * U) % af.ncol == 0;
+        const bool stationary = colrun && (kBlock * VEC) % af.ncol == 0;   // (the stride between ANY two of its vectors)
         // the thread's first vector starts at column run_col of row run_rl (relative to the tile's first
         // row); consecutive vectors of a thread lie kBlock * VEC elements apart = sub_rl rows and
         // sub_col columns, so rows and columns advance without a division per vector

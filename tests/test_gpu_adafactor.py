@@ -18,9 +18,10 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 # matrices with rows longer and shorter than a tile, single rows and columns, 3-D and 4-D tensors,
-# vectors (unfactored), tiny and prime sizes
+# vectors (unfactored), tiny and prime sizes, row lengths that are 1/2, 2 and 8 times the 1024 elements
+# a CTA covers with one vector per thread
 SHAPES = [(1,), (7,), (3, 3, 16, 32), (64, 128), (1031,), (5, 1, 9), (4099, 3), (300, 301), (32,), (20011,),
-          (2, 9001), (1, 4500), (4500, 1), (6, 5000)]
+          (2, 9001), (1, 4500), (4500, 1), (6, 5000), (24, 2048), (3, 8192), (40, 512)]
 
 
 def _hyper(**kw):

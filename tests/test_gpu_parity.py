@@ -472,6 +472,45 @@ def test_empty_tensors_in_the_list(opt):
         assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb", "lars"])
+def test_empty_tensors_in_the_concatenated_layout(opt):
+    # empty tensors first, in the middle and last; 4 x 32-element alignment units in total, so with
+    # R = 4 the concatenation fills the shards exactly and the trailing empty tensor owns no tile at all
+    shapes = [(0,), (32,), (5, 0, 2), (64,), (0, 7), (32,), (100, 0)]
+    R = 4
+    wl, w, m, v, g = _model(shapes, R, seed=19)
+    plan = B.Plan(shapes, R, 32, layout="concat")
+    oplan = O.FlatPlan(wl.numels, R, 32)
+    assert plan.S == oplan.S == 32
+    h = _lars_hyper() if opt == "lars" else _hyper(opt)
+    has_v = opt in ("adam", "lamb")
+    ow, om, ov, _ = _oracle_unsharded(opt, h, w, m, v, g)
+    nan = float("nan")
+    pw, pm, pv = (torch.full((plan.G,), nan, device=DEV) for _ in range(3))
+    for src, dst in ((w, pw), (m, pm), (v, pv)):
+        B.ws_pack(plan, src, dst)                       # must overwrite every element of the flat buffer
+    assert bool(torch.isfinite(pw).all())
+    pg = []
+    for gk in g:
+        b = torch.full((plan.G,), nan, device=DEV)
+        B.ws_pack(plan, gk, b)
+        pg.append(b)
+    fw, fm, fv = pw.clone(), pm.clone(), pv.clone()
+    ws = torch.full((max(16, plan.workspace_bytes(opt)),), 0xFF, dtype=torch.uint8, device=DEV)
+    B.ws_shard_update(plan, -1, pg, pw, pm, pv if has_v else None, B.make_hyper(opt, h), None, ws)
+    tol = TOL_LAMB if opt in ("lamb", "lars") else TOL_FP32
+    for t, (a, b) in enumerate(zip(O.unpack_flat(oplan, to_np(pw)), ow)):
+        assert err(a, b) <= tol, t
+    outs = [torch.full_like(x, 3.0) for x in w]
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), fw, fm, fv if has_v else None, B.make_hyper(opt, h),
+                      B.TensorTable(plan, [outs]), torch.full_like(ws, 0xFF))
+    assert torch.equal(fw, pw) and torch.equal(fm, pm)
+    back = [torch.empty_like(x) for x in w]
+    B.ws_unpack(plan, pw, back)
+    for a, b in zip(outs, back):
+        assert torch.equal(a, b)
+
+
 def test_step_can_be_captured_in_a_cuda_graph():
     # calls take pointers and a stream, allocate nothing and never synchronise, so a whole step
     # (here: the fused update, and pack + update + unpack) can be captured once and replayed
