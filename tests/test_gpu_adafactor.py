@@ -221,3 +221,66 @@ def test_argument_errors():
     lay = plan.factored_layout()
     rows, cols, foff, tot = O.factor_shapes(SHAPES[:4])
     assert [tuple(x) for x in lay] == list(zip(foff.tolist(), rows.tolist(), cols.tolist())) and plan.factored_elems == tot
+
+
+@pytest.mark.parametrize("case", range(32))
+def test_randomised_matrix_shapes_on_both_routes(case):
+    """Random lists of 0- to 4-dimensional tensors (row lengths below, at and above what a CTA covers
+    with one vector per thread; scalars; empty tensors), shard and copy counts, alignments, tile sizes,
+    layouts and dtypes: both routes against the oracle's whole-tensor definition."""
+    rng = np.random.default_rng(7000 + case)
+    pool = [1, 2, 3, 4, 5, 7, 8, 9, 16, 31, 32, 33, 64, 100, 127, 128, 255, 256, 300, 512, 1000, 1024, 1025, 2048, 4097]
+
+    def shape():
+        nd = int(rng.choice([0, 1, 1, 2, 2, 2, 3, 4]))
+        s = tuple(int(rng.choice(pool)) for _ in range(nd))
+        while int(np.prod(s)) > 400000:
+            s = tuple(max(1, d // 2) for d in s)
+        if nd and rng.random() < 0.05:
+            s = s[:-1] + (0,)
+        return s
+    shapes = [shape() for _ in range(int(rng.integers(1, 12)))]
+    if sum(int(np.prod(s)) for s in shapes) == 0:
+        shapes.append((24, 2048))
+    R = int(rng.choice([1, 2, 3, 4, 5, 8, 9, 16, 33]))
+    K = R if rng.random() < 0.8 else int(rng.choice([1, 2, 6]))
+    A, tile = int(rng.choice([8, 16, 32, 64])), int(rng.choice([0, 1024, 2048, 4096]))
+    layout = str(rng.choice(["per_tensor", "concat"]))
+    gdt = torch.bfloat16 if rng.random() < 0.3 else torch.float32
+    odt = torch.bfloat16 if rng.random() < 0.3 else torch.float32
+    wl, plan, w, g, f0 = _setup(shapes, R, gdt, seed=case, A=A, tile=tile, layout=layout, K=K)
+    h = _hyper(step=int(rng.integers(1, 20)), grad_scale=float(rng.choice([1.0, 0.5])),
+               clip_threshold=float(rng.choice([1.0, 0.3])))
+    numels = wl.numels
+    hs = O.make_hyper("adafactor", h)
+    of = to_np(f0)
+    ow = [to_np(x) for x in w]
+    og = [[to_np(x) for x in gk] for gk in g]
+    for t, (off, rows, cols) in enumerate(plan.factored_layout()):
+        if numels[t]:
+            ref = ow[t].reshape(shapes[t]) if len(shapes[t]) else ow[t]
+            O.adafactor_tensor(hs, [gk[t] for gk in og], ref, of[off:off + rows],
+                               of[off + rows:off + rows + cols] if cols else None)
+            ow[t] = ref.ravel()
+    hy = B.make_hyper("adafactor", h)
+    for route in ("separate", "fused"):
+        pw, = _pack(plan, [w])
+        fs = f0.clone()
+        ws = torch.full((plan.workspace_bytes("adafactor"),), 0xFF, dtype=torch.uint8, device=DEV)
+        outs = [torch.full((n,), 9.0, dtype=odt, device=DEV) for n in numels]
+        if route == "separate":
+            gath = torch.empty(plan.G, dtype=odt, device=DEV)
+            B.ws_shard_update(plan, -1, _pack(plan, g), pw, None, fs, hy, gath, ws)
+            B.ws_unpack(plan, gath, outs)
+        else:
+            B.ws_fused_update(plan, -1, B.TensorTable(plan, g), pw, None, fs, hy, B.TensorTable(plan, [outs]), ws)
+        gs = to_np(fs)
+        for t, (off, rows, cols) in enumerate(plan.factored_layout()):
+            if numels[t] == 0:
+                continue
+            a = to_np(outs[t])
+            a = bf16_to_f64(a) if odt == torch.bfloat16 else a
+            # a handful of elements has no tensor-wide scale to be measured against
+            tol = TOL_BF16 if odt == torch.bfloat16 else (TOL_LAMB if numels[t] >= 32 else 1e-4)
+            assert err(a, ow[t]) <= tol, (route, t, shapes[t])
+            assert err(gs[off:off + rows + cols], of[off:off + rows + cols]) <= 10 * TOL_LAMB, (route, t, shapes[t])

@@ -49,16 +49,18 @@ def _guards_intact(big, n, fill):
 
 
 def _pack_all(plan, w, m, v, g):
-    pw = torch.empty(plan.G, dtype=torch.float32, device=DEV)
-    pm, pv = torch.empty_like(pw), torch.empty_like(pw)
+    # the flat buffers start as NaN: ws_pack has to overwrite every element, pads included
+    pw = torch.full((plan.G,), float("nan"), dtype=torch.float32, device=DEV)
+    pm, pv = pw.clone(), pw.clone()
     B.ws_pack(plan, w, pw)
     B.ws_pack(plan, m, pm)
     B.ws_pack(plan, v, pv)
     pg = []
     for gk in g:
-        b = torch.empty(plan.G, dtype=gk[0].dtype, device=DEV)
+        b = torch.full((plan.G,), float("nan"), dtype=gk[0].dtype, device=DEV)
         B.ws_pack(plan, gk, b)
         pg.append(b)
+    assert bool(torch.isfinite(pw).all()) and all(bool(torch.isfinite(b).all()) for b in pg)
     return pw, pm, pv, pg
 
 
