@@ -296,7 +296,12 @@ ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_grads* grads,
  * paper has the combined scalar all-reduce (Section 5.2), so call it after
  * phase 1 of ALL shards.  Phase 2 for shard r recomputes u from w, m', v' and
  * applies w' = w - lr rho u, writing the gathered slot.  `grads` is ignored
- * by ws_lamb_apply and may be NULL there. */
+ * by ws_lamb_apply and may be NULL there.
+ * The shard-by-shard form gives bit for bit the result of the all-shard call
+ * when every shard slice handed in is 32-byte aligned (S * element size a
+ * multiple of 32: any A for fp32, A >= 16 for bf16 gradient slices);
+ * otherwise the kernels fall back to 128-bit accesses for that shard, the
+ * partial sums are formed in another order and the ratios agree to rounding. */
 ws_status ws_lamb_partial(const ws_plan* plan, int32_t r, const ws_grads* grads,
                           const ws_state* state, const ws_hyper* hyper, void* workspace,
                           size_t workspace_bytes, void* stream);
