@@ -66,6 +66,10 @@ def parse_args():
                     help="fused: one kernel reads the gradient tensors and writes the weight tensors; "
                          "unfused: pack, update, unpack as separate kernels; both: time both, headline = fused")
     ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--route", default="replicas", choices=["replicas", "nccl", "peer"],
+                    help="replicas (default): every rank updates its own independent tensor set, no collective; "
+                         "nccl: ONE model over the ranks, NCCL reduce-scatter / all-gather around the single-shard "
+                         "kernels; peer: ONE model, one kernel per rank over symmetric-memory tensors")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-large", action="store_true",
@@ -318,9 +322,85 @@ def job_value(n_params_per_rank: int, world: int, ms_per_step: float) -> float:
 # ----------------------------------------------------------------------------
 # GPU arm
 # ----------------------------------------------------------------------------
+def run_real_replicas(args):
+    """--route nccl | peer: the ranks are the replicas of ONE model (shard count = number of ranks).
+    Each step is the whole weight update of the model: with nccl, pack + reduce-scatter + update of the
+    rank's shard + all-gather + unpack; with peer, one kernel per rank over symmetric-memory tensors
+    between two stream-ordered barriers.  The work per step is fixed (N parameters), so scaling is strong."""
+    import socket
+    import torch
+    import torch.distributed as dist
+    from paper_2004_13336_b200 import build as ws_build
+    from paper_2004_13336_b200 import workloads as W
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    else:
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1, device_id=dev)
+    if rank == 0 and not ws_build.up_to_date():
+        ws_build.build()
+    dist.barrier()
+    from paper_2004_13336_b200.collective import PeerShardedUpdate, ShardedUpdate
+    wl = get_workload(args)
+    wl.R = world
+    w, m, v = W.make_state(wl, dev)                       # same seed on every rank: one model
+    g = W.make_grads_one(wl, rank, dev)                   # this replica's own gradients
+    kw = dict(out_dtype=wl.out_dtype, grad_dtype=wl.grad_dtype, align_elems=args.align, device=dev)
+    if args.route == "nccl":
+        su = ShardedUpdate(wl.shapes, wl.opt, wl.hyper, **kw)
+        su.load_state(w, m, v)
+        outs = [torch.empty(n, dtype=wl.out_dtype, device=dev) for n in wl.numels]
+        step = lambda: su.step(g, outs)
+        launches = {"sgdm": 3, "adam": 3, "lamb": 5, "lars": 5}[wl.opt]      # ours: pack, update phases, unpack
+    else:
+        su = PeerShardedUpdate(wl.shapes, wl.opt, wl.hyper, **kw)
+        su.load_state(w, m, v)
+        for dst, src in zip(su.grads, g):
+            dst.copy_(src)
+        step = su.step
+        launches = 1
+    K, W_ = args.steps, max(3, args.warmup)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    for _ in range(W_):
+        step()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    dist.barrier()
+    torch.cuda.synchronize()
+    t0 = time.time()
+    e0.record()
+    for _ in range(K):
+        step()
+    e1.record()
+    dist.barrier()
+    torch.cuda.synchronize()
+    t1 = time.time()
+    ms = reduce_max(e0.elapsed_time(e1), dev) / K
+    sampler.stop()
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": wl.N / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W_,
+            "ms_per_step": ms, "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": f"{wl.name}: one model of {wl.N} params over {world} replica(s), {wl.opt}",
+                       "route": args.route, "inputs": "larger than L2" if wl.N * 12 > 256e6 else "fit in L2"},
+            "roofline": None, "clocks": sampler.summary(t0, t1), "gpu_launches": K * launches}))
+    dist.destroy_process_group()
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
+    if args.route != "replicas":
+        return run_real_replicas(args)
 
     from paper_2004_13336_b200 import binding as B
     from paper_2004_13336_b200 import build as ws_build
