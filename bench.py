@@ -358,7 +358,7 @@ def run_real_replicas(args):
         su.load_state(w, m, v)
         outs = [torch.empty(n, dtype=wl.out_dtype, device=dev) for n in wl.numels]
         step = lambda: su.step(g, outs)
-        launches = {"sgdm": 3, "adam": 3, "lamb": 5, "lars": 5}[wl.opt]      # ours: pack, update phases, unpack
+        launches = {"sgdm": 3, "adam": 3, "lamb": 5, "lars": 5, "adafactor": 8}[wl.opt]   # ours: pack, update phases, unpack
     else:
         su = PeerShardedUpdate(wl.shapes, wl.opt, wl.hyper, **kw)
         su.load_state(w, m, v)

@@ -329,6 +329,39 @@ ws_status ws_lars_apply(const ws_plan* plan, int32_t r, const ws_state* state,
                         const ws_hyper* hyper, const ws_out* out, void* workspace,
                         size_t workspace_bytes, void* stream);
 
+/* Adafactor stage by stage, for one shard r >= 0 or all shards (r == -1): what
+ * ws_shard_update(WS_ADAFACTOR) runs in this order.  On real replicas each
+ * runs the per-shard stages for its own shard and exchanges the reduce results
+ * between them - the case of Section 4.1 where "sharding affects the collapsed
+ * dimensions": every replica reduces what its shard holds, then the replicas
+ * combine their results with an all-reduce.
+ *   WS_AF_BEGIN    clears this step's row / column sums (no shard argument)
+ *   WS_AF_SUMS     shard r: reduce the gradients, keep the sum (ghat slot r),
+ *                  add the shard's partial row / column sums of g^2 + eps into
+ *                  the sums, leave per-tile sums of w^2
+ *                  -> exchange: all-reduce (sum) the float region
+ *                     ws_workspace_adafactor_sums() names; share the partial
+ *                     rows (ws_workspace_partials)
+ *   WS_AF_MOMENTS  Rv', Cv' (state->v, the same on every replica) and the
+ *                  1/sqrt factors
+ *   WS_AF_SUMSQ    shard r: per-tile sums of U^2
+ *                  -> exchange: share the partial rows again
+ *   WS_AF_CLIP     step sizes alpha_t / max(1, RMS(U_t)/d) for every tensor
+ *   WS_AF_APPLY    shard r: w' = w - step size * U, gathered slot r
+ * Arguments a stage does not use may be NULL (grads outside WS_AF_SUMS, out
+ * outside WS_AF_APPLY, state in WS_AF_BEGIN / SUMSQ / CLIP).  The workspace has
+ * ws_workspace_bytes(plan, WS_ADAFACTOR) bytes and persists through the stages. */
+typedef enum {
+    WS_AF_BEGIN = 0, WS_AF_SUMS = 1, WS_AF_MOMENTS = 2, WS_AF_SUMSQ = 3, WS_AF_CLIP = 4, WS_AF_APPLY = 5
+} ws_af_stage;
+ws_status ws_adafactor_stage(const ws_plan* plan, ws_af_stage stage, int32_t r, const ws_grads* grads,
+                             const ws_state* state, const ws_hyper* hyper, const ws_out* out,
+                             void* workspace, size_t workspace_bytes, void* stream);
+/* Byte offset and size of the float array of row / column sums inside the
+ * Adafactor workspace (the all-reduce operand between WS_AF_SUMS and
+ * WS_AF_MOMENTS).  Host only. */
+ws_status ws_workspace_adafactor_sums(const ws_plan* plan, size_t* offset_bytes, size_t* bytes);
+
 /* ------------------------------------- formatting fused into the update ---
  * Section 5.1: padding the gradient before the reduce-scatter costs every
  * replica a read and a write of the full data, so the paper fuses the

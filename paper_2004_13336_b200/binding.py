@@ -84,6 +84,7 @@ EXPORTS = [
     "ws_plan_create_layout", "ws_plan_layout", "ws_pack_sets",
     "ws_plan_factored_elems", "ws_plan_factored_layout", "ws_workspace_partials",
     "ws_lars_partial", "ws_lars_finalize", "ws_lars_apply",
+    "ws_adafactor_stage", "ws_workspace_adafactor_sums",
 ]
 
 _lib = None
@@ -147,6 +148,11 @@ def lib() -> C.CDLL:
     L.ws_lars_apply.restype = C.c_int
     L.ws_lars_apply.argtypes = [vp, C.c_int32, C.POINTER(ws_state), C.POINTER(ws_hyper), C.POINTER(ws_out),
                                 vp, C.c_size_t, vp]
+    L.ws_adafactor_stage.restype = C.c_int
+    L.ws_adafactor_stage.argtypes = [vp, C.c_int, C.c_int32, C.POINTER(ws_grads), C.POINTER(ws_state),
+                                     C.POINTER(ws_hyper), C.POINTER(ws_out), vp, C.c_size_t, vp]
+    L.ws_workspace_adafactor_sums.restype = C.c_int
+    L.ws_workspace_adafactor_sums.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     L.ws_workspace_partials.restype = C.c_int
     L.ws_workspace_partials.argtypes = [vp, C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
     L.ws_plan_factored_elems.restype = C.c_int64
@@ -384,6 +390,27 @@ def ws_lars_apply(plan: Plan, r: int, w, m, hyper: ws_hyper, workspace: torch.Te
     _check(lib().ws_lars_apply(plan.handle, r, C.byref(s), C.byref(hyper), C.byref(o) if o is not None else None,
                                workspace.data_ptr(), workspace.numel() * workspace.element_size(), _stream()),
            "ws_lars_apply")
+
+
+AF_BEGIN, AF_SUMS, AF_MOMENTS, AF_SUMSQ, AF_CLIP, AF_APPLY = range(6)
+
+
+def ws_adafactor_stage(plan: Plan, stage: int, r: int, hyper: ws_hyper, workspace: torch.Tensor, gbufs=None,
+                       w=None, fstate=None, gathered: Optional[torch.Tensor] = None, slice_mode: int = 0):
+    """One stage of Adafactor (AF_BEGIN ... AF_APPLY) for shard r, or all shards with r = -1."""
+    g = _grads(gbufs, slice_mode) if gbufs is not None else None
+    s = ws_state(w.data_ptr() if w is not None else None, None, fstate.data_ptr() if fstate is not None else None)
+    o = _out(gathered)
+    _check(lib().ws_adafactor_stage(plan.handle, stage, r, C.byref(g) if g is not None else None, C.byref(s),
+                                    C.byref(hyper), C.byref(o) if o is not None else None, workspace.data_ptr(),
+                                    workspace.numel() * workspace.element_size(), _stream()), "ws_adafactor_stage")
+
+
+def adafactor_sums(plan: Plan, workspace: torch.Tensor) -> torch.Tensor:
+    """Float view of this step's row / column sums inside an Adafactor workspace (the all-reduce operand)."""
+    off, nb = C.c_size_t(), C.c_size_t()
+    _check(lib().ws_workspace_adafactor_sums(plan.handle, C.byref(off), C.byref(nb)), "ws_workspace_adafactor_sums")
+    return workspace[off.value: off.value + nb.value].view(torch.float32)
 
 
 def lamb_partials(plan: Plan, workspace: torch.Tensor) -> torch.Tensor:

@@ -4,7 +4,8 @@ shard-major layout, a reduce-scatter leaves replica r the summed shard r, replic
 its 1/R of the weights and of the optimizer slots (which stay sharded between steps), and an
 all-gather of the updated shards rebuilds the full weights - in bfloat16 when asked, while
 the update stays fp32 (Section 4.2).  LAMB and LARS add the combination of the replicas'
-partial norm sums between their two phases (Section 4.1, "Non-elementwise operators").
+partial norm sums between their two phases, Adafactor the all-reduce of its row / column sums
+(Section 4.1, "Non-elementwise operators").
 
 This module is plumbing only: the collectives are ``torch.distributed`` calls (NCCL on GPUs)
 and every arithmetic step is a call into the C-ABI library through ``binding``.  The receive
@@ -14,7 +15,7 @@ own input and output layout, so no extra copy sits between a collective and a ke
 
 ``ops`` names the module that supplies ``Plan``, ``ws_pack``, ``ws_unpack``,
 ``ws_shard_update``, ``ws_lamb_partial / _finalize / _apply``, ``ws_lars_partial / _finalize /
-_apply``, ``lamb_partials`` and ``make_hyper``; it is the CUDA binding unless a test passes a
+_apply``, ``ws_adafactor_stage``, ``lamb_partials``, ``adafactor_sums`` and ``make_hyper``; it is the CUDA binding unless a test passes a
 stand-in to run the choreography on CPU ranks.
 """
 from __future__ import annotations
@@ -34,8 +35,8 @@ class ShardedUpdate:
                  align_elems: int = 32, device=None, group=None, ops=None):
         if ops is None:
             from . import binding as ops      # fails loudly without the built CUDA library
-        if opt not in ("sgdm", "adam", "lamb", "lars"):
-            raise ValueError("shard-by-shard updates exist for sgdm, adam, lamb and lars")
+        if opt not in ("sgdm", "adam", "lamb", "lars", "adafactor"):
+            raise ValueError(f"unknown optimizer {opt}")
         self.ops, self.opt, self.hyper_dict, self.group = ops, opt, dict(hyper), group
         self.rank, self.world = dist.get_rank(group), dist.get_world_size(group)
         self.device = torch.device(device) if device is not None else torch.device("cuda", torch.cuda.current_device())
@@ -47,9 +48,12 @@ class ShardedUpdate:
         self.recv = torch.empty(S, dtype=grad_dtype, device=self.device)      # ... and output
         self.gathered = torch.zeros(G, dtype=out_dtype, device=self.device)   # all-gather buffer
         self.workspace = None
-        if opt in ("lamb", "lars"):
+        if opt in ("lamb", "lars", "adafactor"):
             self.workspace = torch.zeros(max(16, self.plan.workspace_bytes(opt)), dtype=torch.uint8,
                                          device=self.device)
+        self.fstate = None                                                    # Adafactor: replicated, small
+        if opt == "adafactor":
+            self.fstate = torch.zeros(self.plan.factored_elems, **z)
 
     # -- sharding program (Section 4.2): every replica starts from the same full state -----
     def load_state(self, w: Sequence[torch.Tensor], m: Sequence[torch.Tensor], v: Sequence[torch.Tensor]):
@@ -81,6 +85,20 @@ class ShardedUpdate:
             dist.all_gather_into_tensor(rows.view(-1), rows[r], group=self.group)
             ops.ws_lamb_finalize(plan, self.workspace)                          # same sums, same order, every rank
             ops.ws_lamb_apply(plan, r, self.w, self.m, self.v, hy, self.workspace, self.gathered)
+        elif self.opt == "adafactor":
+            # Section 4.1, reduces over a sharded dimension: every replica reduces what its shard holds,
+            # then the results are combined with an all-reduce (here also the per-tile scalar sums)
+            st, ws = ops.ws_adafactor_stage, self.workspace
+            rows = ops.lamb_partials(plan, ws)
+            st(plan, ops.AF_BEGIN, -1, hy, ws)
+            st(plan, ops.AF_SUMS, r, hy, ws, gbufs=[self.recv], w=self.w, slice_mode=1)
+            dist.all_reduce(ops.adafactor_sums(plan, ws), group=self.group)
+            dist.all_gather_into_tensor(rows.view(-1), rows[r], group=self.group)
+            st(plan, ops.AF_MOMENTS, -1, hy, ws, fstate=self.fstate)
+            st(plan, ops.AF_SUMSQ, r, hy, ws)
+            dist.all_gather_into_tensor(rows.view(-1), rows[r], group=self.group)
+            st(plan, ops.AF_CLIP, -1, hy, ws)
+            st(plan, ops.AF_APPLY, r, hy, ws, w=self.w, gathered=self.gathered)
         elif self.opt == "lars":
             ops.ws_lars_partial(plan, r, [self.recv], self.w, self.m, hy, self.workspace, slice_mode=1)
             rows = ops.lamb_partials(plan, self.workspace)

@@ -336,6 +336,14 @@ extern "C" ws_status ws_workspace_partials(const ws_plan* p, size_t* offset_byte
     return WS_OK;
 }
 
+extern "C" ws_status ws_workspace_adafactor_sums(const ws_plan* p, size_t* offset_bytes, size_t* bytes) {
+    if (!p || !offset_bytes || !bytes) return WS_ERR_INVALID_ARG;
+    const WsLambWs L = ws_lamb_layout(p, nullptr);
+    *offset_bytes = (size_t)((char*)L.acc - (char*)nullptr);
+    *bytes = sizeof(float) * (size_t)p->Fi;
+    return WS_OK;
+}
+
 extern "C" size_t ws_workspace_bytes(const ws_plan* p, ws_opt opt) {
     if (!p) return 0;
     if (opt == WS_LAMB) return ws_lamb_layout(p, nullptr).bytes;

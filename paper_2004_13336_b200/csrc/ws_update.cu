@@ -1347,76 +1347,105 @@ ws_status fused_phase(const ws_plan* plan, int32_t r, const ws_tensor_table* gra
 // Adafactor, all shards: zero the row / column sums, pass 1 (reduce, keep the sum, partial row and
 // column sums), moments + step size, pass 2 (sum U^2), clipping, pass 3 (apply).  Either the
 // packed-buffer arguments (grads, out) or the tensor tables (gtab, wtab) are given.
-ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_tensor_table* gtab,
-                    const ws_state* state, const ws_hyper* hyper, const ws_out* out, const ws_tensor_table* wtab,
-                    void* workspace, size_t workspace_bytes, cudaStream_t st) {
-    if (!plan || !state || !hyper) return WS_ERR_INVALID_ARG;
+// One stage of Adafactor for shard r (or all shards with r == -1); see ws_adafactor_stage in ws.h.
+// Either the packed-buffer arguments (grads, out) or the tensor tables (gtab, wtab) are given.
+ws_status af_stage(const ws_plan* plan, int stage, int32_t r, const ws_grads* grads, const ws_tensor_table* gtab,
+                   const ws_state* state, const ws_hyper* hyper, const ws_out* out, const ws_tensor_table* wtab,
+                   void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (!plan || !hyper) return WS_ERR_INVALID_ARG;
     if (!plan->d_tiles) return WS_ERR_NOT_UPLOADED;
-    if (r != -1) return WS_ERR_INVALID_ARG;
-    if (hyper->weight_decay != 0.0 || !(hyper->clip_threshold > 0.0) || !(hyper->decay_exponent > 0.0) ||
-        !(hyper->eps >= 0.0) || !(hyper->eps2 >= 0.0) || hyper->step < 1)
+    if (r < -1 || r >= plan->R) return WS_ERR_INVALID_ARG;
+    if (hyper->opt != WS_ADAFACTOR || hyper->weight_decay != 0.0 || !(hyper->clip_threshold > 0.0) ||
+        !(hyper->decay_exponent > 0.0) || !(hyper->eps >= 0.0) || !(hyper->eps2 >= 0.0) || hyper->step < 1)
         return WS_ERR_INVALID_ARG;
-    if (!state->v) return WS_ERR_INVALID_ARG;
-    if (!ws_aligned16(state->v)) return WS_ERR_ALIGNMENT;
     ws_status s = check_ws(plan, workspace, workspace_bytes, WS_ADAFACTOR);
     if (s != WS_OK) return s;
     const WsLambWs L = ws_lamb_layout(plan, workspace);
     const bool fused = gtab != nullptr;
-    const double beta = 1.0 - pow((double)hyper->step, -hyper->decay_exponent);
-    const double inv_sqrt_t = 1.0 / sqrt((double)hyper->step);
-    const double rho_step = hyper->lr < inv_sqrt_t ? hyper->lr : inv_sqrt_t;
-    const int reps = finalize_reps(plan);
-
-    cudaError_t e = cudaMemsetAsync(L.acc, 0, L.acc_bytes, st);
-    if (e != cudaSuccess) return ws_cuda_fail(e, "adafactor(clear sums)");
     UpdParams P;
     int ok;
     bool gbf;
-    if (fused) {
-        if ((s = fused_phase(plan, -1, gtab, state, hyper, wtab, K_AF1, workspace, st)) != WS_OK) return s;
-    } else {
-        if ((s = prepare(plan, -1, grads, state, hyper, nullptr, K_AF1, P, ok, gbf)) != WS_OK) return s;
-        P.partials = L.partials;
-        P.ghat = L.ghat;
-        P.af_acc = L.acc;
-        std::vector<const void*> gp;
-        offset_grad_ptrs(plan, -1, grads, gp);
-        if ((s = launch_any(K_AF1, gbf, O_NONE, P, gp.data(), st)) != WS_OK) return s;
+    switch (stage) {
+        case WS_AF_BEGIN: {
+            cudaError_t e = cudaMemsetAsync(L.acc, 0, L.acc_bytes, st);
+            return e == cudaSuccess ? WS_OK : ws_cuda_fail(e, "adafactor(clear sums)");
+        }
+        case WS_AF_SUMS: {
+            if (fused) return fused_phase(plan, r, gtab, state, hyper, wtab, K_AF1, workspace, st);
+            if ((s = prepare(plan, r, grads, state, hyper, nullptr, K_AF1, P, ok, gbf)) != WS_OK) return s;
+            P.partials = L.partials;
+            P.ghat = L.ghat;
+            P.af_acc = L.acc;
+            std::vector<const void*> gp;
+            offset_grad_ptrs(plan, r, grads, gp);
+            return launch_any(K_AF1, gbf, O_NONE, P, gp.data(), st);
+        }
+        case WS_AF_MOMENTS: {
+            if (!state || !state->v) return WS_ERR_INVALID_ARG;
+            if (!ws_aligned16(state->v)) return WS_ERR_ALIGNMENT;
+            const double beta = 1.0 - pow((double)hyper->step, -hyper->decay_exponent);
+            const unsigned nchunks = (unsigned)plan->afchunks.size();
+            if (nchunks == 0) return WS_OK;
+            af_moments_kernel<<<nchunks, kBlock, 0, st>>>(plan->d_afchunks, plan->d_segaf, (float*)state->v, L.acc, L.rsum, beta);
+            if ((s = ws_check_launch("adafactor(moments)")) != WS_OK) return s;
+            af_factors_kernel<<<nchunks, kBlock, 0, st>>>(plan->d_afchunks, plan->d_segaf, (const float*)state->v, L.rsum, L.fac);
+            return ws_check_launch("adafactor(factors)");
+        }
+        case WS_AF_SUMSQ: {
+            // (the pass reads only the workspace; `state` is not touched, w stands in for the argument checks)
+            ws_state dummy = {workspace, nullptr, nullptr};
+            if ((s = prepare(plan, r, nullptr, &dummy, hyper, nullptr, K_AF2, P, ok, gbf)) != WS_OK) return s;
+            P.partials = L.partials;
+            P.ghat = L.ghat;
+            P.af_fac = L.fac;
+            if (P.nitems < 1) return WS_OK;
+            int dev = 0, sms = 148;
+            cudaGetDevice(&dev);
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+            const long long cap = (long long)sms * WS_TUNE_AF2_CTAS;
+            af_sumsq_kernel<<<(unsigned)(P.nitems < cap ? P.nitems : cap), kBlock, 0, st>>>(P);
+            return ws_check_launch("adafactor(pass 2)");
+        }
+        case WS_AF_CLIP: {
+            const double inv_sqrt_t = 1.0 / sqrt((double)hyper->step);
+            const double rho_step = hyper->lr < inv_sqrt_t ? hyper->lr : inv_sqrt_t;
+            af_finalize_clip_kernel<<<plan->T, kBlock, 0, st>>>(plan->d_segtiles, plan->d_segaf, L.partials, plan->ntiles,
+                                                               finalize_reps(plan), L.alpha, L.rho, L.norms, hyper->eps2,
+                                                               rho_step, hyper->clip_threshold);
+            return ws_check_launch("adafactor(clipping)");
+        }
+        case WS_AF_APPLY: {
+            if (fused) return fused_phase(plan, r, gtab, state, hyper, wtab, K_AF3, workspace, st);
+            if ((s = prepare(plan, r, nullptr, state, hyper, out, K_AF3, P, ok, gbf)) != WS_OK) return s;
+            P.rho = L.rho;
+            P.ghat = L.ghat;
+            P.af_fac = L.fac;
+            return launch_any(K_AF3, false, ok, P, nullptr, st);
+        }
+        default: return WS_ERR_INVALID_ARG;
     }
-    const unsigned nchunks = (unsigned)plan->afchunks.size();
-    if (nchunks > 0) {
-        af_moments_kernel<<<nchunks, kBlock, 0, st>>>(plan->d_afchunks, plan->d_segaf, (float*)state->v, L.acc, L.rsum, beta);
-        if ((s = ws_check_launch("adafactor(moments)")) != WS_OK) return s;
-        af_factors_kernel<<<nchunks, kBlock, 0, st>>>(plan->d_afchunks, plan->d_segaf, (const float*)state->v, L.rsum, L.fac);
-        if ((s = ws_check_launch("adafactor(factors)")) != WS_OK) return s;
-    }
+}
 
-    if ((s = prepare(plan, -1, nullptr, state, hyper, nullptr, K_AF2, P, ok, gbf)) != WS_OK) return s;
-    P.partials = L.partials;
-    P.ghat = L.ghat;
-    P.af_fac = L.fac;
-    if (P.nitems > 0) {
-        int dev = 0, sms = 148;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        const long long cap = (long long)sms * WS_TUNE_AF2_CTAS;
-        af_sumsq_kernel<<<(unsigned)(P.nitems < cap ? P.nitems : cap), kBlock, 0, st>>>(P);
-        if ((s = ws_check_launch("adafactor(pass 2)")) != WS_OK) return s;
+// Adafactor, all shards: the six stages in order.
+ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_tensor_table* gtab,
+                    const ws_state* state, const ws_hyper* hyper, const ws_out* out, const ws_tensor_table* wtab,
+                    void* workspace, size_t workspace_bytes, cudaStream_t st) {
+    if (r != -1 || !state) return WS_ERR_INVALID_ARG;
+    for (int stage = WS_AF_BEGIN; stage <= WS_AF_APPLY; ++stage) {
+        const ws_status s = af_stage(plan, stage, -1, grads, gtab, state, hyper, out, wtab, workspace, workspace_bytes, st);
+        if (s != WS_OK) return s;
     }
-    af_finalize_clip_kernel<<<plan->T, kBlock, 0, st>>>(plan->d_segtiles, plan->d_segaf, L.partials, plan->ntiles, reps,
-                                                       L.alpha, L.rho, L.norms, hyper->eps2, rho_step,
-                                                       hyper->clip_threshold);
-    if ((s = ws_check_launch("adafactor(clipping)")) != WS_OK) return s;
-
-    if (fused) return fused_phase(plan, -1, gtab, state, hyper, wtab, K_AF3, workspace, st);
-    if ((s = prepare(plan, -1, nullptr, state, hyper, out, K_AF3, P, ok, gbf)) != WS_OK) return s;
-    P.rho = L.rho;
-    P.ghat = L.ghat;
-    P.af_fac = L.fac;
-    return launch_any(K_AF3, false, ok, P, nullptr, st);
+    return WS_OK;
 }
 
 }  // namespace
+
+extern "C" ws_status ws_adafactor_stage(const ws_plan* plan, ws_af_stage stage, int32_t r, const ws_grads* grads,
+                                        const ws_state* state, const ws_hyper* hyper, const ws_out* out,
+                                        void* workspace, size_t workspace_bytes, void* stream) {
+    return af_stage(plan, (int)stage, r, grads, nullptr, state, hyper, out, nullptr, workspace, workspace_bytes,
+                    (cudaStream_t)stream);
+}
 
 extern "C" ws_status ws_fused_update(const ws_plan* plan, int32_t r, const ws_tensor_table* grads, const ws_state* state,
                                      const ws_hyper* hyper, const ws_tensor_table* weights, void* workspace,

@@ -284,3 +284,36 @@ def test_randomised_matrix_shapes_on_both_routes(case):
             tol = TOL_BF16 if odt == torch.bfloat16 else (TOL_LAMB if numels[t] >= 32 else 1e-4)
             assert err(a, ow[t]) <= tol, (route, t, shapes[t])
             assert err(gs[off:off + rows + cols], of[off:off + rows + cols]) <= 10 * TOL_LAMB, (route, t, shapes[t])
+
+
+@pytest.mark.parametrize("R", [1, 3, 8])
+@pytest.mark.parametrize("slice_mode", [0, 1])
+def test_stage_by_stage_per_shard_matches_oracle(R, slice_mode):
+    """What R replicas would run: the per-shard stages for every shard with the finalize stages in
+    between (on one GPU the sums of all shards already meet in the one workspace)."""
+    wl, plan, w, g, f0 = _setup(SHAPES, R, seed=R + 31)
+    h = _hyper(step=6)
+    ow, of, oinfo = _oracle(SHAPES, h, w, g, f0)
+    hy = B.make_hyper("adafactor", h)
+    pw, = _pack(plan, [w])
+    pg = _pack(plan, g)
+    fs = f0.clone()
+    ws = torch.full((plan.workspace_bytes("adafactor"),), 0xFF, dtype=torch.uint8, device=DEV)
+    gath = torch.zeros(plan.G, dtype=torch.bfloat16, device=DEV)
+    S = plan.S
+    sl = [slice(r * S, (r + 1) * S) for r in range(R)]
+    gr = (lambda r: [b[sl[r]] for b in pg]) if slice_mode else (lambda r: pg)
+    B.ws_adafactor_stage(plan, B.AF_BEGIN, -1, hy, ws)
+    for r in range(R):
+        B.ws_adafactor_stage(plan, B.AF_SUMS, r, hy, ws, gbufs=gr(r), w=pw[sl[r]], slice_mode=slice_mode)
+    B.ws_adafactor_stage(plan, B.AF_MOMENTS, -1, hy, ws, fstate=fs)
+    for r in range(R):
+        B.ws_adafactor_stage(plan, B.AF_SUMSQ, r, hy, ws)
+    B.ws_adafactor_stage(plan, B.AF_CLIP, -1, hy, ws)
+    for r in range(R):
+        B.ws_adafactor_stage(plan, B.AF_APPLY, r, hy, ws, w=pw[sl[r]], gathered=gath)
+    _check(plan, SHAPES, pw, fs, ws, ow, of, oinfo)
+    assert torch.equal(gath, pw.to(torch.bfloat16))
+    with pytest.raises(B.WsError) as e:               # a stage number outside the list
+        B.ws_adafactor_stage(plan, 9, -1, hy, ws)
+    assert e.value.status == 1

@@ -96,3 +96,28 @@ def test_one_kernel_route_over_symmetric_memory(world_of_one, opt, out_dtype, gd
             assert err(bf16_to_f64(to_np(a)), b) <= TOL_BF16, t
         else:
             assert err(to_np(a), b) <= TOL_FP32, t
+
+
+def test_adafactor_on_a_one_rank_group(world_of_one):
+    """Adafactor on the NCCL route: per-shard stages with the all-reduce of the row / column sums and the
+    exchange of the per-tile sums between them (real NCCL calls, one rank)."""
+    shapes = SHAPES + [(24, 2048)]
+    wl = W.Workload("t", list(shapes), R=1, opt="adafactor", hyper={}, grad_std=1e-2, seed=37)
+    w, m, v = W.make_state(wl, DEV)
+    g = W.make_grads(wl, DEV)[0]
+    hyper = dict(lr=1e-2, beta1=0.0, beta2=0.0, eps=1e-30, weight_decay=0.0, momentum=0.0, grad_scale=1.0, step=3,
+                 eps2=1e-3, clip_threshold=1.0, decay_exponent=0.8)
+    su = ShardedUpdate(shapes, "adafactor", hyper, device=DEV)
+    su.load_state(w, m, v)
+    f0 = W.make_factored_state(wl, su.plan.factored_elems, DEV)
+    su.fstate.copy_(f0)
+    outs = [torch.zeros(n, device=DEV) for n in wl.numels]
+    su.step(g, outs)
+    torch.cuda.synchronize()
+    hs = O.make_hyper("adafactor", hyper)
+    of = to_np(f0)
+    for t, (off, rows, cols) in enumerate(su.plan.factored_layout()):
+        ref = to_np(w[t]).reshape(shapes[t])
+        O.adafactor_tensor(hs, [to_np(g[t])], ref, of[off:off + rows], of[off + rows:off + rows + cols] if cols else None)
+        assert err(to_np(outs[t]), ref) <= TOL_LAMB, t
+        assert err(to_np(su.fstate)[off:off + rows + cols], of[off:off + rows + cols]) <= TOL_LAMB, t
