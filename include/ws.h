@@ -16,6 +16,10 @@
  *   - Nothing throws or aborts across this boundary; every failure is a
  *     ws_status.  Argument errors are found on the host before any launch.
  *   - The caller owns every buffer.  The library owns only ws_plan objects.
+ *   - The update kernels use programmatic dependent launch: a kernel may start
+ *     while the preceding kernel of the stream drains, but before it waits for
+ *     that kernel it reads nothing except the plan's tables and the
+ *     tensor-pointer tables (which are written once, by copies).
  *   - dtype arguments say how 2- or 4-byte elements are interpreted.
  *
  * Layout vocabulary (Section 4.1 "Sharding representation", Section 5.2
