@@ -539,10 +539,10 @@ def run_ours(args):
     if rank == 0:
         sampler.start()
     res = {}
+    if run_fused:       # the headline route first: a long run of the other route leaves the GPU at its power cap
+        res["fused"] = time_path(step_fused, 2)
     if run_unfused:
         res["unfused"] = time_path(step_unfused, 4)
-    if run_fused:
-        res["fused"] = time_path(step_fused, 2)
     primary = "fused" if run_fused else "unfused"
     ms_per_step, _, window, step_stats = res[primary]
     value = job_value(N, world, ms_per_step)
