@@ -317,3 +317,28 @@ def test_stage_by_stage_per_shard_matches_oracle(R, slice_mode):
     with pytest.raises(B.WsError) as e:               # a stage number outside the list
         B.ws_adafactor_stage(plan, 9, -1, hy, ws)
     assert e.value.status == 1
+
+
+def test_step_can_be_captured_in_a_cuda_graph():
+    # clear + six kernels of an Adafactor step inside a captured graph: replays track the eager calls
+    # (to rounding: the row / column sums are atomic adds)
+    R = 3
+    wl, plan, w, g, f0 = _setup(SHAPES, R, seed=44)
+    hy = B.make_hyper("adafactor", _hyper(step=7))
+    pw, = _pack(plan, [w])
+    pg = B.PtrList(_pack(plan, g))
+    ew, ef, fs = pw.clone(), f0.clone(), f0.clone()
+    ws = torch.zeros(plan.workspace_bytes("adafactor"), dtype=torch.uint8, device=DEV)
+    for _ in range(2):
+        B.ws_shard_update(plan, -1, pg, ew, None, ef, hy, None, ws)
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            B.ws_shard_update(plan, -1, pg, pw, None, fs, hy, None, ws)
+    torch.cuda.current_stream().wait_stream(side)
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.allclose(pw, ew, rtol=2e-5, atol=1e-8) and torch.allclose(fs, ef, rtol=2e-4, atol=0)

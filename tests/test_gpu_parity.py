@@ -545,6 +545,34 @@ def test_step_can_be_captured_in_a_cuda_graph():
         assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("opt", ["lamb", "lars"])
+def test_multi_launch_steps_can_be_captured_in_a_cuda_graph(opt):
+    # the norm-based optimizers are three launches joined by programmatic dependent launch: the
+    # captured graph replays to the same bits as the eager calls (fixed-order sums)
+    wl, w, m, v, g = _model(SHAPES, 3, seed=14, gstd=1e-3)
+    plan = B.Plan(SHAPES, 3, 32)
+    h = _lars_hyper() if opt == "lars" else _hyper(opt)
+    hy = B.make_hyper(opt, h)
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    ew, em, ev = pw.clone(), pm.clone(), pv.clone()
+    gl = B.PtrList(pg)
+    ws = torch.zeros(plan.workspace_bytes(opt), dtype=torch.uint8, device=DEV)
+    sv, esv = (pv, ev) if opt == "lamb" else (None, None)
+    for _ in range(2):                                           # eager reference: two steps
+        B.ws_shard_update(plan, -1, gl, ew, em, esv, hy, None, ws)
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            B.ws_shard_update(plan, -1, gl, pw, pm, sv, hy, None, ws)
+    torch.cuda.current_stream().wait_stream(side)
+    graph.replay()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(pw, ew) and torch.equal(pm, em)
+
+
 @pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb"])
 @pytest.mark.parametrize("groups,M", [(2, 4), (5, 2), (3, 1)])
 def test_partial_sharding_more_gradient_copies_than_shards(opt, groups, M):
