@@ -19,7 +19,23 @@
  *   - The update kernels use programmatic dependent launch: a kernel may start
  *     while the preceding kernel of the stream drains, but before it waits for
  *     that kernel it reads nothing except the plan's tables and the
- *     tensor-pointer tables (which are written once, by copies).
+ *     tensor-pointer tables.  Those tables must therefore be complete before
+ *     the kernel that precedes an update call on the stream is launched:
+ *     upload them with ws_plan_upload / ws_tensor_table_upload (copies, which
+ *     a later kernel never overtakes) and do not rewrite them from a kernel
+ *     of your own directly in front of an update call.
+ *   - Accuracy a caller may expect against the same update in exact
+ *     arithmetic, per tensor, as max_i |x_i - ref_i| / max(|ref_i|, RMS(ref)):
+ *     1e-6 for the fp32 outputs of WS_SGDM and WS_ADAM, 1e-5 for WS_LAMB,
+ *     WS_LARS and WS_ADAFACTOR (their per-tensor norms are fp32 sums), one
+ *     bf16 ulp (2^-8 relative) for bf16 outputs.  These hold for gradients of
+ *     the scale of the state they update (the library's test recipe: standard
+ *     deviation 1e-3, up to 1024 copies).  Single elements can reach 1e-5
+ *     under WS_ADAM when gradient copies ten times larger are summed (not
+ *     averaged) over 8 or more replicas, the copies cancel and the element's
+ *     second moment starts at (almost) zero: the fp32 sum then carries an
+ *     error that is large against the cancelled total.  That is a property of
+ *     fp32 summation, not of the sharding.
  *   - dtype arguments say how 2- or 4-byte elements are interpreted.
  *
  * Layout vocabulary (Section 4.1 "Sharding representation", Section 5.2
@@ -257,7 +273,9 @@ ws_status ws_plan_factored_layout(const ws_plan* plan, int64_t* layout);
  *   float  fac[F']           1/sqrt factors of V for the two elementwise passes
  *   float  alpha[T]          max(eps2, RMS(w_t)) min(lr, 1/sqrt(step))
  * where F' is F = ws_plan_factored_elems() with every tensor's row part and
- * column part padded to a multiple of 8 floats. */
+ * column part padded to a multiple of 8 floats.  The WS_ADAFACTOR workspace
+ * must be 32-byte aligned (its second pass reads ghat with 256-bit loads);
+ * a workspace that is only 16-byte aligned is refused with WS_ERR_ALIGNMENT. */
 size_t ws_workspace_bytes(const ws_plan* plan, ws_opt opt);
 
 /* Where the per-tile partial sums live inside the workspace: byte offset of
@@ -299,8 +317,8 @@ ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_grads* grads,
  * partials in a fixed order in double and writes rho[T]; it stands where the
  * paper has the combined scalar all-reduce (Section 5.2), so call it after
  * phase 1 of ALL shards.  Phase 2 for shard r recomputes u from w, m', v' and
- * applies w' = w - lr rho u, writing the gathered slot.  `grads` is ignored
- * by ws_lamb_apply and may be NULL there.
+ * applies w' = w - lr rho u, writing the gathered slot.  hyper->opt must be
+ * WS_LAMB.
  * The shard-by-shard form gives bit for bit the result of the all-shard call
  * when every shard slice handed in is 32-byte aligned (S * element size a
  * multiple of 32: any A for fp32, A >= 16 for bf16 gradient slices);
@@ -490,7 +508,10 @@ ws_status ws_step_host(const ws_plan* plan, const ws_host_io* io, const ws_state
  *     exits, whether or not this entry point is ever called.
  *   - The first call on each device looks up the array's device address (with
  *     that device current) and caches it; make that first call outside any
- *     stream capture.  Later calls on the same device skip the lookup.
+ *     stream capture.  Later calls on the same device skip the lookup.  The
+ *     cached address belongs to the device's primary context: do not reset
+ *     the device (cudaDeviceReset) while the library stays loaded, the next
+ *     call would hand the kernels the old context's address.
  *   - All calls on one device share the one array, and it keeps whatever the
  *     previous call left in it.  Nothing in it needs clearing (each call
  *     overwrites every entry it later reads), but two calls whose kernels can

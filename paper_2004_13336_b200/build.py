@@ -53,7 +53,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(_OBJ, exist_ok=True)
     nvcc = _nvcc()
     extra = ["-Xptxas", "-v"] if verbose else []
-    extra += os.environ.get("WS_NVCC_EXTRA", "").split()       # development only: -DWS_TUNE_* overrides
     hdr_mtime = max(os.path.getmtime(os.path.join(_CSRC, f)) for f in os.listdir(_CSRC) if f.endswith(".h"))
     hdr_mtime = max(hdr_mtime, os.path.getmtime(os.path.join(_ROOT, "include", "ws.h")))
 

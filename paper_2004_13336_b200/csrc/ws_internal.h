@@ -101,6 +101,10 @@ struct WsLambWs {
 };
 WsLambWs ws_lamb_layout(const ws_plan* plan, void* workspace);
 
+// Argument checks of LAMB's apply phase for an all-shard call, with no launch (so that a sequence of
+// launches can refuse bad arguments before its first one).
+ws_status ws_lamb_check_apply_args(const ws_plan* plan, const ws_state* state, const ws_hyper* hyper, const ws_out* out);
+
 // error bookkeeping
 ws_status ws_cuda_fail(cudaError_t e, const char* what);
 ws_status ws_check_launch(const char* what);

@@ -56,9 +56,11 @@ extern "C" ws_status ws_lamb_update_static_scratch(const ws_plan* plan, const ws
     if (hyper->opt != WS_LAMB) return WS_ERR_INVALID_ARG;
     const size_t need = ws_workspace_bytes(plan, WS_LAMB);
     if (need > kStaticScratchBytes) return WS_ERR_TOO_LARGE;   // refuse before touching the device
-    void* scratch = nullptr;
-    ws_status s = scratch_for_current_device(&scratch);
+    // all three launches' arguments are checked before the first one
+    ws_status s = ws_lamb_check_apply_args(plan, state, hyper, out);
     if (s != WS_OK) return s;
+    void* scratch = nullptr;
+    if ((s = scratch_for_current_device(&scratch)) != WS_OK) return s;
     // Nothing in the scratch has to start at zero: phase 1 overwrites the partial
     // of every (shard, tile) and the finalize step overwrites every ratio and norm.
     s = ws_lamb_partial(plan, -1, grads, state, hyper, scratch, kStaticScratchBytes, stream);

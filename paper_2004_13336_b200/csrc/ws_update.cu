@@ -24,55 +24,25 @@
 // gradients come straight from the replicas' tensor lists and the updated
 // weights go straight to the weight tensors.
 //
-// The WS_TUNE_* macros are build-time tuning constants; their defaults are the
-// values measured best on a B200.
+// The k* constants below are the values measured best on a B200.
 #include <cuda_bf16.h>
 #include <math.h>
 
 #include "ws_internal.h"
 
-#ifndef WS_TUNE_MINB
-#define WS_TUNE_MINB 3   // resident CTAs per SM the compiler must allow for (register budget);
-                         // the bf16-gradient wide kernel on packed buffers is given WS_TUNE_MINB8 = 2
-                         // (measured faster with more registers; the fused variant is faster with 3)
-#endif
-#ifndef WS_TUNE_MINB8
-#define WS_TUNE_MINB8 2
-#endif
-#ifndef WS_TUNE_U8
-#define WS_TUNE_U8 1
-#endif
-#ifndef WS_TUNE_RBL
-#define WS_TUNE_RBL 16   // gradients per tree block when R > 32
-#endif
-#ifndef WS_TUNE_U4
-#define WS_TUNE_U4 1     // 128-bit accesses per thread per pass
-#endif
-#ifndef WS_TUNE_PDL
-#define WS_TUNE_PDL 1    // programmatic dependent launch: an update kernel lets the stream's next kernel start
-                         // early, and itself reads the plan and pointer tables before it waits for the
-                         // previous kernel (measured: LARS on the ResNet-50 set 2 % faster, others unchanged)
-#endif
-#ifndef WS_TUNE_AF2_UNROLL
-#define WS_TUNE_AF2_UNROLL 2
-#endif
-#ifndef WS_TUNE_AF2_CTAS
-#define WS_TUNE_AF2_CTAS 4   // CTAs per SM of Adafactor's pass 2 (a persistent grid)
-#endif
-#ifndef WS_TUNE_UAF2
-#define WS_TUNE_UAF2 2   // ... in Adafactor's pass 1 with up to 2 / up to 4 / more gradient copies
-#endif
-#ifndef WS_TUNE_UAF4
-#define WS_TUNE_UAF4 2
-#endif
-#ifndef WS_TUNE_UAF8
-#define WS_TUNE_UAF8 1
-#endif
-
 namespace {
 
 constexpr int kBlock = 256;
-constexpr int kAf2Unroll = WS_TUNE_AF2_UNROLL;
+// Resident CTAs per SM the compiler must allow for (register budget): 3 measured best (4 forces
+// spills, 2 leaves bandwidth unused); the bf16-gradient wide kernel on packed buffers and the
+// many-replica kernel are faster with the registers of 2.
+constexpr int kMinBlocks = 3;
+constexpr int kMinBlocksWide = 2;
+constexpr int kTreeBlockLarge = 16;   // gradients per tree block when R > 32
+constexpr int kAf2Unroll = 2;         // Adafactor's pass 2: vectors in flight per thread
+constexpr int kAf2Ctas = 4;           // ... and its resident CTAs per SM (a persistent grid)
+// 128-bit accesses per thread per pass in Adafactor's pass 1 with up to 2 / up to 4 / more copies
+constexpr int kUAf2 = 2, kUAf4 = 2, kUAf8 = 1;
 // Kernel flavours.  The norm-based optimizers run as two phases around a finalize step:
 // phase 1 (K_LAMB1, K_LARS1) reduces the gradients and leaves per-tile partial sums of the
 // two norms; phase 2 (K_LAMB2, K_LARS2) applies the step with the per-tensor ratio.
@@ -130,13 +100,6 @@ struct Fv {
     float f[VEC];
 };
 
-#ifndef WS_TUNE_LD8
-#define WS_TUNE_LD8 "ld.global.L1::no_allocate.L2::evict_first.v8.b32"
-#endif
-#ifndef WS_TUNE_ST8
-#define WS_TUNE_ST8 "st.global.v8.b32"
-#endif
-
 template <int VEC>
 __device__ __forceinline__ Fv<VEC> load_f32(const float* p) {
     Fv<VEC> o;
@@ -145,7 +108,7 @@ __device__ __forceinline__ Fv<VEC> load_f32(const float* p) {
         o.f[0] = v.x; o.f[1] = v.y; o.f[2] = v.z; o.f[3] = v.w;
     } else {
         unsigned r[8];
-        asm volatile(WS_TUNE_LD8 " {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+        asm volatile("ld.global.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
                      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
                      : "l"(p));
 #pragma unroll
@@ -159,7 +122,7 @@ __device__ __forceinline__ void store_f32(float* p, const Fv<VEC>& x) {
     if (VEC == 4) {
         __stcs(reinterpret_cast<float4*>(p), make_float4(x.f[0], x.f[1], x.f[2], x.f[3]));
     } else {
-        asm volatile(WS_TUNE_ST8 " [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+        asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
                      :: "l"(p), "r"(__float_as_uint(x.f[0])), "r"(__float_as_uint(x.f[1])), "r"(__float_as_uint(x.f[2])),
                         "r"(__float_as_uint(x.f[3])), "r"(__float_as_uint(x.f[4 % VEC])), "r"(__float_as_uint(x.f[5 % VEC])),
                         "r"(__float_as_uint(x.f[6 % VEC])), "r"(__float_as_uint(x.f[7 % VEC]))
@@ -360,7 +323,7 @@ __device__ __forceinline__ void red_add_vec(float* p, const float* x) {
 // One CTA handles one (shard, tile) work item; the grid is the item count, so the
 // hardware CTA scheduler walks the buffers front to back.
 template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED>
-__global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8) ? WS_TUNE_MINB8 : WS_TUNE_MINB) update_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp) {
+__global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8) ? kMinBlocksWide : kMinBlocks) update_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp) {
     constexpr bool HAS_V = (OPT == K_ADAM || OPT == K_LAMB1 || OPT == K_LAMB2);
     constexpr bool READS_G = !is_phase2(OPT);     // phase 2 works from state (and the stored gradient sum)
     constexpr bool READS_W = true;
@@ -378,10 +341,8 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
     // of Section 2.2 written straight into every replica's tensors), the tile's further output pointers
     __shared__ void* swp[(FUSED && READS_G && writes_weights(OPT)) ? NP : 1];
 
-#if WS_TUNE_PDL
     // the next kernel of the stream may start its prologue while this grid's last CTAs run
     asm volatile("griddepcontrol.launch_dependents;");
-#endif
     for (long long item = blockIdx.x; item < P.nitems; item += gridDim.x) {
         long long rs = P.concat ? 0 : item / P.ntiles;     // shard index inside this launch
         const long long ti = P.concat ? P.tile_lo + item : item - rs * P.ntiles;
@@ -410,11 +371,9 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
             }
         }
         const int nvec = tl.len / VEC;
-#if WS_TUNE_PDL
         // the plan's tables and the tensor-pointer tables do not depend on the previous kernel of the
         // stream; everything read from here on may
         asm volatile("griddepcontrol.wait;" ::: "memory");
-#endif
         float lr_rho = 0.f;
         if (OPT == K_LAMB2 || OPT == K_LARS2) lr_rho = P.c.lr * P.rho[tl.seg];
         if (OPT == K_AF3) lr_rho = P.rho[tl.seg];         // alpha_t / max(1, RMS(U_t)/d)
@@ -779,10 +738,8 @@ __global__ void __launch_bounds__(kBlock) lamb_finalize_kernel(const WsSegTiles*
     const int t = blockIdx.x;
     double a, b;
     const WsSegTiles mine = segtiles[t];
-#if WS_TUNE_PDL
     asm volatile("griddepcontrol.launch_dependents;");
     asm volatile("griddepcontrol.wait;" ::: "memory");
-#endif
     sum_partials(mine, partials, ntiles, R, a, b);
     if (threadIdx.x == 0) {
         norms[2 * t] = a;
@@ -863,7 +820,7 @@ __global__ void __launch_bounds__(kBlock) af_finalize_clip_kernel(const WsSegTil
 // one tile would spend most of its life waiting for the tile descriptor, then the matrix view,
 // then the row factor; here a CTA walks many tiles and fetches the next tile's descriptor and
 // matrix view while it works on the current one.
-__global__ void __launch_bounds__(kBlock, WS_TUNE_AF2_CTAS) af_sumsq_kernel(const UpdParams P) {
+__global__ void __launch_bounds__(kBlock, kAf2Ctas) af_sumsq_kernel(const UpdParams P) {
     long long item = blockIdx.x;
     if (item >= P.nitems) return;
     auto tile_of = [&](long long it, long long& rs) {
@@ -972,7 +929,6 @@ __global__ void __launch_bounds__(kBlock, WS_TUNE_AF2_CTAS) af_sumsq_kernel(cons
 // -------------------------------------------------------------- dispatch ---
 void launch_lamb_finalize(int T, cudaStream_t st, const WsSegTiles* segtiles, const float2* partials, long long ntiles,
                           int R, float* rho, double* norms, int lars, double eta, double beta) {
-#if WS_TUNE_PDL
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)T);
     cfg.blockDim = dim3(kBlock);
@@ -983,9 +939,6 @@ void launch_lamb_finalize(int T, cudaStream_t st, const WsSegTiles* segtiles, co
     cfg.attrs = at;
     cfg.numAttrs = 1;
     cudaLaunchKernelEx(&cfg, lamb_finalize_kernel, segtiles, partials, ntiles, R, rho, norms, lars, eta, beta);
-#else
-    lamb_finalize_kernel<<<T, kBlock, 0, st>>>(segtiles, partials, ntiles, R, rho, norms, lars, eta, beta);
-#endif
 }
 
 template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED>
@@ -995,22 +948,18 @@ ws_status launch(const UpdParams& P, const void* const* gptrs, cudaStream_t st) 
     long long grid = P.nitems;
     if (grid < 1) return WS_OK;
     if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;
-#if WS_TUNE_PDL
-    {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3((unsigned)grid);
-        cfg.blockDim = dim3(kBlock);
-        cfg.stream = st;
-        cudaLaunchAttribute at[1];
-        at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        at[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.attrs = at;
-        cfg.numAttrs = 1;
-        cudaLaunchKernelEx(&cfg, update_kernel<OPT, GBF, OUT, VEC, U, RB, NP, FUSED>, P, gp);
-        return ws_check_launch(FUSED ? "ws_fused_update" : "ws_shard_update");
-    }
-#endif
-    update_kernel<OPT, GBF, OUT, VEC, U, RB, NP, FUSED><<<(unsigned)grid, kBlock, 0, st>>>(P, gp);
+    // programmatic dependent launch: the kernel may start while the previous kernel of the stream drains
+    // (it reads only the plan and pointer tables before it waits for that kernel)
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kBlock);
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, update_kernel<OPT, GBF, OUT, VEC, U, RB, NP, FUSED>, P, gp);
     return ws_check_launch(FUSED ? "ws_fused_update" : "ws_shard_update");
 }
 
@@ -1021,26 +970,26 @@ template <int OPT, bool GBF, int OUT, bool FUSED>
 ws_status launch_r(const UpdParams& P, const void* const* gptrs, bool wide_ok, cudaStream_t st) {
     if constexpr (is_phase2(OPT)) {
         if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 1, 1, FUSED>(P, gptrs, st);
-        return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 1, 1, FUSED>(P, gptrs, st);
+        return launch<OPT, GBF, OUT, 4, 1, 1, 1, FUSED>(P, gptrs, st);
     } else {
         if (P.R <= 2) {
             if constexpr (OPT != K_AF1) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 2, 2, FUSED>(P, gptrs, st);
-            return launch<OPT, GBF, OUT, 4, OPT == K_AF1 ? WS_TUNE_UAF2 : WS_TUNE_U4, 2, 2, FUSED>(P, gptrs, st);
+            return launch<OPT, GBF, OUT, 4, OPT == K_AF1 ? kUAf2 : 1, 2, 2, FUSED>(P, gptrs, st);
         }
         if (P.R <= 4) {
-            if constexpr (GBF && OPT != K_AF1) if (wide_ok) return launch<OPT, GBF, OUT, 8, WS_TUNE_U8, 4, 4, FUSED>(P, gptrs, st);
-            return launch<OPT, GBF, OUT, 4, OPT == K_AF1 ? WS_TUNE_UAF4 : WS_TUNE_U4, 4, 4, FUSED>(P, gptrs, st);
+            if constexpr (GBF && OPT != K_AF1) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 4, 4, FUSED>(P, gptrs, st);
+            return launch<OPT, GBF, OUT, 4, OPT == K_AF1 ? kUAf4 : 1, 4, 4, FUSED>(P, gptrs, st);
         }
         if (P.R <= 8) {
             if constexpr (GBF && OPT != K_AF1) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 8, 8, FUSED>(P, gptrs, st);
-            return launch<OPT, GBF, OUT, 4, OPT == K_AF1 ? WS_TUNE_UAF8 : WS_TUNE_U4, 8, 8, FUSED>(P, gptrs, st);
+            return launch<OPT, GBF, OUT, 4, OPT == K_AF1 ? kUAf8 : 1, 8, 8, FUSED>(P, gptrs, st);
         }
         if (P.R <= 32) {
             if constexpr (GBF && OPT != K_AF1) if (wide_ok) return launch<OPT, GBF, OUT, 8, 1, 8, 32, FUSED>(P, gptrs, st);
-            return launch<OPT, GBF, OUT, 4, WS_TUNE_U4, 8, 32, FUSED>(P, gptrs, st);
+            return launch<OPT, GBF, OUT, 4, 1, 8, 32, FUSED>(P, gptrs, st);
         }
         // many replicas make small shards and few CTAs: more loads in flight per thread
-        if (P.R <= 1024) return launch<OPT, GBF, OUT, 4, 1, WS_TUNE_RBL, 1024, FUSED>(P, gptrs, st);
+        if (P.R <= 1024) return launch<OPT, GBF, OUT, 4, 1, kTreeBlockLarge, 1024, FUSED>(P, gptrs, st);
         return WS_ERR_TOO_LARGE;
     }
 }
@@ -1201,6 +1150,7 @@ ws_status check_ws(const ws_plan* p, void* workspace, size_t bytes, ws_opt opt =
 
 extern "C" ws_status ws_lamb_partial(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_state* state,
                                      const ws_hyper* hyper, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!hyper || hyper->opt != WS_LAMB) return WS_ERR_INVALID_ARG;
     UpdParams P;
     int ok;
     bool gbf;
@@ -1226,6 +1176,7 @@ extern "C" ws_status ws_lamb_finalize(const ws_plan* plan, void* workspace, size
 
 extern "C" ws_status ws_lamb_apply(const ws_plan* plan, int32_t r, const ws_state* state, const ws_hyper* hyper,
                                    const ws_out* out, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!hyper || hyper->opt != WS_LAMB) return WS_ERR_INVALID_ARG;
     UpdParams P;
     int ok;
     bool gbf;
@@ -1285,6 +1236,19 @@ namespace {
 ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_tensor_table* gtab,
                     const ws_state* state, const ws_hyper* hyper, const ws_out* out, const ws_tensor_table* wtab,
                     void* workspace, size_t workspace_bytes, cudaStream_t st);
+
+// The argument checks of the apply phase (state pointers, `out` dtype and alignment), with no launch.
+ws_status check_phase2_args(const ws_plan* plan, const ws_state* state, const ws_hyper* hyper, const ws_out* out,
+                            int phase) {
+    UpdParams P;
+    int ok;
+    bool gbf;
+    return prepare(plan, -1, nullptr, state, hyper, out, phase, P, ok, gbf);
+}
+}
+
+ws_status ws_lamb_check_apply_args(const ws_plan* plan, const ws_state* state, const ws_hyper* hyper, const ws_out* out) {
+    return check_phase2_args(plan, state, hyper, out, K_LAMB2);
 }
 
 extern "C" ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_state* state,
@@ -1295,8 +1259,11 @@ extern "C" ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_gr
         return af_update(plan, r, grads, nullptr, state, hyper, out, nullptr, workspace, workspace_bytes, (cudaStream_t)stream);
     if (hyper->opt == WS_LAMB) {
         if (r != -1) return WS_ERR_INVALID_ARG;
-        ws_status s = ws_lamb_partial(plan, -1, grads, state, hyper, workspace, workspace_bytes, stream);
+        // every phase's arguments are checked before the first launch: an error must not leave the
+        // moments advanced and the weights not
+        ws_status s = check_phase2_args(plan, state, hyper, out, K_LAMB2);
         if (s != WS_OK) return s;
+        if ((s = ws_lamb_partial(plan, -1, grads, state, hyper, workspace, workspace_bytes, stream)) != WS_OK) return s;
         if ((s = ws_lamb_finalize(plan, workspace, workspace_bytes, stream)) != WS_OK) return s;
         return ws_lamb_apply(plan, -1, state, hyper, out, workspace, workspace_bytes, stream);
     }
@@ -1305,8 +1272,9 @@ extern "C" ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_gr
         // keeps the sum in the workspace and leaves partial sums of ||w||^2 and ||g||^2; the finalize
         // step forms each tensor's local rate; phase 2 applies the momentum step.
         if (r != -1) return WS_ERR_INVALID_ARG;
-        ws_status s = ws_lars_partial(plan, -1, grads, state, hyper, workspace, workspace_bytes, stream);
+        ws_status s = check_phase2_args(plan, state, hyper, out, K_LARS2);
         if (s != WS_OK) return s;
+        if ((s = ws_lars_partial(plan, -1, grads, state, hyper, workspace, workspace_bytes, stream)) != WS_OK) return s;
         if ((s = ws_lars_finalize(plan, hyper, workspace, workspace_bytes, stream)) != WS_OK) return s;
         return ws_lars_apply(plan, -1, state, hyper, out, workspace, workspace_bytes, stream);
     }
@@ -1412,6 +1380,8 @@ ws_status af_stage(const ws_plan* plan, int stage, int32_t r, const ws_grads* gr
         return WS_ERR_INVALID_ARG;
     ws_status s = check_ws(plan, workspace, workspace_bytes, WS_ADAFACTOR);
     if (s != WS_OK) return s;
+    // pass 2 reads the stored gradient sum (256 bytes into the workspace and onwards) with 256-bit loads
+    if (!aligned32(workspace)) return WS_ERR_ALIGNMENT;
     const WsLambWs L = ws_lamb_layout(plan, workspace);
     const bool fused = gtab != nullptr;
     UpdParams P;
@@ -1454,7 +1424,7 @@ ws_status af_stage(const ws_plan* plan, int stage, int32_t r, const ws_grads* gr
             int dev = 0, sms = 148;
             cudaGetDevice(&dev);
             cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-            const long long cap = (long long)sms * WS_TUNE_AF2_CTAS;
+            const long long cap = (long long)sms * kAf2Ctas;
             af_sumsq_kernel<<<(unsigned)(P.nitems < cap ? P.nitems : cap), kBlock, 0, st>>>(P);
             return ws_check_launch("adafactor(pass 2)");
         }

@@ -218,6 +218,17 @@ def test_argument_errors():
     with pytest.raises(B.WsError) as e:
         B.ws_shard_update(plan, -1, pg, pw, None, f0, ok, None, small)
     assert e.value.status == 4
+    # a workspace that is 16- but not 32-byte aligned: the second pass reads the stored gradient sum with
+    # 256-bit loads, so the call is refused on the host and nothing is launched
+    big = torch.zeros(plan.workspace_bytes("adafactor") + 64, dtype=torch.uint8, device=DEV)
+    shifted = big[16:16 + plan.workspace_bytes("adafactor")]
+    assert shifted.data_ptr() % 32 == 16
+    w_before = pw.clone()
+    with pytest.raises(B.WsError) as e:
+        B.ws_shard_update(plan, -1, pg, pw, None, f0, ok, None, shifted)
+    assert e.value.status == 2
+    torch.cuda.synchronize()
+    assert torch.equal(pw, w_before) and float(big.sum()) == 0.0
     lay = plan.factored_layout()
     rows, cols, foff, tot = O.factor_shapes(SHAPES[:4])
     assert [tuple(x) for x in lay] == list(zip(foff.tolist(), rows.tolist(), cols.tolist())) and plan.factored_elems == tot

@@ -344,6 +344,42 @@ def test_argument_errors_are_status_codes():
     assert float(buf.abs().sum()) == 0.0                                     # nothing was launched
 
 
+@pytest.mark.parametrize("opt", ["lamb", "lars"])
+def test_bad_output_argument_leaves_the_state_untouched(opt):
+    # the norm-based optimizers run three launches; a bad `out` (found by the checks of the last one)
+    # must be refused before the first launch, or a retry would advance the moments twice
+    import ctypes as C
+    R = 4
+    wl, w, m, v, g = _model(SHAPES[:6], R, seed=9)
+    plan = B.Plan(SHAPES[:6], R, 32)
+    pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+    before = [pw.clone(), pm.clone(), pv.clone()]
+    ws = torch.zeros(plan.workspace_bytes(opt), dtype=torch.uint8, device=DEV)
+    h = _lars_hyper() if opt == "lars" else _hyper("lamb")
+    hy = B.make_hyper(opt, h)
+    gathered = torch.zeros(plan.G + 8, dtype=torch.bfloat16, device=DEV)
+    ptrs = (C.c_void_p * R)(*[b.data_ptr() for b in pg])
+    gr = B.ws_grads(C.cast(ptrs, C.POINTER(C.c_void_p)), R, 0, 0)
+    st = B.ws_state(pw.data_ptr(), pm.data_ptr(), pv.data_ptr() if opt == "lamb" else None)
+    for out, status in ((B.ws_out(gathered.data_ptr() + 2, B.WS_BF16), 2), (B.ws_out(gathered.data_ptr(), 9), 3)):
+        rc = B.lib().ws_shard_update(plan.handle, -1, C.byref(gr), C.byref(st), C.byref(hy), C.byref(out),
+                                     ws.data_ptr(), ws.numel(), None)
+        assert rc == status
+        if opt == "lamb":
+            rc = B.lib().ws_lamb_update_static_scratch(plan.handle, C.byref(gr), C.byref(st), C.byref(hy), C.byref(out), None)
+            assert rc == status
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, b) for a, b in zip((pw, pm, pv), before))
+    if opt == "lamb":      # the shard-by-shard LAMB calls refuse another optimizer's hyper-parameters
+        ha = B.make_hyper("adam", _hyper("adam"))
+        with pytest.raises(B.WsError) as e:
+            B.ws_lamb_partial(plan, 0, pg, pw[:plan.S], pm[:plan.S], pv[:plan.S], ha, ws)
+        assert e.value.status == 1
+        with pytest.raises(B.WsError) as e:
+            B.ws_lamb_apply(plan, 0, pw[:plan.S], pm[:plan.S], pv[:plan.S], ha, ws)
+        assert e.value.status == 1
+
+
 # ------------------------------------------------- fused formatting path ---
 def _views_with_guards(numels, dtype, fill, misalign):
     """One buffer per tensor with 64-element guards; `misalign` shifts the view by 16 bytes so

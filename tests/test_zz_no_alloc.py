@@ -15,8 +15,10 @@ import ctypes as C
 import pytest
 import torch
 
+from oracle import ws_oracle as O
 from paper_2004_13336_b200 import binding as B
 from paper_2004_13336_b200 import workloads as W
+from tests._util import TOL_BF16, TOL_LAMB, bf16_to_f64, err, to_np
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -49,11 +51,16 @@ def test_static_scratch_lamb_equals_workspace_lamb_on_two_steps(R, gdtype):
     wl, plan, (w, m, v) = _setup(R, seed=21, gdtype=gdtype)
     assert plan.workspace_bytes("lamb") <= B.lib().ws_static_scratch_bytes()
     ref = [w.clone(), m.clone(), v.clone()]
+    # ... and, directly, against the CPU oracle's sharded route on the same packed buffers
+    oplan = O.Plan(wl.numels, R, 32)
+    ow, om, ov = to_np(w), to_np(m), to_np(v)
     ws = torch.zeros(plan.workspace_bytes("lamb"), dtype=torch.uint8, device=DEV)
     for step in (1, 2):
-        hy = B.make_hyper("lamb", dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-6, weight_decay=0.01,
-                                       momentum=0.0, grad_scale=1.0, step=step))
+        hd = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-6, weight_decay=0.01, momentum=0.0, grad_scale=1.0,
+                  step=step)
+        hy = B.make_hyper("lamb", hd)
         pg = _grads(wl, plan, seed=100 + step)          # fresh gradients every step
+        og, _, _ = O.sharded_update(O.make_hyper("lamb", hd), oplan, [to_np(b) for b in pg], ow, om, ov, O.BF16)
         g_ref = torch.zeros(plan.G, dtype=torch.bfloat16, device=DEV)
         g_new = torch.zeros_like(g_ref)
         B.ws_shard_update(plan, -1, pg, ref[0], ref[1], ref[2], hy, g_ref, ws)
@@ -62,6 +69,11 @@ def test_static_scratch_lamb_equals_workspace_lamb_on_two_steps(R, gdtype):
         assert torch.equal(w, ref[0]) and torch.equal(m, ref[1]) and torch.equal(v, ref[2]), f"step {step}"
         assert torch.equal(g_new, g_ref), f"step {step}"
         assert bool(torch.isfinite(w).all())
+        for name, got, exp in (("w", w, ow), ("m", m, om), ("v", v, ov)):
+            for t, (a, b) in enumerate(zip(O.unpack(oplan, to_np(got)), O.unpack(oplan, exp))):
+                assert err(a, b) <= TOL_LAMB, f"step {step} {name}[{t}]"
+        for a, b in zip(O.unpack(oplan, to_np(g_new)), O.unpack(oplan, og)):
+            assert err(bf16_to_f64(a), bf16_to_f64(b)) <= TOL_BF16, f"step {step} gathered"
 
 
 def test_static_scratch_rejects_plans_beyond_its_size():
