@@ -2,15 +2,25 @@
 """Benchmark of the sharded weight update (one JSON line on stdout).
 
 A step is one pass of the whole hot path over one model-shaped set of synthetic
-tensors: pack each of the R replicas' gradient lists into the shard-major
-layout, run the fused reduce + optimizer update for all R shards, unpack the
-updated weights back to the tensor list.  `value` is updated (valid)
-parameters per second with everything resident in HBM; `e2e` is the same step
-through the host-buffer entry point with host<->device copies inside the timed
-region; `roofline` is the dominant kernel against the measured HBM copy
-bandwidth; `cpu_baseline` is the CPU oracle timed on this machine's host cores.
+tensors: the R replicas' gradients are reduced shard by shard, the optimizer
+updates every 1/R slice of weights and slots, and the updated weights arrive in
+the weight tensors.  `value` is updated (valid) parameters per second with
+everything resident in HBM; `e2e` is the same step through the host-buffer
+entry point with host<->device copies inside the timed region; `roofline` is
+the dominant kernel's algorithmic bytes over its measured time against the
+measured HBM copy bandwidth; `cpu_baseline` is the CPU oracle timed on this
+box's host cores.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Without --workload the line is the largest single-GPU workload (decoder_1p5b:
+1.56 G parameters, bf16 gradients, R = 4) and carries, under `configs`, one full
+record for each of the other named workloads, under `transformer_r_sweep` the
+Transformer set at R = 1 ... 1024 and alignments 8 and 32, and under
+`next_workloads` the LARS, Adafactor and concatenated-layout runs.
+
+Whatever K is, the timed region lasts at least half a second: it covers
+K x `inner_repeats` back-to-back steps and `ms_per_step` is their mean.
 
 With N > 1 (launched by torch.distributed.run) every rank runs the same
 workload on its own independently seeded tensor set: the update has no
@@ -20,6 +30,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import subprocess
 import sys
@@ -33,29 +44,34 @@ if ROOT not in sys.path:
 METRIC = "updated_params_per_sec"
 UNIT = "params/s"
 FALLBACK_HBM_GBS = 6650.0
+HEADLINE = "decoder_1p5b"
+MIN_TIMED_S = 0.5
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu
-# captures summarised under profiles/, keyed by (workload, kernel); None = not captured.
-NCU_TRAFFIC_BYTES = {
-    ("resnet50", "fused"): 1.2987e9,        # profiles/fused_update_kernel_resnet50_sgdm_R8.md
-    ("decoder_1p5b", "fused"): 52.55e9,     # profiles/fused_update_kernel_bf16_transformer_R4.md, scaled by parameter count
+# DRAM bytes per valid parameter (dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's
+# launches ÷ parameters) from the ncu captures summarised under profiles/, taken on a clipped copy of
+# the workload (a few GB on the device) and scaled here by the parameter count: the kernels' traffic
+# is proportional to the elements they process.  Keyed by (workload, R, path).
+NCU_DRAM_BYTES_PER_PARAM = {
 }
 
 
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="resnet50",
-                    choices=["tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b", "resnet50_lars",
-                             "transformer_adafactor"])
+    ap.add_argument("--workload", default="all",
+                    choices=["all", "tiny", "resnet50", "transformer", "bert_large", "decoder_1p5b", "resnet50_lars",
+                             "transformer_adafactor"],
+                    help="all (default): headline decoder_1p5b plus one record per other workload and the sweeps")
     ap.add_argument("--R", type=int, default=0, help="override the workload's replica count")
     ap.add_argument("--opt", default="", choices=["", "sgdm", "adam", "lamb", "lars", "adafactor"],
                     help="override the workload's optimizer (profiling of small cases)")
     ap.add_argument("--grad-dtype", default="", choices=["", "f32", "bf16"], help="override the gradient dtype")
     ap.add_argument("--out-dtype", default="", choices=["", "f32", "bf16"], help="override the emitted weight dtype")
+    ap.add_argument("--clip", type=int, default=0,
+                    help="clip every tensor dimension to this size (a small copy of the workload for profiler captures)")
     ap.add_argument("--shards", type=int, default=0,
                     help="shard count of the plan when it differs from the replica count (partial sharding)")
     ap.add_argument("--layout", default="per_tensor", choices=["per_tensor", "concat"],
@@ -65,36 +81,45 @@ def parse_args():
     ap.add_argument("--path", default="both", choices=["both", "fused", "unfused"],
                     help="fused: one kernel reads the gradient tensors and writes the weight tensors; "
                          "unfused: pack, update, unpack as separate kernels; both: time both, headline = fused")
-    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--min-timed-s", type=float, default=MIN_TIMED_S,
+                    help="shortest timed region; steps are repeated back to back to reach it")
     ap.add_argument("--route", default="replicas", choices=["replicas", "nccl", "peer"],
                     help="replicas (default): every rank updates its own independent tensor set, no collective; "
                          "nccl: ONE model over the ranks, NCCL reduce-scatter / all-gather around the single-shard "
                          "kernels; peer: ONE model, one kernel per rank over symmetric-memory tensors")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-large", action="store_true",
-                    help="skip the short fused-route runs of the large workloads that are appended to the line")
+    ap.add_argument("--no-side-rows", action="store_true",
+                    help="with --workload all: only the headline record, none of the other workloads or sweeps")
     return ap.parse_args()
 
 
-def get_workload(args):
+def get_workload(name, R=0, opt="", grad_dtype="", out_dtype="", clip=0):
     from paper_2004_13336_b200 import workloads as W
-    wl = W.WORKLOADS[args.workload]()
-    if args.R:
-        wl.R = args.R
-    if args.opt or args.grad_dtype or args.out_dtype:
+    wl = W.WORKLOADS[name]()
+    if R:
+        wl.R = R
+    if opt or grad_dtype or out_dtype:
         import torch
         dt = {"f32": torch.float32, "bf16": torch.bfloat16}
-        if args.opt and args.opt != wl.opt:
-            wl.opt = args.opt
+        if opt and opt != wl.opt:
+            wl.opt = opt
             wl.hyper = dict(W.WORKLOADS[{"sgdm": "resnet50", "adam": "transformer", "lamb": "bert_large",
-                                         "lars": "resnet50_lars", "adafactor": "transformer_adafactor"}[args.opt]]().hyper)
-        if args.grad_dtype:
-            wl.grad_dtype = dt[args.grad_dtype]
-        if args.out_dtype:
-            wl.out_dtype = dt[args.out_dtype]
+                                         "lars": "resnet50_lars", "adafactor": "transformer_adafactor"}[opt]]().hyper)
+        if grad_dtype:
+            wl.grad_dtype = dt[grad_dtype]
+        if out_dtype:
+            wl.out_dtype = dt[out_dtype]
         wl.name += "*"          # not one of the named workloads any more
+    if clip:
+        wl = W.scaled_down(wl, clip)
     return wl
+
+
+def workload_from_args(args):
+    name = HEADLINE if args.workload == "all" else args.workload
+    return get_workload(name, args.R, args.opt, args.grad_dtype, args.out_dtype, args.clip)
 
 
 def measured_peak():
@@ -107,23 +132,28 @@ def measured_peak():
 
 
 def bytes_per_param(wl):
-    """Algorithmic bytes per valid parameter of the fused update (read R gradients, the weight
-    and its slots once; write weight and slots once; plus the gathered copy when it is a
-    separate bf16 buffer) and of one pack / unpack launch."""
+    """Bytes per valid parameter.
+
+    `algorithmic`: what the method must move, every operand once (Section 2.2: read the gradient
+    copies, the weight and the auxiliaries; write the weight and the auxiliaries): SGD-momentum
+    g R + 16, Adam g R + 24 (+2 for a bf16 copy next to the fp32 master), LAMB g R + 24 (its phase 2
+    re-reads are not algorithmic), LARS g R + 16, Adafactor g R + 8, with g = gradient element bytes.
+    `update` / `fused`: what the separate-kernel update and the fused-formatting update move by design.
+    `pack` / `unpack`: one formatting launch."""
     gb = 2 if str(wl.grad_dtype).endswith("bfloat16") else 4
     slots = {"sgdm": 1, "lars": 1, "adafactor": 0}.get(wl.opt, 2)
-    upd = gb * wl.R + 4 * (1 + slots) * 2
+    out_b = 2 if str(wl.out_dtype).endswith("bfloat16") else 0
+    alg = gb * wl.R + 4 * (1 + slots) * 2 + out_b
+    upd = alg
     if wl.opt == "lamb":
-        upd += 12          # plain two-pass: phase 2 reads w, m', v' again and rewrites w
+        upd += 12          # two passes: phase 2 reads w, m', v' again
     if wl.opt == "lars":
         upd += 12          # phase 1 reads w and stores the summed gradient; phase 2 reads it back
     if wl.opt == "adafactor":
         upd += 16          # pass 1 stores the summed gradient, passes 2 and 3 read it back, pass 3 reads w again
-    out_b = 2 if str(wl.out_dtype).endswith("bfloat16") else 0
-    # fused formatting: same reads and state writes, plus the weight tensors written directly
-    fused = upd + (2 if out_b else 4)
-    upd += out_b
-    return {"update": upd, "fused": fused, "pack": 2 * gb, "unpack": 2 * (2 if out_b else 4)}
+    # fused formatting: same reads and state writes; an fp32 weight list is written next to the fp32 shard state
+    fused = upd + (0 if out_b else 4)
+    return {"algorithmic": alg, "update": upd, "fused": fused, "pack": 2 * gb, "unpack": 2 * (2 if out_b else 4)}
 
 
 # ----------------------------------------------------------------------------
@@ -165,7 +195,7 @@ class ClockSampler:
     def summary(self, t0, t1):
         def parse(window):
             sm, mx, reasons = [], [], set()
-            for ts, line in self.samples:
+            for ts, line in list(self.samples):
                 if not (window[0] <= ts <= window[1]):
                     continue
                 p = [x.strip() for x in line.split(",")]
@@ -183,8 +213,8 @@ class ClockSampler:
         sm, mx, reasons = parse((t0, t1))
         window = "timed"
         if len(sm) < 3 and self.samples:
-            sm, mx, reasons = parse((self.samples[0][0], t1 + 1.0))
-            window = "warmup+timed"
+            sm, mx, reasons = parse((t0 - 1.0, t1 + 1.0))
+            window = "timed +-1 s"
         if not sm:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": window}
         sm.sort()
@@ -196,11 +226,12 @@ class ClockSampler:
 # CPU oracle legs
 # ----------------------------------------------------------------------------
 def oracle_step_inputs(wl, stride, align):
-    """Host copies of every `stride`-th tensor of the workload (the bounded sample)."""
+    """Host copies of every `stride`-th tensor of the workload (the bounded sample), starting in the
+    middle of the first stride so that the sample is not dominated by the embedding at index 0."""
     import torch
     from oracle import ws_oracle as O
     from paper_2004_13336_b200 import workloads as W
-    idx = list(range(0, wl.T, stride))
+    idx = list(range(stride // 2 if stride < wl.T else 0, wl.T, stride))
     sub = W.Workload(**{**wl.__dict__})
     sub.shapes = [wl.shapes[i] for i in idx]
     w, m, v = W.make_state(sub, "cpu")
@@ -235,19 +266,33 @@ def oracle_one_step(sub, plan, g, pw, pm, pv):
     return time.perf_counter() - t0
 
 
-def cpu_baseline(wl, align, target_params=26_000_000, min_seconds=10.0, max_steps=20):
+def cpu_baseline(wl, align, target_params=0, min_seconds=10.0, max_steps=20):
+    """The oracle's sharded route, as it stands, on this machine's host cores: once on one thread and once
+    on all of them (the loops over independent (shard, tensor) pairs are split; results do not depend on
+    the thread count).  `value` is the all-core rate."""
     from oracle import ws_oracle as O
+    target_params = target_params or int(2e8 / (wl.R + 3))      # bounds the sample's host memory and set-up time
     stride = max(1, round(wl.N / target_params))
     sub, plan, g, pw, pm, pv = oracle_step_inputs(wl, stride, align)
-    dt, steps = 0.0, 0
-    while steps < max_steps and (steps == 0 or dt < min_seconds):
-        dt += oracle_one_step(sub, plan, g, pw, pm, pv)
-        steps += 1
-    return {"value": sub.N * steps / dt, "unit": UNIT, "cores": 1, "kind": "oracle",
-            "sample": f"{steps} step(s) (pack {sub.R} gradient sets, sharded update, unpack) over every "
-                      f"{stride}-th tensor of {wl.name}: {sub.T} tensors, {sub.N} params, {dt:.2f} s; "
-                      f"the sharded route of the oracle runs on one thread",
-            "host_cores": len(os.sched_getaffinity(0))}
+    host_cores = len(os.sched_getaffinity(0))
+    runs = {}
+    for label, nthreads, secs in (("single_thread", 1, min_seconds * 0.6), ("all_cores", host_cores, min_seconds * 0.4)):
+        prev = O.set_num_threads(nthreads)
+        try:
+            used = O.num_threads()
+            oracle_one_step(sub, plan, g, pw, pm, pv)        # first touch
+            dt, steps = 0.0, 0
+            while steps < max_steps and (steps == 0 or dt < secs):
+                dt += oracle_one_step(sub, plan, g, pw, pm, pv)
+                steps += 1
+        finally:
+            O.set_num_threads(prev)
+        runs[label] = {"value": sub.N * steps / dt, "unit": UNIT, "cores": used, "steps": steps, "seconds": round(dt, 2)}
+    return {"value": runs["all_cores"]["value"], "unit": UNIT, "cores": runs["all_cores"]["cores"], "kind": "oracle",
+            "sample": f"whole path (pack {sub.R} gradient sets, sharded update, unpack) over every {stride}-th tensor of "
+                      f"{wl.name}: {sub.T} tensors, {sub.N} params, {runs['all_cores']['steps']} step(s) in "
+                      f"{runs['all_cores']['seconds']} s on {runs['all_cores']['cores']} threads",
+            "single_thread": runs["single_thread"], "host_cores": host_cores}
 
 
 def run_reference(args):
@@ -257,37 +302,37 @@ def run_reference(args):
         return
     from oracle import ws_oracle as O
     O.build()
-    wl = get_workload(args)
-    stride = max(1, round(wl.N / 1_500_000))
+    wl = workload_from_args(args)
+    stride = max(1, round(wl.N / 6_000_000))
     sub, plan, g, pw, pm, pv = oracle_step_inputs(wl, stride, args.align)
-    for _ in range(args.warmup):
+    cores = O.num_threads()
+    for _ in range(max(1, args.warmup)):
         oracle_one_step(sub, plan, g, pw, pm, pv)
     t = 0.0
     for _ in range(args.steps):
         t += oracle_one_step(sub, plan, g, pw, pm, pv)
     val = sub.N * args.steps / t
     sample = (f"each step = whole path over every {stride}-th tensor of {wl.name} "
-              f"({sub.T} tensors, {sub.N} params)")
+              f"({sub.T} tensors, {sub.N} params) on {cores} threads")
     line = {
         "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
-        "data": "synthetic", "config": config_of(wl, args, extra={"sample": sample}),
-        "cpu_baseline": {"value": val, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "data": "synthetic", "config": config_of(wl, args.align, args.layout, wl.R, extra={"sample": sample}),
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
 
 
-def config_of(wl, args, extra=None, path="unfused"):
+def config_of(wl, align, layout, shards, extra=None, path="fused"):
     steps = {"unfused": "pack R gradient sets + fused reduce/update of all shards + unpack weights (separate kernels)",
              "fused": "one kernel: gradients read from the R replicas' tensor lists (formatting fused in), reduce, "
                       "update of all shards, weights written to the weight tensors"}
     c = {"workload": f"{wl.name}: {wl.T} tensors, {wl.N} params, R={wl.R} replicas, {wl.opt}, "
                      f"grads {str(wl.grad_dtype).split('.')[-1]}, gathered {str(wl.out_dtype).split('.')[-1]}",
-         "R": wl.R, "shards": getattr(args, "shards", 0) or wl.R, "optimizer": wl.opt, "align_elems": args.align,
-         "layout": getattr(args, "layout", "per_tensor"),
+         "R": wl.R, "shards": shards or wl.R, "optimizer": wl.opt, "align_elems": align, "layout": layout,
          "step": steps[path],
          "l2": "inputs exceed L2 (no flush)" if wl.N * 4 * (wl.R + 3) > 256e6 else "flush between steps"}
     if extra:
@@ -319,6 +364,14 @@ def job_value(n_params_per_rank: int, world: int, ms_per_step: float) -> float:
     return world * n_params_per_rank / (ms_per_step * 1e-3)
 
 
+def inner_repeats(est_ms_per_step: float, steps: int, min_timed_s: float) -> int:
+    """Back-to-back repetitions of every counted step so that the timed region lasts at least
+    `min_timed_s` whatever `steps` is."""
+    if est_ms_per_step <= 0:
+        return 1
+    return max(1, min(20000, math.ceil(min_timed_s * 1e3 / (steps * est_ms_per_step))))
+
+
 # ----------------------------------------------------------------------------
 # GPU arm
 # ----------------------------------------------------------------------------
@@ -348,7 +401,7 @@ def run_real_replicas(args):
         ws_build.build()
     dist.barrier()
     from paper_2004_13336_b200.collective import PeerShardedUpdate, ShardedUpdate
-    wl = get_workload(args)
+    wl = workload_from_args(args)
     wl.R = world
     w, m, v = W.make_state(wl, dev)                       # same seed on every rank: one model
     g = W.make_grads_one(wl, rank, dev)                   # this replica's own gradients
@@ -396,56 +449,82 @@ def run_real_replicas(args):
     dist.destroy_process_group()
 
 
-def run_ours(args):
+class Ctx:
+    """What every measurement of a process shares: ranks, device, the clock sampler."""
+
+    def __init__(self, args):
+        import torch
+        import torch.distributed as dist
+        self.args = args
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local = int(os.environ.get("LOCAL_RANK", "0"))
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device: the sharded update has no CPU fallback")
+        torch.cuda.set_device(self.local)
+        self.dev = torch.device("cuda", self.local)
+        if self.world > 1:
+            dist.init_process_group("nccl", device_id=self.dev)
+        from paper_2004_13336_b200 import build as ws_build
+        if self.rank == 0 and not ws_build.up_to_date():
+            ws_build.build()                      # one rank builds; the others wait at the barrier
+        if self.world > 1:
+            dist.barrier()
+        from paper_2004_13336_b200 import binding as B
+        B.lib()
+        self.sampler = ClockSampler(self.local)
+        if self.rank == 0:
+            self.sampler.start()
+
+    def barrier(self):
+        import torch
+        import torch.distributed as dist
+        if self.world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def close(self):
+        import torch.distributed as dist
+        self.sampler.stop()
+        if self.world > 1:
+            dist.destroy_process_group()
+
+
+def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both", e2e=True, cpu=True,
+            steps=20, warmup=5, e2e_steps=3, cpu_seconds=10.0):
+    """One workload on this rank's GPU: the fused route (and the separate-kernel route), the roofline of
+    the dominant kernel, the end-to-end step from host buffers and the CPU oracle beside it.  Returns the
+    record (rank 0) or None."""
     import torch
-    import torch.distributed as dist
-    if args.route != "replicas":
-        return run_real_replicas(args)
-
     from paper_2004_13336_b200 import binding as B
-    from paper_2004_13336_b200 import build as ws_build
     from paper_2004_13336_b200 import workloads as W
-
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device: the sharded update has no CPU fallback")
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
-    if rank == 0 and not ws_build.up_to_date():
-        ws_build.build()                      # one rank builds; the others wait at the barrier
-    if world > 1:
-        dist.barrier()
-    B.lib()
-
-    wl = get_workload(args)
+    args, dev, world, rank = ctx.args, ctx.dev, ctx.world, ctx.rank
     wl.seed = rank_seed(wl.seed, rank)        # every rank owns its own tensor set
     R, T, N = wl.R, wl.T, wl.N
     # partial sharding (Section 5.2): R gradient copies, but the update is sharded only `shards` ways
-    shards = args.shards or R
-    plan = B.Plan(wl.shapes, shards, args.align, args.tile, device=dev, layout=args.layout)
+    shards = shards or R
+    plan = B.Plan(wl.shapes, shards, align, tile, device=dev, layout=layout)
     if shards != R:
-        args.no_e2e = True        # the host-buffer entry point takes one gradient arena per shard
+        e2e = False               # the host-buffer entry point takes one gradient arena per shard
     gdt, odt = wl.grad_dtype, wl.out_dtype
     gb = 2 if gdt == torch.bfloat16 else 4
     wb = 2 if odt == torch.bfloat16 else 4
     numels = wl.numels
     A_el = plan.arena_elems
     total_mem = torch.cuda.get_device_properties(dev).total_memory
-    run_unfused = args.path in ("both", "unfused")
-    run_fused = args.path in ("both", "fused")
+    run_unfused = path in ("both", "unfused")
+    run_fused = path in ("both", "fused")
     need_unfused = R * (A_el + plan.G) * gb + 3 * plan.G * 4 + plan.G * wb + A_el * wb
     if R * A_el * gb + 3 * plan.G * 4 > 0.85 * total_mem:
         # not even the R gradient lists fit on one GPU (Transformer at R = 1024 needs 863 GB)
-        return run_shard_window(args, wl, plan, dev, world, rank)
+        return run_shard_window(ctx, wl, plan, align, layout, steps, warmup)
     unfused_skipped = None
     if run_unfused and need_unfused > 0.85 * total_mem:
         unfused_skipped = f"needs {need_unfused / 1e9:.0f} GB of device memory (tensor lists plus packed gradient buffers)"
         run_unfused = False
         run_fused = True
+    if e2e and need_unfused > 0.85 * total_mem:
+        e2e = False
 
     # ---- device-resident inputs: per replica one gradient arena, viewed tensor by tensor
     w, m, v = W.make_state(wl, dev)
@@ -467,10 +546,10 @@ def run_ours(args):
         del gk
     w_arena = torch.zeros(A_el, dtype=odt, device=dev)
     w_views = B.PtrList(plan.arena_views(w_arena, numels))
-    ws = torch.empty(max(16, plan.workspace_bytes(wl.opt)), dtype=torch.uint8, device=dev)
+    ws = torch.empty(max(32, plan.workspace_bytes(wl.opt)), dtype=torch.uint8, device=dev)
     hy = B.make_hyper(wl.opt, wl.hyper)
     pg = gathered = None
-    if run_unfused:
+    if run_unfused or e2e:
         pg = B.PtrList([torch.empty(plan.G, dtype=gdt, device=dev) for _ in range(R)])
         gathered = torch.empty(plan.G, dtype=odt, device=dev) if odt != torch.float32 else None
     gtab = wtab = gtab_u = None
@@ -507,49 +586,52 @@ def run_ours(args):
         if ev:
             ev[1].record()
 
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize()
-
-    K = args.steps
-    W_ = max(3, args.warmup)
+    K = steps
+    W_ = max(3, warmup)
 
     def time_path(step, nev):
         for _ in range(W_):
             step()
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nev)] for _ in range(K)]
-        barrier()
+        # a first estimate fixes how often every counted step is repeated (same on every rank)
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(nev)]
+        ctx.barrier()
+        est = []
+        for _ in range(3):
+            step(ev)
+            torch.cuda.synchronize()
+            est.append(ev[0].elapsed_time(ev[nev - 1]))
+        inner = inner_repeats(reduce_max(min(est), dev), K, args.min_timed_s)
+        n = K * inner
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nev)] for _ in range(n)]
+        ctx.barrier()
         t0 = time.time()
-        for i in range(K):
+        for i in range(n):
             step(evs[i])
-        barrier()
+        ctx.barrier()
         t1 = time.time()
         total_ms = evs[0][0].elapsed_time(evs[-1][nev - 1])
         if flush is not None:   # leave the L2 flush out of the step time
             total_ms = sum(e[0].elapsed_time(e[nev - 1]) for e in evs)
-        phase_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / K for i in range(nev - 1)]
+        phase_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / n for i in range(nev - 1)]
         total_ms = reduce_max(total_ms, dev)
         per_step = sorted(e[0].elapsed_time(e[nev - 1]) for e in evs)      # each step's own launches
         stats = {"median": per_step[len(per_step) // 2], "min": per_step[0], "max": per_step[-1],
-                 "mean_back_to_back": total_ms / K}
-        return total_ms / K, phase_ms, (t0, t1), stats
+                 "mean_back_to_back": total_ms / n}
+        return {"ms": total_ms / n, "phase_ms": phase_ms, "window": (t0, t1), "stats": stats, "inner": inner,
+                "timed_s": total_ms * 1e-3}
 
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     res = {}
     if run_fused:       # the headline route first: a long run of the other route leaves the GPU at its power cap
         res["fused"] = time_path(step_fused, 2)
     if run_unfused:
         res["unfused"] = time_path(step_unfused, 4)
     primary = "fused" if run_fused else "unfused"
-    ms_per_step, _, window, step_stats = res[primary]
+    ms_per_step = res[primary]["ms"]
     value = job_value(N, world, ms_per_step)
 
     # ---- one replica's work: ws_shard_update for a single shard r (reads slice r of the R packed buffers)
     single = None
-    if run_unfused and wl.opt in ("sgdm", "adam") and args.layout == "per_tensor":
+    if run_unfused and wl.opt in ("sgdm", "adam") and layout == "per_tensor" and shards == R:
         r_mid, S_ = R // 2, plan.S
         sl = slice(r_mid * S_, (r_mid + 1) * S_)
         valid = sum(min(max(sg.numel - r_mid * sg.piece, 0), sg.piece) for sg in plan.segments())
@@ -568,15 +650,12 @@ def run_ours(args):
         med = times[len(times) // 2]
         single = {"call": f"ws_shard_update(r={r_mid}) alone, one launch", "valid_params": valid,
                   "ms_median": med, "ms_min": times[0], "value": valid / (med * 1e-3), "unit": UNIT,
-                  "achieved_gbs": valid * bytes_per_param(wl)["update"] / (med * 1e-3) / 1e9}
+                  "achieved_gbs": valid * bytes_per_param(wl)["algorithmic"] / (med * 1e-3) / 1e9}
         single["frac"] = single["achieved_gbs"] / measured_peak()[0]
 
     # ---- end to end through the host-buffer entry point
-    e2e = None
-    if not args.no_e2e:
-        if pg is None:
-            pg = B.PtrList([torch.empty(plan.G, dtype=gdt, device=dev) for _ in range(R)])
-            gathered = torch.empty(plan.G, dtype=odt, device=dev) if odt != torch.float32 else None
+    e2e_rec = None
+    if e2e:
         host_g = [torch.empty(A_el, dtype=gdt).pin_memory() for _ in range(R)]
         for k in range(R):
             host_g[k].copy_(g_arena[k])
@@ -588,19 +667,18 @@ def run_ours(args):
             B.ws_step_host(plan, host_g, stage, pg, pw, pm, pv, hy, w_arena, host_w, gathered, ws)
         for _ in range(2):
             e2e_step()
-        barrier()
+        ctx.barrier()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
-        for _ in range(args.e2e_steps):
+        for _ in range(e2e_steps):
             e2e_step()
         e1.record()
-        barrier()
-        e2e_ms = e0.elapsed_time(e1)
-        e2e_ms = reduce_max(e2e_ms, dev)
-        e2e = {"value": world * N * args.e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
-               "h2d_bytes_per_step": R * A_el * gb, "d2h_bytes_per_step": A_el * wb,
-               "steps": args.e2e_steps, "ms_per_step": e2e_ms / args.e2e_steps,
-               "api": "ws_step_host (pinned host arenas)"}
+        ctx.barrier()
+        e2e_ms = reduce_max(e0.elapsed_time(e1), dev)
+        e2e_rec = {"value": world * N * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
+                   "h2d_bytes_per_step": R * A_el * gb, "d2h_bytes_per_step": A_el * wb,
+                   "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps,
+                   "api": "ws_step_host (pinned host arenas)"}
         # The fused entry point also takes pinned host tensors as they are: the kernel then pulls the
         # gradients over PCIe itself and writes the weights back the same way (no staging copies).
         try:
@@ -609,27 +687,23 @@ def run_ours(args):
 
             def zc_step():
                 B.ws_fused_update(plan, -1, zg, pw, pm, pv, hy, zw, ws)
-            for _ in range(2):
-                zc_step()
-            barrier()
+            zc_step()
+            ctx.barrier()
             e0.record()
-            for _ in range(args.e2e_steps):
+            for _ in range(e2e_steps):
                 zc_step()
             e1.record()
-            barrier()
+            ctx.barrier()
             zc_ms = reduce_max(e0.elapsed_time(e1), dev)
-            e2e["zero_copy"] = {"value": world * N * args.e2e_steps / (zc_ms * 1e-3), "unit": UNIT,
-                                "ms_per_step": zc_ms / args.e2e_steps,
-                                "api": "ws_fused_update on pinned host tensors (kernel reads and writes host memory)"}
+            e2e_rec["zero_copy"] = {"value": world * N * e2e_steps / (zc_ms * 1e-3), "unit": UNIT,
+                                    "ms_per_step": zc_ms / e2e_steps,
+                                    "api": "ws_fused_update on pinned host tensors (kernel reads and writes host memory)"}
             del zg, zw
         except Exception as ex:
-            e2e["zero_copy"] = {"error": str(ex)[:200]}
+            e2e_rec["zero_copy"] = {"error": str(ex)[:200]}
         del host_g, host_w, stage
-    sampler.stop()
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
+        return None
 
     # ---- per-kernel rates and the roofline of the dominant kernel
     peak, peak_src = measured_peak()
@@ -641,77 +715,87 @@ def run_ours(args):
                 if n_upd_launch == 6 else
                 "update_kernel phase 1 + lamb_finalize_kernel + update_kernel phase 2")
 
-    def kernel_rows(path):
-        ph = res[path][1]
-        if path == "fused":
+    def kernel_rows(pth):
+        ph = res[pth]["phase_ms"]
+        if pth == "fused":
             rows = [{"kernel": upd_name + " (formatting fused in)", "launches_per_step": n_upd_launch,
-                     "ms_per_step": ph[0], "bytes_per_step": N * bpp["fused"]}]
+                     "ms_per_step": ph[0], "algorithmic_bytes_per_step": N * bpp["algorithmic"],
+                     "moved_bytes_per_step": N * bpp["fused"]}]
         else:
             rows = [{"kernel": "pack_sets_kernel (gradients, all R lists)", "launches_per_step": 1,
-                     "ms_per_step": ph[0], "bytes_per_step": R * N * bpp["pack"]},
+                     "ms_per_step": ph[0], "algorithmic_bytes_per_step": R * N * bpp["pack"],
+                     "moved_bytes_per_step": R * N * bpp["pack"]},
                     {"kernel": upd_name, "launches_per_step": n_upd_launch, "ms_per_step": ph[1],
-                     "bytes_per_step": N * bpp["update"]},
+                     "algorithmic_bytes_per_step": N * bpp["algorithmic"], "moved_bytes_per_step": N * bpp["update"]},
                     {"kernel": "pack_kernel (unpack weights)", "launches_per_step": chunks,
-                     "ms_per_step": ph[2], "bytes_per_step": N * bpp["unpack"]}]
+                     "ms_per_step": ph[2], "algorithmic_bytes_per_step": N * bpp["unpack"],
+                     "moved_bytes_per_step": N * bpp["unpack"]}]
         tot = sum(r_["ms_per_step"] for r_ in rows)
         for r_ in rows:
-            r_["achieved_gbs"] = r_["bytes_per_step"] / (r_["ms_per_step"] * 1e-3) / 1e9
+            r_["achieved_gbs"] = r_["algorithmic_bytes_per_step"] / (r_["ms_per_step"] * 1e-3) / 1e9
             r_["frac"] = r_["achieved_gbs"] / peak
+            r_["moved_gbs"] = r_["moved_bytes_per_step"] / (r_["ms_per_step"] * 1e-3) / 1e9
             r_["share"] = r_["ms_per_step"] / tot
         return rows
 
     kernels = kernel_rows(primary)
     dom = max(kernels, key=lambda z: z["ms_per_step"])
-    one_launch = dom["launches_per_step"] if "phase 1" not in dom["kernel"] else 1
+    # the multi-launch optimizers' update is reported as one unit (its launches depend on one another)
+    traffic_pp = NCU_DRAM_BYTES_PER_PARAM.get((wl.name, wl.R, primary))
     roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["achieved_gbs"], "peak": peak,
                 "peak_source": f"{peak_src} copy bandwidth", "unit": "GB/s", "frac": dom["frac"],
-                "algorithmic_bytes_per_launch": dom["bytes_per_step"] / one_launch,
-                "avg_launch_ms": dom["ms_per_step"] / one_launch,
-                "traffic": NCU_TRAFFIC_BYTES.get((wl.name, primary)),
+                "algorithmic_bytes_per_launch": dom["algorithmic_bytes_per_step"],
+                "algorithmic_bytes_per_param": bpp["algorithmic"],
+                "moved_bytes_per_launch": dom["moved_bytes_per_step"],
+                "launch": f"one step's update = {dom['launches_per_step']} dependent launch(es), timed together",
+                "avg_launch_ms": dom["ms_per_step"],
+                "traffic": traffic_pp * N if traffic_pp else None,
                 "frac_of_nominal_8TBs": dom["achieved_gbs"] / 8000.0}
-    clocks = sampler.summary(*window)
-
-    line = {
+    if wl.opt == "lamb":
+        roofline["two_pass"] = {"bytes_per_param": bpp["algorithmic"] + 12,
+                                "achieved": dom["achieved_gbs"] * (bpp["algorithmic"] + 12) / bpp["algorithmic"],
+                                "frac": dom["frac"] * (bpp["algorithmic"] + 12) / bpp["algorithmic"]}
+    pr = res[primary]
+    rec = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": W_, "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": config_of(wl, args, path=primary), "roofline": roofline, "kernels": kernels, "clocks": clocks,
-        "gpu_launches": K * sum(kz["launches_per_step"] for kz in kernels),
-        "step_ms": step_stats,
+        "config": config_of(wl, align, layout, shards, path=primary,
+                            extra={"inner_repeats": pr["inner"], "timed_region_s": round(pr["timed_s"], 3),
+                                   "timed_steps": K * pr["inner"]}),
+        "roofline": roofline, "kernels": kernels, "clocks": ctx.sampler.summary(*pr["window"]),
+        "gpu_launches": K * pr["inner"] * sum(kz["launches_per_step"] for kz in kernels),
+        "step_ms": pr["stats"],
     }
     if "unfused" in res and primary != "unfused":
         rows = kernel_rows("unfused")
-        line["unfused_path"] = {
+        ur = res["unfused"]
+        rec["unfused_path"] = {
             "step": "ws_pack_sets (R gradient lists) + ws_shard_update(all shards) + ws_unpack as separate kernels",
-            "value": world * N / (res["unfused"][0] * 1e-3), "unit": UNIT, "ms_per_step": res["unfused"][0],
-            "kernels": rows, "gpu_launches": K * sum(kz["launches_per_step"] for kz in rows),
-            "step_ms": res["unfused"][3]}
+            "value": world * N / (ur["ms"] * 1e-3), "unit": UNIT, "ms_per_step": ur["ms"],
+            "kernels": rows, "gpu_launches": K * ur["inner"] * sum(kz["launches_per_step"] for kz in rows),
+            "step_ms": ur["stats"], "clocks": ctx.sampler.summary(*ur["window"])}
         if single is not None:
-            line["unfused_path"]["single_shard"] = single
+            rec["unfused_path"]["single_shard"] = single
     if unfused_skipped:
-        line["unfused_path"] = {"skipped": unfused_skipped}
-    if e2e is not None:
-        line["e2e"] = e2e
-    if world == 1 and not args.no_cpu_baseline:
+        rec["unfused_path"] = {"skipped": unfused_skipped}
+    if e2e_rec is not None:
+        rec["e2e"] = e2e_rec
+    if world == 1 and cpu:
         from oracle import ws_oracle as O
         O.build()
-        line["cpu_baseline"] = cpu_baseline(wl, args.align)
-    if world == 1 and not args.no_large and args.workload == "resnet50" and not (args.R or args.opt):
-        del pw, pm, pv, g_arena, g_views, w_arena, w_views, pg, gathered, gtab, wtab, gtab_u
-        torch.cuda.empty_cache()
-        line["large_workloads"] = large_workload_rows(args)
-    print(json.dumps(line))
-    if world > 1:
-        dist.destroy_process_group()
+        rec["cpu_baseline"] = cpu_baseline(wl, align, min_seconds=cpu_seconds)
+    return rec
 
 
-def run_shard_window(args, wl, plan, dev, world, rank):
+def run_shard_window(ctx, wl, plan, align, layout, steps, warmup):
     """Replica counts whose gradients cannot exist on one GPU: time ws_shard_update shard by shard
     on a window of 16 shards, each fed from R S-element slices (what a reduce-scatter receive
     buffer holds), and extrapolate the whole-model step as R x the mean shard time."""
     import numpy as np
     import torch
     from paper_2004_13336_b200 import binding as B
+    dev, world, rank = ctx.dev, ctx.world, ctx.rank
     R, N, S = wl.R, wl.N, plan.S
     rng = np.random.default_rng(wl.seed)
     window = sorted(set([0, 1, R // 2, R - 1] + [int(x) for x in rng.integers(2, R - 1, 12)]))
@@ -722,8 +806,9 @@ def run_shard_window(args, wl, plan, dev, world, rank):
     m = torch.empty(S, device=dev).normal_(0.0, wl.m_std, generator=gen)
     v = torch.empty(S, device=dev).normal_(0.0, wl.v_std, generator=gen).abs_()
     hy = B.make_hyper(wl.opt, wl.hyper)
-    K, W_ = max(1, args.steps // 50), max(3, args.warmup // 5)
+    K, W_ = max(20, steps), max(3, warmup)
     per_shard = []
+    t0 = time.time()
     for r in window:
         for _ in range(W_):
             B.ws_shard_update(plan, r, gl, w, m, v if wl.opt != "sgdm" else None, hy, None, None, slice_mode=1)
@@ -735,48 +820,105 @@ def run_shard_window(args, wl, plan, dev, world, rank):
         e1.record()
         torch.cuda.synchronize()
         per_shard.append(e0.elapsed_time(e1) / K)
+    t1 = time.time()
     mean_ms = reduce_max(float(np.mean(per_shard)), dev)
     if rank != 0:
-        return
+        return None
     peak, peak_src = measured_peak()
-    bpp = bytes_per_param(wl)["update"]
+    bpp = bytes_per_param(wl)["algorithmic"]
     gbs = (N / R) * bpp / (mean_ms * 1e-3) / 1e9
-    line = {
+    return {
         "metric": METRIC, "value": job_value(N, world, R * mean_ms), "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": W_, "ms_per_step": R * mean_ms, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": config_of(wl, args, extra={
+        "config": config_of(wl, align, layout, R, path="unfused", extra={
             "window": f"extrapolated from {len(window)} of {R} shards: whole-model step = R x mean shard time; "
                       f"each shard call reads R slices of S={S} elements (slice mode 1)",
-            "shard_ms_mean": mean_ms, "shard_ms_min": min(per_shard), "shard_ms_max": max(per_shard)}),
+            "shard_ms_mean": mean_ms, "shard_ms_min": min(per_shard), "shard_ms_max": max(per_shard),
+            "padding_pct": 100.0 * (R * S - N) / N}),
         "roofline": {"bound": "hbm", "kernel": "update_kernel (one shard)", "achieved": gbs, "peak": peak,
                      "peak_source": f"{peak_src} copy bandwidth", "unit": "GB/s", "frac": gbs / peak,
                      "algorithmic_bytes_per_launch": (N / R) * bpp, "avg_launch_ms": mean_ms, "traffic": None,
                      "frac_of_nominal_8TBs": gbs / 8000.0},
+        "clocks": ctx.sampler.summary(t0, t1),
         "gpu_launches": K * len(window), "e2e": None,
     }
-    print(json.dumps(line))
 
 
-def large_workload_rows(args):
-    """Short fused-route runs of the large model-shaped workloads (each in its own process so that its
-    memory is returned), summarised next to the headline workload."""
-    rows = []
-    for name, extra in (("transformer", ["--R", "8"]), ("bert_large", []), ("decoder_1p5b", []),
-                        ("transformer_adafactor", [])):
-        cmd = [sys.executable, os.path.abspath(__file__), "--workload", name, *extra, "--path", "fused", "--steps", "30",
-               "--warmup", "5", "--no-e2e", "--no-cpu-baseline", "--no-large", "--align", str(args.align)]
+def short_row(rec):
+    """The few figures of a sweep row."""
+    if rec is None:
+        return None
+    rf = rec["roofline"]
+    row = {"workload": rec["config"]["workload"], "R": rec["config"]["R"], "align_elems": rec["config"]["align_elems"],
+           "layout": rec["config"]["layout"], "value": rec["value"], "unit": UNIT, "ms_per_step": rec["ms_per_step"],
+           "timed_steps": rec["config"].get("timed_steps", rec["steps"]),
+           "algorithmic_bytes_per_param": rf.get("algorithmic_bytes_per_param"),
+           "achieved_gbs": rf["achieved"], "frac_of_measured_peak": rf["frac"],
+           "frac_of_nominal_8TBs": rf["frac_of_nominal_8TBs"], "clocks": rec["clocks"]}
+    for k in ("window", "padding_pct", "shard_ms_mean"):
+        if k in rec["config"]:
+            row[k] = rec["config"][k]
+    if "two_pass" in rf:
+        row["two_pass"] = rf["two_pass"]
+    return row
+
+
+def run_ours(args):
+    import gc
+    import torch
+    if args.route != "replicas":
+        return run_real_replicas(args)
+    ctx = Ctx(args)
+
+    def release():
+        gc.collect()
+        torch.cuda.empty_cache()
+
+    def guarded(fn, what):
         try:
-            r = subprocess.run(cmd, capture_output=True, text=True, timeout=600)
-            j = json.loads(r.stdout.strip().splitlines()[-1])
-            rf = j["roofline"]
-            rows.append({"workload": j["config"]["workload"], "value": j["value"], "unit": UNIT,
-                         "ms_per_step": j["ms_per_step"], "gpu_launches_per_step": j["gpu_launches"] // j["steps"],
-                         "achieved_gbs": rf["achieved"], "frac_of_measured_peak": rf["frac"],
-                         "frac_of_nominal_8TBs": rf["frac_of_nominal_8TBs"], "clocks": j["clocks"]})
+            return fn()
         except Exception as e:      # a failed side run must not lose the headline line
-            rows.append({"workload": name, "error": str(e)[:200]})
-    return rows
+            release()
+            return {"workload": what, "error": f"{type(e).__name__}: {str(e)[:200]}"}
+
+    common = dict(steps=args.steps, warmup=args.warmup, e2e_steps=args.e2e_steps)
+    head = measure(ctx, workload_from_args(args), align=args.align, layout=args.layout, shards=args.shards,
+                   tile=args.tile, path=args.path, e2e=not args.no_e2e, cpu=not args.no_cpu_baseline, **common)
+    release()
+    side = args.workload == "all" and ctx.world == 1 and not args.no_side_rows and not (args.R or args.opt or args.clip)
+    if side:
+        # one full record for each of the other named workloads
+        head["configs"] = []
+        for name in ("tiny", "resnet50", "transformer", "bert_large"):
+            head["configs"].append(guarded(lambda: measure(
+                ctx, get_workload(name), align=args.align, e2e=not args.no_e2e, cpu=not args.no_cpu_baseline,
+                cpu_seconds=4.0, **common), name))
+            release()
+        # Transformer set over the replica counts of the tiny-shard study (Section 5.2), alignments 8 and 32
+        sweep = []
+        for R, A in ((1, 32), (2, 32), (8, 8), (32, 32), (128, 32), (128, 8), (1024, 32), (1024, 8)):
+            sweep.append(guarded(lambda: short_row(measure(
+                ctx, get_workload("transformer", R=R), align=A, path="fused", e2e=False, cpu=False, **common)),
+                f"transformer R={R} A={A}"))
+            release()
+        for r_ in head["configs"]:          # the R = 8, A = 32 point is the full record above
+            if isinstance(r_, dict) and r_.get("config", {}).get("workload", "").startswith("transformer"):
+                sweep.insert(2, short_row(r_))
+        head["transformer_r_sweep"] = sweep
+        nxt = []
+        for name, kw in (("resnet50_lars", {}), ("transformer_adafactor", {}),
+                         ("bert_large", {"layout": "concat"}), ("decoder_1p5b", {"layout": "concat"}),
+                         ("transformer", {"layout": "concat", "R": 1024})):
+            R_ = kw.pop("R", 0)
+            nxt.append(guarded(lambda: short_row(measure(
+                ctx, get_workload(name, R=R_), align=args.align, path="fused", e2e=False, cpu=False, **kw, **common)),
+                name))
+            release()
+        head["next_workloads"] = nxt
+    if ctx.rank == 0:
+        print(json.dumps(head))
+    ctx.close()
 
 
 def main():

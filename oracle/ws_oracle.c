@@ -119,6 +119,8 @@ int64_t wso_plan(const int64_t *numel, int32_t T, int32_t R, int32_t A,
 void wso_pack(const void *const *tensors, const int64_t *numel, const int64_t *piece,
               const int64_t *off, int32_t T, int32_t R, int64_t S, int32_t elem_bytes,
               void *flat) {
+    /* (small inputs stay on the calling thread: waking a team costs more than the copy) */
+#pragma omp parallel for collapse(2) schedule(dynamic) if ((int64_t)R * S > (1 << 18))
     for (int32_t r = 0; r < R; ++r)
         for (int32_t t = 0; t < T; ++t)
             for (int64_t q = 0; q < piece[t]; ++q) {
@@ -136,6 +138,9 @@ void wso_pack(const void *const *tensors, const int64_t *numel, const int64_t *p
 void wso_unpack(const void *flat, const int64_t *numel, const int64_t *piece,
                 const int64_t *off, int32_t T, int64_t S, int32_t elem_bytes,
                 void *const *tensors) {
+    int64_t total = 0;
+    for (int32_t t = 0; t < T; ++t) total += numel[t];
+#pragma omp parallel for schedule(dynamic) if (total > (1 << 18))
     for (int32_t t = 0; t < T; ++t)
         for (int64_t i = 0; i < numel[t]; ++i) {
             int64_t r = i / piece[t], q = i % piece[t];
@@ -257,6 +262,10 @@ void wso_sharded_update(const wso_hyper *h, int32_t T, const int64_t *numel,
         u = (double *)calloc((size_t)R * (size_t)S + 1, sizeof(double));
         part = (double *)calloc((size_t)R * (size_t)T * 2 + 1, sizeof(double));
     }
+    /* (shard, tensor) iterations touch disjoint positions and own one pair of partial sums each,
+     * accumulated in ascending q on whichever thread runs the iteration: the result does not
+     * depend on the number of threads */
+#pragma omp parallel for collapse(2) schedule(dynamic) if ((int64_t)R * S > (1 << 18))
     for (int32_t r = 0; r < R; ++r) {
         for (int32_t t = 0; t < T; ++t) {
             double pa = 0.0, pb = 0.0;
@@ -297,6 +306,8 @@ void wso_sharded_update(const wso_hyper *h, int32_t T, const int64_t *numel,
             }
         }
     }
+    /* per tensor: combine the shards' partials in ascending r, then apply (tensors are independent) */
+#pragma omp parallel for schedule(dynamic) if ((int64_t)R * S > (1 << 18))
     for (int32_t t = 0; t < T; ++t) {
         double ratio = 1.0;
         if (lamb) {
@@ -318,10 +329,12 @@ void wso_sharded_update(const wso_hyper *h, int32_t T, const int64_t *numel,
     if (partials && lamb) memcpy(partials, part, sizeof(double) * (size_t)R * T * 2);
     if (gathered) {
         int64_t G = (int64_t)R * S;
-        if (out_dtype == WSO_BF16)
+        if (out_dtype == WSO_BF16) {
+#pragma omp parallel for schedule(static) if (G > (1 << 18))
             for (int64_t j = 0; j < G; ++j) ((uint16_t *)gathered)[j] = wso_f32_to_bf16(w[j]);
-        else
+        } else {
             memcpy(gathered, w, sizeof(float) * (size_t)G);
+        }
     }
     free(u);
     free(part);
@@ -704,6 +717,21 @@ int32_t wso_num_threads(void) {
     extern int omp_get_max_threads(void);
     return omp_get_max_threads();
 #else
+    return 1;
+#endif
+}
+
+/* Threads the loops with independent iterations may use from now on (1 = the single-thread
+ * timing of the benchmark); returns the previous setting.  Results do not depend on it. */
+int32_t wso_set_num_threads(int32_t n) {
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    extern void omp_set_num_threads(int);
+    int32_t prev = omp_get_max_threads();
+    if (n >= 1) omp_set_num_threads(n);
+    return prev;
+#else
+    (void)n;
     return 1;
 #endif
 }

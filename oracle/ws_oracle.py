@@ -106,6 +106,8 @@ def lib():
         L.wso_bf16_to_double.restype = C.c_double
         L.wso_bf16_to_double.argtypes = [C.c_uint16]
         L.wso_num_threads.restype = C.c_int32
+        L.wso_set_num_threads.restype = C.c_int32
+        L.wso_set_num_threads.argtypes = [C.c_int32]
         _lib = L
     return _lib
 
@@ -283,6 +285,12 @@ def bf16_bits_to_f64(x: np.ndarray) -> np.ndarray:
 
 def num_threads() -> int:
     return int(lib().wso_num_threads())
+
+
+def set_num_threads(n: int) -> int:
+    """Threads for the loops with independent iterations (the results do not depend on it);
+    returns the previous setting."""
+    return int(lib().wso_set_num_threads(int(n)))
 
 
 class FlatPlan:

@@ -366,6 +366,26 @@ def test_sharded_equals_unsharded_bit_identical(opt, R):
             assert a.tobytes() == b.tobytes()
 
 
+@pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb"])
+def test_thread_count_does_not_change_any_bit(opt):
+    # the all-core timing of the benchmark runs the same code on more threads: only loops with
+    # independent iterations are split, every sum keeps its one fixed order
+    numel = [1, 9, 64, 333, 2048, 5000, 70001, 300000]      # large enough for the loops to go parallel
+    prev = O.set_num_threads(1)
+    try:
+        _, _, one = _run_both(opt, 7, 8, numel, momentum=0.9, weight_decay=0.01, bf16=(opt == "adam"), seed=3,
+                              out_dtype=O.BF16)
+        O.set_num_threads(max(2, os.cpu_count() or 2))
+        assert O.num_threads() >= 2
+        _, _, many = _run_both(opt, 7, 8, numel, momentum=0.9, weight_decay=0.01, bf16=(opt == "adam"), seed=3,
+                               out_dtype=O.BF16)
+    finally:
+        O.set_num_threads(prev)
+    for a, b in zip(one, many):
+        if a is not None:
+            assert np.asarray(a).tobytes() == np.asarray(b).tobytes()
+
+
 @pytest.mark.parametrize("R", [1, 3, 8, 64])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_sharded_lamb_equals_unsharded_within_one_ulp(R, bf16):
