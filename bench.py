@@ -151,8 +151,9 @@ def bytes_per_param(wl):
         upd += 12          # phase 1 reads w and stores the summed gradient; phase 2 reads it back
     if wl.opt == "adafactor":
         upd += 16          # pass 1 stores the summed gradient, passes 2 and 3 read it back, pass 3 reads w again
-    # fused formatting: same reads and state writes; an fp32 weight list is written next to the fp32 shard state
-    fused = upd + (0 if out_b else 4)
+    # fused formatting: same reads and state writes; fp32 weight tensors are the master copy themselves
+    # (read and written in place, no sharded w), a bf16 weight list is the copy counted in `alg`
+    fused = upd
     return {"algorithmic": alg, "update": upd, "fused": fused, "pack": 2 * gb, "unpack": 2 * (2 if out_b else 4)}
 
 
@@ -225,6 +226,15 @@ class ClockSampler:
 # ----------------------------------------------------------------------------
 # CPU oracle legs
 # ----------------------------------------------------------------------------
+def sample_stride(n_total, target):
+    """Stride of the bounded tensor sample: about n_total / target, rounded up to a prime so that it does
+    not fall in step with the period of a layer's tensor list (16 tensors per BERT layer)."""
+    k = max(1, round(n_total / target))
+    while k > 2 and any(k % d == 0 for d in range(2, int(k ** 0.5) + 1)):
+        k += 1
+    return k
+
+
 def oracle_step_inputs(wl, stride, align):
     """Host copies of every `stride`-th tensor of the workload (the bounded sample), starting in the
     middle of the first stride so that the sample is not dominated by the embedding at index 0."""
@@ -272,7 +282,7 @@ def cpu_baseline(wl, align, target_params=0, min_seconds=10.0, max_steps=20):
     the thread count).  `value` is the all-core rate."""
     from oracle import ws_oracle as O
     target_params = target_params or int(2e8 / (wl.R + 3))      # bounds the sample's host memory and set-up time
-    stride = max(1, round(wl.N / target_params))
+    stride = sample_stride(wl.N, target_params)
     sub, plan, g, pw, pm, pv = oracle_step_inputs(wl, stride, align)
     host_cores = len(os.sched_getaffinity(0))
     runs = {}
@@ -303,7 +313,7 @@ def run_reference(args):
     from oracle import ws_oracle as O
     O.build()
     wl = workload_from_args(args)
-    stride = max(1, round(wl.N / 6_000_000))
+    stride = sample_stride(wl.N, 6_000_000)
     sub, plan, g, pw, pm, pv = oracle_step_inputs(wl, stride, args.align)
     cores = O.num_threads()
     for _ in range(max(1, args.warmup)):
@@ -329,7 +339,8 @@ def run_reference(args):
 def config_of(wl, align, layout, shards, extra=None, path="fused"):
     steps = {"unfused": "pack R gradient sets + fused reduce/update of all shards + unpack weights (separate kernels)",
              "fused": "one kernel: gradients read from the R replicas' tensor lists (formatting fused in), reduce, "
-                      "update of all shards, weights written to the weight tensors"}
+                      "update of all shards, weights written to the weight tensors (fp32 weights: read from and "
+                      "written to the tensors, which are the master copy)"}
     c = {"workload": f"{wl.name}: {wl.T} tensors, {wl.N} params, R={wl.R} replicas, {wl.opt}, "
                      f"grads {str(wl.grad_dtype).split('.')[-1]}, gathered {str(wl.out_dtype).split('.')[-1]}",
          "R": wl.R, "shards": shards or wl.R, "optimizer": wl.opt, "align_elems": align, "layout": layout,
@@ -536,6 +547,13 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
         pv = None
     if wl.opt == "adafactor":
         pm, pv = None, W.make_factored_state(wl, plan.factored_elems, dev)
+    w_arena = torch.zeros(A_el, dtype=odt, device=dev)
+    w_views = B.PtrList(plan.arena_views(w_arena, numels))
+    # fp32 weights: on the fused route the weight tensors are the master copy (no sharded w is passed)
+    master = odt == torch.float32
+    if master:
+        for dst, src in zip(w_views, w):
+            dst.copy_(src)
     del w, m, v
     g_arena = [torch.zeros(A_el, dtype=gdt, device=dev) for _ in range(R)]
     g_views = [B.PtrList(plan.arena_views(a, numels)) for a in g_arena]
@@ -544,8 +562,6 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
         for dst, src in zip(g_views[k], gk):
             dst.copy_(src)
         del gk
-    w_arena = torch.zeros(A_el, dtype=odt, device=dev)
-    w_views = B.PtrList(plan.arena_views(w_arena, numels))
     ws = torch.empty(max(32, plan.workspace_bytes(wl.opt)), dtype=torch.uint8, device=dev)
     hy = B.make_hyper(wl.opt, wl.hyper)
     pg = gathered = None
@@ -582,7 +598,7 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
             flush.zero_()
         if ev:
             ev[0].record()
-        B.ws_fused_update(plan, -1, gtab, pw, pm, pv, hy, wtab, ws)
+        B.ws_fused_update(plan, -1, gtab, None if master else pw, pm, pv, hy, wtab, ws)
         if ev:
             ev[1].record()
 

@@ -141,6 +141,43 @@ ws_status ws_plan_segments(const ws_plan* plan, const ws_segment** segs, int32_t
 size_t ws_plan_device_bytes(const ws_plan* plan);
 ws_status ws_plan_upload(ws_plan* plan, void* dev_buf, size_t bytes, void* stream);
 
+/* One-launch schedule (optional).  The norm-based optimizers (WS_LAMB, WS_LARS) need every shard's
+ * partial norm sums of a tensor before any shard can apply the step (Section 4.1), so their
+ * all-shard update is phase 1, a combination step, phase 2.  As three launches, phase 2 reads the
+ * weight and the new moments from DRAM again.  A plan whose schedule has been uploaded runs the same
+ * update as ONE persistent kernel instead: the two phases of every tensor are work items ordered so
+ * that a tensor's phase 2 follows its phase 1 closely, while other tensors' phase 1 streams from
+ * DRAM, and phase 2 finds its operands in L2 - every operand crosses HBM once, as the update of
+ * Section 2.2 counts them.  Results: the same as the three-launch form up to the order of the norm
+ * sums (the ratios agree to rounding; they are bit-stable from run to run).
+ *   ws_plan_schedule_bytes   device bytes of the schedule (0: this plan has none - more than
+ *                            65535 shards or 2^30 work items)
+ *   ws_plan_upload_schedule  builds the schedule on first use and copies it into the caller's
+ *                            buffer (16-byte aligned, alive while the plan is in use) with
+ *                            cudaMemcpyAsync on `stream`; call once, before the plan is shared
+ *                            between threads
+ * Afterwards ws_shard_update / ws_fused_update with r == -1 and WS_LAMB or WS_LARS (and
+ * ws_lamb_update_static_scratch) take the one-kernel route when there are at most 32 gradient
+ * copies; the shard-by-shard calls are unchanged.  The kernel's waits (a phase-2 item waits for
+ * its tensor's ratio) are bounded: if one ever runs out, the kernel stops, leaves the update
+ * incomplete and sets the 32-bit status word inside the workspace (ws_workspace_sync_status gives
+ * its byte offset; 0 = completed) - a caller that wants to detect this reads the word after
+ * synchronising the stream.
+ * ws_plan_schedule_view / ws_plan_schedule_item expose the order for inspection (host only):
+ * entry i of `order` is item index * 2 + phase (0: phase 1, 1: phase 2). */
+size_t ws_plan_schedule_bytes(const ws_plan* plan);
+ws_status ws_plan_upload_schedule(ws_plan* plan, void* dev_buf, size_t bytes, void* stream);
+typedef struct {
+    int32_t tensor, shard;
+    int64_t pos;        /* start inside the shard                     */
+    int64_t tensor_off; /* element index of the start in the tensor   */
+    int32_t len;        /* elements of the item                       */
+    int32_t nvalid;     /* how many of them exist in the tensor       */
+} ws_sched_item;
+ws_status ws_plan_schedule_view(ws_plan* plan, const uint32_t** order, int64_t* n_entries);
+ws_status ws_plan_schedule_item(ws_plan* plan, int64_t item, ws_sched_item* out);
+ws_status ws_workspace_sync_status(const ws_plan* plan, size_t* offset_bytes);
+
 /* ------------------------------------------------------- pack / unpack ---
  * ws_pack: flat[r S + off_t + q] = X_t[r p_t + q] where that location exists,
  * +0 (all-zero bits) otherwise.  This is the "sharding program" for weights
@@ -262,8 +299,10 @@ ws_status ws_plan_factored_layout(const ws_plan* plan, int64_t* layout);
  *   double norms[T][2]       squared norms (sum w^2, sum u^2) per tensor
  *   float  partials[R][tiles][2]   per-tile partial sums from phase 1
  *                                  ([tiles][2] for the concatenated layout)
+ *   (scratch of the one-launch route: per-item partial sums, per-tensor
+ *    counters and flags, a ticket counter and the status word)
  * so a caller can read rho and the norms back for logging.  WS_LARS uses the
- * same three arrays (rho holds the local rates, norms sum w^2 and sum g^2)
+ * same arrays (rho holds the local rates, norms sum w^2 and sum g^2)
  * followed, at the next 256-byte boundary, by
  *   float  ghat[R][S]        the summed gradients kept from phase 1 for phase 2
  * WS_ADAFACTOR uses all four (rho holds the applied step size alpha_t / max(1,

@@ -67,6 +67,11 @@ class ws_tensor_table(C.Structure):
                 ("min_align", C.c_int32)]
 
 
+class ws_sched_item(C.Structure):
+    _fields_ = [("tensor", C.c_int32), ("shard", C.c_int32), ("pos", C.c_int64), ("tensor_off", C.c_int64),
+                ("len", C.c_int32), ("nvalid", C.c_int32)]
+
+
 class ws_host_io(C.Structure):
     _fields_ = [("host_grads", C.POINTER(C.c_void_p)), ("grad_dtype", C.c_int32),
                 ("dev_grad_arena", C.c_void_p), ("dev_packed_grads", C.POINTER(C.c_void_p)),
@@ -85,6 +90,8 @@ EXPORTS = [
     "ws_plan_factored_elems", "ws_plan_factored_layout", "ws_workspace_partials",
     "ws_lars_partial", "ws_lars_finalize", "ws_lars_apply",
     "ws_adafactor_stage", "ws_workspace_adafactor_sums",
+    "ws_plan_schedule_bytes", "ws_plan_upload_schedule", "ws_plan_schedule_view", "ws_plan_schedule_item",
+    "ws_workspace_sync_status",
 ]
 
 _lib = None
@@ -179,6 +186,16 @@ def lib() -> C.CDLL:
     L.ws_fused_update.restype = C.c_int
     L.ws_fused_update.argtypes = [vp, C.c_int32, C.POINTER(ws_tensor_table), C.POINTER(ws_state),
                                   C.POINTER(ws_hyper), C.POINTER(ws_tensor_table), vp, C.c_size_t, vp]
+    L.ws_plan_schedule_bytes.restype = C.c_size_t
+    L.ws_plan_schedule_bytes.argtypes = [vp]
+    L.ws_plan_upload_schedule.restype = C.c_int
+    L.ws_plan_upload_schedule.argtypes = [vp, vp, C.c_size_t, vp]
+    L.ws_plan_schedule_view.restype = C.c_int
+    L.ws_plan_schedule_view.argtypes = [vp, C.POINTER(C.POINTER(C.c_uint32)), C.POINTER(C.c_int64)]
+    L.ws_plan_schedule_item.restype = C.c_int
+    L.ws_plan_schedule_item.argtypes = [vp, C.c_int64, C.POINTER(ws_sched_item)]
+    L.ws_workspace_sync_status.restype = C.c_int
+    L.ws_workspace_sync_status.argtypes = [vp, C.POINTER(C.c_size_t)]
     L.ws_status_string.restype = C.c_char_p
     L.ws_status_string.argtypes = [C.c_int]
     L.ws_last_cuda_error.restype = C.c_char_p
@@ -241,7 +258,10 @@ class Plan:
     """Owns a ws_plan and the device buffer that holds its tables."""
 
     def __init__(self, shapes: Sequence[Sequence[int]], R: int, align_elems: int = 32, tile_elems: int = 0,
-                 device: Optional[torch.device] = None, upload: bool = True, layout: str = "per_tensor"):
+                 device: Optional[torch.device] = None, upload: bool = True, layout: str = "per_tensor",
+                 one_launch: bool = True):
+        """``one_launch``: also upload the plan's one-launch schedule, so that the all-shard LAMB and LARS
+        updates run as one persistent kernel (with ``False`` they run as three launches)."""
         T = len(shapes)
         descs = (ws_tensor_desc * max(1, T))()
         for i, s in enumerate(shapes):
@@ -261,8 +281,11 @@ class Plan:
         self.G = self.R * self.S
         self.ntiles = L.ws_plan_num_tiles(self._h)
         self.dev_buf = None
+        self.sched_buf = None
         if upload:
             self.upload(device)
+            if one_launch:
+                self.upload_schedule(device)
 
     @property
     def handle(self):
@@ -277,6 +300,33 @@ class Plan:
         nbytes = lib().ws_plan_device_bytes(self._h)
         self.dev_buf = torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
         _check(lib().ws_plan_upload(self._h, self.dev_buf.data_ptr(), nbytes, _stream()), "ws_plan_upload")
+
+    def upload_schedule(self, device=None):
+        nbytes = lib().ws_plan_schedule_bytes(self._h)
+        if nbytes == 0:          # the plan has no one-launch schedule
+            return
+        self.sched_buf = torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
+        _check(lib().ws_plan_upload_schedule(self._h, self.sched_buf.data_ptr(), nbytes, _stream()),
+               "ws_plan_upload_schedule")
+
+    def schedule(self):
+        """(order, items): the one-launch execution order as a list of (item, phase) and the items as
+        ws_sched_item records.  Host only."""
+        order, n = C.POINTER(C.c_uint32)(), C.c_int64()
+        _check(lib().ws_plan_schedule_view(self._h, C.byref(order), C.byref(n)), "ws_plan_schedule_view")
+        import numpy as np
+        arr = np.ctypeslib.as_array(order, shape=(n.value,)).copy()
+        items = []
+        for i in range(n.value // 2):
+            it = ws_sched_item()
+            _check(lib().ws_plan_schedule_item(self._h, i, C.byref(it)), "ws_plan_schedule_item")
+            items.append(it)
+        return [(int(e) >> 1, int(e) & 1) for e in arr], items
+
+    def sync_status_offset(self) -> int:
+        off = C.c_size_t()
+        _check(lib().ws_workspace_sync_status(self._h, C.byref(off)), "ws_workspace_sync_status")
+        return off.value
 
     @property
     def arena_elems(self) -> int:
@@ -333,7 +383,8 @@ def _grads(gbufs: Sequence[torch.Tensor], slice_mode: int):
 
 
 def _state(w, m, v):
-    return ws_state(w.data_ptr(), m.data_ptr() if m is not None else None, v.data_ptr() if v is not None else None)
+    return ws_state(w.data_ptr() if w is not None else None, m.data_ptr() if m is not None else None,
+                    v.data_ptr() if v is not None else None)
 
 
 def _out(gathered):

@@ -56,6 +56,28 @@ struct WsAfChunk {
     int seg;
 };
 
+// One-launch schedule of the norm-based optimizers (LAMB, LARS): the update of all shards as ONE
+// persistent kernel.  A work item is a run of at most kWsItemElems consecutive shard positions inside
+// one tile; every item appears twice in the schedule, once for phase 1 (reduce, moments, partial
+// norm sums) and once for phase 2 (apply the step with the tensor's ratio).
+constexpr int kWsItemElems = 2048;
+struct __align__(16) WsItem {
+    long long pos;        // start inside the shard, multiple of 8
+    long long toff;       // element index of the first element inside tensor `seg`
+    int seg;              // tensor index
+    int nvalid;           // elements of the item that exist in the tensor (the rest is padding)
+    unsigned short len;   // elements, multiple of 8
+    unsigned short shard;
+    unsigned flags;       // bit 0: the tensor group is small enough to stay in L2 between its phases
+};
+static_assert(sizeof(WsItem) == 32, "WsItem is read as two 16-byte words");
+// Items are numbered tensor by tensor (then shard by shard), so a tensor's items - and with them its
+// partial norm sums - are one contiguous range.
+struct WsItemSeg {
+    int first;
+    int count;
+};
+
 struct ws_plan {
     int T = 0, R = 0, A = 0, K = 0;
     int layout = 0;                           // ws_layout
@@ -77,6 +99,14 @@ struct ws_plan {
     long long Fi = 0;                         // floats of the padded workspace layout
     const WsSegAf* d_segaf = nullptr;
     const WsAfChunk* d_afchunks = nullptr;
+    // one-launch schedule: counted at creation, built and uploaded by ws_plan_upload_schedule
+    long long n_items = 0;                    // work items (0: the plan has no one-launch schedule)
+    std::vector<WsItem> items;
+    std::vector<WsItemSeg> itemsegs;          // [T]
+    std::vector<unsigned> sched;              // [2 n_items]: item index * 2 + phase, in execution order
+    const WsItem* d_items = nullptr;
+    const WsItemSeg* d_itemsegs = nullptr;
+    const unsigned* d_sched = nullptr;
 };
 
 // Optimizer constants narrowed to fp32 for the kernels.
@@ -89,7 +119,15 @@ struct WsLambWs {
     float* rho;        // [T]
     double* norms;     // [T][2]
     float2* partials;  // [R][ntiles]
-    size_t bytes;      // through the partials: what LAMB needs
+    // one-launch update: per-item partial sums, per-tensor arrival counters and ready flags, the
+    // ticket counter and the status word (sync_bytes from `count` on are cleared before every launch)
+    float2* ipart;     // [n_items]
+    int* count;        // [T]
+    int* flag;         // [T]
+    unsigned long long* ticket;
+    int* status;
+    size_t sync_bytes;
+    size_t bytes;      // through the one-launch scratch: what LAMB needs
     float* ghat;       // LARS only: [R][S] summed gradients, 256-byte aligned after the partials
     size_t bytes_lars; // through ghat: what LARS needs
     float* acc;        // Adafactor: [Fi] this step's row / column sums (padded layout)

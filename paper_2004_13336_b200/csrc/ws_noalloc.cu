@@ -61,11 +61,9 @@ extern "C" ws_status ws_lamb_update_static_scratch(const ws_plan* plan, const ws
     if (s != WS_OK) return s;
     void* scratch = nullptr;
     if ((s = scratch_for_current_device(&scratch)) != WS_OK) return s;
-    // Nothing in the scratch has to start at zero: phase 1 overwrites the partial
-    // of every (shard, tile) and the finalize step overwrites every ratio and norm.
-    s = ws_lamb_partial(plan, -1, grads, state, hyper, scratch, kStaticScratchBytes, stream);
-    if (s != WS_OK) return s;
-    s = ws_lamb_finalize(plan, scratch, kStaticScratchBytes, stream);
-    if (s != WS_OK) return s;
-    return ws_lamb_apply(plan, -1, state, hyper, out, scratch, kStaticScratchBytes, stream);
+    // The update itself is ws_shard_update's all-shard LAMB with the library's array as its workspace:
+    // three launches, or one when the plan carries its one-launch schedule.  What has to start at zero
+    // (the one-launch route's counters, flags, ticket and status word) is cleared on the stream by that
+    // route itself; everything else in the scratch is overwritten before it is read.
+    return ws_shard_update(plan, -1, grads, state, hyper, out, scratch, kStaticScratchBytes, stream);
 }

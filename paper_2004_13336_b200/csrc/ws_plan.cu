@@ -78,6 +78,18 @@ static void ws_matrix_views(ws_plan* p, const ws_tensor_desc* descs) {
     p->Fi = ioff;
 }
 
+// Work items of the one-launch schedule: every tile cut into runs of kWsItemElems elements, for every
+// shard it serves.  Plans beyond the item fields' ranges get no schedule (n_items stays 0).
+static void ws_count_items(ws_plan* p) {
+    p->n_items = 0;
+    if (p->R > 65535) return;
+    long long per_shard = 0;
+    for (const WsTile& tl : p->tiles) per_shard += (tl.len + kWsItemElems - 1) / kWsItemElems;
+    const long long n = p->layout == WS_LAYOUT_CONCAT ? per_shard : per_shard * p->R;
+    if (n > 0x3fffffffLL) return;
+    p->n_items = n;
+}
+
 extern "C" ws_status ws_plan_create(const ws_tensor_desc* descs, int32_t T, int32_t R,
                                     int32_t align_elems, int32_t tile_elems, ws_plan** out) {
     return ws_plan_create_layout(descs, T, R, align_elems, tile_elems, WS_LAYOUT_PER_TENSOR, out);
@@ -187,6 +199,7 @@ extern "C" ws_status ws_plan_create_layout(const ws_tensor_desc* descs, int32_t 
                 if (!seen[k])
                     p->segtiles[k].tile_begin = k > 0 ? p->segtiles[k - 1].tile_begin + p->segtiles[k - 1].tile_count : 0;
             ws_matrix_views(p, descs);
+            ws_count_items(p);
             *out = p;
             return WS_OK;
         }
@@ -228,6 +241,7 @@ extern "C" ws_status ws_plan_create_layout(const ws_tensor_desc* descs, int32_t 
         p->S = off;
         p->ntiles = (long long)p->tiles.size();
         ws_matrix_views(p, descs);
+        ws_count_items(p);
     } catch (...) {
         delete p;
         return WS_ERR_INVALID_ARG;
@@ -309,6 +323,18 @@ WsLambWs ws_lamb_layout(const ws_plan* p, void* workspace) {
     o = round16(o + sizeof(double) * 2 * (size_t)p->T);
     L.partials = (float2*)(b + o);
     o = round16(o + sizeof(float2) * (size_t)(p->layout == WS_LAYOUT_CONCAT ? 1 : p->R) * (size_t)p->ntiles);
+    L.ipart = (float2*)(b + o);
+    o = round16(o + sizeof(float2) * (size_t)p->n_items);
+    L.count = (int*)(b + o);
+    const size_t sync0 = o;
+    o += sizeof(int) * (size_t)p->T;
+    L.flag = (int*)(b + o);
+    o = (o + sizeof(int) * (size_t)p->T + 7) & ~(size_t)7;
+    L.ticket = (unsigned long long*)(b + o);
+    o += sizeof(unsigned long long);
+    L.status = (int*)(b + o);
+    o = round16(o + sizeof(int));
+    L.sync_bytes = o - sync0;
     L.bytes = o;
     o = (o + 255) & ~(size_t)255;
     L.ghat = (float*)(b + o);
@@ -350,4 +376,186 @@ extern "C" size_t ws_workspace_bytes(const ws_plan* p, ws_opt opt) {
     if (opt == WS_LARS) return ws_lamb_layout(p, nullptr).bytes_lars;
     if (opt == WS_ADAFACTOR) return ws_lamb_layout(p, nullptr).bytes_af;
     return 0;
+}
+
+// ------------------------------------------------------ one-launch schedule ---
+// Order of execution for the one-kernel LAMB / LARS update.  Tensors are taken in groups of a few
+// megabytes of state; a group's phase-2 items follow its phase-1 items at a distance of at least
+// kLag schedule entries (by then every CTA that worked on the group's phase 1 has finished and the
+// tensors' ratios are known, so no CTA waits), interleaved one to one with the phase-1 items of the
+// following groups: phase 2 then reads w, m', v' out of L2 while phase 1 of the next tensors streams
+// from DRAM, and each operand crosses HBM once (Section 2.2).  When more than kLag eligible phase-2
+// items are waiting (a tensor larger than L2 has just finished) they run first.
+namespace {
+constexpr long long kGroupBytes = 6LL << 20;    // state bytes (12 per element) that close a group
+constexpr long long kKeepLo = 16LL << 20;       // groups between these sizes ask L2 to keep their lines;
+constexpr long long kKeepHi = 80LL << 20;       //   smaller ones stay resident anyway, larger ones cannot
+constexpr int kLag = 512;
+
+void ws_build_schedule(ws_plan* p) {
+    const int T = p->T, R = p->R;
+    const bool concat = p->layout == WS_LAYOUT_CONCAT;
+    p->items.clear();
+    p->items.reserve((size_t)p->n_items);
+    p->itemsegs.assign(T, WsItemSeg{0, 0});
+    std::vector<long long> seg_bytes(T, 0);
+    for (int t = 0; t < T; ++t) {
+        p->itemsegs[t].first = (int)p->items.size();
+        const WsSegTiles st = p->segtiles[t];
+        for (int r = 0; r < (concat ? 1 : R); ++r)
+            for (int k = 0; k < st.tile_count; ++k) {
+                const WsTile& tl = p->tiles[st.tile_begin + k];
+                const long long toff0 = concat ? tl.poff : (long long)r * tl.piece + tl.poff;
+                const long long valid0 = concat ? tl.vt : tl.vt - (long long)r * tl.piece;
+                for (int so = 0; so < tl.len; so += kWsItemElems) {
+                    WsItem it;
+                    memset(&it, 0, sizeof(it));
+                    const int len = tl.len - so < kWsItemElems ? tl.len - so : kWsItemElems;
+                    long long nv = valid0 - so;
+                    it.pos = tl.pos + so;
+                    it.toff = toff0 + so;
+                    it.seg = t;
+                    it.nvalid = (int)(nv < 0 ? 0 : (nv > len ? len : nv));
+                    it.len = (unsigned short)len;
+                    it.shard = (unsigned short)(concat ? tl.shard : r);
+                    p->items.push_back(it);
+                    seg_bytes[t] += 12LL * len;
+                }
+            }
+        p->itemsegs[t].count = (int)p->items.size() - p->itemsegs[t].first;
+    }
+    // groups of consecutive tensors
+    struct Group { int first, end; };     // item range
+    std::vector<Group> groups;
+    {
+        long long acc = 0;
+        int gfirst = 0, t0 = 0;
+        for (int t = 0; t < T; ++t) {
+            acc += seg_bytes[t];
+            const bool last = t == T - 1;
+            if (acc >= kGroupBytes || last) {
+                const int gend = p->itemsegs[t].first + p->itemsegs[t].count;
+                if (gend > gfirst) {
+                    groups.push_back(Group{gfirst, gend});
+                    const unsigned keep = (acc > kKeepLo && acc < kKeepHi) ? 1u : 0u;
+                    for (int i = gfirst; i < gend; ++i) p->items[i].flags = keep;
+                }
+                gfirst = gend;
+                acc = 0;
+                t0 = t + 1;
+            }
+        }
+        (void)t0;
+    }
+    // merge the phase-1 stream and the phase-2 stream
+    const long long n = (long long)p->items.size();
+    p->sched.clear();
+    p->sched.reserve((size_t)(2 * n));
+    const int G = (int)groups.size();
+    std::vector<long long> p1_done_at(G, -1);     // schedule position of each group's last phase-1 item
+    int ag = 0, eg = 0;                           // group of the next phase-1 item; first group not yet eligible
+    long long ai = 0, bi = 0;                     // next phase-1 / phase-2 item
+    long long eligible = 0;                       // phase-2 items of groups whose phase 1 ended >= kLag entries ago
+    int last_kind = 1;
+    while (bi < n) {
+        const long long pos = (long long)p->sched.size();
+        while (eg < ag && pos - p1_done_at[eg] >= kLag) {
+            eligible += groups[eg].end - groups[eg].first;
+            ++eg;
+        }
+        const long long backlog = eligible - bi;
+        const bool may2 = backlog > 0;
+        if (ai < n && !(may2 && (last_kind == 0 || backlog > kLag))) {
+            p->sched.push_back((unsigned)(ai << 1));
+            last_kind = 0;
+            if (++ai == groups[ag].end) {
+                p1_done_at[ag] = pos;
+                ++ag;
+            }
+        } else {
+            // (at the very end the last groups' phase 2 follows their phase 1 directly: the scheduling
+            // warps then wait for the ratios, a few microseconds once per launch)
+            p->sched.push_back((unsigned)(bi << 1) | 1u);
+            last_kind = 1;
+            ++bi;
+            if (!may2) eligible = bi;             // keep the backlog arithmetic consistent in the tail
+        }
+    }
+}
+
+size_t schedule_bytes(const ws_plan* p) {
+    return round16((size_t)p->n_items * sizeof(WsItem)) + round16((size_t)p->T * sizeof(WsItemSeg)) +
+           round16((size_t)p->n_items * 2 * sizeof(unsigned));
+}
+}  // namespace
+
+extern "C" size_t ws_plan_schedule_bytes(const ws_plan* p) {
+    if (!p || p->n_items <= 0) return 0;
+    return schedule_bytes(p);
+}
+
+extern "C" ws_status ws_plan_upload_schedule(ws_plan* p, void* dev_buf, size_t bytes, void* stream) {
+    if (!p || !dev_buf) return WS_ERR_INVALID_ARG;
+    if (p->n_items <= 0) return WS_ERR_TOO_LARGE;
+    if (!ws_aligned16(dev_buf)) return WS_ERR_ALIGNMENT;
+    if (bytes < schedule_bytes(p)) return WS_ERR_WORKSPACE;
+    try {
+        if (p->sched.empty()) ws_build_schedule(p);
+    } catch (...) {
+        return WS_ERR_INVALID_ARG;
+    }
+    if ((long long)p->items.size() != p->n_items) return WS_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    char* base = (char*)dev_buf;
+    const size_t ib = (size_t)p->n_items * sizeof(WsItem), sb = (size_t)p->T * sizeof(WsItemSeg);
+    cudaError_t e = cudaMemcpyAsync(base, p->items.data(), ib, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return ws_cuda_fail(e, "ws_plan_upload_schedule(items)");
+    e = cudaMemcpyAsync(base + round16(ib), p->itemsegs.data(), sb, cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return ws_cuda_fail(e, "ws_plan_upload_schedule(tensor ranges)");
+    e = cudaMemcpyAsync(base + round16(ib) + round16(sb), p->sched.data(), p->sched.size() * sizeof(unsigned),
+                        cudaMemcpyHostToDevice, st);
+    if (e != cudaSuccess) return ws_cuda_fail(e, "ws_plan_upload_schedule(order)");
+    p->d_items = (const WsItem*)base;
+    p->d_itemsegs = (const WsItemSeg*)(base + round16(ib));
+    p->d_sched = (const unsigned*)(base + round16(ib) + round16(sb));
+    return WS_OK;
+}
+
+extern "C" ws_status ws_plan_schedule_view(ws_plan* p, const uint32_t** order, int64_t* n_entries) {
+    if (!p || !order || !n_entries) return WS_ERR_INVALID_ARG;
+    if (p->n_items <= 0) return WS_ERR_TOO_LARGE;
+    try {
+        if (p->sched.empty()) ws_build_schedule(p);
+    } catch (...) {
+        return WS_ERR_INVALID_ARG;
+    }
+    *order = p->sched.data();
+    *n_entries = (int64_t)p->sched.size();
+    return WS_OK;
+}
+
+extern "C" ws_status ws_plan_schedule_item(ws_plan* p, int64_t item, ws_sched_item* out) {
+    if (!p || !out) return WS_ERR_INVALID_ARG;
+    if (p->n_items <= 0) return WS_ERR_TOO_LARGE;
+    try {
+        if (p->sched.empty()) ws_build_schedule(p);
+    } catch (...) {
+        return WS_ERR_INVALID_ARG;
+    }
+    if (item < 0 || item >= p->n_items) return WS_ERR_INVALID_ARG;
+    const WsItem& it = p->items[(size_t)item];
+    out->tensor = it.seg;
+    out->shard = it.shard;
+    out->pos = it.pos;
+    out->tensor_off = it.toff;
+    out->len = it.len;
+    out->nvalid = it.nvalid;
+    return WS_OK;
+}
+
+extern "C" ws_status ws_workspace_sync_status(const ws_plan* p, size_t* offset_bytes) {
+    if (!p || !offset_bytes) return WS_ERR_INVALID_ARG;
+    const WsLambWs L = ws_lamb_layout(p, nullptr);
+    *offset_bytes = (size_t)((char*)L.status - (char*)nullptr);
+    return WS_OK;
 }

@@ -173,3 +173,72 @@ def test_factored_layout_matches_oracle_view():
     assert plan.factored_elems == tot == 12 + 0 + 0 + 100 + 29 + 1 + 10 + 10
     assert plan.factored_layout() == list(zip(foff.tolist(), rows.tolist(), cols.tolist()))
     assert plan.workspace_bytes("adafactor") >= plan.workspace_bytes("lars") + 8 * tot + 4 * plan.T
+
+
+@pytest.mark.parametrize("layout", ["per_tensor", "concat"])
+@pytest.mark.parametrize("R,tile", [(1, 0), (3, 1024), (16, 4096), (40, 0)])
+def test_one_launch_schedule_invariants(layout, R, tile):
+    """The execution order of the one-kernel LAMB / LARS update (host logic): every element of every shard
+    is covered by exactly one item, every item appears once per phase, an item's phase 2 comes after ALL
+    phase-1 items of its tensor (the ratio needs every shard's partial sums, Section 4.1) and, except in
+    the tail of the order, at least 512 entries after the last of them (no CTA waits for a ratio)."""
+    shapes = [(1,), (7,), (3, 3, 16, 32), (64, 128), (0,), (1031,), (4099, 3), (300, 301), (32,), (70001,),
+              (512, 1024), (1024, 2048), (1024,), (9,)]
+    plan = B.Plan(shapes, R, 32, tile, upload=False, layout=layout)
+    order, items = plan.schedule()
+    n = len(items)
+    assert len(order) == 2 * n and B.lib().ws_plan_schedule_bytes(plan.handle) >= 32 * n + 8 * n + 8 * len(shapes)
+    # coverage of the [R][S] layout
+    cover = np.zeros(plan.G, dtype=np.int32)
+    numels = [int(np.prod(s)) for s in shapes]
+    valid = 0
+    for it in items:
+        assert 0 < it.len <= 2048 and it.len % 8 == 0 and it.pos % 8 == 0 and 0 <= it.nvalid <= it.len
+        assert it.nvalid == min(max(numels[it.tensor] - it.tensor_off, 0), it.len)
+        cover[it.shard * plan.S + it.pos: it.shard * plan.S + it.pos + it.len] += 1
+        valid += it.nvalid
+    assert (cover == 1).all() and valid == plan.N
+    # items are numbered tensor by tensor
+    tens = [it.tensor for it in items]
+    assert tens == sorted(tens)
+    # each item once per phase; phase 2 after every phase-1 item of the tensor
+    pos1, pos2 = {}, {}
+    for p, (i, ph) in enumerate(order):
+        d = pos1 if ph == 0 else pos2
+        assert i not in d
+        d[i] = p
+    assert len(pos1) == len(pos2) == n
+    last1 = {}
+    for i, p in pos1.items():
+        last1[tens[i]] = max(last1.get(tens[i], -1), p)
+    early = 0
+    for i, p in pos2.items():
+        assert p > last1[tens[i]]
+        if p - last1[tens[i]] < 512:
+            early += 1
+    # phase-1 items run in item order, so do phase-2 items (tickets are handed out in this order)
+    assert [i for i, ph in order if ph == 0] == list(range(n)) and [i for i, ph in order if ph == 1] == list(range(n))
+    # only the tail (after the last phase-1 entry) may hold phase-2 items that follow their tensor closely
+    end1 = max(pos1.values())
+    assert all(p > end1 for i, p in pos2.items() if p - last1[tens[i]] < 512)
+
+
+def test_one_launch_schedule_on_bert_large_keeps_phase_two_close():
+    """On the BERT-large set (R = 16) the state a phase-2 item reads was written a bounded distance earlier:
+    except for the embedding (larger than L2) and the few tensors whose phase 2 queues behind the
+    embedding's, the phase-1 to phase-2 distance of an item, in bytes of state touched in between, stays
+    below 150 MB."""
+    wl = W.bert_large()
+    plan = B.Plan(wl.shapes, wl.R, 32, upload=False)
+    order, items = plan.schedule()
+    n = len(items)
+    touched = np.cumsum([12 * items[i].len for i, _ in order])       # bytes of state moved up to entry p
+    p1 = np.zeros(n, dtype=np.int64)
+    p2 = np.zeros(n, dtype=np.int64)
+    for p, (i, ph) in enumerate(order):
+        (p1 if ph == 0 else p2)[i] = p
+    dist = touched[p2] - touched[p1]
+    big = np.array([wl.numels[it.tensor] * 12 > 200e6 for it in items])
+    assert np.quantile(dist[~big], 0.98) < 150e6
+    assert np.median(dist[~big]) < 80e6
+    assert plan.workspace_bytes("lamb") <= 4 * 1024 * 1024            # fits the library's static scratch
