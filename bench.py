@@ -88,6 +88,8 @@ def parse_args():
                     help="replicas (default): every rank updates its own independent tensor set, no collective; "
                          "nccl: ONE model over the ranks, NCCL reduce-scatter / all-gather around the single-shard "
                          "kernels; peer: ONE model, one kernel per rank over symmetric-memory tensors")
+    ap.add_argument("--three-launch", action="store_true",
+                    help="LAMB / LARS as three launches (phase 1, combination, phase 2) instead of the one persistent kernel")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-side-rows", action="store_true",
@@ -514,7 +516,7 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
     R, T, N = wl.R, wl.T, wl.N
     # partial sharding (Section 5.2): R gradient copies, but the update is sharded only `shards` ways
     shards = shards or R
-    plan = B.Plan(wl.shapes, shards, align, tile, device=dev, layout=layout)
+    plan = B.Plan(wl.shapes, shards, align, tile, device=dev, layout=layout, one_launch=not args.three_launch)
     if shards != R:
         e2e = False               # the host-buffer entry point takes one gradient arena per shard
     gdt, odt = wl.grad_dtype, wl.out_dtype
@@ -724,9 +726,11 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
     # ---- per-kernel rates and the roofline of the dominant kernel
     peak, peak_src = measured_peak()
     bpp = bytes_per_param(wl)
-    n_upd_launch = {"lamb": 3, "lars": 3, "adafactor": 6}.get(wl.opt, 1)
+    one_kernel = wl.opt in ("lamb", "lars") and plan.sched_buf is not None and R <= 32
+    n_upd_launch = 1 if one_kernel else {"lamb": 3, "lars": 3, "adafactor": 6}.get(wl.opt, 1)
     chunks = -(-T // 1024)
-    upd_name = ("update_kernel" if n_upd_launch == 1 else
+    upd_name = ("two_phase_kernel (phase 1 and phase 2 of every tensor as items of one persistent kernel)" if one_kernel else
+                "update_kernel" if n_upd_launch == 1 else
                 "update_kernel pass 1 + af_moments_kernel + af_factors_kernel + pass 2 + af_finalize_clip_kernel + pass 3"
                 if n_upd_launch == 6 else
                 "update_kernel phase 1 + lamb_finalize_kernel + update_kernel phase 2")

@@ -554,6 +554,104 @@ void wso_sharded_update_map(const wso_hyper *h, int32_t T, const int32_t *tmap, 
     free(part);
 }
 
+/* ------------------------------------------- one replica's share, phase by phase -- */
+
+/* The sharded LAMB / LARS update as ONE replica runs it on real replicas (Section 2.2: after the
+ * reduce-scatter replica r holds the fully reduced gradient of shard r; Section 4.1: every replica
+ * reduces what its shard holds, masking pads by location, and the replicas then combine their
+ * partial results).  These are wso_sharded_update / wso_lars_sharded cut at the two points where
+ * the replicas exchange data; running them for r = 0..R-1 around a sum of the partials over r
+ * (ascending) gives bit for bit the same result.
+ *   gslice : the reduced gradient of shard r, S elements (what the reduce-scatter delivered)
+ *   w, m, v: the replica's S-element shards
+ *   part   : [T][2] this shard's partial sums (sum w^2, sum u^2; LARS: sum w^2, sum g^2)
+ *   u      : S doubles kept between the two phases (LAMB: the step direction; LARS: the scaled gradient) */
+void wso_lamb_shard_partial(const wso_hyper *h, int32_t T, const int64_t *numel, const int64_t *piece,
+                            const int64_t *off, int32_t r, const void *gslice, int32_t g_dtype,
+                            const float *w, float *m, float *v, double *part, double *u) {
+    bias_corr b = bias_of(h);
+    for (int32_t t = 0; t < T; ++t) {
+        double pa = 0.0, pb = 0.0;
+        for (int64_t q = 0; q < piece[t]; ++q) {
+            int64_t j = off[t] + q;
+            if ((int64_t)r * piece[t] + q >= numel[t]) {     /* pad: identity / +0 */
+                m[j] = 0.0f;
+                v[j] = 0.0f;
+                u[j] = 0.0;
+                continue;
+            }
+            double g = load_grad(gslice, g_dtype, j) * h->grad_scale;
+            double wd = (double)w[j], md = (double)m[j], vd = (double)v[j];
+            double dir = adam_moments(h, b, g, &md, &vd);
+            double uu = dir + h->weight_decay * wd;
+            m[j] = (float)md;
+            v[j] = (float)vd;
+            u[j] = uu;
+            pa += wd * wd;
+            pb += uu * uu;
+        }
+        part[2 * t + 0] = pa;
+        part[2 * t + 1] = pb;
+    }
+}
+
+void wso_lars_shard_partial(const wso_hyper *h, int32_t T, const int64_t *numel, const int64_t *piece,
+                            const int64_t *off, int32_t r, const void *gslice, int32_t g_dtype,
+                            const float *w, double *part, double *u) {
+    for (int32_t t = 0; t < T; ++t) {
+        double pa = 0.0, pb = 0.0;
+        for (int64_t q = 0; q < piece[t]; ++q) {
+            int64_t j = off[t] + q;
+            if ((int64_t)r * piece[t] + q >= numel[t]) {
+                u[j] = 0.0;
+                continue;
+            }
+            double g = load_grad(gslice, g_dtype, j) * h->grad_scale;
+            u[j] = g;
+            pa += (double)w[j] * (double)w[j];
+            pb += g * g;
+        }
+        part[2 * t + 0] = pa;
+        part[2 * t + 1] = pb;
+    }
+}
+
+/* The per-tensor ratio from the combined sums: LAMB's trust ratio or LARS's local rate. */
+double wso_norm_ratio(const wso_hyper *h, double a, double b) {
+    if (h->opt == WSO_LARS) return lars_rate(h, a, b);
+    return (a > 0.0 && b > 0.0) ? sqrt(a) / sqrt(b) : 1.0;
+}
+
+/* Phase 2 for shard r with the tensors' ratios; writes the shard's slot of the gathered layout
+ * (S elements of out_dtype) when slot != NULL.  m is read and written by LARS only. */
+void wso_norm_shard_apply(const wso_hyper *h, int32_t T, const int64_t *numel, const int64_t *piece,
+                          const int64_t *off, int64_t S, int32_t r, const double *ratio, const double *u,
+                          float *w, float *m, void *slot, int32_t out_dtype) {
+    for (int32_t t = 0; t < T; ++t)
+        for (int64_t q = 0; q < piece[t]; ++q) {
+            int64_t j = off[t] + q;
+            if ((int64_t)r * piece[t] + q >= numel[t]) {
+                w[j] = 0.0f;
+                if (h->opt == WSO_LARS) m[j] = 0.0f;
+                continue;
+            }
+            double wd = (double)w[j];
+            if (h->opt == WSO_LARS) {
+                double vn = h->momentum * (double)m[j] + h->lr * ratio[t] * (u[j] + h->weight_decay * wd);
+                m[j] = (float)vn;
+                w[j] = (float)(wd - vn);
+            } else {
+                w[j] = (float)(wd - h->lr * ratio[t] * u[j]);
+            }
+        }
+    if (slot) {
+        if (out_dtype == WSO_BF16)
+            for (int64_t j = 0; j < S; ++j) ((uint16_t *)slot)[j] = wso_f32_to_bf16(w[j]);
+        else
+            memcpy(slot, w, sizeof(float) * (size_t)S);
+    }
+}
+
 /* ------------------------------------------------------------- Adafactor -- */
 
 static double af_decay(const wso_hyper *h) { return 1.0 - pow((double)h->step, -h->decay_exponent); }

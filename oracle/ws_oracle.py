@@ -101,6 +101,18 @@ def lib():
         L.wso_shard_reduce.restype = None
         L.wso_shard_reduce.argtypes = [C.c_int32, i64p, i64p, i64p, C.c_int64, C.c_int32,
                                        C.c_int32, vpp, C.c_int32, C.c_double, C.c_void_p]
+        dp = C.POINTER(C.c_double)
+        L.wso_lamb_shard_partial.restype = None
+        L.wso_lamb_shard_partial.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p, C.c_int32, C.c_void_p,
+                                             C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p, dp, dp]
+        L.wso_lars_shard_partial.restype = None
+        L.wso_lars_shard_partial.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p, C.c_int32, C.c_void_p,
+                                             C.c_int32, C.c_void_p, dp, dp]
+        L.wso_norm_ratio.restype = C.c_double
+        L.wso_norm_ratio.argtypes = [C.POINTER(Hyper), C.c_double, C.c_double]
+        L.wso_norm_shard_apply.restype = None
+        L.wso_norm_shard_apply.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p, C.c_int64, C.c_int32, dp, dp,
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]
         L.wso_f32_to_bf16.restype = C.c_uint16
         L.wso_f32_to_bf16.argtypes = [C.c_float]
         L.wso_bf16_to_double.restype = C.c_double
@@ -213,6 +225,47 @@ def sharded_update(h: Hyper, plan: Plan, gpacked: Sequence[np.ndarray], w: np.nd
         rho.ctypes.data_as(C.POINTER(C.c_double)),
         partials.ctypes.data_as(C.POINTER(C.c_double)))
     return gathered, rho, partials
+
+
+def _dp(a: np.ndarray):
+    assert a.dtype == np.float64 and a.flags["C_CONTIGUOUS"]
+    return a.ctypes.data_as(C.POINTER(C.c_double))
+
+
+def norm_shard_partial(h: Hyper, plan: Plan, r: int, gslice: np.ndarray, w: np.ndarray, m: np.ndarray,
+                       v: Optional[np.ndarray]):
+    """Phase 1 of LAMB / LARS as ONE replica runs it: shard r's S-element state and its reduced gradient
+    slice.  LAMB updates m, v in place.  Returns (part[T][2], u[S]): the shard's partial sums and the
+    per-element quantity phase 2 needs (LAMB: the step direction, LARS: the scaled gradient)."""
+    part = np.zeros((plan.T, 2), dtype=np.float64)
+    u = np.zeros(plan.S, dtype=np.float64)
+    if h.opt == LARS:
+        lib().wso_lars_shard_partial(C.byref(h), plan.T, _p(plan.numel), _p(plan.piece), _p(plan.off), r,
+                                     gslice.ctypes.data, _dtype_code(gslice), w.ctypes.data, _dp(part), _dp(u))
+    else:
+        lib().wso_lamb_shard_partial(C.byref(h), plan.T, _p(plan.numel), _p(plan.piece), _p(plan.off), r,
+                                     gslice.ctypes.data, _dtype_code(gslice), w.ctypes.data, m.ctypes.data,
+                                     v.ctypes.data, _dp(part), _dp(u))
+    return part, u
+
+
+def norm_ratio(h: Hyper, a: float, b: float) -> float:
+    """LAMB's trust ratio / LARS's local rate from a tensor's combined sums."""
+    return float(lib().wso_norm_ratio(C.byref(h), float(a), float(b)))
+
+
+def norm_shard_apply(h: Hyper, plan: Plan, r: int, ratio: np.ndarray, u: np.ndarray, w: np.ndarray,
+                     m: Optional[np.ndarray], out_dtype: Optional[int] = None):
+    """Phase 2 for shard r, in place; returns the shard's slot of the gathered layout (or None)."""
+    ratio = np.ascontiguousarray(ratio, dtype=np.float64)
+    slot = None
+    if out_dtype is not None:
+        slot = np.empty(plan.S, dtype=np.uint16 if out_dtype == BF16 else np.float32)
+    lib().wso_norm_shard_apply(C.byref(h), plan.T, _p(plan.numel), _p(plan.piece), _p(plan.off), plan.S, r,
+                               _dp(ratio), _dp(u), w.ctypes.data, m.ctypes.data if m is not None else None,
+                               slot.ctypes.data if slot is not None else None,
+                               out_dtype if out_dtype is not None else F32)
+    return slot
 
 
 def factor_shapes(shapes):

@@ -14,8 +14,11 @@ class Plan:
         self.o = O.Plan(self.numels, R, align_elems)
         self.S, self.G, self.T, self.R = self.o.S, self.o.G, self.o.T, R
 
+        self._u = {}          # shard -> what phase 1 keeps for phase 2 (the kernels recompute or store it)
+
     def workspace_bytes(self, opt):
-        return 0
+        """Stand-in workspace for the norm-based optimizers: double rho[T] | double partials[R][T][2]."""
+        return 8 * (self.T + self.R * 2 * self.T) if opt in ("lamb", "lars") else 0
 
 
 def make_hyper(opt, hyper):
@@ -67,3 +70,70 @@ def ws_shard_update(plan, r, gbufs, w, m, v, hyper, gathered=None, workspace=Non
             slot.copy_(torch.from_numpy(O.f32_to_bf16_bits(wn).view(np.int16)).view(torch.bfloat16))
         else:
             slot.copy_(w)
+
+
+# ---------------------------------------------------------------- LAMB / LARS on CPU ranks ---
+# Phase 1 for the rank's own shard, the exchange of the partial rows, the combination (every rank,
+# same order) and phase 2: the oracle's per-replica phase functions behind the binding's call names.
+def lamb_partials(plan, workspace):
+    """The [R][T * 2] view of the per-shard partial sums (doubles here) inside the stand-in workspace."""
+    return workspace[8 * plan.T:].view(torch.float64).view(plan.R, 2 * plan.T)
+
+
+def lamb_ratios(plan, workspace):
+    return workspace[:8 * plan.T].view(torch.float64)
+
+
+def _partial(plan, r, gbufs, w, m, v, hyper, workspace, slice_mode):
+    assert slice_mode == 1 and len(gbufs) == 1 and 0 <= r < plan.R
+    part, u = O.norm_shard_partial(hyper, plan.o, r, _np(gbufs[0]), _np(w), _np(m) if m is not None else None,
+                                   _np(v) if v is not None else None)
+    plan._u[r] = u
+    lamb_partials(plan, workspace)[r].copy_(torch.from_numpy(part.reshape(-1)))
+
+
+def ws_lamb_partial(plan, r, gbufs, w, m, v, hyper, workspace, slice_mode=0):
+    _partial(plan, r, gbufs, w, m, v, hyper, workspace, slice_mode)
+
+
+def ws_lars_partial(plan, r, gbufs, w, m, hyper, workspace, slice_mode=0):
+    _partial(plan, r, gbufs, w, None, None, hyper, workspace, slice_mode)
+
+
+def _finalize(plan, hyper, workspace):
+    rows = lamb_partials(plan, workspace).numpy().reshape(plan.R, plan.T, 2)
+    tot = np.zeros((plan.T, 2))
+    for r in range(plan.R):                   # ascending r on every rank: identical ratios everywhere
+        tot += rows[r]
+    lamb_ratios(plan, workspace).copy_(torch.tensor([O.norm_ratio(hyper, a, b) for a, b in tot], dtype=torch.float64))
+
+
+def ws_lamb_finalize(plan, workspace, hyper=None):
+    _finalize(plan, O.make_hyper("lamb", dict(lr=0, beta1=0, beta2=0, eps=0, weight_decay=0, momentum=0,
+                                                 grad_scale=1, step=1)), workspace)
+
+
+def ws_lars_finalize(plan, hyper, workspace):
+    _finalize(plan, hyper, workspace)
+
+
+def _apply(plan, r, w, m, hyper, workspace, gathered):
+    out_dt = None
+    if gathered is not None:
+        out_dt = O.BF16 if gathered.dtype == torch.bfloat16 else O.F32
+    slot = O.norm_shard_apply(hyper, plan.o, r, lamb_ratios(plan, workspace).numpy(), plan._u.pop(r), _np(w),
+                              _np(m) if m is not None else None, out_dt)
+    if gathered is not None:
+        dst = gathered[r * plan.S:(r + 1) * plan.S]
+        if gathered.dtype == torch.bfloat16:
+            dst.copy_(torch.from_numpy(slot.view(np.int16)).view(torch.bfloat16))
+        else:
+            dst.copy_(torch.from_numpy(slot))
+
+
+def ws_lamb_apply(plan, r, w, m, v, hyper, workspace, gathered=None):
+    _apply(plan, r, w, None, hyper, workspace, gathered)
+
+
+def ws_lars_apply(plan, r, w, m, hyper, workspace, gathered=None):
+    _apply(plan, r, w, m, hyper, workspace, gathered)

@@ -252,8 +252,9 @@ def test_per_shard_calls_equal_all_shard_launch(opt, R, slice_mode):
 
 @pytest.mark.parametrize("R", [1, 3, 8])
 def test_lamb_shard_by_shard_phases(R):
+    # (the plan carries no one-launch schedule: the all-shard call runs the same three launches)
     wl, w, m, v, g = _model(SHAPES, R, seed=6)
-    plan = B.Plan(SHAPES, R, 32)
+    plan = B.Plan(SHAPES, R, 32, one_launch=False)
     h = B.make_hyper("lamb", _hyper("lamb"))
     pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
     aw, am, av = pw.clone(), pm.clone(), pv.clone()
@@ -668,11 +669,60 @@ def test_lars_matches_oracle_and_fused_equals_unfused(R, gdtype):
         assert torch.equal(a, b)
 
 
+@pytest.mark.parametrize("opt", ["lamb", "lars"])
+@pytest.mark.parametrize("R", [1, 2, 3, 8, 16, 32, 40])
+@pytest.mark.parametrize("gdtype,layout,fused", [(torch.float32, "per_tensor", False), (torch.bfloat16, "per_tensor", True),
+                                                 (torch.float32, "concat", True), (torch.bfloat16, "concat", False)])
+def test_one_launch_update_equals_three_launches(opt, R, gdtype, layout, fused):
+    # The all-shard LAMB / LARS update as ONE persistent kernel (plan with its one-launch schedule) against
+    # the three launches (phase 1, combination, phase 2): same elementwise arithmetic, the norm sums grouped
+    # by 2048-element item instead of by tile, so ratios agree to rounding; the status word stays 0; two
+    # steps in a row (the second finds the first's counters and flags in the workspace).  More than 32
+    # gradient copies (R = 40) take the three launches on both plans.
+    shapes = SHAPES + [(1024, 512), (0,), (70001,)]
+    wl, w, m, v, g = _model(shapes, R, gdtype, seed=R + 31, gstd=1e-3 if opt == "lars" else 1e-2)
+    p1 = B.Plan(shapes, R, 32, layout=layout)
+    p3 = B.Plan(shapes, R, 32, layout=layout, one_launch=False)
+    assert p1.sched_buf is not None and p3.sched_buf is None
+    h = _lars_hyper() if opt == "lars" else _hyper("lamb")
+    has_v = opt == "lamb"
+    bufs = {}
+    for name, plan in (("one", p1), ("three", p3)):
+        pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
+        ws = torch.full((max(32, plan.workspace_bytes(opt)),), 0xA5, dtype=torch.uint8, device=DEV)   # dirty workspace
+        outs = [torch.zeros(n, dtype=torch.bfloat16, device=DEV) for n in wl.numels]
+        gathered = torch.zeros(plan.G, dtype=torch.bfloat16, device=DEV)
+        gt = B.TensorTable(plan, g) if fused else None
+        wt = B.TensorTable(plan, [outs]) if fused else None
+        for step in (10, 11):
+            hy = B.make_hyper(opt, dict(h, step=step))
+            if fused:
+                B.ws_fused_update(plan, -1, gt, pw, pm, pv if has_v else None, hy, wt, ws)
+            else:
+                B.ws_shard_update(plan, -1, pg, pw, pm, pv if has_v else None, hy, gathered, ws)
+        torch.cuda.synchronize()
+        if not fused:
+            B.ws_unpack(plan, gathered, outs)
+        bufs[name] = (pw, pm, pv, outs, B.lamb_ratios(plan, ws).clone(), ws)
+    off = p1.sync_status_offset()
+    assert int(bufs["one"][5][off:off + 4].view(torch.int32).item()) == 0
+    a, b = bufs["one"], bufs["three"]
+    tol = 3e-7
+    assert err(to_np(a[0]), to_np(b[0])) <= tol and err(to_np(a[1]), to_np(b[1])) <= tol
+    if has_v:
+        assert torch.equal(a[2], b[2])
+    ra, rb = a[4].cpu().numpy().astype(np.float64), b[4].cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(ra / rb - 1.0) <= 1e-6)
+    for x, y in zip(a[3], b[3]):
+        assert err(to_np(x.float()), to_np(y.float())) <= TOL_BF16
+    assert _pads_are_zero(O.Plan(wl.numels, R, 32), a[0]) if layout == "per_tensor" else True
+
+
 @pytest.mark.parametrize("R", [1, 3, 8])
 def test_lars_shard_by_shard_phases(R):
     # what R replicas would run (phase 1 per shard, finalize, phase 2 per shard) equals the all-shard call
     wl, w, m, v, g = _model(SHAPES, R, seed=16, gstd=1e-3)
-    plan = B.Plan(SHAPES, R, 32)
+    plan = B.Plan(SHAPES, R, 32, one_launch=False)
     h = B.make_hyper("lars", _lars_hyper())
     pw, pm, _, pg = _pack_all(plan, w, m, v, g)
     aw, am = pw.clone(), pm.clone()

@@ -386,6 +386,41 @@ def test_thread_count_does_not_change_any_bit(opt):
             assert np.asarray(a).tobytes() == np.asarray(b).tobytes()
 
 
+@pytest.mark.parametrize("opt", ["lamb", "lars"])
+@pytest.mark.parametrize("R", [1, 3, 8])
+def test_one_replicas_phases_compose_to_the_sharded_update(opt, R):
+    # Section 4.1: every replica reduces what its shard holds, the partial results are combined, then
+    # every replica applies.  The per-replica phase functions, run for r = 0..R-1 around a sum of the
+    # partials in ascending r, must give bit for bit what the all-shard routine gives (one gradient copy:
+    # the reduce-scatter has already summed the replicas' copies).
+    rng = np.random.default_rng(40 + R)
+    numel = [1, 9, 64, 333, 2048, 5000]
+    hs, _ = _hyper(opt, momentum=0.9, weight_decay=0.01, trust_coeff=0.02, lr=0.5 if opt == "lars" else 1e-3)
+    w, m, v, g = _rand_model(rng, numel, 1)
+    p = O.Plan(numel, R, 8)
+    pw, pm, pv, pg = O.pack(p, w), O.pack(p, m), O.pack(p, v), O.pack(p, g[0])
+    aw, am, av = pw.copy(), pm.copy(), pv.copy()
+    gathered, rho, _ = O.sharded_update(hs, p, [pg], aw, am, av if opt == "lamb" else None, O.BF16)
+    S = p.S
+    parts, us = [], []
+    for r in range(R):
+        sl = slice(r * S, (r + 1) * S)
+        part, u = O.norm_shard_partial(hs, p, r, pg[sl], pw[sl], pm[sl], pv[sl] if opt == "lamb" else None)
+        parts.append(part)
+        us.append(u)
+    tot = np.zeros((p.T, 2))
+    for part in parts:                       # ascending r
+        tot += part
+    ratio = np.array([O.norm_ratio(hs, a, b) for a, b in tot])
+    assert ratio.tobytes() == np.asarray(rho).tobytes()
+    slots = [O.norm_shard_apply(hs, p, r, ratio, us[r], pw[r * S:(r + 1) * S], pm[r * S:(r + 1) * S], O.BF16)
+             for r in range(R)]
+    assert pw.tobytes() == aw.tobytes() and pm.tobytes() == am.tobytes()
+    if opt == "lamb":
+        assert pv.tobytes() == av.tobytes()
+    assert np.concatenate(slots).tobytes() == gathered.tobytes()
+
+
 @pytest.mark.parametrize("R", [1, 3, 8, 64])
 @pytest.mark.parametrize("bf16", [False, True])
 def test_sharded_lamb_equals_unsharded_within_one_ulp(R, bf16):
