@@ -32,6 +32,17 @@ def _inputs(world):
     return wl, w, m, v, g
 
 
+def _hyper_for(opt, world):
+    h = dict(lr=1e-3, beta1=0.9, beta2=0.999, eps=1e-8, weight_decay=0.0, momentum=0.9, grad_scale=1.0 / world, step=3)
+    if opt == "sgdm":
+        h.update(lr=0.1, weight_decay=5e-5)
+    if opt == "lamb":
+        h.update(eps=1e-6, weight_decay=0.01)
+    if opt == "lars":
+        h.update(lr=2.0, weight_decay=5e-5, trust_coeff=0.02)
+    return h
+
+
 def _worker(rank, world, port, opt, out_bf16, out):
     from oracle import ws_oracle as O
     from paper_2004_13336_b200.collective import ShardedUpdate
@@ -39,8 +50,7 @@ def _worker(rank, world, port, opt, out_bf16, out):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
     dist.init_process_group("gloo", rank=rank, world_size=world)
     wl, w, m, v, g = _inputs(world)
-    hyper = dict(lr=1e-3 if opt == "adam" else 0.1, beta1=0.9, beta2=0.999, eps=1e-8,
-                 weight_decay=0.0 if opt == "adam" else 5e-5, momentum=0.9, grad_scale=1.0 / world, step=3)
+    hyper = _hyper_for(opt, world)
     su = ShardedUpdate(SHAPES, opt, hyper, out_dtype=torch.bfloat16 if out_bf16 else torch.float32,
                        device="cpu", ops=_oracle_ops)
     su.load_state(w, m, v)
@@ -48,8 +58,9 @@ def _worker(rank, world, port, opt, out_bf16, out):
     su.step(g[rank], outs)                       # this rank's own gradients only
     m_full = [torch.zeros(n) for n in wl.numels]
     su.gather_slot(su.m, m_full)
+    ratios = _oracle_ops.lamb_ratios(su.plan, su.workspace).numpy().copy() if opt in ("lamb", "lars") else None
     out[rank] = ([o.view(torch.int16).numpy().copy() if out_bf16 else o.numpy().copy() for o in outs],
-                 [x.numpy().copy() for x in m_full])
+                 [x.numpy().copy() for x in m_full], ratios)
     dist.barrier()
     dist.destroy_process_group()
 
@@ -66,8 +77,7 @@ def test_every_rank_ends_with_the_unsharded_result(world, opt, out_bf16):
     # expected: the plain update of whole tensors from the all-reduced gradient (summed in fp32 in
     # rank order, as the collective does for world 2; for world 3 the association may differ by an ulp)
     wl, w, m, v, g = _inputs(world)
-    hyper = dict(lr=1e-3 if opt == "adam" else 0.1, beta1=0.9, beta2=0.999, eps=1e-8,
-                 weight_decay=0.0 if opt == "adam" else 5e-5, momentum=0.9, grad_scale=1.0 / world, step=3)
+    hyper = _hyper_for(opt, world)
     hs = O.make_hyper(opt, hyper)
     for t in range(wl.T):
         gs = g[0][t].clone()
@@ -90,3 +100,41 @@ def test_every_rank_ends_with_the_unsharded_result(world, opt, out_bf16):
     for rank in range(1, world):                 # all ranks hold identical full weights
         for a, b in zip(res[0][0], res[rank][0]):
             np.testing.assert_array_equal(a, b)
+
+
+@pytest.mark.parametrize("world", [2, 3])
+@pytest.mark.parametrize("opt,out_bf16", [("lamb", False), ("lars", True)])
+def test_norm_based_optimizers_exchange_their_partial_sums(world, opt, out_bf16):
+    """LAMB and LARS on CPU ranks (Section 4.1: every replica reduces what its shard holds, then the
+    replicas combine their partial reduce results): phase 1 on the rank's own shard, all-gather of the
+    partial rows, the same combination on every rank, phase 2, all-gather of the weights.  Every rank
+    must end with the unsharded oracle result and all ranks with identical ratios."""
+    from oracle import ws_oracle as O
+    port = _free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_worker, args=(world, port, opt, out_bf16, out), nprocs=world, join=True)
+        res = dict(out)
+    wl, w, m, v, g = _inputs(world)
+    hs = O.make_hyper(opt, _hyper_for(opt, world))
+    for rank in range(1, world):                 # identical weights, slots and ratios everywhere
+        for a, b in zip(res[0][0], res[rank][0]):
+            np.testing.assert_array_equal(a, b)
+        np.testing.assert_array_equal(res[0][2], res[rank][2])
+    for t in range(wl.T):
+        gs = g[0][t].clone()
+        for k in range(1, world):                # the collective's fp32 sum in rank order
+            gs += g[k][t]
+        ew, em = w[t].numpy().copy(), m[t].numpy().copy()
+        ev = v[t].numpy().copy() if opt == "lamb" else None
+        rho = O.update_tensor(hs, [gs.numpy()], ew, em, ev)
+        # (the sharded route sums a tensor's norm shard by shard: the ratio agrees to double rounding, the
+        # weights to one fp32 ulp; with three ranks the collective may also associate the sum differently)
+        assert abs(res[0][2][t] / rho - 1.0) < 1e-6
+        got_w, got_m = res[0][0][t], res[0][1][t]
+        if out_bf16:
+            exp = O.f32_to_bf16_bits(ew)
+            assert (np.abs(got_w.view(np.uint16).astype(np.int64) - exp.astype(np.int64)) <= 1).all()
+        else:
+            np.testing.assert_allclose(got_w, ew, rtol=0, atol=2e-7)
+        np.testing.assert_allclose(got_m, em, rtol=1e-5, atol=1e-9)
