@@ -810,6 +810,101 @@ void wso_adafactor_sharded(const wso_hyper *h, int32_t T, const int64_t *numel, 
     free(u);
 }
 
+/* Sharded Adafactor as ONE replica runs it, stage by stage (wso_adafactor_sharded cut where the
+ * replicas exchange data; for r = 0..R-1 with the sums taken over r in ascending order the result is
+ * bit for bit the same).  gslice / w: shard r's reduced gradient and weights (S elements).
+ *   sums  : adds shard r's partial row / column sums of g^2 + eps1 into acc (laid out like the
+ *           factored state: tensor t at foff[t], rows then columns) and leaves sum w^2 per tensor in
+ *           pw[T]; keeps the scaled gradient in gk[S]
+ *           -> the replicas add their acc arrays (all-reduce) and share their pw rows
+ *   moments: from the combined acc: st = beta state + (1 - beta) acc (doubles, kept for the later
+ *           stages), the fp32 state, and every tensor's sum of row accumulators
+ *   sumsq : u = g / sqrt(V) on shard r, partial sums of u^2 per tensor
+ *           -> the replicas share their rows again
+ *   step  : alpha and the clipping divisor of a tensor from its combined sums
+ *   apply : w' = w - alpha u / clip on shard r */
+void wso_af_shard_sums(const wso_hyper *h, int32_t T, const int64_t *numel, const int64_t *piece,
+                       const int64_t *off, int32_t r, const void *gslice, int32_t g_dtype, const float *w,
+                       const int64_t *rows, const int64_t *cols, const int64_t *foff, double *acc, double *pw,
+                       double *gk) {
+    for (int32_t t = 0; t < T; ++t) {
+        const int64_t n = numel[t], nr = rows[t], nc = cols[t];
+        double sw = 0.0;
+        for (int64_t q = 0; q < piece[t]; ++q) {
+            const int64_t e = (int64_t)r * piece[t] + q, j = off[t] + q;
+            gk[j] = 0.0;
+            if (e >= n) continue;
+            gk[j] = load_grad(gslice, g_dtype, j) * h->grad_scale;
+            const double x = gk[j] * gk[j] + h->eps;
+            if (nc > 0) {
+                acc[foff[t] + e / nc] += x;
+                acc[foff[t] + nr + e % nc] += x;
+            } else {
+                acc[foff[t] + e] += x;
+            }
+            sw += (double)w[j] * (double)w[j];
+        }
+        pw[t] = sw;
+    }
+}
+
+void wso_af_moments(const wso_hyper *h, int32_t T, const int64_t *rows, const int64_t *cols, const int64_t *foff,
+                    const double *acc, float *fstate, double *st, double *sum_r) {
+    const double beta = af_decay(h);
+    for (int32_t t = 0; t < T; ++t) {
+        const int64_t nr = rows[t], nc = cols[t], nstate = nc > 0 ? nr + nc : nr;
+        double s = 0.0;
+        for (int64_t i = 0; i < nstate; ++i) {
+            const double x = beta * (double)fstate[foff[t] + i] + (1.0 - beta) * acc[foff[t] + i];
+            st[foff[t] + i] = x;
+            fstate[foff[t] + i] = (float)x;
+            if (nc > 0 && i < nr) s += x;
+        }
+        sum_r[t] = s;
+    }
+}
+
+void wso_af_shard_sumsq(int32_t T, const int64_t *numel, const int64_t *piece, const int64_t *off, int32_t r,
+                        const int64_t *rows, const int64_t *cols, const int64_t *foff, const double *st,
+                        const double *sum_r, const double *gk, double *u, double *pu) {
+    for (int32_t t = 0; t < T; ++t) {
+        const int64_t n = numel[t], nr = rows[t], nc = cols[t];
+        double p = 0.0;
+        for (int64_t q = 0; q < piece[t]; ++q) {
+            const int64_t e = (int64_t)r * piece[t] + q, j = off[t] + q;
+            u[j] = 0.0;
+            if (e >= n) continue;
+            const double V = nc > 0 ? st[foff[t] + e / nc] * st[foff[t] + nr + e % nc] / sum_r[t] : st[foff[t] + e];
+            u[j] = gk[j] / sqrt(V);
+            p += u[j] * u[j];
+        }
+        pu[t] = p;
+    }
+}
+
+void wso_af_step(const wso_hyper *h, int64_t n, double sw, double su, double *alpha, double *clip) {
+    const double rms_u = n > 0 ? sqrt(su / (double)n) : 0.0;
+    const double rms_w = n > 0 ? sqrt(sw / (double)n) : 0.0;
+    *clip = rms_u / h->clip_threshold > 1.0 ? rms_u / h->clip_threshold : 1.0;
+    *alpha = (h->eps2 > rms_w ? h->eps2 : rms_w) * af_rho(h);
+}
+
+void wso_af_shard_apply(int32_t T, const int64_t *numel, const int64_t *piece, const int64_t *off, int64_t S,
+                        int32_t r, const double *alpha, const double *clip, const double *u, float *w, void *slot,
+                        int32_t out_dtype) {
+    for (int32_t t = 0; t < T; ++t)
+        for (int64_t q = 0; q < piece[t]; ++q) {
+            const int64_t e = (int64_t)r * piece[t] + q, j = off[t] + q;
+            w[j] = e < numel[t] ? (float)((double)w[j] - alpha[t] * (u[j] / clip[t])) : 0.0f;
+        }
+    if (slot) {
+        if (out_dtype == WSO_BF16)
+            for (int64_t j = 0; j < S; ++j) ((uint16_t *)slot)[j] = wso_f32_to_bf16(w[j]);
+        else
+            memcpy(slot, w, sizeof(float) * (size_t)S);
+    }
+}
+
 int32_t wso_num_threads(void) {
 #ifdef _OPENMP
     extern int omp_get_max_threads(void);

@@ -113,6 +113,18 @@ def lib():
         L.wso_norm_shard_apply.restype = None
         L.wso_norm_shard_apply.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p, C.c_int64, C.c_int32, dp, dp,
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32]
+        L.wso_af_shard_sums.restype = None
+        L.wso_af_shard_sums.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p, C.c_int32, C.c_void_p, C.c_int32,
+                                        C.c_void_p, i64p, i64p, i64p, dp, dp, dp]
+        L.wso_af_moments.restype = None
+        L.wso_af_moments.argtypes = [C.POINTER(Hyper), C.c_int32, i64p, i64p, i64p, dp, C.c_void_p, dp, dp]
+        L.wso_af_shard_sumsq.restype = None
+        L.wso_af_shard_sumsq.argtypes = [C.c_int32, i64p, i64p, i64p, C.c_int32, i64p, i64p, i64p, dp, dp, dp, dp, dp]
+        L.wso_af_step.restype = None
+        L.wso_af_step.argtypes = [C.POINTER(Hyper), C.c_int64, C.c_double, C.c_double, dp, dp]
+        L.wso_af_shard_apply.restype = None
+        L.wso_af_shard_apply.argtypes = [C.c_int32, i64p, i64p, i64p, C.c_int64, C.c_int32, dp, dp, dp, C.c_void_p,
+                                         C.c_void_p, C.c_int32]
         L.wso_f32_to_bf16.restype = C.c_uint16
         L.wso_f32_to_bf16.argtypes = [C.c_float]
         L.wso_bf16_to_double.restype = C.c_double
@@ -315,6 +327,64 @@ def adafactor_sharded(h: Hyper, plan: Plan, shapes, gpacked: Sequence[np.ndarray
         w.ctypes.data, fstate.ctypes.data, gathered.ctypes.data if gathered is not None else None,
         out_dtype if out_dtype is not None else F32, info.ctypes.data_as(C.POINTER(C.c_double)))
     return gathered, info
+
+
+class AdafactorReplica:
+    """Adafactor as ONE replica runs it (shard r of a plan), stage by stage; the caller moves the partial
+    results between replicas.  ``acc`` (this replica's row / column sums, F doubles, to be added over the
+    replicas), ``pw`` / ``pu`` (its per-tensor sums of w^2 and u^2)."""
+
+    def __init__(self, h: Hyper, plan: Plan, shapes, r: int):
+        self.h, self.plan, self.r = h, plan, r
+        self.rows, self.cols, self.foff, self.F = factor_shapes(shapes)
+        self.acc = np.zeros(self.F, dtype=np.float64)
+        self.pw = np.zeros(plan.T, dtype=np.float64)
+        self.pu = np.zeros(plan.T, dtype=np.float64)
+        self.gk = np.zeros(plan.S, dtype=np.float64)
+        self.u = np.zeros(plan.S, dtype=np.float64)
+        self.st = np.zeros(self.F, dtype=np.float64)
+        self.sum_r = np.zeros(plan.T, dtype=np.float64)
+
+    def _plan(self):
+        p = self.plan
+        return p.T, _p(p.numel), _p(p.piece), _p(p.off)
+
+    def sums(self, gslice: np.ndarray, w: np.ndarray):
+        T, n, pc, off = self._plan()
+        self.acc[:] = 0.0
+        lib().wso_af_shard_sums(C.byref(self.h), T, n, pc, off, self.r, gslice.ctypes.data, _dtype_code(gslice),
+                                w.ctypes.data, _p(self.rows), _p(self.cols), _p(self.foff), _dp(self.acc), _dp(self.pw),
+                                _dp(self.gk))
+
+    def moments(self, acc_total: np.ndarray, fstate: np.ndarray):
+        acc_total = np.ascontiguousarray(acc_total, dtype=np.float64)
+        lib().wso_af_moments(C.byref(self.h), self.plan.T, _p(self.rows), _p(self.cols), _p(self.foff), _dp(acc_total),
+                             fstate.ctypes.data, _dp(self.st), _dp(self.sum_r))
+
+    def sumsq(self):
+        T, n, pc, off = self._plan()
+        lib().wso_af_shard_sumsq(T, n, pc, off, self.r, _p(self.rows), _p(self.cols), _p(self.foff), _dp(self.st),
+                                 _dp(self.sum_r), _dp(self.gk), _dp(self.u), _dp(self.pu))
+
+    def step_sizes(self, sw_total: np.ndarray, su_total: np.ndarray):
+        alpha, clip = np.zeros(self.plan.T), np.zeros(self.plan.T)
+        a, c = C.c_double(), C.c_double()
+        for t in range(self.plan.T):
+            lib().wso_af_step(C.byref(self.h), int(self.plan.numel[t]), float(sw_total[t]), float(su_total[t]),
+                              C.byref(a), C.byref(c))
+            alpha[t], clip[t] = a.value, c.value
+        return alpha, clip
+
+    def apply(self, alpha: np.ndarray, clip: np.ndarray, w: np.ndarray, out_dtype: Optional[int] = None):
+        T, n, pc, off = self._plan()
+        slot = None
+        if out_dtype is not None:
+            slot = np.empty(self.plan.S, dtype=np.uint16 if out_dtype == BF16 else np.float32)
+        lib().wso_af_shard_apply(T, n, pc, off, self.plan.S, self.r, _dp(np.ascontiguousarray(alpha)),
+                                 _dp(np.ascontiguousarray(clip)), _dp(self.u), w.ctypes.data,
+                                 slot.ctypes.data if slot is not None else None,
+                                 out_dtype if out_dtype is not None else F32)
+        return slot
 
 
 def shard_reduce(plan: Plan, r: int, gpacked: Sequence[np.ndarray], grad_scale: float = 1.0):

@@ -704,8 +704,9 @@ def test_one_launch_update_equals_three_launches(opt, R, gdtype, layout, fused):
         if not fused:
             B.ws_unpack(plan, gathered, outs)
         bufs[name] = (pw, pm, pv, outs, B.lamb_ratios(plan, ws).clone(), ws)
-    off = p1.sync_status_offset()
-    assert int(bufs["one"][5][off:off + 4].view(torch.int32).item()) == 0
+    if R <= 32:                                # (beyond that both plans run the three launches)
+        off = p1.sync_status_offset()
+        assert int(bufs["one"][5][off:off + 4].view(torch.int32).item()) == 0
     a, b = bufs["one"], bufs["three"]
     tol = 3e-7
     assert err(to_np(a[0]), to_np(b[0])) <= tol and err(to_np(a[1]), to_np(b[1])) <= tol

@@ -208,3 +208,50 @@ def test_poisoned_pads_never_leak():
     _, _, dirty = _run_both(7, 32, 2, False, seed=1, out_dtype=O.F32, poison=True)
     for a, b in zip(clean, dirty):
         assert a.tobytes() == b.tobytes()
+
+
+@pytest.mark.parametrize("R", [1, 3, 8])
+def test_one_replicas_stages_compose_to_the_sharded_update(R):
+    """Section 4.1, reduces that collapse a dimension the sharding cuts: every replica reduces what its
+    shard holds and the replicas combine their results.  The per-replica stage functions, run for
+    r = 0..R-1 with the row / column sums and the scalar sums added over r in ascending order, must give
+    bit for bit what the all-shard routine gives (one gradient copy: the reduce-scatter has summed them)."""
+    shapes = [(7,), (5, 9), (64, 33), (3, 3, 4, 8), (1031,), (1, 40), (40, 1)]
+    numel = [int(np.prod(s)) for s in shapes]
+    rng = np.random.default_rng(70 + R)
+    h = dict(lr=1e-2, beta1=0.0, beta2=0.0, eps=1e-30, weight_decay=0.0, momentum=0.0, grad_scale=0.5, step=7,
+             eps2=1e-3, clip_threshold=1.0, decay_exponent=0.8)
+    hs = O.make_hyper("adafactor", h)
+    w = [rng.normal(0, 0.02, n).astype(np.float32) for n in numel]
+    g = [rng.normal(0, 1e-2, n).astype(np.float32) for n in numel]
+    p = O.Plan(numel, R, 8)
+    rows, cols, foff, F = O.factor_shapes(shapes)
+    f0 = rng.uniform(1e-6, 1e-3, F).astype(np.float32)
+    pw, pg = O.pack(p, w), O.pack(p, g)
+    aw, af = pw.copy(), f0.copy()
+    gathered, info = O.adafactor_sharded(hs, p, shapes, [pg], aw, af, O.BF16)
+    S = p.S
+    reps = [O.AdafactorReplica(hs, p, shapes, r) for r in range(R)]
+    for r, rep in enumerate(reps):
+        rep.sums(pg[r * S:(r + 1) * S], pw[r * S:(r + 1) * S])
+    acc, sw = np.zeros(F), np.zeros(p.T)
+    for rep in reps:                           # ascending r
+        acc += rep.acc
+        sw += rep.pw
+    fs = f0.copy()
+    for rep in reps:                           # the small factored state is replicated
+        fr = f0.copy()
+        rep.moments(acc, fr)
+        fs = fr
+        rep.sumsq()
+    su = np.zeros(p.T)
+    for rep in reps:
+        su += rep.pu
+    slots = []
+    for r, rep in enumerate(reps):
+        alpha, clip = rep.step_sizes(sw, su)
+        slots.append(rep.apply(alpha, clip, pw[r * S:(r + 1) * S], O.BF16))
+    assert fs.tobytes() == af.tobytes()
+    assert pw.tobytes() == aw.tobytes()
+    assert np.concatenate(slots).tobytes() == gathered.tobytes()
+    assert alpha.tobytes() == np.ascontiguousarray(info[:, 0]).tobytes()
