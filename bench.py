@@ -89,7 +89,7 @@ def parse_args():
                          "nccl: ONE model over the ranks, NCCL reduce-scatter / all-gather around the single-shard "
                          "kernels; peer: ONE model, one kernel per rank over symmetric-memory tensors")
     ap.add_argument("--three-launch", action="store_true",
-                    help="LAMB / LARS as three launches (phase 1, combination, phase 2) instead of the one persistent kernel")
+                    help="LAMB as three launches (phase 1, combination, phase 2) instead of the one kernel")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-side-rows", action="store_true",
@@ -726,10 +726,10 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
     # ---- per-kernel rates and the roofline of the dominant kernel
     peak, peak_src = measured_peak()
     bpp = bytes_per_param(wl)
-    one_kernel = wl.opt in ("lamb", "lars") and plan.sched_buf is not None and R <= 32
+    one_kernel = wl.opt == "lamb" and plan.sched_buf is not None and 8 <= R <= 32
     n_upd_launch = 1 if one_kernel else {"lamb": 3, "lars": 3, "adafactor": 6}.get(wl.opt, 1)
     chunks = -(-T // 1024)
-    upd_name = ("two_phase_kernel (phase 1 and phase 2 of every tensor as items of one persistent kernel)" if one_kernel else
+    upd_name = ("two_phase_kernel (phase 1 and phase 2 of every tensor as work items of one kernel)" if one_kernel else
                 "update_kernel" if n_upd_launch == 1 else
                 "update_kernel pass 1 + af_moments_kernel + af_factors_kernel + pass 2 + af_finalize_clip_kernel + pass 3"
                 if n_upd_launch == 6 else

@@ -141,28 +141,29 @@ ws_status ws_plan_segments(const ws_plan* plan, const ws_segment** segs, int32_t
 size_t ws_plan_device_bytes(const ws_plan* plan);
 ws_status ws_plan_upload(ws_plan* plan, void* dev_buf, size_t bytes, void* stream);
 
-/* One-launch schedule (optional).  The norm-based optimizers (WS_LAMB, WS_LARS) need every shard's
- * partial norm sums of a tensor before any shard can apply the step (Section 4.1), so their
- * all-shard update is phase 1, a combination step, phase 2.  As three launches, phase 2 reads the
- * weight and the new moments from DRAM again.  A plan whose schedule has been uploaded runs the same
- * update as ONE persistent kernel instead: the two phases of every tensor are work items ordered so
- * that a tensor's phase 2 follows its phase 1 closely, while other tensors' phase 1 streams from
- * DRAM, and phase 2 finds its operands in L2 - every operand crosses HBM once, as the update of
- * Section 2.2 counts them.  Results: the same as the three-launch form up to the order of the norm
- * sums (the ratios agree to rounding; they are bit-stable from run to run).
+/* One-launch schedule (optional).  The norm-based optimizers need every shard's partial norm sums
+ * of a tensor before any shard can apply the step (Section 4.1), so their all-shard update is
+ * phase 1, a combination step, phase 2.  As three launches, phase 2 reads the weight and the new
+ * moments from DRAM again.  A plan whose schedule has been uploaded runs WS_LAMB's all-shard update
+ * as ONE kernel instead: the two phases of every tensor are work items (runs of up to 8192 shard
+ * positions) ordered so that a tensor's phase 2 follows its phase 1 at a short distance, while other
+ * tensors' phase 1 streams from DRAM, and phase 2 finds part of its operands in L2 (toward the
+ * update of Section 2.2, where every operand crosses HBM once).  Results: the same as the
+ * three-launch form up to the order of the norm sums (the ratios agree to rounding; they are
+ * bit-stable from run to run).
  *   ws_plan_schedule_bytes   device bytes of the schedule (0: this plan has none - more than
  *                            65535 shards or 2^30 work items)
  *   ws_plan_upload_schedule  builds the schedule on first use and copies it into the caller's
  *                            buffer (16-byte aligned, alive while the plan is in use) with
  *                            cudaMemcpyAsync on `stream`; call once, before the plan is shared
  *                            between threads
- * Afterwards ws_shard_update / ws_fused_update with r == -1 and WS_LAMB or WS_LARS (and
- * ws_lamb_update_static_scratch) take the one-kernel route when there are at most 32 gradient
- * copies; the shard-by-shard calls are unchanged.  The kernel's waits (a phase-2 item waits for
- * its tensor's ratio) are bounded: if one ever runs out, the kernel stops, leaves the update
- * incomplete and sets the 32-bit status word inside the workspace (ws_workspace_sync_status gives
- * its byte offset; 0 = completed) - a caller that wants to detect this reads the word after
- * synchronising the stream.
+ * Afterwards ws_shard_update / ws_fused_update with r == -1 and WS_LAMB (and
+ * ws_lamb_update_static_scratch) take the one-kernel route when there are 8 to 32 gradient copies -
+ * where it measured faster on a B200; other cases, WS_LARS and the shard-by-shard calls run as
+ * before.  The kernel's waits (a phase-2 item waits for its tensor's ratio) are bounded: if one
+ * ever runs out, the kernel leaves the update incomplete and sets the 32-bit status word inside
+ * the workspace (ws_workspace_sync_status gives its byte offset; 0 = completed) - a caller that
+ * wants to detect this reads the word after synchronising the stream.
  * ws_plan_schedule_view / ws_plan_schedule_item expose the order for inspection (host only):
  * entry i of `order` is item index * 2 + phase (0: phase 1, 1: phase 2). */
 size_t ws_plan_schedule_bytes(const ws_plan* plan);

@@ -15,6 +15,7 @@ extern "C" ws_status ws_plan_arena_offsets(const ws_plan* p, const int64_t** off
 extern "C" ws_status ws_step_host(const ws_plan* p, const ws_host_io* io, const ws_state* state,
                                   const ws_hyper* hyper, const ws_out* out, void* workspace,
                                   size_t workspace_bytes, void* stream) {
+    WsRange range_("ws_step_host");
     if (!p || !io || !state || !hyper) return WS_ERR_INVALID_ARG;
     if (!io->host_grads || !io->dev_grad_arena || !io->dev_packed_grads || !io->dev_weight_arena ||
         !io->host_weights)

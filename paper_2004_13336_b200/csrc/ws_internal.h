@@ -2,11 +2,21 @@
 // Nothing here is part of the public ABI (see include/ws.h).
 #pragma once
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 #include <stdint.h>
 
 #include <vector>
 
 #include "ws.h"
+
+// A named range around an entry point for timeline tools (NVTX; costs a few nanoseconds when no tool
+// is attached).  Covers the host side of the call: argument checks and launches.
+struct WsRange {
+    explicit WsRange(const char* name) { nvtxRangePushA(name); }
+    ~WsRange() { nvtxRangePop(); }
+    WsRange(const WsRange&) = delete;
+    WsRange& operator=(const WsRange&) = delete;
+};
 
 // One work tile: a run of at most `tile_elems` consecutive shard positions that
 // lies inside one tensor's piece.  A tile carries everything a kernel needs to
@@ -60,7 +70,7 @@ struct WsAfChunk {
 // persistent kernel.  A work item is a run of at most kWsItemElems consecutive shard positions inside
 // one tile; every item appears twice in the schedule, once for phase 1 (reduce, moments, partial
 // norm sums) and once for phase 2 (apply the step with the tensor's ratio).
-constexpr int kWsItemElems = 2048;
+constexpr int kWsItemElems = 8192;
 struct __align__(16) WsItem {
     long long pos;        // start inside the shard, multiple of 8
     long long toff;       // element index of the first element inside tensor `seg`
@@ -123,10 +133,10 @@ struct WsLambWs {
     // ticket counter and the status word (sync_bytes from `count` on are cleared before every launch)
     float2* ipart;     // [n_items]
     int* count;        // [T]
-    int* flag;         // [T]
+    unsigned long long* flag;   // [T] ready words
     unsigned long long* ticket;
     int* status;
-    size_t sync_bytes;
+    size_t sync_bytes; // from count on
     size_t bytes;      // through the one-launch scratch: what LAMB needs
     float* ghat;       // LARS only: [R][S] summed gradients, 256-byte aligned after the partials
     size_t bytes_lars; // through ghat: what LARS needs

@@ -282,17 +282,8 @@ struct ItemCtx {
     bool keep;           // HINT only: the state this item touches is read again soon (keep it in L2)
 };
 
-// CTA-wide barrier of the kBlock worker threads: the whole CTA, or (NAMED) the workers of a CTA that
-// also runs a scheduling warp.
-template <bool NAMED>
-__device__ __forceinline__ void worker_sync() {
-    if constexpr (NAMED) asm volatile("bar.sync 1, %0;" :: "n"(kBlock) : "memory");
-    else __syncthreads();
-}
-
-// Sums two values over the kBlock workers at once (one pair of barriers for both); the totals are
-// valid in thread 0.  The order of the additions is fixed, so the result is run-to-run bit-stable.
-template <bool NAMED>
+// Sums two values over the CTA at once (one pair of barriers for both); the totals are valid in
+// thread 0.  The order of the additions is fixed, so the result is run-to-run bit-stable.
 __device__ __forceinline__ float2 block_sum2(float x, float y, float2* smem /* kBlock/32 entries */) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
@@ -300,9 +291,9 @@ __device__ __forceinline__ float2 block_sum2(float x, float y, float2* smem /* k
         y += __shfl_xor_sync(0xffffffffu, y, o);
     }
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    worker_sync<NAMED>();
+    __syncthreads();
     if (lane == 0) smem[warp] = make_float2(x, y);
-    worker_sync<NAMED>();
+    __syncthreads();
     float2 t = make_float2(0.f, 0.f);
     if (threadIdx.x < 32) {
         if (lane < kBlock / 32) t = smem[lane];
@@ -361,11 +352,11 @@ __device__ __forceinline__ Fv<VEC> load_f32_partial(const float* p, int n) {
 // weight tensors, so no packed gradient buffer and no gathered buffer exist.  With
 // OUT == O_F32M the fp32 weight tensors are the master copy themselves: the weight is read
 // from its tensor and written back there, and no sharded copy of w exists.
-// NAMED: the kBlock workers are part of a larger CTA (barriers by name).  HINT: see ItemCtx::keep.
+// HINT: see ItemCtx::keep.
 // sgp: this item's R gradient tensor pointers (FUSED), swp: its weight tensor pointers when the
 // result goes to several weight lists, wt: its first weight tensor; red: kBlock/32 float2 of
 // shared memory.
-template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED, bool NAMED, bool HINT>
+template <int OPT, bool GBF, int OUT, int VEC, int U, int RB, int NP, bool FUSED, bool HINT>
 __device__ __forceinline__ void process_item(const UpdParams& P, const GradPtrs<NP>& gp, const ItemCtx& it,
                                              const void* const* sgp, void* const* swp, char* wt, float lr_rho,
                                              float2* red) {
@@ -700,7 +691,7 @@ __device__ __forceinline__ void process_item(const UpdParams& P, const GradPtrs<
     }
     if (leaves_partials(OPT)) {
         // (Adafactor's passes leave one sum each)
-        const float2 ab = block_sum2<NAMED>(sw, su, red);
+        const float2 ab = block_sum2(sw, su, red);
         if (threadIdx.x == 0) *it.partial = make_float2(ab.x, ab.y);   // (Adafactor's pass 1: y = 0, pass 2 adds its sum there)
     }
 }
@@ -717,14 +708,14 @@ struct OneLaunch {
     int T;
     float2* ipart;               // [items] partial norm sums of every item's phase 1
     int* count;                  // [T] finished phase-1 items per tensor        (cleared before the launch)
-    int* flag;                   // [T] 1 once the tensor's ratio is published    (cleared before the launch)
+    unsigned long long* flag;    // [T] (ratio bits << 32) | 1 once the ratio is known (cleared before the launch)
     unsigned long long* ticket;  // next schedule entry to hand out              (cleared before the launch)
     int* status;                 // 0, or 1 after a wait ran out                  (cleared before the launch)
     float* rho;                  // [T] ratios
     double* norms;               // [T][2]
     double eta, beta;            // LARS: trust coefficient and weight decay
 };
-bool one_launch_supports(int R);
+bool one_launch_supports(int pair, int R);
 // pair 0: LAMB, 1: LARS.  P carries the arguments of both phases (gradient sources, state, outputs).
 ws_status launch_one_launch(int pair, bool gbf, int out, bool fused, bool wide, const UpdParams& P,
                             const void* const* gptrs, const OneLaunch& Q, cudaStream_t st);

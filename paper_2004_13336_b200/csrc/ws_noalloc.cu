@@ -52,6 +52,7 @@ extern "C" size_t ws_static_scratch_bytes(void) { return kStaticScratchBytes; }
 
 extern "C" ws_status ws_lamb_update_static_scratch(const ws_plan* plan, const ws_grads* grads, const ws_state* state,
                                                    const ws_hyper* hyper, const ws_out* out, void* stream) {
+    WsRange range_("ws_lamb_update_static_scratch");
     if (!plan || !hyper) return WS_ERR_INVALID_ARG;
     if (hyper->opt != WS_LAMB) return WS_ERR_INVALID_ARG;
     const size_t need = ws_workspace_bytes(plan, WS_LAMB);

@@ -218,15 +218,18 @@ ws_status run(const ws_plan* p, void* const* tensor_ptrs, ws_dtype dtype, void* 
 
 extern "C" ws_status ws_pack(const ws_plan* plan, const void* const* tensor_ptrs, ws_dtype dtype, void* flat,
                              void* stream) {
+    WsRange range_("ws_pack");
     return run<true>(plan, (void* const*)tensor_ptrs, dtype, flat, stream);
 }
 
 extern "C" ws_status ws_unpack(const ws_plan* plan, const void* flat, ws_dtype dtype, void* const* tensor_ptrs,
                                void* stream) {
+    WsRange range_("ws_unpack");
     return run<false>(plan, tensor_ptrs, dtype, (void*)flat, stream);
 }
 
 extern "C" ws_status ws_pack_sets(const ws_plan* p, const ws_tensor_table* table, void* const* flats, void* stream) {
+    WsRange range_("ws_pack_sets");
     if (!p || !table || !table->dev || !flats) return WS_ERR_INVALID_ARG;
     if (!p->d_tiles) return WS_ERR_NOT_UPLOADED;
     if (table->T != p->T || table->nsets < 1 || table->nsets > kPtrChunk) return WS_ERR_INVALID_ARG;

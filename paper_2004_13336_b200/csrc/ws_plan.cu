@@ -325,11 +325,11 @@ WsLambWs ws_lamb_layout(const ws_plan* p, void* workspace) {
     o = round16(o + sizeof(float2) * (size_t)(p->layout == WS_LAYOUT_CONCAT ? 1 : p->R) * (size_t)p->ntiles);
     L.ipart = (float2*)(b + o);
     o = round16(o + sizeof(float2) * (size_t)p->n_items);
-    L.count = (int*)(b + o);
     const size_t sync0 = o;
-    o += sizeof(int) * (size_t)p->T;
-    L.flag = (int*)(b + o);
+    L.count = (int*)(b + o);
     o = (o + sizeof(int) * (size_t)p->T + 7) & ~(size_t)7;
+    L.flag = (unsigned long long*)(b + o);
+    o += sizeof(unsigned long long) * (size_t)p->T;
     L.ticket = (unsigned long long*)(b + o);
     o += sizeof(unsigned long long);
     L.status = (int*)(b + o);
@@ -388,8 +388,7 @@ extern "C" size_t ws_workspace_bytes(const ws_plan* p, ws_opt opt) {
 // items are waiting (a tensor larger than L2 has just finished) they run first.
 namespace {
 constexpr long long kGroupBytes = 6LL << 20;    // state bytes (12 per element) that close a group
-constexpr long long kKeepLo = 16LL << 20;       // groups between these sizes ask L2 to keep their lines;
-constexpr long long kKeepHi = 80LL << 20;       //   smaller ones stay resident anyway, larger ones cannot
+constexpr long long kKeepHi = 200LL << 20;      // larger groups cannot stay in L2: their state is streamed
 constexpr int kLag = 512;
 
 void ws_build_schedule(ws_plan* p) {
@@ -437,7 +436,7 @@ void ws_build_schedule(ws_plan* p) {
                 const int gend = p->itemsegs[t].first + p->itemsegs[t].count;
                 if (gend > gfirst) {
                     groups.push_back(Group{gfirst, gend});
-                    const unsigned keep = (acc > kKeepLo && acc < kKeepHi) ? 1u : 0u;
+                    const unsigned keep = acc < kKeepHi ? 1u : 0u;
                     for (int i = gfirst; i < gend; ++i) p->items[i].flags = keep;
                 }
                 gfirst = gend;

@@ -83,7 +83,7 @@ __global__ void __launch_bounds__(kBlock, ((VEC == 8 && GBF && !FUSED) || RB > 8
         float lr_rho = 0.f;
         if (OPT == K_LAMB2 || OPT == K_LARS2) lr_rho = P.c.lr * P.rho[tl.seg];
         if (OPT == K_AF3) lr_rho = P.rho[tl.seg];         // alpha_t / max(1, RMS(U_t)/d)
-        process_item<OPT, GBF, OUT, VEC, U, RB, NP, FUSED, false, false>(P, gp, it, sgp, swp, wt, lr_rho, red);
+        process_item<OPT, GBF, OUT, VEC, U, RB, NP, FUSED, false>(P, gp, it, sgp, swp, wt, lr_rho, red);
     }
 }
 
@@ -543,6 +543,7 @@ ws_status check_ws(const ws_plan* p, void* workspace, size_t bytes, ws_opt opt =
 
 extern "C" ws_status ws_lamb_partial(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_state* state,
                                      const ws_hyper* hyper, void* workspace, size_t workspace_bytes, void* stream) {
+    WsRange range_("ws_lamb_partial");
     if (!hyper || hyper->opt != WS_LAMB) return WS_ERR_INVALID_ARG;
     UpdParams P;
     int ok;
@@ -557,6 +558,7 @@ extern "C" ws_status ws_lamb_partial(const ws_plan* plan, int32_t r, const ws_gr
 }
 
 extern "C" ws_status ws_lamb_finalize(const ws_plan* plan, void* workspace, size_t workspace_bytes, void* stream) {
+    WsRange range_("ws_lamb_finalize");
     if (!plan) return WS_ERR_INVALID_ARG;
     if (!plan->d_tiles) return WS_ERR_NOT_UPLOADED;
     ws_status s = check_ws(plan, workspace, workspace_bytes);
@@ -569,6 +571,7 @@ extern "C" ws_status ws_lamb_finalize(const ws_plan* plan, void* workspace, size
 
 extern "C" ws_status ws_lamb_apply(const ws_plan* plan, int32_t r, const ws_state* state, const ws_hyper* hyper,
                                    const ws_out* out, void* workspace, size_t workspace_bytes, void* stream) {
+    WsRange range_("ws_lamb_apply");
     if (!hyper || hyper->opt != WS_LAMB) return WS_ERR_INVALID_ARG;
     UpdParams P;
     int ok;
@@ -582,6 +585,7 @@ extern "C" ws_status ws_lamb_apply(const ws_plan* plan, int32_t r, const ws_stat
 
 extern "C" ws_status ws_lars_partial(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_state* state,
                                      const ws_hyper* hyper, void* workspace, size_t workspace_bytes, void* stream) {
+    WsRange range_("ws_lars_partial");
     if (!hyper || hyper->opt != WS_LARS) return WS_ERR_INVALID_ARG;
     UpdParams P;
     int ok;
@@ -599,6 +603,7 @@ extern "C" ws_status ws_lars_partial(const ws_plan* plan, int32_t r, const ws_gr
 
 extern "C" ws_status ws_lars_finalize(const ws_plan* plan, const ws_hyper* hyper, void* workspace,
                                       size_t workspace_bytes, void* stream) {
+    WsRange range_("ws_lars_finalize");
     if (!plan || !hyper || hyper->opt != WS_LARS) return WS_ERR_INVALID_ARG;
     if (!plan->d_tiles) return WS_ERR_NOT_UPLOADED;
     ws_status s = check_ws(plan, workspace, workspace_bytes, WS_LARS);
@@ -612,6 +617,7 @@ extern "C" ws_status ws_lars_finalize(const ws_plan* plan, const ws_hyper* hyper
 
 extern "C" ws_status ws_lars_apply(const ws_plan* plan, int32_t r, const ws_state* state, const ws_hyper* hyper,
                                    const ws_out* out, void* workspace, size_t workspace_bytes, void* stream) {
+    WsRange range_("ws_lars_apply");
     if (!hyper || hyper->opt != WS_LARS) return WS_ERR_INVALID_ARG;
     UpdParams P;
     int ok;
@@ -641,7 +647,7 @@ ws_status try_one_launch(const ws_plan* plan, int pair, const ws_grads* grads, c
     if (!plan || !plan->d_sched) return WS_OK;
     const bool fused = gtab != nullptr;
     const int copies = fused ? gtab->nsets : (grads ? grads->R : 0);
-    if (!one_launch_supports(copies)) return WS_OK;
+    if (!one_launch_supports(pair, copies)) return WS_OK;
     UpdParams P;
     int out_kind;
     bool gbf;
@@ -687,7 +693,7 @@ ws_status try_one_launch(const ws_plan* plan, int pair, const ws_grads* grads, c
     Q.norms = L.norms;
     Q.eta = hyper->trust_coeff;
     Q.beta = hyper->weight_decay;
-    cudaError_t e = cudaMemsetAsync(L.count, 0, L.sync_bytes, st);     // counters, flags, ticket, status
+    cudaError_t e = cudaMemsetAsync(L.count, 0, L.sync_bytes, st);     // counters, ready words, ticket, status
     if (e != cudaSuccess) return ws_cuda_fail(e, "one-launch update (clear counters)");
     s = launch_one_launch(pair, gbf, out_kind, fused, wide, P, fused ? nullptr : gp.data(), Q, st);
     if (s == WS_OK) done = true;
@@ -711,6 +717,7 @@ ws_status ws_lamb_check_apply_args(const ws_plan* plan, const ws_state* state, c
 extern "C" ws_status ws_shard_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const ws_state* state,
                                      const ws_hyper* hyper, const ws_out* out, void* workspace,
                                      size_t workspace_bytes, void* stream) {
+    WsRange range_("ws_shard_update");
     if (!hyper) return WS_ERR_INVALID_ARG;
     if (hyper->opt == WS_ADAFACTOR)
         return af_update(plan, r, grads, nullptr, state, hyper, out, nullptr, workspace, workspace_bytes, (cudaStream_t)stream);
@@ -931,6 +938,7 @@ ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const
 extern "C" ws_status ws_adafactor_stage(const ws_plan* plan, ws_af_stage stage, int32_t r, const ws_grads* grads,
                                         const ws_state* state, const ws_hyper* hyper, const ws_out* out,
                                         void* workspace, size_t workspace_bytes, void* stream) {
+    WsRange range_("ws_adafactor_stage");
     return af_stage(plan, (int)stage, r, grads, nullptr, state, hyper, out, nullptr, workspace, workspace_bytes,
                     (cudaStream_t)stream);
 }
@@ -938,6 +946,7 @@ extern "C" ws_status ws_adafactor_stage(const ws_plan* plan, ws_af_stage stage, 
 extern "C" ws_status ws_fused_update(const ws_plan* plan, int32_t r, const ws_tensor_table* grads, const ws_state* state,
                                      const ws_hyper* hyper, const ws_tensor_table* weights, void* workspace,
                                      size_t workspace_bytes, void* stream) {
+    WsRange range_("ws_fused_update");
     if (!plan || !grads || !weights || !hyper || !state) return WS_ERR_INVALID_ARG;
     if (!grads->dev || !weights->dev) return WS_ERR_INVALID_ARG;
     if (grads->T != plan->T || weights->T != plan->T || grads->nsets < 1 || weights->nsets < 1) return WS_ERR_INVALID_ARG;

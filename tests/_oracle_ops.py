@@ -10,6 +10,8 @@ from oracle import ws_oracle as O
 
 class Plan:
     def __init__(self, shapes, R, align_elems=32, tile_elems=0, device=None, upload=True, layout="per_tensor"):
+        self.shapes = [tuple(int(d) for d in s) for s in shapes]
+        self.factored_elems = int(O.factor_shapes(self.shapes)[3])
         self.numels = [int(np.prod(s)) for s in shapes]
         self.o = O.Plan(self.numels, R, align_elems)
         self.S, self.G, self.T, self.R = self.o.S, self.o.G, self.o.T, R
@@ -18,6 +20,8 @@ class Plan:
 
     def workspace_bytes(self, opt):
         """Stand-in workspace for the norm-based optimizers: double rho[T] | double partials[R][T][2]."""
+        if opt == "adafactor":               # ... followed by double acc[F], this step's row / column sums
+            return 8 * (self.T + self.R * 2 * self.T + self.factored_elems)
         return 8 * (self.T + self.R * 2 * self.T) if opt in ("lamb", "lars") else 0
 
 
@@ -77,7 +81,7 @@ def ws_shard_update(plan, r, gbufs, w, m, v, hyper, gathered=None, workspace=Non
 # same order) and phase 2: the oracle's per-replica phase functions behind the binding's call names.
 def lamb_partials(plan, workspace):
     """The [R][T * 2] view of the per-shard partial sums (doubles here) inside the stand-in workspace."""
-    return workspace[8 * plan.T:].view(torch.float64).view(plan.R, 2 * plan.T)
+    return workspace[8 * plan.T: 8 * (plan.T + plan.R * 2 * plan.T)].view(torch.float64).view(plan.R, 2 * plan.T)
 
 
 def lamb_ratios(plan, workspace):
@@ -137,3 +141,49 @@ def ws_lamb_apply(plan, r, w, m, v, hyper, workspace, gathered=None):
 
 def ws_lars_apply(plan, r, w, m, hyper, workspace, gathered=None):
     _apply(plan, r, w, m, hyper, workspace, gathered)
+
+
+# ------------------------------------------------------------------ Adafactor on CPU ranks ---
+AF_BEGIN, AF_SUMS, AF_MOMENTS, AF_SUMSQ, AF_CLIP, AF_APPLY = range(6)
+
+
+def adafactor_sums(plan, workspace):
+    """This step's row / column sums (the all-reduce operand between AF_SUMS and AF_MOMENTS)."""
+    return workspace[8 * (plan.T + plan.R * 2 * plan.T):].view(torch.float64)
+
+
+def ws_adafactor_stage(plan, stage, r, hyper, workspace, gbufs=None, w=None, fstate=None, gathered=None, slice_mode=0):
+    """One stage for the rank's own shard (or a replicated stage, r = -1): the oracle's per-replica stage
+    functions behind the binding's call."""
+    rows = lamb_partials(plan, workspace)
+    if stage == AF_BEGIN:
+        adafactor_sums(plan, workspace).zero_()
+    elif stage == AF_SUMS:
+        assert slice_mode == 1 and len(gbufs) == 1 and 0 <= r < plan.R
+        rep = O.AdafactorReplica(hyper, plan.o, plan.shapes, r)
+        rep.sums(_np(gbufs[0]), _np(w))
+        adafactor_sums(plan, workspace).copy_(torch.from_numpy(rep.acc))
+        rows[r][0::2] = torch.from_numpy(rep.pw)
+        plan._af = rep
+    elif stage == AF_MOMENTS:
+        plan._af.moments(adafactor_sums(plan, workspace).numpy(), _np(fstate))
+    elif stage == AF_SUMSQ:
+        plan._af.sumsq()
+        rows[r][1::2] = torch.from_numpy(plan._af.pu)
+    elif stage == AF_CLIP:
+        sw, su = np.zeros(plan.T), np.zeros(plan.T)
+        for k in range(plan.R):                       # ascending shard order on every rank
+            sw += rows[k][0::2].numpy()
+            su += rows[k][1::2].numpy()
+        plan._af_step = plan._af.step_sizes(sw, su)
+    elif stage == AF_APPLY:
+        out_dt = None if gathered is None else (O.BF16 if gathered.dtype == torch.bfloat16 else O.F32)
+        slot = plan._af.apply(plan._af_step[0], plan._af_step[1], _np(w), out_dt)
+        if gathered is not None:
+            dst = gathered[r * plan.S:(r + 1) * plan.S]
+            if gathered.dtype == torch.bfloat16:
+                dst.copy_(torch.from_numpy(slot.view(np.int16)).view(torch.bfloat16))
+            else:
+                dst.copy_(torch.from_numpy(slot))
+    else:
+        raise ValueError(stage)

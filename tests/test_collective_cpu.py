@@ -40,7 +40,14 @@ def _hyper_for(opt, world):
         h.update(eps=1e-6, weight_decay=0.01)
     if opt == "lars":
         h.update(lr=2.0, weight_decay=5e-5, trust_coeff=0.02)
+    if opt == "adafactor":
+        h.update(lr=1e-2, beta1=0.0, beta2=0.0, eps=1e-30, eps2=1e-3, clip_threshold=1.0, decay_exponent=0.8)
     return h
+
+
+def _fstate0(n):
+    gen = torch.Generator().manual_seed(5)
+    return torch.rand(n, generator=gen) * 1e-3 + 1e-6
 
 
 def _worker(rank, world, port, opt, out_bf16, out):
@@ -54,13 +61,17 @@ def _worker(rank, world, port, opt, out_bf16, out):
     su = ShardedUpdate(SHAPES, opt, hyper, out_dtype=torch.bfloat16 if out_bf16 else torch.float32,
                        device="cpu", ops=_oracle_ops)
     su.load_state(w, m, v)
+    if opt == "adafactor":
+        su.fstate.copy_(_fstate0(su.plan.factored_elems))
     outs = [torch.zeros(n, dtype=su.gathered.dtype) for n in wl.numels]
     su.step(g[rank], outs)                       # this rank's own gradients only
     m_full = [torch.zeros(n) for n in wl.numels]
     su.gather_slot(su.m, m_full)
+    if opt == "adafactor":
+        m_full = [su.fstate.numpy().copy()]      # the (replicated) factored state instead of a momentum
     ratios = _oracle_ops.lamb_ratios(su.plan, su.workspace).numpy().copy() if opt in ("lamb", "lars") else None
     out[rank] = ([o.view(torch.int16).numpy().copy() if out_bf16 else o.numpy().copy() for o in outs],
-                 [x.numpy().copy() for x in m_full], ratios)
+                 [np.asarray(x).copy() for x in m_full], ratios)
     dist.barrier()
     dist.destroy_process_group()
 
@@ -138,3 +149,35 @@ def test_norm_based_optimizers_exchange_their_partial_sums(world, opt, out_bf16)
         else:
             np.testing.assert_allclose(got_w, ew, rtol=0, atol=2e-7)
         np.testing.assert_allclose(got_m, em, rtol=1e-5, atol=1e-9)
+
+
+@pytest.mark.parametrize("world", [2, 3])
+def test_adafactor_combines_row_and_column_sums_across_ranks(world):
+    """Adafactor on CPU ranks (Section 4.1: a reduce whose collapsed dimension the sharding cuts - every
+    replica reduces what its shard holds, then the replicas combine their results with an all-reduce):
+    the stages of one replica around the all-reduce of the row / column sums and the exchange of the
+    scalar partial sums.  Every rank must end with the unsharded oracle result and the same factored state."""
+    from oracle import ws_oracle as O
+    port = _free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_worker, args=(world, port, "adafactor", False, out), nprocs=world, join=True)
+        res = dict(out)
+    wl, w, m, v, g = _inputs(world)
+    hs = O.make_hyper("adafactor", _hyper_for("adafactor", world))
+    for rank in range(1, world):
+        for a, b in zip(res[0][0], res[rank][0]):
+            np.testing.assert_array_equal(a, b)
+        np.testing.assert_array_equal(res[0][1][0], res[rank][1][0])
+    rows, cols, foff, F = O.factor_shapes(SHAPES)
+    f = _fstate0(F).numpy().copy()
+    for t in range(wl.T):
+        gs = g[0][t].clone()
+        for k in range(1, world):
+            gs += g[k][t]
+        ew = w[t].numpy().copy().reshape(SHAPES[t])
+        vr = f[foff[t]:foff[t] + rows[t]]
+        vc = f[foff[t] + rows[t]:foff[t] + rows[t] + cols[t]] if cols[t] else None
+        O.adafactor_tensor(hs, [gs.numpy()], ew, vr, vc)
+        np.testing.assert_allclose(res[0][0][t], ew.ravel(), rtol=0, atol=2e-7)
+    np.testing.assert_allclose(res[0][1][0], f, rtol=2e-7, atol=0)

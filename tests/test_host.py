@@ -193,7 +193,7 @@ def test_one_launch_schedule_invariants(layout, R, tile):
     numels = [int(np.prod(s)) for s in shapes]
     valid = 0
     for it in items:
-        assert 0 < it.len <= 2048 and it.len % 8 == 0 and it.pos % 8 == 0 and 0 <= it.nvalid <= it.len
+        assert 0 < it.len <= 8192 and it.len % 8 == 0 and it.pos % 8 == 0 and 0 <= it.nvalid <= it.len
         assert it.nvalid == min(max(numels[it.tensor] - it.tensor_off, 0), it.len)
         cover[it.shard * plan.S + it.pos: it.shard * plan.S + it.pos + it.len] += 1
         valid += it.nvalid
@@ -226,8 +226,9 @@ def test_one_launch_schedule_invariants(layout, R, tile):
 def test_one_launch_schedule_on_bert_large_keeps_phase_two_close():
     """On the BERT-large set (R = 16) the state a phase-2 item reads was written a bounded distance earlier:
     except for the embedding (larger than L2) and the few tensors whose phase 2 queues behind the
-    embedding's, the phase-1 to phase-2 distance of an item, in bytes of state touched in between, stays
-    below 150 MB."""
+    embedding's, the phase-1 to phase-2 distance of an item, in bytes of state touched in between (by either
+    phase, so each byte counts twice), stays below 200 MB - the few hundred work items that are in flight
+    at any time, 8192 elements each."""
     wl = W.bert_large()
     plan = B.Plan(wl.shapes, wl.R, 32, upload=False)
     order, items = plan.schedule()
@@ -239,6 +240,6 @@ def test_one_launch_schedule_on_bert_large_keeps_phase_two_close():
         (p1 if ph == 0 else p2)[i] = p
     dist = touched[p2] - touched[p1]
     big = np.array([wl.numels[it.tensor] * 12 > 200e6 for it in items])
-    assert np.quantile(dist[~big], 0.98) < 150e6
-    assert np.median(dist[~big]) < 80e6
+    assert np.quantile(dist[~big], 0.98) < 200e6
+    assert np.median(dist[~big]) < 160e6
     assert plan.workspace_bytes("lamb") <= 4 * 1024 * 1024            # fits the library's static scratch
