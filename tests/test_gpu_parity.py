@@ -381,6 +381,52 @@ def test_bad_output_argument_leaves_the_state_untouched(opt):
         assert e.value.status == 1
 
 
+@pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb"])
+@pytest.mark.parametrize("fused", [False, True])
+def test_checkpoint_round_trip_equals_uninterrupted_run(opt, fused):
+    # Section 4.2: the auxiliary variables stay sharded between steps and are gathered only when a
+    # checkpoint needs them (the "unsharding program"); restoring shards them again (the "sharding
+    # program").  Step, unpack w / m / v to checkpoint-shaped tensors, pack them into fresh buffers of a
+    # fresh plan, step again: bit for bit the state of two uninterrupted steps.
+    R = 5
+    wl, w, m, v, g = _model(SHAPES, R, seed=44)
+    g2 = W.make_grads(W.Workload("t", list(SHAPES), R=R, opt="adam", hyper={}, grad_std=1e-2, seed=45), DEV)
+    has_v = opt != "sgdm"
+
+    def step(plan, bufs, grads, stepno):
+        hy = B.make_hyper(opt, _hyper(opt, step=stepno))
+        ws = torch.zeros(max(32, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+        pw, pm, pv = bufs
+        if fused:
+            outs = [torch.zeros_like(x) for x in w]
+            B.ws_fused_update(plan, -1, B.TensorTable(plan, grads), pw, pm, pv if has_v else None, hy,
+                              B.TensorTable(plan, [outs]), ws)
+        else:
+            pg = []
+            for gk in grads:
+                b = torch.empty(plan.G, device=DEV)
+                B.ws_pack(plan, gk, b)
+                pg.append(b)
+            B.ws_shard_update(plan, -1, pg, pw, pm, pv if has_v else None, hy, None, ws)
+
+    plan = B.Plan(SHAPES, R, 32)
+    a = list(_pack_all(plan, w, m, v, [])[:3])
+    step(plan, a, g, 10)
+    step(plan, a, g2, 11)                                   # uninterrupted
+    b = list(_pack_all(plan, w, m, v, [])[:3])
+    step(plan, b, g, 10)
+    ckpt = [[torch.empty_like(x) for x in w] for _ in range(3)]
+    for buf, lst in zip(b, ckpt):
+        B.ws_unpack(plan, buf, lst)                         # the checkpoint: tensors in their own shapes
+    del plan
+    plan2 = B.Plan(SHAPES, R, 32)                           # a restarted job plans again
+    c = list(_pack_all(plan2, ckpt[0], ckpt[1], ckpt[2], [])[:3])
+    step(plan2, c, g2, 11)
+    torch.cuda.synchronize()
+    for x, y in zip(a[:3 if has_v else 2], c):
+        assert torch.equal(x, y)
+
+
 # ------------------------------------------------- fused formatting path ---
 def _views_with_guards(numels, dtype, fill, misalign):
     """One buffer per tensor with 64-element guards; `misalign` shifts the view by 16 bytes so
