@@ -565,6 +565,25 @@ ws_status ws_lamb_update_static_scratch(const ws_plan* plan, const ws_grads* gra
                                         const ws_state* state, const ws_hyper* hyper,
                                         const ws_out* out, void* stream);
 
+/* ---------------------------------------------- bounds-checking debug build ---
+ * (Test infrastructure of the library, no counterpart in the paper.)  A copy of the library
+ * compiled with -DWS_DEBUG_BOUNDS (`python -m paper_2004_13336_b200.build --debug` builds it as
+ * libws_debug.so; the Python binding loads it when the environment variable WS_DEBUG_BOUNDS is 1)
+ * makes every kernel compare the range of each work item with the extents of the buffers it was
+ * given before it touches them.  A range outside them ORs a bit into a status word and the item is
+ * skipped; nothing traps or asserts.
+ *   ws_debug_bounds_enabled   1 in the debug build, 0 in the regular one
+ *   ws_debug_bounds_read      synchronises the device, returns the bits (1: w / m / v, 2: a packed
+ *                             gradient buffer, 4: the gathered buffer or the stored gradient sum,
+ *                             8: the flat buffer of ws_pack / ws_unpack, 0x40000000: the self-test)
+ *                             and clears them when `clear` is non-zero; WS_ERR_INVALID_ARG in the
+ *                             regular build
+ *   ws_debug_bounds_selftest  runs the check on an index outside its extent (no memory is
+ *                             accessed), so a test can see the bit arrive */
+int32_t ws_debug_bounds_enabled(void);
+ws_status ws_debug_bounds_read(uint32_t* bits, int32_t clear);
+ws_status ws_debug_bounds_selftest(void* stream);
+
 /* Static, never NULL. */
 const char* ws_status_string(ws_status s);
 /* Text of the last CUDA error seen by the calling thread inside this library

@@ -14,7 +14,9 @@ from typing import List, Optional, Sequence
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libws.so")
+# WS_DEBUG_BOUNDS=1 selects the bounds-checking debug build of the library (see ws.h)
+DEBUG_BOUNDS = os.environ.get("WS_DEBUG_BOUNDS", "") == "1"
+LIB_PATH = os.path.join(_PKG, "libws_debug.so" if DEBUG_BOUNDS else "libws.so")
 
 WS_OK = 0
 WS_F32, WS_BF16 = 0, 1
@@ -92,6 +94,7 @@ EXPORTS = [
     "ws_adafactor_stage", "ws_workspace_adafactor_sums",
     "ws_plan_schedule_bytes", "ws_plan_upload_schedule", "ws_plan_schedule_view", "ws_plan_schedule_item",
     "ws_workspace_sync_status",
+    "ws_debug_bounds_enabled", "ws_debug_bounds_read", "ws_debug_bounds_selftest",
 ]
 
 _lib = None
@@ -196,12 +199,25 @@ def lib() -> C.CDLL:
     L.ws_plan_schedule_item.argtypes = [vp, C.c_int64, C.POINTER(ws_sched_item)]
     L.ws_workspace_sync_status.restype = C.c_int
     L.ws_workspace_sync_status.argtypes = [vp, C.POINTER(C.c_size_t)]
+    L.ws_debug_bounds_enabled.restype = C.c_int32
+    L.ws_debug_bounds_enabled.argtypes = []
+    L.ws_debug_bounds_read.restype = C.c_int
+    L.ws_debug_bounds_read.argtypes = [C.POINTER(C.c_uint32), C.c_int32]
+    L.ws_debug_bounds_selftest.restype = C.c_int
+    L.ws_debug_bounds_selftest.argtypes = [vp]
     L.ws_status_string.restype = C.c_char_p
     L.ws_status_string.argtypes = [C.c_int]
     L.ws_last_cuda_error.restype = C.c_char_p
     L.ws_last_cuda_error.argtypes = []
     _lib = L
     return L
+
+
+def debug_bounds_read(clear: bool = True) -> int:
+    """Bits of the bounds-checking debug build's status word (synchronises the device)."""
+    bits = C.c_uint32()
+    _check(lib().ws_debug_bounds_read(C.byref(bits), 1 if clear else 0), "ws_debug_bounds_read")
+    return bits.value
 
 
 def _check(status: int, what: str):

@@ -1,10 +1,11 @@
 """Builds libws.so (the C-ABI CUDA library) in-tree with nvcc for sm_100a.
 
-    python -m paper_2004_13336_b200.build [--force] [--verbose]
+    python -m paper_2004_13336_b200.build [--force] [--verbose] [--debug]
 
 Each .cu file is compiled to an object in csrc/build/ (in parallel) and the
 objects are linked into paper_2004_13336_b200/libws.so.  nvcc cross-compiles
-without a GPU.
+without a GPU.  --debug builds the bounds-checking copy instead
+(-DWS_DEBUG_BOUNDS, objects in csrc/build_debug/, libws_debug.so).
 """
 from __future__ import annotations
 
@@ -17,7 +18,9 @@ _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 _CSRC = os.path.join(_PKG, "csrc")
 _OBJ = os.path.join(_CSRC, "build")
+_OBJ_DEBUG = os.path.join(_CSRC, "build_debug")
 LIB_PATH = os.path.join(_PKG, "libws.so")
+DEBUG_LIB_PATH = os.path.join(_PKG, "libws_debug.so")
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -43,21 +46,25 @@ def _deps_mtime() -> float:
     return max(os.path.getmtime(p) for p in paths)
 
 
-def up_to_date() -> bool:
-    return os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= _deps_mtime()
+def up_to_date(debug: bool = False) -> bool:
+    lib = DEBUG_LIB_PATH if debug else LIB_PATH
+    return os.path.exists(lib) and os.path.getmtime(lib) >= _deps_mtime()
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and up_to_date():
-        return LIB_PATH
-    os.makedirs(_OBJ, exist_ok=True)
+def build(force: bool = False, verbose: bool = False, debug: bool = False) -> str:
+    lib_path, obj_dir = (DEBUG_LIB_PATH, _OBJ_DEBUG) if debug else (LIB_PATH, _OBJ)
+    if not force and up_to_date(debug):
+        return lib_path
+    os.makedirs(obj_dir, exist_ok=True)
     nvcc = _nvcc()
     extra = ["-Xptxas", "-v"] if verbose else []
+    if debug:
+        extra.append("-DWS_DEBUG_BOUNDS")
     hdr_mtime = max(os.path.getmtime(os.path.join(_CSRC, f)) for f in os.listdir(_CSRC) if f.endswith(".h"))
     hdr_mtime = max(hdr_mtime, os.path.getmtime(os.path.join(_ROOT, "include", "ws.h")))
 
     def compile_one(src: str) -> str:
-        obj = os.path.join(_OBJ, src[:-3] + ".o")
+        obj = os.path.join(obj_dir, src[:-3] + ".o")
         spath = os.path.join(_CSRC, src)
         if (not force and os.path.exists(obj)
                 and os.path.getmtime(obj) >= max(os.path.getmtime(spath), hdr_mtime)):
@@ -72,13 +79,13 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
     with cf.ThreadPoolExecutor(max_workers=min(8, os.cpu_count() or 1)) as ex:
         objs = list(ex.map(compile_one, _sources()))
-    cmd = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", LIB_PATH, *objs]
+    cmd = [nvcc, "-shared", "-gencode", "arch=compute_100a,code=sm_100a", "-o", lib_path, *objs]
     res = subprocess.run(cmd, capture_output=True, text=True)
     if res.returncode != 0:
         raise RuntimeError(f"link failed:\n{res.stdout}\n{res.stderr}")
-    return LIB_PATH
+    return lib_path
 
 
 if __name__ == "__main__":
-    path = build(force="--force" in sys.argv, verbose="--verbose" in sys.argv)
+    path = build(force="--force" in sys.argv, verbose="--verbose" in sys.argv, debug="--debug" in sys.argv)
     print(path)

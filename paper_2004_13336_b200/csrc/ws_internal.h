@@ -153,6 +153,20 @@ WsLambWs ws_lamb_layout(const ws_plan* plan, void* workspace);
 // launches can refuse bad arguments before its first one).
 ws_status ws_lamb_check_apply_args(const ws_plan* plan, const ws_state* state, const ws_hyper* hyper, const ws_out* out);
 
+// Debug build (-DWS_DEBUG_BOUNDS): before a kernel touches a work item it compares the item's range
+// with the extents of the buffers it was given; a range outside them sets a bit in a status word that
+// the caller can read (ws_debug_bounds_read) and the item is skipped - no trap, no assert, no access.
+enum {
+    WS_BOUNDS_STATE = 1,      // w / m / v
+    WS_BOUNDS_GRAD = 2,       // a packed gradient buffer
+    WS_BOUNDS_OUT = 4,        // the gathered buffer or the stored gradient sum
+    WS_BOUNDS_FLAT = 8,       // the flat buffer of ws_pack / ws_unpack
+    WS_BOUNDS_SELFTEST = 0x40000000
+};
+#ifdef WS_DEBUG_BOUNDS
+unsigned* ws_bounds_word();   // device address of the status word on the current device, or null
+#endif
+
 // error bookkeeping
 ws_status ws_cuda_fail(cudaError_t e, const char* what);
 ws_status ws_check_launch(const char* what);

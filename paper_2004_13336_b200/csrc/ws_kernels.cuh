@@ -68,6 +68,12 @@ struct UpdParams {
     float* af_acc;          // Adafactor pass 1: [F] row / column sums of g^2 + eps1 (atomic adds)
     const float* af_fac;    // Adafactor passes 2, 3: [F] 1/sqrt factors of V
     WsConsts c;
+#ifdef WS_DEBUG_BOUNDS
+    unsigned* bounds;       // status word of the bounds checks
+    long long state_elems;  // elements of w / m / v as this launch addresses them
+    long long grad_elems;   // ... of every packed gradient buffer
+    long long out_elems;    // ... of the gathered buffer and of the stored gradient sum
+#endif
 };
 
 // ---------------------------------------------------------------- memory ---
@@ -373,6 +379,20 @@ __device__ __forceinline__ void process_item(const UpdParams& P, const GradPtrs<
     const int nvalid = it.nvalid;
     const long long gbase = it.gbase, sbase = it.sbase, obase = it.obase, toff = it.toff;
     const int nvec = it.len / VEC;
+#ifdef WS_DEBUG_BOUNDS
+    {
+        // every access of the item lies in [base, base + len) of its buffer: check the three ranges once
+        unsigned bits = 0;
+        if (sbase < 0 || sbase + it.len > P.state_elems) bits |= WS_BOUNDS_STATE;
+        if (READS_G && !FUSED && (gbase < 0 || gbase + it.len > P.grad_elems)) bits |= WS_BOUNDS_GRAD;
+        const bool uses_out = (WRITES_W && !FUSED && OUT != O_NONE) || READS_GHAT || WRITES_GHAT;
+        if (uses_out && (obase < 0 || obase + it.len > P.out_elems)) bits |= WS_BOUNDS_OUT;
+        if (bits) {                                    // uniform over the CTA: the item is skipped
+            if (threadIdx.x == 0 && P.bounds) atomicOr(P.bounds, bits);
+            return;
+        }
+    }
+#endif
     float sw = 0.f, su = 0.f;
     // Adafactor: where the tile starts inside its tensor's rows x cols matrix
     WsSegAf af = {};

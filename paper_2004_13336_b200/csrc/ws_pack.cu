@@ -27,6 +27,10 @@ struct PackParams {
     long long S;
     int seg_lo;           // tensor index of PtrChunk::p[0]
     int concat;           // concatenated layout: every tile names its own shard
+#ifdef WS_DEBUG_BOUNDS
+    unsigned* bounds;     // status word of the bounds checks
+    long long flat_elems; // elements of the flat buffer
+#endif
 };
 
 // VB-byte vector (16 or 32) moved with streaming accesses
@@ -78,6 +82,12 @@ __global__ void __launch_bounds__(kBlock) pack_kernel(PackParams P, const __grid
         const long long src0 = r * tl.piece + tl.poff;      // element index in the tensor
         long long nv = tl.vt - r * tl.piece;                // valid elements in this tile
         nv = nv < 0 ? 0 : (nv > tl.len ? (long long)tl.len : nv);
+#ifdef WS_DEBUG_BOUNDS
+        if (r * P.S + tl.pos < 0 || r * P.S + tl.pos + tl.len > P.flat_elems) {
+            if (threadIdx.x == 0 && P.bounds) atomicOr(P.bounds, (unsigned)WS_BOUNDS_FLAT);
+            continue;
+        }
+#endif
         char* fl = flat + (r * P.S + tl.pos) * EB;
         char* tn = tensor + src0 * EB;
         const int nvec = tl.len / EPV;
@@ -132,6 +142,12 @@ __global__ void __launch_bounds__(kBlock) pack_sets_kernel(PackParams P, const v
         const char* tn = (const char*)table[(long long)tl.seg * nsets + k] + (r * tl.piece + tl.poff) * EB;
         long long nv = tl.vt - r * tl.piece;
         nv = nv < 0 ? 0 : (nv > tl.len ? (long long)tl.len : nv);
+#ifdef WS_DEBUG_BOUNDS
+        if (r * P.S + tl.pos < 0 || r * P.S + tl.pos + tl.len > P.flat_elems) {
+            if (threadIdx.x == 0 && P.bounds) atomicOr(P.bounds, (unsigned)WS_BOUNDS_FLAT);
+            continue;
+        }
+#endif
         char* fl = (char*)flats.p[k] + (r * P.S + tl.pos) * EB;
         const int nvec = tl.len / EPV;
 #pragma unroll 4
@@ -197,6 +213,10 @@ ws_status run(const ws_plan* p, void* const* tensor_ptrs, ws_dtype dtype, void* 
         P.nitems = P.concat ? P.ntl : P.ntl * p->R;
         P.S = p->S;
         P.seg_lo = seg_lo;
+#ifdef WS_DEBUG_BOUNDS
+        P.bounds = ws_bounds_word();
+        P.flat_elems = (long long)p->R * p->S;
+#endif
         long long grid = P.nitems;   // one CTA per (shard, tile): the CTA scheduler walks the buffers in order
         if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;
         if (grid < 1) continue;
@@ -248,6 +268,10 @@ extern "C" ws_status ws_pack_sets(const ws_plan* p, const ws_tensor_table* table
     P.nitems = P.concat ? P.ntl : P.ntl * p->R;
     P.S = p->S;
     P.seg_lo = 0;
+#ifdef WS_DEBUG_BOUNDS
+    P.bounds = ws_bounds_word();
+    P.flat_elems = (long long)p->R * p->S;
+#endif
     long long grid = P.nitems * table->nsets;
     if (grid < 1) return WS_OK;
     if (grid > 0x7fffffffLL) grid = 0x7fffffffLL;

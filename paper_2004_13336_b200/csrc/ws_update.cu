@@ -514,6 +514,13 @@ ws_status prepare(const ws_plan* p, int32_t r, const ws_grads* g, const ws_state
     P.rho = nullptr;
     P.ghat = nullptr;
     P.c = make_consts(h);
+#ifdef WS_DEBUG_BOUNDS
+    P.bounds = ws_bounds_word();
+    P.state_elems = (long long)nshards * p->S;
+    // (one shard of a packed buffer: the pointers are advanced to the shard, S elements remain in view)
+    P.grad_elems = (g && g->slice_mode == 0 && r < 0) ? (long long)p->R * p->S : p->S;
+    P.out_elems = (long long)p->R * p->S;
+#endif
     return WS_OK;
 }
 
