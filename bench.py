@@ -47,11 +47,20 @@ FALLBACK_HBM_GBS = 6650.0
 HEADLINE = "decoder_1p5b"
 MIN_TIMED_S = 0.5
 
-# DRAM bytes per valid parameter (dram__bytes_read.sum + dram__bytes_write.sum of the dominant kernel's
-# launches ÷ parameters) from the ncu captures summarised under profiles/, taken on a clipped copy of
-# the workload (a few GB on the device) and scaled here by the parameter count: the kernels' traffic
-# is proportional to the elements they process.  Keyed by (workload, R, path).
+# DRAM bytes per valid parameter (dram__bytes_read.sum + dram__bytes_write.sum of the update's launches
+# ÷ parameters) from the ncu captures summarised under profiles/.  Workloads too large for a multi-pass
+# capture were captured on a smaller copy (every dimension clipped, or a few layers at full size) and are
+# scaled here by the parameter count: the kernels' traffic is proportional to the elements they process.
+# Keyed by (workload, R, path): (bytes per parameter, which capture).
 NCU_DRAM_BYTES_PER_PARAM = {
+    ("resnet50", 8, "fused"): (47.06, "profiles/fused_update_kernel_resnet50_sgdm_R8.md (full size)"),
+    ("decoder_1p5b", 4, "fused"): (33.73, "profiles/fused_update_kernel_decoder_bf16_R4.md (dimensions clipped to 1024)"),
+    ("transformer", 8, "fused"): (55.70, "profiles/fused_update_kernel_transformer_adam.md (dimensions clipped to 1024)"),
+    ("transformer", 1, "fused"): (27.46, "profiles/fused_update_kernel_transformer_adam.md (dimensions clipped to 1024)"),
+    ("bert_large", 16, "fused"): (89.4, "profiles/lamb_one_kernel_bert_large_R16.md (six layers at full size: 88.2; the "
+                                        "embeddings, a tenth of the parameters, counted at the two-pass 100)"),
+    ("resnet50_lars", 8, "fused"): (57.2, "profiles/fused_lars_kernels_resnet50_R8.md (full size)"),
+    ("transformer_adafactor", 8, "fused"): (55.5, "profiles/fused_adafactor_kernels_transformer.md (dimensions clipped to 1024)"),
 }
 
 
@@ -72,6 +81,8 @@ def parse_args():
     ap.add_argument("--out-dtype", default="", choices=["", "f32", "bf16"], help="override the emitted weight dtype")
     ap.add_argument("--clip", type=int, default=0,
                     help="clip every tensor dimension to this size (a small copy of the workload for profiler captures)")
+    ap.add_argument("--tensors", default="",
+                    help="A:B - keep only tensors A..B-1 of the workload's list (a few layers at full size, for profiler captures)")
     ap.add_argument("--shards", type=int, default=0,
                     help="shard count of the plan when it differs from the replica count (partial sharding)")
     ap.add_argument("--layout", default="per_tensor", choices=["per_tensor", "concat"],
@@ -97,7 +108,7 @@ def parse_args():
     return ap.parse_args()
 
 
-def get_workload(name, R=0, opt="", grad_dtype="", out_dtype="", clip=0):
+def get_workload(name, R=0, opt="", grad_dtype="", out_dtype="", clip=0, tensors=""):
     from paper_2004_13336_b200 import workloads as W
     wl = W.WORKLOADS[name]()
     if R:
@@ -116,12 +127,16 @@ def get_workload(name, R=0, opt="", grad_dtype="", out_dtype="", clip=0):
         wl.name += "*"          # not one of the named workloads any more
     if clip:
         wl = W.scaled_down(wl, clip)
+    if tensors:
+        a, b = (int(x) for x in tensors.split(":"))
+        wl.shapes = wl.shapes[a:b]
+        wl.name += f"[{a}:{b}]"
     return wl
 
 
 def workload_from_args(args):
     name = HEADLINE if args.workload == "all" else args.workload
-    return get_workload(name, args.R, args.opt, args.grad_dtype, args.out_dtype, args.clip)
+    return get_workload(name, args.R, args.opt, args.grad_dtype, args.out_dtype, args.clip, args.tensors)
 
 
 def measured_peak():
@@ -761,7 +776,9 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
     kernels = kernel_rows(primary)
     dom = max(kernels, key=lambda z: z["ms_per_step"])
     # the multi-launch optimizers' update is reported as one unit (its launches depend on one another)
-    traffic_pp = NCU_DRAM_BYTES_PER_PARAM.get((wl.name, wl.R, primary))
+    traffic_pp, traffic_src = NCU_DRAM_BYTES_PER_PARAM.get((wl.name, wl.R, primary), (None, None))
+    if layout != "per_tensor" or shards != R or (wl.opt == "lamb" and not one_kernel):
+        traffic_pp, traffic_src = None, None
     roofline = {"bound": "hbm", "kernel": dom["kernel"], "achieved": dom["achieved_gbs"], "peak": peak,
                 "peak_source": f"{peak_src} copy bandwidth", "unit": "GB/s", "frac": dom["frac"],
                 "algorithmic_bytes_per_launch": dom["algorithmic_bytes_per_step"],
@@ -769,7 +786,7 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
                 "moved_bytes_per_launch": dom["moved_bytes_per_step"],
                 "launch": f"one step's update = {dom['launches_per_step']} dependent launch(es), timed together",
                 "avg_launch_ms": dom["ms_per_step"],
-                "traffic": traffic_pp * N if traffic_pp else None,
+                "traffic": traffic_pp * N if traffic_pp else None, "traffic_source": traffic_src,
                 "frac_of_nominal_8TBs": dom["achieved_gbs"] / 8000.0}
     if wl.opt == "lamb":
         roofline["two_pass"] = {"bytes_per_param": bpp["algorithmic"] + 12,
@@ -906,7 +923,8 @@ def run_ours(args):
     head = measure(ctx, workload_from_args(args), align=args.align, layout=args.layout, shards=args.shards,
                    tile=args.tile, path=args.path, e2e=not args.no_e2e, cpu=not args.no_cpu_baseline, **common)
     release()
-    side = args.workload == "all" and ctx.world == 1 and not args.no_side_rows and not (args.R or args.opt or args.clip)
+    side = (args.workload == "all" and ctx.world == 1 and not args.no_side_rows
+            and not (args.R or args.opt or args.clip or args.tensors))
     if side:
         # one full record for each of the other named workloads
         head["configs"] = []
