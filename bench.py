@@ -518,6 +518,46 @@ class Ctx:
             dist.destroy_process_group()
 
 
+def copy_floor(torch, dev, nbytes):
+    """What a plain device-to-device copy that moves `nbytes` (half read, half written) achieves when it is
+    timed like a short kernel here: back to back over rotating buffer pairs larger than L2 together, and
+    alone on a drained GPU.  A launch of tens of microseconds cannot beat this by much: it is the ramp and
+    tail of any grid, not the kernel's code, that separates it from the copy bandwidth of a long launch."""
+    n = max(nbytes // 8, 1)
+    pairs = max(1, min(8, int(512e6 // max(nbytes, 1)) + 1))
+    try:
+        bufs = [(torch.empty(n, dtype=torch.float32, device=dev), torch.empty(n, dtype=torch.float32, device=dev))
+                for _ in range(pairs)]
+    except RuntimeError:
+        return None
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for a, b in bufs:
+        b.copy_(a)
+    torch.cuda.synchronize()
+    reps = max(2, min(40, int(4e-3 / (nbytes / 6.5e12)) // pairs + 1))
+    e0.record()
+    for _ in range(reps):
+        for a, b in bufs:
+            b.copy_(a)
+    e1.record()
+    torch.cuda.synchronize()
+    b2b = e0.elapsed_time(e1) / (reps * pairs)
+    iso = []
+    for i in range(15):
+        a, b = bufs[i % pairs]
+        e0.record()
+        b.copy_(a)
+        e1.record()
+        torch.cuda.synchronize()
+        iso.append(e0.elapsed_time(e1))
+    iso.sort()
+    pk = measured_peak()[0]
+    return {"what": "cudaMemcpyAsync device to device moving the same bytes, timed the same two ways",
+            "bytes": nbytes, "ms_back_to_back": b2b, "frac_back_to_back": nbytes / (b2b * 1e-3) / 1e9 / pk,
+            "ms_isolated_median": iso[len(iso) // 2],
+            "frac_isolated": nbytes / (iso[len(iso) // 2] * 1e-3) / 1e9 / pk}
+
+
 def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both", e2e=True, cpu=True,
             steps=20, warmup=5, e2e_steps=3, cpu_seconds=10.0):
     """One workload on this rank's GPU: the fused route (and the separate-kernel route), the roofline of
@@ -685,6 +725,30 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
                   "ms_median": med, "ms_min": times[0], "value": valid / (med * 1e-3), "unit": UNIT,
                   "achieved_gbs": valid * bytes_per_param(wl)["algorithmic"] / (med * 1e-3) / 1e9}
         single["frac"] = single["achieved_gbs"] / measured_peak()[0]
+        # The isolated figure carries the idle-to-first-CTA latency of a launch on a drained GPU (an empty
+        # kernel timed this way takes ~10 us).  Steady state: every shard's launch in turn, back to back, so
+        # that each reads different memory (R launches together read the whole model: nothing comes from L2).
+        if N * 4 * (R + 3) > 256e6:
+            def one_of_each():
+                for r_ in range(R):
+                    s_ = slice(r_ * S_, (r_ + 1) * S_)
+                    B.ws_shard_update(plan, r_, pg, pw[s_], pm[s_], pv[s_] if pv is not None else None, hy,
+                                      gathered, ws)
+            one_of_each()
+            rounds = max(2, min(50, int(2000 / (med * 1e3 * R)) + 1))
+            torch.cuda.synchronize()
+            ev[0].record()
+            for _ in range(rounds):
+                one_of_each()
+            ev[1].record()
+            torch.cuda.synchronize()
+            ss_ms = ev[0].elapsed_time(ev[1]) / (rounds * R)
+            ss_bytes = N / R * bytes_per_param(wl)["algorithmic"]
+            single["steady_state"] = {
+                "what": f"the {R} shards' launches in turn, back to back, {rounds} rounds; mean per launch",
+                "ms": ss_ms, "achieved_gbs": ss_bytes / (ss_ms * 1e-3) / 1e9,
+                "frac": ss_bytes / (ss_ms * 1e-3) / 1e9 / measured_peak()[0]}
+            single["copy_floor"] = copy_floor(torch, dev, int(ss_bytes))
 
     # ---- end to end through the host-buffer entry point
     e2e_rec = None
@@ -765,6 +829,8 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
                     {"kernel": "pack_kernel (unpack weights)", "launches_per_step": chunks,
                      "ms_per_step": ph[2], "algorithmic_bytes_per_step": N * bpp["unpack"],
                      "moved_bytes_per_step": N * bpp["unpack"]}]
+        if pth == "unfused" and rows[2]["ms_per_step"] < 0.2:
+            rows[2]["copy_floor"] = copy_floor(torch, dev, int(N * bpp["unpack"]))
         tot = sum(r_["ms_per_step"] for r_ in rows)
         for r_ in rows:
             r_["achieved_gbs"] = r_["algorithmic_bytes_per_step"] / (r_["ms_per_step"] * 1e-3) / 1e9

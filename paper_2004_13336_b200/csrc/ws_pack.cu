@@ -69,16 +69,36 @@ __device__ __forceinline__ Vec<VB> zero_vec() {
     return v;
 }
 
+// Programmatic dependent launch: the grid may become resident while the previous kernel of the stream
+// drains; the kernels read only tables that were uploaded once before their griddepcontrol.wait.
+template <typename... KArgs, typename... Args>
+static void launch_pdl(void (*kernel)(KArgs...), long long grid, int block, cudaStream_t st, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3((unsigned)block);
+    cfg.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // EB = element bytes (4 or 2); PACK = true: tensors -> flat, false: flat -> tensors; VB = vector bytes
 template <int EB, bool PACK, int VB>
 __global__ void __launch_bounds__(kBlock) pack_kernel(PackParams P, const __grid_constant__ PtrChunk tab,
                                                       char* __restrict__ flat) {
     constexpr int EPV = VB / EB;  // elements per vector
+    // the next kernel of the stream may start its prologue while this grid's last CTAs run
+    asm volatile("griddepcontrol.launch_dependents;");
     for (long long item = blockIdx.x; item < P.nitems; item += gridDim.x) {
         long long r = P.concat ? 0 : item / P.ntl;
         const WsTile tl = P.tiles[P.tile_lo + (item - r * P.ntl)];
         if (P.concat) r = tl.shard;
         char* tensor = (char*)tab.p[tl.seg - P.seg_lo];
+        // the plan's tile table does not depend on the previous kernel of the stream; the data does
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         const long long src0 = r * tl.piece + tl.poff;      // element index in the tensor
         long long nv = tl.vt - r * tl.piece;                // valid elements in this tile
         nv = nv < 0 ? 0 : (nv > tl.len ? (long long)tl.len : nv);
@@ -133,6 +153,7 @@ __global__ void __launch_bounds__(kBlock) pack_sets_kernel(PackParams P, const v
                                                            const __grid_constant__ FlatPtrs flats) {
     constexpr int EPV = VB / EB;
     const long long total = P.nitems * nsets;
+    asm volatile("griddepcontrol.launch_dependents;");
     for (long long gi = blockIdx.x; gi < total; gi += gridDim.x) {
         const int k = (int)(gi / P.nitems);
         const long long item = gi - (long long)k * P.nitems;
@@ -140,6 +161,8 @@ __global__ void __launch_bounds__(kBlock) pack_sets_kernel(PackParams P, const v
         const WsTile tl = P.tiles[item - r * P.ntl];
         if (P.concat) r = tl.shard;
         const char* tn = (const char*)table[(long long)tl.seg * nsets + k] + (r * tl.piece + tl.poff) * EB;
+        // tile and pointer tables were uploaded once; the previous kernel of the stream may own the data
+        asm volatile("griddepcontrol.wait;" ::: "memory");
         long long nv = tl.vt - r * tl.piece;
         nv = nv < 0 ? 0 : (nv > tl.len ? (long long)tl.len : nv);
 #ifdef WS_DEBUG_BOUNDS
@@ -222,11 +245,11 @@ ws_status run(const ws_plan* p, void* const* tensor_ptrs, ws_dtype dtype, void* 
         if (grid < 1) continue;
         const int nb = pack_block(p, eb, wide ? 32 : 16);
         if (wide) {
-            if (dtype == WS_F32) pack_kernel<4, PACK, 32><<<(unsigned)grid, nb, 0, st>>>(P, tab, (char*)flat);
-            else                 pack_kernel<2, PACK, 32><<<(unsigned)grid, nb, 0, st>>>(P, tab, (char*)flat);
+            if (dtype == WS_F32) launch_pdl(pack_kernel<4, PACK, 32>, grid, nb, st, P, tab, (char*)flat);
+            else                 launch_pdl(pack_kernel<2, PACK, 32>, grid, nb, st, P, tab, (char*)flat);
         } else {
-            if (dtype == WS_F32) pack_kernel<4, PACK, 16><<<(unsigned)grid, nb, 0, st>>>(P, tab, (char*)flat);
-            else                 pack_kernel<2, PACK, 16><<<(unsigned)grid, nb, 0, st>>>(P, tab, (char*)flat);
+            if (dtype == WS_F32) launch_pdl(pack_kernel<4, PACK, 16>, grid, nb, st, P, tab, (char*)flat);
+            else                 launch_pdl(pack_kernel<2, PACK, 16>, grid, nb, st, P, tab, (char*)flat);
         }
         ws_status s = ws_check_launch(PACK ? "ws_pack" : "ws_unpack");
         if (s != WS_OK) return s;
@@ -281,12 +304,13 @@ extern "C" ws_status ws_pack_sets(const ws_plan* p, const ws_tensor_table* table
     for (int k = 0; k < table->nsets; ++k) wide = wide && (reinterpret_cast<uintptr_t>(flats[k]) & 31u) == 0;
     const void* const* tb = (const void* const*)table->dev;
     const int nb = pack_block(p, eb, wide ? 32 : 16);
+    const int ns = table->nsets;
     if (wide) {
-        if (table->dtype == WS_F32) pack_sets_kernel<4, 32><<<(unsigned)grid, nb, 0, st>>>(P, tb, table->nsets, fp);
-        else                        pack_sets_kernel<2, 32><<<(unsigned)grid, nb, 0, st>>>(P, tb, table->nsets, fp);
+        if (table->dtype == WS_F32) launch_pdl(pack_sets_kernel<4, 32>, grid, nb, st, P, tb, ns, fp);
+        else                        launch_pdl(pack_sets_kernel<2, 32>, grid, nb, st, P, tb, ns, fp);
     } else {
-        if (table->dtype == WS_F32) pack_sets_kernel<4, 16><<<(unsigned)grid, nb, 0, st>>>(P, tb, table->nsets, fp);
-        else                        pack_sets_kernel<2, 16><<<(unsigned)grid, nb, 0, st>>>(P, tb, table->nsets, fp);
+        if (table->dtype == WS_F32) launch_pdl(pack_sets_kernel<4, 16>, grid, nb, st, P, tb, ns, fp);
+        else                        launch_pdl(pack_sets_kernel<2, 16>, grid, nb, st, P, tb, ns, fp);
     }
     return ws_check_launch("ws_pack_sets");
 }
