@@ -880,6 +880,12 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
             "step_ms": ur["stats"], "clocks": ctx.sampler.summary(*ur["window"])}
         if single is not None:
             rec["unfused_path"]["single_shard"] = single
+    if one_kernel:
+        # the one-kernel route's waits are bounded; a wait that ran out leaves 1 in the workspace's status word
+        off = plan.sync_status_offset()
+        rec["config"]["one_kernel_wait_status"] = int(ws[off:off + 4].view(torch.int32).item())
+        if rec["config"]["one_kernel_wait_status"] != 0:
+            raise RuntimeError("one-kernel LAMB: a bounded wait ran out (status word set); the update is incomplete")
     if unfused_skipped:
         rec["unfused_path"] = {"skipped": unfused_skipped}
     if e2e_rec is not None:

@@ -60,7 +60,7 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
     extra = ["-Xptxas", "-v"] if verbose else []
     if debug:
         extra.append("-DWS_DEBUG_BOUNDS")
-    hdr_mtime = max(os.path.getmtime(os.path.join(_CSRC, f)) for f in os.listdir(_CSRC) if f.endswith(".h"))
+    hdr_mtime = max(os.path.getmtime(os.path.join(_CSRC, f)) for f in os.listdir(_CSRC) if f.endswith((".h", ".cuh")))
     hdr_mtime = max(hdr_mtime, os.path.getmtime(os.path.join(_ROOT, "include", "ws.h")))
 
     def compile_one(src: str) -> str:

@@ -61,6 +61,8 @@ struct UpdParams {
     const void* const* gtab; // fused formatting: device table [T][R] of gradient tensor pointers
     void* const* wtab;       // fused formatting: device table [T][nw] of weight tensor pointers (outputs)
     int nw;                  // number of weight lists written (1, or one per replica)
+    int keep;                // norm pairs, phase 1: leave w and what phase 2 reads again in L2 (small models)
+    int reverse;             // norm pairs, phase 2: walk the items back to front (phase 1's last items are still in L2)
     float2* partials;       // phase 1: [R][ntiles] partial sums of the two norms
     const float* rho;       // phase 2: [T] trust ratio (LAMB) / local rate (LARS)
     float* ghat;            // LARS, Adafactor: [R][S] summed gradients, written by phase 1, read afterwards
