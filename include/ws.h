@@ -16,14 +16,15 @@
  *   - Nothing throws or aborts across this boundary; every failure is a
  *     ws_status.  Argument errors are found on the host before any launch.
  *   - The caller owns every buffer.  The library owns only ws_plan objects.
- *   - The update kernels use programmatic dependent launch: a kernel may start
- *     while the preceding kernel of the stream drains, but before it waits for
- *     that kernel it reads nothing except the plan's tables and the
- *     tensor-pointer tables.  Those tables must therefore be complete before
- *     the kernel that precedes an update call on the stream is launched:
+ *   - The pack, unpack and update kernels use programmatic dependent launch:
+ *     a kernel may start while the preceding kernel of the stream drains, but
+ *     before it waits for that kernel it reads nothing except the plan's
+ *     tables and the tensor-pointer tables.  Those tables must therefore be
+ *     complete before the kernel that precedes such a call on the stream is
+ *     launched:
  *     upload them with ws_plan_upload / ws_tensor_table_upload (copies, which
  *     a later kernel never overtakes) and do not rewrite them from a kernel
- *     of your own directly in front of an update call.
+ *     of your own directly in front of such a call.
  *   - Accuracy a caller may expect against the same update in exact
  *     arithmetic, per tensor, as max_i |x_i - ref_i| / max(|ref_i|, RMS(ref)):
  *     1e-6 for the fp32 outputs of WS_SGDM and WS_ADAM, 1e-5 for WS_LAMB,
