@@ -798,6 +798,14 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
             del zg, zw
         except Exception as ex:
             e2e_rec["zero_copy"] = {"error": str(ex)[:200]}
+        # Both are public calls that take host buffers; the headline is the faster one (the staged copies
+        # run one direction of PCIe at a time, the kernel that reads and writes host memory uses both).
+        zc = e2e_rec["zero_copy"]
+        if "ms_per_step" in zc and zc["ms_per_step"] < e2e_rec["ms_per_step"]:
+            staged = {k_: e2e_rec[k_] for k_ in ("value", "ms_per_step", "api")}
+            e2e_rec.update({"value": zc["value"], "ms_per_step": zc["ms_per_step"], "api": zc["api"],
+                            "staged_copies": staged})
+            del e2e_rec["zero_copy"]
         del host_g, host_w, stage
     if rank != 0:
         return None

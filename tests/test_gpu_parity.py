@@ -857,6 +857,42 @@ def test_step_host_from_pinned_arenas_matches_oracle(opt, gdtype, odtype):
         assert err(bf16_to_f64(got) if odtype == torch.bfloat16 else got, ref) <= tol
 
 
+@pytest.mark.parametrize("opt,gdtype,odtype", [("sgdm", torch.float32, torch.float32),
+                                               ("adam", torch.bfloat16, torch.bfloat16),
+                                               ("lamb", torch.float32, torch.float32)])
+def test_fused_update_on_pinned_host_tensors_matches_oracle(opt, gdtype, odtype):
+    # the end-to-end step without staging copies: the gradient and weight tensors are pinned host memory,
+    # the kernel reads and writes them over PCIe; the sharded state stays on the device
+    R = 8 if opt == "lamb" else 3
+    wl, w, m, v, g = _model(SHAPES, R, gdtype, seed=37)
+    plan = B.Plan(SHAPES, R, 32)
+    h = _hyper(opt)
+    ow, om, _, _ = _oracle_unsharded(opt, h, w, m, v, g)
+    pw, pm, pv, _ = _pack_all(plan, w, m, v, [])
+    n_el, numels = plan.arena_elems, wl.numels
+    host_g = []
+    for gk in g:
+        a = torch.zeros(n_el, dtype=gdtype).pin_memory()
+        for dst, src in zip(plan.arena_views(a, numels), gk):
+            dst.copy_(src)
+        host_g.append(a)
+    host_w = torch.zeros(n_el, dtype=odtype).pin_memory()
+    master = odtype == torch.float32
+    if master:                                     # fp32 weights: the host tensors are the master copy
+        for dst, src in zip(plan.arena_views(host_w, numels), w):
+            dst.copy_(src)
+    gt = B.TensorTable(plan, [plan.arena_views(a, numels) for a in host_g], device=DEV)
+    wt = B.TensorTable(plan, [plan.arena_views(host_w, numels)], device=DEV)
+    ws = torch.zeros(max(32, plan.workspace_bytes(opt)), dtype=torch.uint8, device=DEV)
+    B.ws_fused_update(plan, -1, gt, None if master else pw, pm, pv if opt != "sgdm" else None,
+                      B.make_hyper(opt, h), wt, ws)
+    torch.cuda.synchronize()
+    tol = TOL_BF16 if odtype == torch.bfloat16 else (TOL_LAMB if opt == "lamb" else TOL_FP32)
+    for got, ref in zip(plan.arena_views(host_w, numels), ow):
+        got = to_np(got)
+        assert err(bf16_to_f64(got) if odtype == torch.bfloat16 else got, ref) <= tol
+
+
 def test_more_than_1024_tensors():
     # tensor pointers travel in kernel parameters in chunks of 1024: a list longer than that
     # takes several pack launches; the update and the fused route see one table
