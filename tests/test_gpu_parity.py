@@ -628,12 +628,13 @@ def test_step_can_be_captured_in_a_cuda_graph():
         assert torch.equal(a, b)
 
 
-@pytest.mark.parametrize("opt", ["lamb", "lars"])
-def test_multi_launch_steps_can_be_captured_in_a_cuda_graph(opt):
-    # the norm-based optimizers are three launches joined by programmatic dependent launch: the
-    # captured graph replays to the same bits as the eager calls (fixed-order sums)
-    wl, w, m, v, g = _model(SHAPES, 3, seed=14, gstd=1e-3)
-    plan = B.Plan(SHAPES, 3, 32)
+@pytest.mark.parametrize("opt,R", [("lamb", 3), ("lamb", 8), ("lars", 3)])
+def test_multi_launch_steps_can_be_captured_in_a_cuda_graph(opt, R):
+    # the norm-based optimizers are three launches joined by programmatic dependent launch - or, for LAMB
+    # with 8 copies, a clear of the counters and the one kernel: the captured graph replays to the same
+    # bits as the eager calls (fixed-order sums)
+    wl, w, m, v, g = _model(SHAPES, R, seed=14, gstd=1e-3)
+    plan = B.Plan(SHAPES, R, 32)
     h = _lars_hyper() if opt == "lars" else _hyper(opt)
     hy = B.make_hyper(opt, h)
     pw, pm, pv, pg = _pack_all(plan, w, m, v, g)
@@ -654,6 +655,9 @@ def test_multi_launch_steps_can_be_captured_in_a_cuda_graph(opt):
     graph.replay()
     torch.cuda.synchronize()
     assert torch.equal(pw, ew) and torch.equal(pm, em)
+    if opt == "lamb" and R == 8:
+        off = plan.sync_status_offset()
+        assert int(ws[off:off + 4].view(torch.int32).item()) == 0
 
 
 @pytest.mark.parametrize("opt", ["sgdm", "adam", "lamb"])
