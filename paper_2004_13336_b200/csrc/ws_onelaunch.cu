@@ -70,7 +70,7 @@ two_phase_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp, con
     __shared__ unsigned long long s_word;      // the ticket, later the tensor's ready word
     __shared__ const void* sgp[FUSED ? NP : 1];
     __shared__ float2 red[kBlock / 32];
-    __shared__ double fin_a[kBlock], fin_b[kBlock];
+    __shared__ double fin_a[kBlock / 32], fin_b[kBlock / 32];   // (small on purpose: shared memory comes out of the L1)
     __shared__ int s_last;
     const int tid = threadIdx.x;
 
@@ -134,19 +134,23 @@ two_phase_kernel(const UpdParams P, const __grid_constant__ GradPtrs<NP> gp, con
             a += (double)p.x;
             b += (double)p.y;
         }
-        fin_a[tid] = a;
-        fin_b[tid] = b;
-        __syncthreads();
-        for (int h = kBlock / 2; h > 0; h >>= 1) {
-            if (tid < h) {
-                fin_a[tid] += fin_a[tid + h];
-                fin_b[tid] += fin_b[tid + h];
-            }
-            __syncthreads();
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {                    // fixed tree inside the warp ...
+            a += __shfl_xor_sync(0xffffffffu, a, o);
+            b += __shfl_xor_sync(0xffffffffu, b, o);
         }
+        if ((tid & 31) == 0) {
+            fin_a[tid >> 5] = a;
+            fin_b[tid >> 5] = b;
+        }
+        __syncthreads();
         if (tid == 0) {
-            a = fin_a[0];
-            b = fin_b[0];
+            a = 0.0;
+            b = 0.0;
+            for (int i = 0; i < kBlock / 32; ++i) {           // ... and the warps in order
+                a += fin_a[i];
+                b += fin_b[i];
+            }
             Q.norms[2 * it.seg] = a;
             Q.norms[2 * it.seg + 1] = b;
             float ratio = 1.0f;
