@@ -675,17 +675,37 @@ def measure(ctx, wl, align=32, layout="per_tensor", shards=0, tile=0, path="both
             est.append(ev[0].elapsed_time(ev[nev - 1]))
         inner = inner_repeats(reduce_max(min(est), dev), K, args.min_timed_s)
         n = K * inner
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nev)] for _ in range(n)]
-        ctx.barrier()
-        t0 = time.time()
-        for i in range(n):
-            step(evs[i])
-        ctx.barrier()
-        t1 = time.time()
-        total_ms = evs[0][0].elapsed_time(evs[-1][nev - 1])
-        if flush is not None:   # leave the L2 flush out of the step time
+        if flush is None:
+            # the timed region: n steps back to back between two events, nothing else on the stream
+            e_start, e_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            ctx.barrier()
+            t0 = time.time()
+            e_start.record()
+            for i in range(n):
+                step()
+            e_end.record()
+            ctx.barrier()
+            t1 = time.time()
+            total_ms = e_start.elapsed_time(e_end)
+            # afterwards, a short pass with events around every kernel: the kernels' shares and each step's
+            # own duration (an event between two launches keeps the second from starting under the first's tail)
+            evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nev)] for _ in range(min(n, 64))]
+            for e in evs:
+                step(e)
+            torch.cuda.synchronize()
+        else:
+            # small inputs: the L2 is flushed in front of every step, so every step is timed by itself
+            evs = [[torch.cuda.Event(enable_timing=True) for _ in range(nev)] for _ in range(n)]
+            ctx.barrier()
+            t0 = time.time()
+            for i in range(n):
+                step(evs[i])
+            ctx.barrier()
+            t1 = time.time()
             total_ms = sum(e[0].elapsed_time(e[nev - 1]) for e in evs)
-        phase_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / n for i in range(nev - 1)]
+        phase_ms = [sum(e[i].elapsed_time(e[i + 1]) for e in evs) / len(evs) for i in range(nev - 1)]
+        if nev == 2 and flush is None:
+            phase_ms = [total_ms / n]          # one update per step: its duration is the region's mean
         total_ms = reduce_max(total_ms, dev)
         per_step = sorted(e[0].elapsed_time(e[nev - 1]) for e in evs)      # each step's own launches
         stats = {"median": per_step[len(per_step) // 2], "min": per_step[0], "max": per_step[-1],
