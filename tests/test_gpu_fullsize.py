@@ -260,6 +260,48 @@ def test_bert_large_lamb_whole_tensors():
     assert worst_rho <= TOL_LAMB and worst_w <= TOL_LAMB and worst_mv <= TOL_FP32
 
 
+@pytest.mark.parametrize("name", ["resnet50", "transformer", "bert_large"])
+def test_benchmark_configuration_fp32_master_weights_full_size(name):
+    """What bench.py times for the fp32 workloads: ws_fused_update on all shards with the weight tensors as
+    the master copy (no sharded w), for BERT-large as one kernel.  Every weight tensor, m and v must equal
+    the separate-kernel route bit for bit (which the tests above tie to the oracle), two steps in a row."""
+    wl = W.WORKLOADS[name]()
+    torch.cuda.empty_cache()
+    plan = B.Plan(wl.shapes, wl.R, A)
+    w, m, v = W.make_state(wl, DEV)
+    has_v = wl.opt in ("adam", "lamb")
+    pw = torch.empty(plan.G, device=DEV)
+    pm, pv = torch.empty_like(pw), torch.empty_like(pw)
+    for src, dst in ((w, pw), (m, pm), (v, pv)):
+        B.ws_pack(plan, src, dst)
+    fm, fv = pm.clone(), pv.clone()
+    del m, v
+    glists = [W.make_grads_one(wl, k, DEV) for k in range(wl.R)]
+    gtab, wtab = B.TensorTable(plan, glists), B.TensorTable(plan, [w])
+    ws = torch.full((max(32, plan.workspace_bytes(wl.opt)),), 0x5A, dtype=torch.uint8, device=DEV)
+    ws2 = torch.full_like(ws, 0xA5)
+    pg = []
+    for gk in glists:
+        b = torch.empty(plan.G, device=DEV)
+        B.ws_pack(plan, gk, b)
+        pg.append(b)
+    for step in (10, 11):
+        hy = B.make_hyper(wl.opt, dict(wl.hyper, step=step))
+        B.ws_shard_update(plan, -1, pg, pw, pm, pv if has_v else None, hy, None, ws)
+        B.ws_fused_update(plan, -1, gtab, None, fm, fv if has_v else None, hy, wtab, ws2)
+    torch.cuda.synchronize()
+    del pg
+    assert torch.equal(fm, pm) and (not has_v or torch.equal(fv, pv))
+    ref = [torch.empty_like(x) for x in w]
+    B.ws_unpack(plan, pw, ref)
+    for t, (a, b) in enumerate(zip(w, ref)):
+        assert torch.equal(a, b), f"tensor {t}"
+    if wl.opt == "lamb":
+        assert torch.equal(B.lamb_ratios(plan, ws), B.lamb_ratios(plan, ws2))
+        off = plan.sync_status_offset()
+        assert int(ws2[off:off + 4].view(torch.int32).item()) == 0
+
+
 def test_bert_large_lamb_fused_equals_unfused():
     """The benchmark's configuration for config 4: ws_fused_update (three launches) from the 16
     gradient lists.  Same arithmetic and same tiling as the packed path, so every output is
