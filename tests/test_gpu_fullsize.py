@@ -260,7 +260,7 @@ def test_bert_large_lamb_whole_tensors():
     assert worst_rho <= TOL_LAMB and worst_w <= TOL_LAMB and worst_mv <= TOL_FP32
 
 
-@pytest.mark.parametrize("name", ["resnet50", "transformer", "bert_large"])
+@pytest.mark.parametrize("name", ["resnet50", "transformer", "bert_large", "resnet50_lars"])
 def test_benchmark_configuration_fp32_master_weights_full_size(name):
     """What bench.py times for the fp32 workloads: ws_fused_update on all shards with the weight tensors as
     the master copy (no sharded w), for BERT-large as one kernel.  Every weight tensor, m and v must equal
