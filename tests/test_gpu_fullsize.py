@@ -409,6 +409,20 @@ def test_transformer_adafactor_whole_tensors():
         worst_f = max(worst_f, err(got_f[off:off + nr + nc], ref_f[off:off + nr + nc]))
     print(f"transformer Adafactor: err w {worst_w:.2e} factored state {worst_f:.2e} step size {worst_c:.2e}")
     assert worst_w <= TOL_LAMB and worst_f <= TOL_LAMB and worst_c <= TOL_LAMB
+    # the form the benchmark times: the fp32 weight tensors are the master copy (no sharded w); the row and
+    # column sums are combined by atomic adds, so the two runs agree to rounding, not bit for bit
+    master = [x.clone() for x in w]
+    fs2 = f0.clone()
+    ws2 = torch.empty_like(ws)
+    B.ws_fused_update(plan, -1, B.TensorTable(plan, g), None, None, fs2, hy, B.TensorTable(plan, [master]), ws2)
+    worst_m = max(err(to_np(master[t]), ref_w[t]) for t in chosen)
+    worst_mf = max(err(to_np(fs2)[lay[t][0]:lay[t][0] + lay[t][1] + lay[t][2]],
+                       ref_f[lay[t][0]:lay[t][0] + lay[t][1] + lay[t][2]]) for t in chosen)
+    print(f"transformer Adafactor, weight tensors as master: err w {worst_m:.2e} factored state {worst_mf:.2e}")
+    assert worst_m <= TOL_LAMB and worst_mf <= TOL_LAMB
+    for t in range(wl.T):
+        if wl.numels[t]:
+            assert err(to_np(master[t]), to_np(outs[t]).astype(np.float64)) <= 1e-6
     # the sharded weight state and the weight tensors hold the same values
     B.ws_unpack(plan, pw, w)
     for t in chosen:
