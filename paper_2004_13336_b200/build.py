@@ -40,6 +40,13 @@ def _sources():
     return sorted(f for f in os.listdir(_CSRC) if f.endswith(".cu"))
 
 
+def _headers():
+    """Every header a .cu file may include: a change to any of them recompiles every object."""
+    hs = [os.path.join(_CSRC, f) for f in sorted(os.listdir(_CSRC)) if f.endswith((".h", ".cuh"))]
+    hs.append(os.path.join(_ROOT, "include", "ws.h"))
+    return hs
+
+
 def _deps_mtime() -> float:
     paths = [os.path.join(_CSRC, f) for f in os.listdir(_CSRC) if f.endswith((".cu", ".h", ".cuh"))]
     paths.append(os.path.join(_ROOT, "include", "ws.h"))
@@ -60,8 +67,7 @@ def build(force: bool = False, verbose: bool = False, debug: bool = False) -> st
     extra = ["-Xptxas", "-v"] if verbose else []
     if debug:
         extra.append("-DWS_DEBUG_BOUNDS")
-    hdr_mtime = max(os.path.getmtime(os.path.join(_CSRC, f)) for f in os.listdir(_CSRC) if f.endswith((".h", ".cuh")))
-    hdr_mtime = max(hdr_mtime, os.path.getmtime(os.path.join(_ROOT, "include", "ws.h")))
+    hdr_mtime = max(os.path.getmtime(h) for h in _headers())
 
     def compile_one(src: str) -> str:
         obj = os.path.join(obj_dir, src[:-3] + ".o")

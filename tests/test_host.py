@@ -243,3 +243,18 @@ def test_one_launch_schedule_on_bert_large_keeps_phase_two_close():
     assert np.quantile(dist[~big], 0.98) < 200e6
     assert np.median(dist[~big]) < 160e6
     assert plan.workspace_bytes("lamb") <= 4 * 1024 * 1024            # fits the library's static scratch
+
+
+def test_build_tracks_every_header_the_kernels_include():
+    """A change to any header of the kernel sources (.h and .cuh, and the public ws.h) must recompile every
+    object: objects built against different versions of a shared struct would still link."""
+    import re
+    from paper_2004_13336_b200 import build as WB
+    tracked = {os.path.basename(h) for h in WB._headers()}
+    csrc = os.path.join(ROOT, "paper_2004_13336_b200", "csrc")
+    included = set()
+    for f in os.listdir(csrc):
+        if f.endswith((".cu", ".cuh", ".h")):
+            with open(os.path.join(csrc, f)) as fh:
+                included |= set(re.findall(r'#include\s+"([^"]+)"', fh.read()))
+    assert included and {os.path.basename(i) for i in included} <= tracked
