@@ -277,7 +277,7 @@ class Plan:
                  device: Optional[torch.device] = None, upload: bool = True, layout: str = "per_tensor",
                  one_launch: bool = True):
         """``one_launch``: also upload the plan's one-launch schedule, so that the all-shard LAMB and LARS
-        updates run as one persistent kernel (with ``False`` they run as three launches)."""
+        updates run as one kernel (with ``False`` they run as three launches)."""
         T = len(shapes)
         descs = (ws_tensor_desc * max(1, T))()
         for i, s in enumerate(shapes):

@@ -67,7 +67,7 @@ struct WsAfChunk {
 };
 
 // One-launch schedule of the norm-based optimizers (LAMB, LARS): the update of all shards as ONE
-// persistent kernel.  A work item is a run of at most kWsItemElems consecutive shard positions inside
+// kernel.  A work item is a run of at most kWsItemElems consecutive shard positions inside
 // one tile; every item appears twice in the schedule, once for phase 1 (reduce, moments, partial
 // norm sums) and once for phase 2 (apply the step with the tensor's ratio).
 constexpr int kWsItemElems = 8192;

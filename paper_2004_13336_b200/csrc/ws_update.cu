@@ -657,7 +657,7 @@ ws_status af_update(const ws_plan* plan, int32_t r, const ws_grads* grads, const
                     const ws_state* state, const ws_hyper* hyper, const ws_out* out, const ws_tensor_table* wtab,
                     void* workspace, size_t workspace_bytes, cudaStream_t st);
 
-// LAMB (pair 0) or LARS (pair 1) for all shards as one persistent kernel, when the plan's one-launch
+// LAMB (pair 0) or LARS (pair 1) for all shards as one kernel, when the plan's one-launch
 // schedule is on the device and the number of gradient copies is supported; `done` says whether the
 // update was enqueued here (false: the caller runs the separate launches).  Either the packed-buffer
 // arguments (grads, out) or the tensor tables (gtab, wtab) are given.

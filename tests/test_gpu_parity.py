@@ -724,7 +724,7 @@ def test_lars_matches_oracle_and_fused_equals_unfused(R, gdtype):
 @pytest.mark.parametrize("gdtype,layout,fused", [(torch.float32, "per_tensor", False), (torch.bfloat16, "per_tensor", True),
                                                  (torch.float32, "concat", True), (torch.bfloat16, "concat", False)])
 def test_one_launch_update_equals_three_launches(opt, R, gdtype, layout, fused):
-    # The all-shard LAMB / LARS update as ONE persistent kernel (plan with its one-launch schedule) against
+    # The all-shard LAMB / LARS update as ONE kernel (plan with its one-launch schedule) against
     # the three launches (phase 1, combination, phase 2): same elementwise arithmetic, the norm sums grouped
     # by work item instead of by tile, so ratios agree to rounding; the status word stays 0; two steps in
     # a row (the second finds the first's counters and flags in the workspace).  The one-kernel route is
