@@ -456,6 +456,12 @@ void ws_build_schedule(ws_plan* p) {
     long long ai = 0, bi = 0;                     // next phase-1 / phase-2 item
     long long eligible = 0;                       // phase-2 items of groups whose phase 1 ended >= kLag entries ago
     int last_kind = 1;
+    // phase 2 walks every group back to front: the items phase 1 wrote last are the ones most likely to be
+    // in L2 still, and a group larger than the L2 then keeps its tail instead of nothing (reading it front
+    // to back would evict each line just before its turn)
+    std::vector<unsigned> p2item((size_t)n);
+    for (const Group& g : groups)
+        for (int i = g.first; i < g.end; ++i) p2item[(size_t)i] = (unsigned)(g.end - 1 - (i - g.first));
     while (bi < n) {
         const long long pos = (long long)p->sched.size();
         while (eg < ag && pos - p1_done_at[eg] >= kLag) {
@@ -474,7 +480,7 @@ void ws_build_schedule(ws_plan* p) {
         } else {
             // (at the very end the last groups' phase 2 follows their phase 1 directly: the scheduling
             // warps then wait for the ratios, a few microseconds once per launch)
-            p->sched.push_back((unsigned)(bi << 1) | 1u);
+            p->sched.push_back((p2item[(size_t)bi] << 1) | 1u);
             last_kind = 1;
             ++bi;
             if (!may2) eligible = bi;             // keep the backlog arithmetic consistent in the tail

@@ -216,8 +216,22 @@ def test_one_launch_schedule_invariants(layout, R, tile):
         assert p > last1[tens[i]]
         if p - last1[tens[i]] < 512:
             early += 1
-    # phase-1 items run in item order, so do phase-2 items (tickets are handed out in this order)
-    assert [i for i, ph in order if ph == 0] == list(range(n)) and [i for i, ph in order if ph == 1] == list(range(n))
+    # phase-1 items run in item order (tickets are handed out in this order); phase 2 takes the groups of
+    # tensors in the same order but walks each group back to front (its last items are the freshest in L2):
+    # the sequence is a chain of descending runs, each a contiguous block of indices, blocks ascending
+    assert [i for i, ph in order if ph == 0] == list(range(n))
+    seq2 = [i for i, ph in order if ph == 1]
+    assert sorted(seq2) == list(range(n))
+    lo_expected, k = 0, 0
+    while k < n:
+        hi = seq2[k]
+        j = k
+        while j + 1 < n and seq2[j + 1] == seq2[j] - 1:
+            j += 1
+        assert seq2[j] == lo_expected and hi >= seq2[j]
+        lo_expected = hi + 1
+        k = j + 1
+    assert lo_expected == n
     # only the tail (after the last phase-1 entry) may hold phase-2 items that follow their tensor closely
     end1 = max(pos1.values())
     assert all(p > end1 for i, p in pos2.items() if p - last1[tens[i]] < 512)
@@ -227,7 +241,7 @@ def test_one_launch_schedule_on_bert_large_keeps_phase_two_close():
     """On the BERT-large set (R = 16) the state a phase-2 item reads was written a bounded distance earlier:
     except for the embedding (larger than L2) and the few tensors whose phase 2 queues behind the
     embedding's, the phase-1 to phase-2 distance of an item, in bytes of state touched in between (by either
-    phase, so each byte counts twice), stays below 200 MB - the few hundred work items that are in flight
+    phase, so each byte counts twice), stays below 260 MB - the few hundred work items that are in flight
     at any time, 8192 elements each."""
     wl = W.bert_large()
     plan = B.Plan(wl.shapes, wl.R, 32, upload=False)
@@ -240,8 +254,11 @@ def test_one_launch_schedule_on_bert_large_keeps_phase_two_close():
         (p1 if ph == 0 else p2)[i] = p
     dist = touched[p2] - touched[p1]
     big = np.array([wl.numels[it.tensor] * 12 > 200e6 for it in items])
-    assert np.quantile(dist[~big], 0.98) < 200e6
+    # (phase 2 walks a group back to front: the items written last are read first - a tenth of all items at
+    # less than 100 MB - and the first-written ones last)
+    assert np.quantile(dist[~big], 0.98) < 260e6
     assert np.median(dist[~big]) < 160e6
+    assert np.quantile(dist[~big], 0.10) < 100e6
     assert plan.workspace_bytes("lamb") <= 4 * 1024 * 1024            # fits the library's static scratch
 
 
