@@ -233,10 +233,11 @@ ws_status launch_o(const UpdParams& P, const void* const* gptrs, const OneLaunch
 }  // namespace
 
 // Where the one-kernel route measured faster than the three launches on a B200: LAMB with 8 to 32
-// gradient copies (BERT-large set, R = 16: 4.91 ms against 5.16 ms; Transformer set under LAMB: 2 %
-// faster at R = 8, 3 % at R = 32).  With few copies phase 1 is as short as phase 2 and the three
-// launches win (Transformer set, R = 2: 1.38 ms against 1.47 ms), and so they do for LARS on the
-// ResNet-50 set, whose 161 mostly tiny tensors make a step of 0.25 ms.
+// gradient copies (BERT-large set, R = 16: 4.87 ms against 5.13 ms, R = 8: 3.27 against 3.46 ms;
+// Transformer set under LAMB: 5 % faster at R = 8, 3.6 % at R = 32).  With few copies phase 1 is as
+// short as phase 2 and the three launches win (Transformer set, R = 4: 1.64 ms against 1.67 ms, R = 2:
+// 1.38 against 1.49 ms), and so they do for LARS on the ResNet-50 set, whose 161 mostly tiny tensors
+// make a step of 0.24 ms.
 bool one_launch_supports(int pair, int R) { return pair == 0 && R >= 8 && R <= 32; }
 
 ws_status launch_one_launch(int pair, bool gbf, int out, bool fused, bool wide, const UpdParams& P,

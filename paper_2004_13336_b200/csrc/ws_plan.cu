@@ -388,7 +388,6 @@ extern "C" size_t ws_workspace_bytes(const ws_plan* p, ws_opt opt) {
 // items are waiting (a tensor larger than L2 has just finished) they run first.
 namespace {
 constexpr long long kGroupBytes = 6LL << 20;    // state bytes (12 per element) that close a group
-constexpr long long kKeepHi = 200LL << 20;      // larger groups cannot stay in L2: their state is streamed
 constexpr int kLag = 512;
 
 void ws_build_schedule(ws_plan* p) {
@@ -436,7 +435,9 @@ void ws_build_schedule(ws_plan* p) {
                 const int gend = p->itemsegs[t].first + p->itemsegs[t].count;
                 if (gend > gfirst) {
                     groups.push_back(Group{gfirst, gend});
-                    const unsigned keep = acc < kKeepHi ? 1u : 0u;
+                    // (every group leaves its state in L2 at normal priority: phase 2 reads a group back to
+                    // front, so even a tensor many times the L2 finds its last-written part there)
+                    const unsigned keep = 1u;
                     for (int i = gfirst; i < gend; ++i) p->items[i].flags = keep;
                 }
                 gfirst = gend;
