@@ -17,7 +17,7 @@ Without --workload the line is the largest single-GPU workload (decoder_1p5b:
 1.56 G parameters, bf16 gradients, R = 4) and carries, under `configs`, one full
 record for each of the other named workloads, under `transformer_r_sweep` the
 Transformer set at R = 1 ... 1024 and alignments 8 and 32, and under
-`next_workloads` the LARS, Adafactor and concatenated-layout runs.
+`next_workloads` the LARS, Adafactor, concatenated-layout and partial-sharding runs.
 
 Whatever K is, the timed region lasts at least half a second: it covers
 K x `inner_repeats` back-to-back steps and `ms_per_step` is their mean.
@@ -988,7 +988,8 @@ def short_row(rec):
         return None
     rf = rec["roofline"]
     row = {"workload": rec["config"]["workload"], "R": rec["config"]["R"], "align_elems": rec["config"]["align_elems"],
-           "layout": rec["config"]["layout"], "value": rec["value"], "unit": UNIT, "ms_per_step": rec["ms_per_step"],
+           "layout": rec["config"]["layout"], "shards": rec["config"].get("shards", rec["config"]["R"]),
+           "value": rec["value"], "unit": UNIT, "ms_per_step": rec["ms_per_step"],
            "timed_steps": rec["config"].get("timed_steps", rec["steps"]),
            "algorithmic_bytes_per_param": rf.get("algorithmic_bytes_per_param"),
            "achieved_gbs": rf["achieved"], "frac_of_measured_peak": rf["frac"],
@@ -1047,7 +1048,9 @@ def run_ours(args):
         nxt = []
         for name, kw in (("resnet50_lars", {}), ("transformer_adafactor", {}),
                          ("bert_large", {"layout": "concat"}), ("decoder_1p5b", {"layout": "concat"}),
-                         ("transformer", {"layout": "concat", "R": 1024})):
+                         ("transformer", {"layout": "concat", "R": 1024}),
+                         # partial sharding (Section 5.2): 8 gradient copies, the update sharded 2 ways
+                         ("transformer", {"shards": 2, "R": 8})):
             R_ = kw.pop("R", 0)
             nxt.append(guarded(lambda: short_row(measure(
                 ctx, get_workload(name, R=R_), align=args.align, path="fused", e2e=False, cpu=False, **kw, **common)),
