@@ -32,11 +32,13 @@
  *     bf16 ulp (2^-8 relative) for bf16 outputs.  These hold for gradients of
  *     the scale of the state they update (the library's test recipe: standard
  *     deviation 1e-3, up to 1024 copies).  Single elements can reach 1e-5
- *     under WS_ADAM when gradient copies ten times larger are summed (not
- *     averaged) over 8 or more replicas, the copies cancel and the element's
- *     second moment starts at (almost) zero: the fp32 sum then carries an
- *     error that is large against the cancelled total.  That is a property of
- *     fp32 summation, not of the sharding.
+ *     (2.4e-5 seen) under WS_ADAM when gradient copies ten times larger are
+ *     summed (not averaged) over 8 or more replicas, the copies cancel and
+ *     the element's second moment starts at (almost) zero: the fp32 sum then
+ *     carries an error that is large against the cancelled total, and the
+ *     step divides by its root.  That is a property of fp32 summation (a
+ *     pairwise fp32 sum of the same copies gives the library's value bit for
+ *     bit), not of the sharding.
  *   - dtype arguments say how 2- or 4-byte elements are interpreted.
  *
  * Layout vocabulary (Section 4.1 "Sharding representation", Section 5.2
